@@ -1,0 +1,252 @@
+/*
+ * pcm_b200.h - C ABI of the B200 (sm_100a) GRPO actor update with Probabilistic Chunk Masking.
+ *
+ * One training iteration of Algorithm 1 maps onto five calls, in this order:
+ *
+ *   pcm_score_phases       Eq. 1 (advantages) and Eq. 5 (success-failure action variance per phase)
+ *   pcm_update_keep_probs  Eq. 7-9 (score buffer, share / max normalisation, floor p_min)
+ *   pcm_sample_chunks      Eq. 10 (fixed-budget weighted sampling without replacement)
+ *   grpo_pack_chunks       Sec. 4.5 "physical shrinking": dense batch of the kept chunks only
+ *   grpo_actor_fwd_bwd     Eq. 11 (masked GRPO objective, with the PPO clip of App. E): loss + gradients
+ *
+ * Conventions
+ *   - Every pointer named "device" is device memory owned by the caller; the library neither frees
+ *     nor reallocates it.  Host pointers are marked "host".  `stream` is a cudaStream_t.
+ *   - All device work is enqueued on `stream`; calls return without synchronising unless stated.
+ *   - Return value: PCM_OK (0) or a negative pcm_status.  Nothing is printed; no exception crosses
+ *     the boundary.  Bad arguments are rejected on the host before anything is launched.
+ *     Device-side problems (a phase label >= n_phases, a trajectory longer than max_len, a bounded
+ *     wait that ran out) are latched in a status word read by pcm_poll_status().
+ *   - Trajectories g*G .. g*G+G-1 form rollout group g (G = group_size).
+ *   - Chunks are stored CSR style: trajectory i owns chunks traj_off[i] .. traj_off[i+1]-1.
+ *   - A chunk is 56 action tokens (8 actions x 7 degrees of freedom, Sec. 5.1) over 256 bins.
+ *   - Every linear weight is stored row-major [out_features][in_features] (y = x W^T).
+ */
+#ifndef PCM_B200_H
+#define PCM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PCM_ACT_DIM 56
+#define PCM_N_BINS 256
+#define PCM_MAX_PHASES 32
+#define PCM_MAX_TRC 16
+
+typedef enum {
+  PCM_OK = 0,
+  PCM_ERR_ARG = -1,            /* null pointer, value out of range                                */
+  PCM_ERR_SHAPE = -2,          /* sizes the kernels do not support (see each call)                */
+  PCM_ERR_WORKSPACE = -3,      /* workspace too small or misaligned                               */
+  PCM_ERR_CUDA = -4,           /* a CUDA runtime / driver call failed                             */
+  PCM_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired                              */
+  PCM_ERR_STATE = -6,          /* state blob of the wrong size / version                          */
+  PCM_ERR_DEVICE_DATA = -7     /* device-side data check failed, e.g. phase label >= n_phases     */
+} pcm_status;
+
+typedef void* pcm_stream;      /* cudaStream_t */
+typedef struct pcm_ctx pcm_ctx;
+
+typedef struct {
+  int32_t n_phases;            /* the paper's K, 1..PCM_MAX_PHASES                                */
+  int32_t budget;              /* the paper's B: chunks kept per trajectory, >= 1                 */
+  int32_t group_size;          /* G rollouts per group, >= 1                                      */
+  int32_t t_rc;                /* refresh window T_rc, 1..PCM_MAX_TRC                             */
+  double p_min;                /* keep-probability floor, in (0, 1]                               */
+  double adv_eps;              /* epsilon of Eq. 1                                                */
+  uint64_t seed;               /* Philox key of the sampler                                       */
+} pcm_config;
+
+typedef struct {
+  int32_t n_traj;              /* multiple of group_size                                          */
+  int32_t n_chunks;            /* traj_off[n_traj]                                                */
+  int32_t max_len;             /* upper bound on chunks per trajectory (sizes shared memory)      */
+  int32_t reserved;
+  const int32_t* traj_off;     /* device [n_traj+1]                                               */
+  const uint8_t* tok;          /* device [n_chunks][56], 4-byte aligned                           */
+  const uint8_t* phase;        /* device [n_chunks], labels < n_phases, any order                 */
+  const uint8_t* reward;       /* device [n_traj], 0 or 1                                         */
+  const void* obs;             /* device [n_chunks][P][d] in the model dtype; pack only           */
+  const float* logp_old;       /* device [n_chunks][56]; pack only                                */
+} pcm_batch;
+
+/* ---- context: configuration, persistent keep-probability state, small scratch ---------------- */
+
+/* Creates a context on the current device.  Allocates device memory for the keep-probability
+ * state, the status word and per-group score scratch: about 9 * n_phases bytes per group for
+ * max_traj / group_size groups, plus a few KB.  Batches passed later may hold at most max_traj
+ * trajectories. */
+int pcm_create(pcm_ctx** out, const pcm_config* cfg, int32_t max_traj);
+int pcm_destroy(pcm_ctx* ctx);
+
+/* Reads and clears the device status word (synchronises `stream`).  Returns PCM_OK,
+ * PCM_ERR_DEVICE_TIMEOUT or PCM_ERR_DEVICE_DATA. */
+int pcm_poll_status(pcm_ctx* ctx, pcm_stream stream);
+
+/* Keep-probability state (buffers B_c, step counter, p_c) as a flat host blob, so that a chain of
+ * iterations can be stopped and resumed bit-exactly.  Both calls synchronise the device.
+ * pcm_state_export: *bytes in = capacity of host_buf, out = bytes needed / written; with
+ * host_buf == NULL only the size is reported. */
+int pcm_state_export(pcm_ctx* ctx, void* host_buf, size_t* bytes);
+int pcm_state_import(pcm_ctx* ctx, const void* host_buf, size_t bytes);
+
+/* ---- Eq. 1 + Eq. 5 ---------------------------------------------------------------------------
+ * For every group with both outcomes present and every phase c that has chunks from a successful
+ * and from a failed rollout of that group:
+ *     C_{c,g} = || mean_{success chunks in c} a - mean_{failure chunks in c} a ||_2
+ * with a the 56-vector of bin-centre values a = -1 + (tok + 1/2) * 2/256.  C[c] is the mean of
+ * C_{c,g} over the groups where it is defined (ascending g); valid[c] = 0 and C[c] = 0 when there
+ * is none (uniform-reward groups are ignored, a phase missing from one outcome is skipped).
+ * Token sums are exact integers; the remaining fp64 operations are individually rounded IEEE
+ * operations in a fixed order, so the result does not depend on the launch shape.
+ * adv (may be NULL) receives Eq. 1 with population variance: A_i = (r_i - mu) / (sigma + adv_eps).
+ * Outputs: device C[n_phases] f64, valid[n_phases] u8, n_valid_groups[n_phases] i32 (may be NULL),
+ * adv[n_traj] f32. */
+int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* batch, double* C, uint8_t* valid,
+                     int32_t* n_valid_groups, float* adv, pcm_stream stream);
+
+/* ---- Eq. 7-9, Algorithm 1 ---------------------------------------------------------------------
+ * Appends C (0 where valid[c] == 0) to the phase buffers.  On the first call, or when the buffers
+ * hold t_rc entries: S_c = sum of buffer, rho_c = S_c / sum S, rho~_c = rho_c / max rho,
+ * p_c = max(p_min, rho~_c); buffers cleared.  If every S_c is 0 the previous p_c is kept.
+ * Otherwise p_c is unchanged.  The state lives in the context (device memory).
+ * Outputs: device p[n_phases] f32 and q[n_phases] u32 = round-half-even(p_c * 2^24), the integer
+ * chunk weight used by pcm_sample_chunks. */
+int pcm_update_keep_probs(pcm_ctx* ctx, const double* C, const uint8_t* valid, float* p, uint32_t* q,
+                          pcm_stream stream);
+
+/* ---- Eq. 10 -----------------------------------------------------------------------------------
+ * For every trajectory draws m_i = min(budget, N_i) chunks by successive sampling without
+ * replacement (Plackett-Luce) with integer weights w_ik = q[phase(i,k)].  Draw r of trajectory i
+ * takes 64 bits from Philox4x32-10 with key (seed lo, seed hi) and counter (iter lo, i, r, iter hi),
+ * maps them to x = floor(bits * W_remaining / 2^64) and selects the first remaining chunk, in index
+ * order, whose running weight sum exceeds x.  When m_i = N_i every chunk is kept and no random
+ * numbers are consumed.  max_len <= 12000.
+ * Outputs: device kept_idx[sum m_i] i32 global chunk ids, trajectory-major and ascending within a
+ * trajectory (capacity n_traj*budget is always enough); kept_off[n_traj+1] i32;
+ * kept_per_phase[n_phases] i32 (may be NULL). */
+int pcm_sample_chunks(pcm_ctx* ctx, const pcm_batch* batch, const uint32_t* q, uint64_t iter,
+                      int32_t* kept_idx, int32_t* kept_off, int32_t* kept_per_phase, pcm_stream stream);
+
+/* ---- model ----------------------------------------------------------------------------------- */
+typedef enum { GRPO_F32 = 0, GRPO_BF16 = 1 } grpo_dtype;
+
+typedef struct {
+  int32_t d;                   /* model width, multiple of 8                                      */
+  int32_t n_layers;            /* 1..128                                                          */
+  int32_t n_heads;             /* head dim d / n_heads in {32, 64, 128}                           */
+  int32_t prefix_len;          /* P observation-prefix tokens per chunk, >= 1; S = P + 56 <= 384  */
+  int32_t dtype;               /* grpo_dtype of weights, observations and activations             */
+  int32_t reserved;
+} grpo_model_cfg;
+
+/* Decoder-only policy: per layer RMSNorm(g1) -> fused QKV -> rotary embedding (base 10000, pairs
+ * (i, i + dh/2)) -> causal attention within the chunk -> W_o + residual -> RMSNorm(g2) -> SwiGLU
+ * (gate rows first, then up rows, hidden 4d) -> W_d + residual; then RMSNorm(gf) and the 256-bin
+ * head.  RMSNorm epsilon 1e-5.  All tensors device, in cfg.dtype. */
+typedef struct {
+  grpo_model_cfg cfg;
+  const void* w_qkv;           /* [L][3d][d]                                                      */
+  const void* w_o;             /* [L][d][d]                                                       */
+  const void* w_gu;            /* [L][8d][d]                                                      */
+  const void* w_d;             /* [L][d][4d]                                                      */
+  const void* g1;              /* [L][d]                                                          */
+  const void* g2;              /* [L][d]                                                          */
+  const void* gf;              /* [d]                                                             */
+  const void* w_h;             /* [256][d]                                                        */
+  const void* e_act;           /* [256][d]                                                        */
+} grpo_model;
+
+/* fp32 gradients with the shapes of grpo_model (device). */
+typedef struct {
+  float* w_qkv; float* w_o; float* w_gu; float* w_d; float* g1; float* g2; float* gf; float* w_h; float* e_act;
+} grpo_grads;
+
+/* Dense batch of kept chunks, caller-allocated device views. */
+typedef struct {
+  int32_t n_kept;
+  int32_t reserved;
+  void* X;                     /* [n_kept][S][d] model dtype: prefix rows then E_act[token] rows  */
+  uint8_t* tgt;                /* [n_kept][56] action tokens                                      */
+  float* lpo;                  /* [n_kept][56] behaviour-policy log-probs                         */
+  float* adv_c;                /* [n_kept] advantage of the owning trajectory                     */
+  int32_t* src;                /* [n_kept] global chunk id                                        */
+} grpo_packed;
+
+/* ---- Sec. 4.5 physical shrinking ----------------------------------------------------------------
+ * Copies the kept chunks, in kept_idx order, into the dense batch: X[j] = [obs[kept_idx[j]] ;
+ * E_act[tok[kept_idx[j]][0..55]]], plus targets, old log-probs, advantage and source id.  A pure
+ * byte copy (bit-exact).  Requires d * sizeof(dtype) to be a multiple of 16 and at most 32768, and
+ * 16-byte aligned obs, E_act and X.  n_kept = out->n_kept must equal kept_off[n_traj] (<= 65535). */
+int grpo_pack_chunks(pcm_ctx* ctx, const pcm_batch* batch, const grpo_model_cfg* cfg,
+                     const int32_t* kept_idx, const int32_t* kept_off, const void* e_act,
+                     const float* adv, grpo_packed* out, pcm_stream stream);
+
+/* ---- Eq. 11 ------------------------------------------------------------------------------------ */
+#define GRPO_FWD_ONLY 1u       /* forward only: writes logp (and loss), touches no gradient       */
+#define GRPO_ACCUMULATE 2u     /* add into grads instead of overwriting them                      */
+
+typedef struct {
+  float eps_low;               /* clip range [1 - eps_low, 1 + eps_high]                          */
+  float eps_high;
+  float loss_scale;            /* <= 0: token mean 1 / (56 * n_kept)                              */
+  int32_t mb_chunks;           /* chunks per micro-batch, >= 1                                    */
+  uint32_t flags;
+  int32_t reserved;
+} grpo_loss_cfg;
+
+typedef struct {
+  float loss;
+  float clip_frac;             /* fraction of action tokens whose surrogate gradient is clipped   */
+  float mean_ratio;
+  int32_t n_launches;          /* kernels launched by this call                                   */
+  uint64_t workspace_high_water;
+} grpo_stats;
+
+/* Bytes of workspace grpo_actor_fwd_bwd needs for micro-batches of mb_chunks chunks (activations
+ * are kept, not recomputed).  0 when cfg is not supported. */
+size_t grpo_workspace_bytes(const grpo_model_cfg* cfg, int32_t mb_chunks, uint32_t flags);
+
+/* Forward and backward of the policy on the packed batch under
+ *     loss = -loss_scale * sum_{kept chunks} sum_{j<56} min(r_j A, clip(r_j, 1-eps_low, 1+eps_high) A),
+ *     r_j = exp(logp_j - lpo_j), logp_j = log softmax(z_j)[tgt_j], z_j = head(position P-1+j).
+ * A term's gradient is r_j A when (A >= 0 and r_j <= 1+eps_high) or (A < 0 and r_j >= 1-eps_low),
+ * else 0.  The batch is processed in micro-batches of mb_chunks chunks; gradients accumulate in
+ * fp32, so the micro-batch size only changes the rounding order.  No gradient reaches the
+ * observation prefix.
+ * Outputs: device loss[1] f32; device logp[n_kept][56] f32 (may be NULL); grads (ignored with
+ * GRPO_FWD_ONLY); host stats (may be NULL; when given the call synchronises `stream` and returns
+ * PCM_ERR_DEVICE_TIMEOUT if a bounded device-side wait expired).
+ * workspace: device, 256-byte aligned, >= grpo_workspace_bytes(). */
+int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* batch, const grpo_loss_cfg* loss_cfg,
+                       grpo_grads* grads, float* loss, float* logp, grpo_stats* stats,
+                       void* workspace, size_t workspace_bytes, pcm_stream stream);
+
+/* ---- diagnostic entry points (per-kernel tests and measurements; not part of Algorithm 1) -------
+ * grpo_gemm: C[m][n] = sum_k A(m,k) B(n,k) (+ R[m][n]) with the GEMM kernels the actor update uses.
+ * a_kmajor != 0: A is stored [M][K] with row stride lda, else [K][M]; likewise B ([N][K] / [K][N]).
+ * ab_dtype / c_dtype are grpo_dtype values; R (fp32, may be NULL) may alias C to accumulate (C fp32).
+ * backend: 0 = automatic, 1 = SIMT kernel, 2 = tcgen05 kernel (PCM_ERR_SHAPE when it cannot take the
+ * problem).  Synchronises `stream`; returns PCM_ERR_DEVICE_TIMEOUT when a bounded wait expired. */
+int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_kmajor, const void* B,
+              int64_t ldb, int32_t b_kmajor, int32_t ab_dtype, void* C, int64_t ldc, int32_t c_dtype,
+              const float* R, int64_t ldr, int32_t backend, pcm_stream stream);
+
+/* grpo_attention: causal attention inside each of n_seq sequences of S tokens, as used by the actor
+ * update.  qkv [n_seq*S][3d] holds q | k | v (rotary embedding already applied), out [n_seq*S][d],
+ * lse [n_seq][H][S] fp32.  With dout != NULL also runs the backward pass: dqkv [n_seq*S][3d],
+ * scratch [n_seq][H][S] fp32.  Synchronises `stream`. */
+int grpo_attention(int32_t dtype, const void* qkv, void* out, float* lse, const void* dout, void* dqkv,
+                   float* scratch, int32_t n_seq, int32_t S, int32_t n_heads, int32_t head_dim, pcm_stream stream);
+
+/* Number of kernels this library has launched in the calling process (for accounting). */
+int64_t pcm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PCM_B200_H */

@@ -1,0 +1,39 @@
+// Internal interfaces between the translation units of the library (not part of the C ABI).
+#pragma once
+#include "common.cuh"
+
+namespace pcm {
+
+enum { DT_F32 = 0, DT_BF16 = 1 };
+
+// C[m][n] = sum_k A(m,k) * B(n,k)  (+ R[m][n] when R != nullptr; R may alias C to accumulate).
+// An operand is "K-major" when its contraction index is contiguous in memory:
+//   a_kmajor: A stored [M][K] with row stride lda;   otherwise A stored [K][M] with row stride lda.
+//   b_kmajor: B stored [N][K] with row stride ldb;   otherwise B stored [K][N] with row stride ldb.
+struct GemmArgs {
+  int M, N, K;
+  const void* A; long long lda; bool a_kmajor;
+  const void* B; long long ldb; bool b_kmajor;
+  int ab_dtype;                 // DT_F32 or DT_BF16 (both operands)
+  void* C; long long ldc; int c_dtype;
+  const float* R; long long ldr;
+};
+
+enum GemmBackend { GEMM_AUTO = 0, GEMM_SIMT = 1, GEMM_TCGEN05 = 2 };
+
+int gemm(const GemmArgs& g, cudaStream_t s, GemmBackend backend = GEMM_AUTO);
+int gemm_simt(const GemmArgs& g, cudaStream_t s);
+int gemm_tcgen05(const GemmArgs& g, cudaStream_t s);
+bool gemm_tcgen05_supported(const GemmArgs& g);
+// Reads and clears the tensor-core kernels' device status word (synchronous copy).
+int tcgen05_poll_status();
+
+// Causal attention within each sequence of S tokens.  qkv [n_seq*S][3d] (q | k | v, heads of dh
+// inside each), out [n_seq*S][d], lse [n_seq][H][S].
+int attention_fwd(int dtype, const void* qkv, void* out, float* lse, int n_seq, int S, int H, int dh,
+                  cudaStream_t s);
+// dqkv [n_seq*S][3d] receives dq | dk | dv.  dsum [n_seq][H][S] is scratch.
+int attention_bwd(int dtype, const void* qkv, const void* out, const void* dout, const float* lse, float* dsum,
+                  void* dqkv, int n_seq, int S, int H, int dh, cudaStream_t s);
+
+}  // namespace pcm

@@ -1,0 +1,494 @@
+// PCM control plane on the device: advantages (Eq. 1), phase scores (Eq. 5), online keep-probability
+// update (Eq. 7-9), fixed-budget weighted sampling on a Philox stream (Eq. 10), and the context that
+// holds the persistent state.
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace pcm {
+std::atomic<long long> g_launches{0};
+
+constexpr int ACT = PCM_ACT_DIM;           // 56 action tokens per chunk
+constexpr int WORDS = ACT / 4;             // 14 32-bit words per chunk
+constexpr int STATE_VERSION = 1;
+
+struct KeepState {                         // persistent, device resident
+  double buf[PCM_MAX_PHASES][PCM_MAX_TRC]; // phase-score buffers B_c
+  double p[PCM_MAX_PHASES];                // keep-probabilities p_c
+  long long step;
+  int count;                               // entries currently in every buffer
+  int n_refresh;
+};
+
+struct StateBlob {                         // host representation for export / import
+  int version;
+  int n_phases;
+  int t_rc;
+  int pad;
+  KeepState st;
+};
+
+}  // namespace pcm
+
+struct pcm_ctx {
+  pcm_config cfg;
+  int max_traj;
+  int device;
+  pcm::KeepState* state;       // device
+  unsigned* status;            // device status word
+  double* c_group;             // device [max_groups][n_phases]
+  uint8_t* valid_group;        // device [max_groups][n_phases]
+};
+
+namespace pcm {
+
+unsigned* ctx_status(pcm_ctx* c) { return c->status; }
+
+// ------------------------------------------------------------------------------------------------
+// Eq. 5, per group: integer token sums per (phase, outcome), then C_{c,g}
+// ------------------------------------------------------------------------------------------------
+// One CTA per group.  A warp walks whole trajectories; lanes 0..27 cover two chunks per step (14
+// words each).  Four tokens travel in one 32-bit word and are accumulated as two words of two 16-bit
+// lanes; a run ends when the phase changes or after 256 chunks (255 * 257 < 2^16), and is then
+// flushed to 32-bit shared-memory counters.  Integer sums are exact, so any order gives the same
+// result.
+__global__ void __launch_bounds__(256)
+score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restrict__ tok,
+                    const uint8_t* __restrict__ phase, const uint8_t* __restrict__ reward, int G,
+                    int n_phases, double* __restrict__ c_group, uint8_t* __restrict__ valid_group,
+                    unsigned* __restrict__ status) {
+  extern __shared__ unsigned sm[];
+  unsigned* sums = sm;                                   // [n_phases][2][56]
+  unsigned* cnt = sm + n_phases * 2 * ACT;               // [n_phases][2]
+  const int g = blockIdx.x;
+  for (int i = threadIdx.x; i < n_phases * 2 * (ACT + 1); i += blockDim.x) sm[i] = 0;
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int sub = lane / WORDS;                          // 0, 1 active; 2 idle
+  const int word = lane - sub * WORDS;
+  const uint32_t* tokw = reinterpret_cast<const uint32_t*>(tok);
+
+  for (int i = g * G + warp; i < (g + 1) * G; i += nwarps) {
+    const int o = reward[i] ? 1 : 0;
+    const int a = traj_off[i], b = traj_off[i + 1];
+    unsigned acc_lo = 0, acc_hi = 0, run = 0;
+    int cur = -1;
+    auto flush = [&]() {
+      if (run) {
+        unsigned* s = sums + (cur * 2 + o) * ACT + word * 4;
+        atomicAdd(s + 0, acc_lo & 0xFFFFu);
+        atomicAdd(s + 1, acc_hi & 0xFFFFu);
+        atomicAdd(s + 2, acc_lo >> 16);
+        atomicAdd(s + 3, acc_hi >> 16);
+        if (word == 0) atomicAdd(cnt + cur * 2 + o, run);
+      }
+      acc_lo = acc_hi = run = 0;
+    };
+    if (sub < 2) {
+      for (int ch0 = a + sub; ch0 < b; ch0 += 8) {       // four chunk pairs per iteration
+        uint32_t wv[4];
+        int ph[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int ch = ch0 + 2 * u;
+          if (ch < b) {
+            wv[u] = __ldg(tokw + (size_t)ch * WORDS + word);
+            ph[u] = __ldg(phase + ch);
+          } else {
+            wv[u] = 0;
+            ph[u] = -1;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (ph[u] < 0) continue;
+          if (ph[u] >= n_phases) {
+            atomicOr(status, STATUS_BAD_PHASE);
+            continue;
+          }
+          if (ph[u] != cur || run == 256) {
+            flush();
+            cur = ph[u];
+          }
+          acc_lo += wv[u] & 0x00FF00FFu;
+          acc_hi += (wv[u] >> 8) & 0x00FF00FFu;
+          ++run;
+        }
+      }
+      flush();
+    }
+  }
+  __syncthreads();
+
+  // C_{c,g}: individually rounded fp64 operations in ascending-dimension order
+  for (int c = threadIdx.x; c < n_phases; c += blockDim.x) {
+    const unsigned n_succ = cnt[c * 2 + 1], n_fail = cnt[c * 2 + 0];
+    double val = 0.0;
+    uint8_t ok = 0;
+    if (n_succ && n_fail) {
+      double acc = 0.0;
+      const unsigned* s1 = sums + (c * 2 + 1) * ACT;
+      const unsigned* s0 = sums + (c * 2 + 0) * ACT;
+      for (int dim = 0; dim < ACT; ++dim) {
+        const double m1 = __ddiv_rn((double)s1[dim], (double)n_succ);
+        const double m0 = __ddiv_rn((double)s0[dim], (double)n_fail);
+        const double diff = __dsub_rn(m1, m0);
+        acc = __dadd_rn(acc, __dmul_rn(diff, diff));
+      }
+      val = __dmul_rn(__dsqrt_rn(acc), 2.0 / 256.0);
+      ok = 1;
+    }
+    c_group[(size_t)g * n_phases + c] = val;
+    valid_group[(size_t)g * n_phases + c] = ok;
+  }
+}
+
+// Block 0: mean of C_{c,g} over valid groups in ascending g (one thread per phase).
+// Blocks 1..: Eq. 1 advantages, one thread per group.
+__global__ void score_finalize_kernel(const double* __restrict__ c_group,
+                                      const uint8_t* __restrict__ valid_group, int n_groups, int n_phases,
+                                      double* __restrict__ C, uint8_t* __restrict__ valid,
+                                      int32_t* __restrict__ n_valid, const uint8_t* __restrict__ reward,
+                                      int G, double eps, float* __restrict__ adv) {
+  if (blockIdx.x == 0) {
+    const int c = threadIdx.x;
+    if (c < n_phases) {
+      double s = 0.0;
+      int k = 0;
+      for (int g = 0; g < n_groups; ++g) {
+        if (valid_group[(size_t)g * n_phases + c]) {
+          s = __dadd_rn(s, c_group[(size_t)g * n_phases + c]);
+          ++k;
+        }
+      }
+      C[c] = k ? __ddiv_rn(s, (double)k) : 0.0;
+      valid[c] = k ? 1 : 0;
+      if (n_valid) n_valid[c] = k;
+    }
+    return;
+  }
+  if (!adv) return;
+  const int g = (blockIdx.x - 1) * blockDim.x + threadIdx.x;
+  if (g >= n_groups) return;
+  double s = 0.0;
+  for (int j = 0; j < G; ++j) s = __dadd_rn(s, reward[g * G + j] ? 1.0 : 0.0);
+  const double mu = __ddiv_rn(s, (double)G);
+  double v = 0.0;
+  for (int j = 0; j < G; ++j) {
+    const double dl = __dsub_rn(reward[g * G + j] ? 1.0 : 0.0, mu);
+    v = __dadd_rn(v, __dmul_rn(dl, dl));
+  }
+  const double denom = __dadd_rn(__dsqrt_rn(__ddiv_rn(v, (double)G)), eps);
+  for (int j = 0; j < G; ++j)
+    adv[g * G + j] = (float)__ddiv_rn(__dsub_rn(reward[g * G + j] ? 1.0 : 0.0, mu), denom);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Eq. 7-9: online update (one thread; O(n_phases * t_rc) scalar fp64 operations in a fixed order)
+// ------------------------------------------------------------------------------------------------
+__global__ void update_keep_probs_kernel(KeepState* st, const double* __restrict__ C,
+                                         const uint8_t* __restrict__ valid, int n_phases, int t_rc,
+                                         double p_min, float* __restrict__ p_out, uint32_t* __restrict__ q_out) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  for (int c = 0; c < n_phases; ++c) st->buf[c][st->count] = valid[c] ? C[c] : 0.0;
+  st->count += 1;
+  if (st->step == 0 || st->count == t_rc) {
+    double S[PCM_MAX_PHASES];
+    double tot = 0.0;
+    for (int c = 0; c < n_phases; ++c) {
+      double s = 0.0;
+      for (int t = 0; t < st->count; ++t) s = __dadd_rn(s, st->buf[c][t]);
+      S[c] = s;
+    }
+    for (int c = 0; c < n_phases; ++c) tot = __dadd_rn(tot, S[c]);
+    if (tot > 0.0) {
+      double rho_max = 0.0;
+      for (int c = 0; c < n_phases; ++c) {
+        S[c] = __ddiv_rn(S[c], tot);                      // share rho_c
+        if (S[c] > rho_max) rho_max = S[c];
+      }
+      for (int c = 0; c < n_phases; ++c) {
+        const double r = __ddiv_rn(S[c], rho_max);        // rho~_c
+        st->p[c] = r > p_min ? r : p_min;
+      }
+    }
+    st->count = 0;
+    st->n_refresh += 1;
+  }
+  st->step += 1;
+  for (int c = 0; c < n_phases; ++c) {
+    p_out[c] = (float)st->p[c];
+    q_out[c] = (uint32_t)__double2ll_rn(__dmul_rn(st->p[c], 16777216.0));   // round half to even
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Eq. 10: sampling
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t& o0, uint32_t& o1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  o0 = c0; o1 = c1;
+}
+
+// kept_off = exclusive prefix sum of min(budget, N_i); single block.
+__global__ void kept_offsets_kernel(const int32_t* __restrict__ traj_off, int n_traj, int budget,
+                                    int32_t* __restrict__ kept_off) {
+  __shared__ int part[1024];
+  const int t = threadIdx.x, nt = blockDim.x;
+  const int per = (n_traj + nt - 1) / nt;
+  const int lo = min(t * per, n_traj), hi = min(lo + per, n_traj);
+  int s = 0;
+  for (int i = lo; i < hi; ++i) s += min(budget, traj_off[i + 1] - traj_off[i]);
+  part[t] = s;
+  __syncthreads();
+  for (int off = 1; off < nt; off <<= 1) {               // Hillis-Steele inclusive scan
+    int v = (t >= off) ? part[t - off] : 0;
+    __syncthreads();
+    part[t] += v;
+    __syncthreads();
+  }
+  int run = part[t] - s;
+  for (int i = lo; i < hi; ++i) {
+    kept_off[i] = run;
+    run += min(budget, traj_off[i + 1] - traj_off[i]);
+  }
+  if (t == nt - 1) kept_off[n_traj] = part[nt - 1];
+}
+
+// One warp per trajectory.  Weights sit in shared memory; bit 31 marks a chunk already drawn.
+__global__ void __launch_bounds__(128)
+sample_chunks_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restrict__ phase,
+                     const uint32_t* __restrict__ q, int n_traj, int n_phases, int budget, int max_len,
+                     uint32_t seed_lo, uint32_t seed_hi, uint32_t it_lo, uint32_t it_hi,
+                     const int32_t* __restrict__ kept_off, int32_t* __restrict__ kept_idx,
+                     int32_t* __restrict__ kept_per_phase, unsigned* __restrict__ status) {
+  extern __shared__ unsigned wsm[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int i = blockIdx.x * (blockDim.x >> 5) + warp;
+  if (i >= n_traj) return;
+  unsigned* w = wsm + (size_t)warp * max_len;
+  const int a = traj_off[i], N = traj_off[i + 1] - a;
+  if (N > max_len || N < 0) {
+    if (lane == 0) atomicOr(status, STATUS_TOO_LONG);
+    return;
+  }
+  const int m = min(budget, N);
+  unsigned long long W = 0;
+  for (int k = lane; k < N; k += 32) {
+    const int ph = phase[a + k];
+    unsigned wk = 0;
+    if (ph < n_phases) wk = q[ph]; else atomicOr(status, STATUS_BAD_PHASE);
+    w[k] = wk;
+    W += wk;
+  }
+#pragma unroll
+  for (int off = 16; off; off >>= 1) W += __shfl_xor_sync(0xffffffffu, W, off);
+  __syncwarp();
+
+  if (m < N) {
+    for (int r = 0; r < m; ++r) {
+      uint32_t b0, b1;
+      philox4x32_10(it_lo, (uint32_t)i, (uint32_t)r, it_hi, seed_lo, seed_hi, b0, b1);
+      const unsigned long long bits = ((unsigned long long)b1 << 32) | b0;
+      const unsigned long long x = __umul64hi(bits, W);
+      unsigned long long base = 0;
+      int pick = -1;
+      for (int k0 = 0; k0 < N; k0 += 32) {
+        const int k = k0 + lane;
+        unsigned v = (k < N) ? (w[k] & 0x7FFFFFFFu) : 0u;
+        unsigned incl = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const unsigned up = __shfl_up_sync(0xffffffffu, incl, off);
+          if (lane >= off) incl += up;
+        }
+        const unsigned tot = __shfl_sync(0xffffffffu, incl, 31);
+        if (base + tot > x) {
+          const unsigned hit = __ballot_sync(0xffffffffu, base + incl > x);
+          pick = k0 + __ffs(hit) - 1;
+          break;
+        }
+        base += tot;
+      }
+      if (pick < 0) {                                    // cannot happen while weights are >= 1
+        if (lane == 0) atomicOr(status, STATUS_BAD_PHASE);
+        break;
+      }
+      const unsigned wp = w[pick] & 0x7FFFFFFFu;
+      __syncwarp();
+      if (lane == 0) w[pick] = 0x80000000u;
+      W -= wp;
+      __syncwarp();
+    }
+  } else {
+    for (int k = lane; k < N; k += 32) w[k] = 0x80000000u;
+    __syncwarp();
+  }
+
+  // compaction in index order = ascending chunk ids
+  int out = kept_off[i];
+  for (int k0 = 0; k0 < N; k0 += 32) {
+    const int k = k0 + lane;
+    const bool kept = (k < N) && (w[k] & 0x80000000u);
+    const unsigned mask = __ballot_sync(0xffffffffu, kept);
+    if (kept) {
+      kept_idx[out + __popc(mask & ((1u << lane) - 1u))] = a + k;
+      if (kept_per_phase) atomicAdd(kept_per_phase + phase[a + k], 1);
+    }
+    out += __popc(mask);
+  }
+}
+
+static int check_batch(const pcm_ctx* ctx, const pcm_batch* b) {
+  if (!ctx || !b || !b->traj_off || !b->phase) return PCM_ERR_ARG;
+  if (b->n_traj <= 0 || b->n_traj > ctx->max_traj || b->n_traj % ctx->cfg.group_size) return PCM_ERR_ARG;
+  if (b->n_chunks < 0 || b->max_len < 0) return PCM_ERR_ARG;
+  return PCM_OK;
+}
+
+}  // namespace pcm
+
+using namespace pcm;
+
+extern "C" {
+
+int pcm_create(pcm_ctx** out, const pcm_config* cfg, int32_t max_traj) {
+  if (!out || !cfg) return PCM_ERR_ARG;
+  if (cfg->n_phases < 1 || cfg->n_phases > PCM_MAX_PHASES || cfg->budget < 1 || cfg->group_size < 1 ||
+      cfg->t_rc < 1 || cfg->t_rc > PCM_MAX_TRC || !(cfg->p_min > 0.0) || cfg->p_min > 1.0 ||
+      !(cfg->adv_eps >= 0.0) || max_traj < cfg->group_size)
+    return PCM_ERR_ARG;
+  pcm_ctx* c = new (std::nothrow) pcm_ctx();
+  if (!c) return PCM_ERR_ARG;
+  c->cfg = *cfg;
+  c->max_traj = max_traj;
+  c->state = nullptr; c->status = nullptr; c->c_group = nullptr; c->valid_group = nullptr;
+  const size_t ng = (size_t)max_traj / cfg->group_size;
+  bool ok = cudaGetDevice(&c->device) == cudaSuccess &&
+            cudaMalloc(&c->state, sizeof(KeepState)) == cudaSuccess &&
+            cudaMalloc(&c->status, 256) == cudaSuccess &&
+            cudaMalloc(&c->c_group, ng * cfg->n_phases * sizeof(double)) == cudaSuccess &&
+            cudaMalloc(&c->valid_group, ng * cfg->n_phases) == cudaSuccess;
+  if (ok) {
+    KeepState init;
+    memset(&init, 0, sizeof(init));
+    for (int k = 0; k < PCM_MAX_PHASES; ++k) init.p[k] = 1.0;
+    ok = cudaMemcpy(c->state, &init, sizeof(init), cudaMemcpyHostToDevice) == cudaSuccess &&
+         cudaMemset(c->status, 0, 256) == cudaSuccess;
+  }
+  if (!ok) {
+    pcm_destroy(c);
+    return PCM_ERR_CUDA;
+  }
+  *out = c;
+  return PCM_OK;
+}
+
+int pcm_destroy(pcm_ctx* c) {
+  if (!c) return PCM_ERR_ARG;
+  cudaFree(c->state); cudaFree(c->status); cudaFree(c->c_group); cudaFree(c->valid_group);
+  delete c;
+  return PCM_OK;
+}
+
+int pcm_poll_status(pcm_ctx* ctx, pcm_stream stream) {
+  if (!ctx) return PCM_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  unsigned h = 0;
+  PCM_CUDA_TRY(cudaMemcpyAsync(&h, ctx->status, sizeof(h), cudaMemcpyDeviceToHost, s));
+  PCM_CUDA_TRY(cudaMemsetAsync(ctx->status, 0, sizeof(unsigned), s));
+  PCM_CUDA_TRY(cudaStreamSynchronize(s));
+  if (h & STATUS_TIMEOUT) return PCM_ERR_DEVICE_TIMEOUT;
+  if (h) return PCM_ERR_DEVICE_DATA;
+  return PCM_OK;
+}
+
+int pcm_state_export(pcm_ctx* ctx, void* host_buf, size_t* bytes) {
+  if (!ctx || !bytes) return PCM_ERR_ARG;
+  const size_t need = sizeof(StateBlob);
+  if (!host_buf || *bytes < need) {
+    *bytes = need;
+    return host_buf ? PCM_ERR_STATE : PCM_OK;
+  }
+  StateBlob* b = (StateBlob*)host_buf;
+  b->version = STATE_VERSION; b->n_phases = ctx->cfg.n_phases; b->t_rc = ctx->cfg.t_rc; b->pad = 0;
+  PCM_CUDA_TRY(cudaDeviceSynchronize());
+  PCM_CUDA_TRY(cudaMemcpy(&b->st, ctx->state, sizeof(KeepState), cudaMemcpyDeviceToHost));
+  *bytes = need;
+  return PCM_OK;
+}
+
+int pcm_state_import(pcm_ctx* ctx, const void* host_buf, size_t bytes) {
+  if (!ctx || !host_buf) return PCM_ERR_ARG;
+  const StateBlob* b = (const StateBlob*)host_buf;
+  if (bytes != sizeof(StateBlob) || b->version != STATE_VERSION || b->n_phases != ctx->cfg.n_phases ||
+      b->t_rc != ctx->cfg.t_rc || b->st.count < 0 || b->st.count >= ctx->cfg.t_rc)
+    return PCM_ERR_STATE;
+  PCM_CUDA_TRY(cudaDeviceSynchronize());
+  PCM_CUDA_TRY(cudaMemcpy(ctx->state, &b->st, sizeof(KeepState), cudaMemcpyHostToDevice));
+  return PCM_OK;
+}
+
+int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* b, double* C, uint8_t* valid, int32_t* n_valid_groups,
+                     float* adv, pcm_stream stream) {
+  int rc = check_batch(ctx, b);
+  if (rc) return rc;
+  if (!b->tok || !b->reward || !C || !valid) return PCM_ERR_ARG;
+  if (((uintptr_t)b->tok) & 3) return PCM_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int G = ctx->cfg.group_size, Kc = ctx->cfg.n_phases, ng = b->n_traj / G;
+  const size_t smem = (size_t)Kc * 2 * (ACT + 1) * sizeof(unsigned);
+  score_groups_kernel<<<ng, 256, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, G, Kc, ctx->c_group,
+                                             ctx->valid_group, ctx->status);
+  PCM_LAUNCH_CHECK();
+  const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
+  score_finalize_kernel<<<1 + adv_blocks, 128, 0, s>>>(ctx->c_group, ctx->valid_group, ng, Kc, C, valid,
+                                                       n_valid_groups, b->reward, G, ctx->cfg.adv_eps, adv);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
+}
+
+int pcm_update_keep_probs(pcm_ctx* ctx, const double* C, const uint8_t* valid, float* p, uint32_t* q,
+                          pcm_stream stream) {
+  if (!ctx || !C || !valid || !p || !q) return PCM_ERR_ARG;
+  update_keep_probs_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->state, C, valid, ctx->cfg.n_phases,
+                                                               ctx->cfg.t_rc, ctx->cfg.p_min, p, q);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
+}
+
+int pcm_sample_chunks(pcm_ctx* ctx, const pcm_batch* b, const uint32_t* q, uint64_t iter, int32_t* kept_idx,
+                      int32_t* kept_off, int32_t* kept_per_phase, pcm_stream stream) {
+  int rc = check_batch(ctx, b);
+  if (rc) return rc;
+  if (!q || !kept_idx || !kept_off) return PCM_ERR_ARG;
+  if (b->max_len < 1 || b->max_len > 12000) return PCM_ERR_SHAPE;     // 4 warps x max_len x 4 B <= 192 KB
+  cudaStream_t s = (cudaStream_t)stream;
+  kept_offsets_kernel<<<1, 1024, 0, s>>>(b->traj_off, b->n_traj, ctx->cfg.budget, kept_off);
+  PCM_LAUNCH_CHECK();
+  if (kept_per_phase) PCM_CUDA_TRY(cudaMemsetAsync(kept_per_phase, 0, ctx->cfg.n_phases * sizeof(int32_t), s));
+  const int warps = 4;
+  const size_t smem = (size_t)warps * b->max_len * sizeof(unsigned);
+  if (smem > 48 * 1024)
+    PCM_CUDA_TRY(cudaFuncSetAttribute(sample_chunks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  sample_chunks_kernel<<<ceil_div(b->n_traj, warps), warps * 32, smem, s>>>(
+      b->traj_off, b->phase, q, b->n_traj, ctx->cfg.n_phases, ctx->cfg.budget, b->max_len,
+      (uint32_t)(ctx->cfg.seed & 0xFFFFFFFFu), (uint32_t)(ctx->cfg.seed >> 32), (uint32_t)(iter & 0xFFFFFFFFu),
+      (uint32_t)(iter >> 32), kept_off, kept_idx, kept_per_phase, ctx->status);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
+}
+
+int64_t pcm_launch_count(void) { return (int64_t)g_launches.load(); }
+
+}  // extern "C"
