@@ -1,0 +1,336 @@
+// bf16 GEMM on the 5th-generation tensor cores: TMA (cp.async.bulk.tensor) fills a shared-memory
+// ring with 128-byte-swizzled operand tiles, one thread issues tcgen05.mma with the fp32
+// accumulator in tensor memory, and four epilogue warps read it back with tcgen05.ld.
+//
+//   C[m][n] = sum_k A(m,k) B(n,k) (+ R[m][n])      store as bf16 / fp32, or
+//   C[m][n] += sum_k A(m,k) B(n,k)                  fp32 reduction (weight gradients, split along k)
+//
+// Either operand may be K-major (contraction index contiguous in memory) or MN-major (the other
+// index contiguous); the layout enters through the tensor map, the shared-memory descriptor and
+// one bit of the instruction descriptor, so forward, input-gradient and weight-gradient GEMMs
+// are the same kernel.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = tensor-memory allocation + MMA issue,
+// warps 2..5 = epilogue.  Every mbarrier wait is bounded; when one runs out the CTA sets a status
+// flag, all roles leave their loops, tensor memory is released and the kernel returns.
+#include <cuda.h>
+
+#include "async_ptx.cuh"
+#include "internal.h"
+
+namespace pcm {
+
+constexpr int TC_BM = 128;
+constexpr int TC_BK = 64;                     // 64 bf16 = one 128-byte swizzle row
+constexpr int TC_STAGES = 4;
+constexpr int TC_THREADS = 192;
+constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per mbarrier wait
+
+__device__ unsigned g_tc_status = 0;          // bit 0: a bounded wait expired
+
+struct TcParams {
+  int M, N, K;
+  int kb_per_split;                           // k-blocks of 64 handled by one blockIdx.z
+  void* C; long long ldc; int c_dtype;        // DT_BF16 / DT_F32
+  const float* R; long long ldr;
+  int reduce;                                 // 1: fp32 reduction into C
+  int a_kmajor, b_kmajor;
+};
+
+// Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets in
+// 16-byte units, descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;                     // version
+  d |= (uint64_t)2 << 61;                     // SWIZZLE_128B
+  return d;
+}
+
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 A and B, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+template <int BN>
+struct TcSmem {
+  static constexpr int A_BYTES = TC_BM * TC_BK * 2;           // 16 KB
+  static constexpr int B_BYTES = BN * TC_BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TOTAL = TC_STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  using SM = TcSmem<BN>;
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t* tiles = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);       // swizzle atoms need 1024-byte alignment
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + TC_STAGES * SM::STAGE_BYTES);
+  uint64_t* full = bars;                      // [TC_STAGES] producer -> MMA
+  uint64_t* empty = bars + TC_STAGES;         // [TC_STAGES] MMA -> producer
+  uint64_t* acc_full = bars + 2 * TC_STAGES;  // MMA -> epilogue
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_STAGES + 1);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * TC_BM;
+  const int num_kb_total = (p.K + TC_BK - 1) / TC_BK;
+  const int kb_lo = blockIdx.z * p.kb_per_split;
+  const int kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
+  const int num_kb = kb_hi - kb_lo;           // >= 1 by construction of the grid
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, BN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_acc = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------ TMA producer ------------------------------
+      for (int i = 0; i < num_kb; ++i) {
+        const int st = i % TC_STAGES;
+        const unsigned ph = (unsigned)(i / TC_STAGES) & 1u;
+        if (*abort_flag) break;
+        if (!mbar_wait_bounded(&empty[st], ph ^ 1u, TC_WAIT_LIMIT_NS)) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); break; }
+        uint8_t* sa = tiles + st * SM::STAGE_BYTES;
+        uint8_t* sb = sa + SM::A_BYTES;
+        mbar_expect_tx(&full[st], SM::STAGE_BYTES);
+        const int k0 = (kb_lo + i) * TC_BK;
+        if (p.a_kmajor) {
+          tma_load_2d(sa, &tmA, k0, m0, &full[st]);                     // box {64 k, 128 m}
+        } else {
+#pragma unroll
+          for (int b = 0; b < TC_BM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, m0 + b * 64, k0, &full[st]);  // box {64 m, 64 k}
+        }
+        if (p.b_kmajor) {
+          tma_load_2d(sb, &tmB, k0, n0, &full[st]);                     // box {64 k, BN n}
+        } else {
+#pragma unroll
+          for (int b = 0; b < BN / 64; ++b) tma_load_2d(sb + b * 8192, &tmB, n0 + b * 64, k0, &full[st]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------ MMA issuer ------------------------------
+      const uint32_t idesc = make_idesc(BN, p.a_kmajor ? 0 : 1, p.b_kmajor ? 0 : 1);
+      // K-major tile: rows of 128 B, 8-row groups 1024 B apart; a k-step of 16 elements is 32 B along the row.
+      // MN-major tile: boxes of 64 (mn) x 64 (k): k-rows of 128 B, 8-row groups 1024 B apart, next 64 mn 8192 B on;
+      //                a k-step of 16 rows is 2048 B.
+      const uint32_t a_lbo = p.a_kmajor ? 16u : 8192u, b_lbo = p.b_kmajor ? 16u : 8192u;
+      const uint32_t a_step = p.a_kmajor ? 32u : 2048u, b_step = p.b_kmajor ? 32u : 2048u;
+      bool ok = true;
+      for (int i = 0; i < num_kb && ok; ++i) {
+        const int st = i % TC_STAGES;
+        const unsigned ph = (unsigned)(i / TC_STAGES) & 1u;
+        if (*abort_flag) { ok = false; break; }
+        if (!mbar_wait_bounded(&full[st], ph, TC_WAIT_LIMIT_NS)) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(tiles + st * SM::STAGE_BYTES);
+        const uint32_t sb = sa + SM::A_BYTES;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k) {
+          const uint64_t da = make_smem_desc(sa + k * a_step, a_lbo, 1024u);
+          const uint64_t db = make_smem_desc(sb + k * b_step, b_lbo, 1024u);
+          umma_bf16(tmem_acc, da, db, idesc, (i | k) ? 1u : 0u);
+        }
+        umma_commit(&empty[st]);              // frees the stage once the MMAs above have read it
+      }
+      if (ok) umma_commit(acc_full);
+    }
+  } else {
+    // ------------------------------ epilogue: warps 2..5 ------------------------------
+    const int quad = warp & 3;                // tensor-memory lane quadrant this warp may access
+    const int row = m0 + quad * 32 + lane;
+    int ok = 1;
+    if (lane == 0) {
+      ok = (mbar_wait_bounded(acc_full, 0u, TC_WAIT_LIMIT_NS * 2ull) && !*abort_flag) ? 1 : 0;
+      if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (ok) {
+      tc_fence_after();
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, r);
+        tmem_ld_wait();
+        const int col = n0 + c0;
+        if (row < p.M && col < p.N) {        // N is a multiple of 32 on this path
+          if (p.reduce) {
+            float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              red_add_v4(dst + e, __uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
+                         __uint_as_float(r[e + 3]));
+          } else {
+            float v[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
+            if (p.R) {
+              const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const float4 t = rp[e];
+                v[4 * e] += t.x; v[4 * e + 1] += t.y; v[4 * e + 2] += t.z; v[4 * e + 3] += t.w;
+              }
+            }
+            if (p.c_dtype == DT_F32) {
+              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+            } else {
+              uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(v[8 * e], v[8 * e + 1]);
+                __nv_bfloat162 h1 = __floats2bfloat162_rn(v[8 * e + 2], v[8 * e + 3]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * e + 4], v[8 * e + 5]);
+                __nv_bfloat162 h3 = __floats2bfloat162_rn(v[8 * e + 6], v[8 * e + 7]);
+                uint4 o;
+                o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+                o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+                dst[e] = o;
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // teardown: on the abort path give copies still in flight time to land before shared memory is released
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_acc, BN);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows][cols] with row stride ld (elements); box {box_cols, box_rows}, 128-byte swizzle,
+// out-of-range elements read as zero.
+static bool make_tmap(CUtensorMap* tm, const void* base, long long rows, long long cols, long long ld, int box_cols,
+                      int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool gemm_tcgen05_supported(const GemmArgs& g) {
+  if (g.ab_dtype != DT_BF16) return false;
+  if (g.M < 1 || g.N < 32 || g.K < 1 || (g.N % 32)) return false;
+  if ((g.lda % 8) || (g.ldb % 8)) return false;
+  if (((uintptr_t)g.A | (uintptr_t)g.B | (uintptr_t)g.C) & 15) return false;
+  if (g.c_dtype == DT_BF16 && (g.ldc % 8)) return false;
+  if (g.c_dtype == DT_F32 && (g.ldc % 4)) return false;
+  if (g.R && (((uintptr_t)g.R & 15) || (g.ldr % 4))) return false;
+  if (g.R && (const void*)g.R == (const void*)g.C && g.c_dtype != DT_F32) return false;
+  if ((g.M + TC_BM - 1) / TC_BM > 65535) return false;
+  return encode_fn() != nullptr;
+}
+
+template <int BN>
+static int launch_tc(const GemmArgs& g, cudaStream_t s) {
+  CUtensorMap tmA, tmB;
+  // K-major operand: tensor [MN][K] -> box {64 k, rows}.  MN-major operand: tensor [K][MN] -> box {64 mn, 64 k}.
+  const bool okA = g.a_kmajor ? make_tmap(&tmA, g.A, g.M, g.K, g.lda, TC_BK, TC_BM)
+                              : make_tmap(&tmA, g.A, g.K, g.M, g.lda, 64, TC_BK);
+  const bool okB = g.b_kmajor ? make_tmap(&tmB, g.B, g.N, g.K, g.ldb, TC_BK, BN)
+                              : make_tmap(&tmB, g.B, g.K, g.N, g.ldb, 64, TC_BK);
+  if (!okA || !okB) return PCM_ERR_CUDA;
+  TcParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  p.C = g.C; p.ldc = g.ldc; p.c_dtype = g.c_dtype;
+  p.reduce = (g.R && (const void*)g.R == (const void*)g.C) ? 1 : 0;
+  p.R = p.reduce ? nullptr : g.R; p.ldr = g.ldr;
+  p.a_kmajor = g.a_kmajor; p.b_kmajor = g.b_kmajor;
+  const int tiles_m = (g.M + TC_BM - 1) / TC_BM, tiles_n = (g.N + BN - 1) / BN;
+  const int num_kb = (g.K + TC_BK - 1) / TC_BK;
+  int splits = 1;
+  if (p.reduce) {
+    // split the contraction until there are about two waves of CTAs, keeping >= 8 k-blocks per split
+    const long long tiles = (long long)tiles_m * tiles_n;
+    long long want = (2 * 148 + tiles - 1) / tiles;
+    long long cap = num_kb / 8 > 0 ? num_kb / 8 : 1;
+    splits = (int)(want < cap ? want : cap);
+    if (splits < 1) splits = 1;
+  }
+  p.kb_per_split = (num_kb + splits - 1) / splits;
+  splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;          // no empty split
+  static bool attr_done = false;
+  if (!attr_done) {
+    PCM_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<BN>::TOTAL));
+    attr_done = true;
+  }
+  dim3 grid(tiles_n, tiles_m, splits);
+  gemm_tc_kernel<BN><<<grid, TC_THREADS, TcSmem<BN>::TOTAL, s>>>(tmA, tmB, p);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
+}
+
+int gemm_tcgen05(const GemmArgs& g, cudaStream_t s) {
+  if (g.N % 256 == 0 || g.N > 256) return launch_tc<256>(g, s);
+  return launch_tc<128>(g, s);
+}
+
+int tcgen05_poll_status() {
+  unsigned h = 0;
+  if (cudaMemcpyFromSymbol(&h, g_tc_status, sizeof(h)) != cudaSuccess) return PCM_ERR_CUDA;
+  if (h) {
+    unsigned z = 0;
+    cudaMemcpyToSymbol(g_tc_status, &z, sizeof(z));
+    return PCM_ERR_DEVICE_TIMEOUT;
+  }
+  return PCM_OK;
+}
+
+}  // namespace pcm
