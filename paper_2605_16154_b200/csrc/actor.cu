@@ -1,0 +1,645 @@
+// grpo_actor_fwd_bwd: forward and backward of the decoder policy on the packed batch of kept
+// chunks under the masked, clipped GRPO objective (Eq. 11).  This file holds the orchestration and
+// the memory-bound kernels (RMSNorm, rotary embedding, SwiGLU, the loss over the 256-bin head,
+// embedding gradient); the contractions live in gemm_*.cu and attention*.cu.
+#include <cstdlib>
+#include <cstring>
+
+#include "internal.h"
+
+namespace pcm {
+
+constexpr int ACT = PCM_ACT_DIM;
+constexpr int NB = PCM_N_BINS;
+constexpr float RMS_EPS = 1e-5f;
+constexpr int NORM_BWD_BLOCKS = 592;         // 4 CTAs per SM on 148 SMs
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p);
+template <> __device__ __forceinline__ float ldf<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void stf(T* p, float v);
+template <> __device__ __forceinline__ void stf<float>(float* p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int off = 16; off; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+
+// Row r of a [rows][d] tensor that holds only the scored positions maps to token row
+// (r / 56) * S + P - 1 + r % 56 of the full activation; map_S == 0 means identity.
+__device__ __forceinline__ long long map_row(long long r, int map_S, int map_P) {
+  if (map_S == 0) return r;
+  const long long j = r / ACT;
+  return j * map_S + map_P - 1 + (r - j * ACT);
+}
+
+// ------------------------------------------------------------------------------------------------
+// packed batch (model dtype) -> fp32 residual stream
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void to_residual_kernel(const T* __restrict__ x, float* __restrict__ y, long long n) {
+  const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i + 3 < n) {
+    float4 o;
+    o.x = ldf(x + i); o.y = ldf(x + i + 1); o.z = ldf(x + i + 2); o.w = ldf(x + i + 3);
+    *reinterpret_cast<float4*>(y + i) = o;
+  } else {
+    for (long long k = i; k < n; ++k) y[k] = ldf(x + k);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// RMSNorm forward: one warp per row.  x fp32 [.][d] (rows optionally gathered), h T [rows][d].
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+rmsnorm_fwd_kernel(const float* __restrict__ x, const T* __restrict__ gamma, T* __restrict__ h,
+                   float* __restrict__ rstd, long long rows, int d, int map_S, int map_P) {
+  const long long r = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= rows) return;
+  const float* xr = x + map_row(r, map_S, map_P) * d;
+  float ss = 0.f;
+  for (int c = lane * 4; c < d; c += 128) {
+    const float4 v = *reinterpret_cast<const float4*>(xr + c);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = warp_sum(ss);
+  const float rs = rsqrtf(ss / (float)d + RMS_EPS);
+  if (lane == 0) rstd[r] = rs;
+  T* hr = h + r * d;
+  for (int c = lane * 4; c < d; c += 128) {
+    const float4 v = *reinterpret_cast<const float4*>(xr + c);
+    stf(hr + c, v.x * rs * ldf(gamma + c));
+    stf(hr + c + 1, v.y * rs * ldf(gamma + c + 1));
+    stf(hr + c + 2, v.z * rs * ldf(gamma + c + 2));
+    stf(hr + c + 3, v.w * rs * ldf(gamma + c + 3));
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// RMSNorm backward.  dy fp32 [rows][d]; x fp32 (rows optionally gathered); dx_out = dx_in + dx is
+// written through the same row map, in fp32 and in T.  Per-CTA partial sums of
+// dgamma = sum_rows dy * x * rstd go to part[blockIdx][d]; a second kernel adds them up in order.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+rmsnorm_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ rstd,
+                   const T* __restrict__ gamma, const float* dx_in, float* dx_out, T* __restrict__ dx_out_t,
+                   float* __restrict__ part, long long rows, int d, int map_S, int map_P) {
+  extern __shared__ float red[];                         // [8 warps][d]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* mine = red + (size_t)warp * d;
+  for (int c = lane; c < d; c += 32) mine[c] = 0.f;
+  __syncwarp();
+  for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
+    const long long xr_i = map_row(r, map_S, map_P);
+    const float* xr = x + xr_i * d;
+    const float* dyr = dy + r * d;
+    const float rs = rstd[r];
+    float dot = 0.f;
+    for (int c = lane * 4; c < d; c += 128) {
+      const float4 xv = *reinterpret_cast<const float4*>(xr + c);
+      const float4 gv = *reinterpret_cast<const float4*>(dyr + c);
+      dot += gv.x * ldf(gamma + c) * xv.x + gv.y * ldf(gamma + c + 1) * xv.y + gv.z * ldf(gamma + c + 2) * xv.z +
+             gv.w * ldf(gamma + c + 3) * xv.w;
+    }
+    dot = warp_sum(dot);
+    const float coef = dot * rs * rs * rs / (float)d;    // mean(dn * n) * rstd, with n = x * rstd
+    for (int c = lane * 4; c < d; c += 128) {
+      const float4 xv = *reinterpret_cast<const float4*>(xr + c);
+      const float4 gv = *reinterpret_cast<const float4*>(dyr + c);
+      const float xa[4] = {xv.x, xv.y, xv.z, xv.w};
+      const float ga[4] = {gv.x, gv.y, gv.z, gv.w};
+      float o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        o[e] = rs * ga[e] * ldf(gamma + c + e) - coef * xa[e];
+        mine[c + e] += ga[e] * xa[e] * rs;
+      }
+      if (dx_in) {
+        const float4 pv = *reinterpret_cast<const float4*>(dx_in + xr_i * d + c);
+        o[0] += pv.x; o[1] += pv.y; o[2] += pv.z; o[3] += pv.w;
+      }
+      *reinterpret_cast<float4*>(dx_out + xr_i * d + c) = make_float4(o[0], o[1], o[2], o[3]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) stf(dx_out_t + xr_i * d + c + e, o[e]);
+    }
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += red[(size_t)w * d + c];
+    part[(size_t)blockIdx.x * d + c] = s;
+  }
+}
+
+// out[c] += sum_b part[b][c] in ascending b
+__global__ void colsum_accumulate_kernel(const float* __restrict__ part, int nblk, int d, float* __restrict__ out) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= d) return;
+  float s = 0.f;
+  for (int b = 0; b < nblk; ++b) s += part[(size_t)b * d + c];
+  out[c] += s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// rotary embedding on the q and k parts of qkv [rows][3d], in place; table [S][dh/2] of (cos, sin)
+// built in fp64.  sign = +1 forward, -1 backward (the transpose of a rotation).
+// ------------------------------------------------------------------------------------------------
+__global__ void rope_table_kernel(float2* __restrict__ tab, int S, int dh) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int half = dh / 2;
+  if (idx >= S * half) return;
+  const int pos = idx / half, i = idx - pos * half;
+  const double inv_freq = pow(10000.0, -(2.0 * (double)i) / (double)dh);
+  const double ang = (double)pos * inv_freq;
+  tab[idx] = make_float2((float)cos(ang), (float)sin(ang));
+}
+
+template <typename T>
+__global__ void rope_kernel(T* __restrict__ qkv, const float2* __restrict__ tab, long long rows, int S, int H,
+                            int dh, float sign) {
+  const int half = dh / 2, d = H * dh;
+  const long long per_row = 2LL * H * half;              // q and k pairs
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * per_row) return;
+  const long long r = idx / per_row;
+  const int rem = (int)(idx - r * per_row);
+  const int which = rem / (H * half);                    // 0 = q, 1 = k
+  const int hh = (rem - which * H * half) / half;
+  const int i = rem % half;
+  const int pos = (int)(r % S);
+  const float2 cs = tab[pos * half + i];
+  T* p = qkv + r * 3LL * d + (long long)which * d + (long long)hh * dh + i;
+  const float a = ldf(p), b = ldf(p + half);
+  const float sn = cs.y * sign;
+  stf(p, a * cs.x - b * sn);
+  stf(p + half, b * cs.x + a * sn);
+}
+
+// ------------------------------------------------------------------------------------------------
+// SwiGLU: gu [rows][8d] = gate | up
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void swiglu_fwd_kernel(const T* __restrict__ gu, T* __restrict__ act, long long rows, int f) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * f) return;
+  const long long r = idx / f;
+  const int c = (int)(idx - r * f);
+  const float g = ldf(gu + r * 2LL * f + c), u = ldf(gu + r * 2LL * f + f + c);
+  stf(act + idx, g / (1.f + __expf(-g)) * u);
+}
+
+template <typename T>
+__global__ void swiglu_bwd_kernel(const T* __restrict__ gu, const T* __restrict__ dact, T* __restrict__ dgu,
+                                  long long rows, int f) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * f) return;
+  const long long r = idx / f;
+  const int c = (int)(idx - r * f);
+  const float g = ldf(gu + r * 2LL * f + c), u = ldf(gu + r * 2LL * f + f + c), da = ldf(dact + idx);
+  const float sg = 1.f / (1.f + __expf(-g));
+  stf(dgu + r * 2LL * f + c, da * u * sg * (1.f + g * (1.f - sg)));
+  stf(dgu + r * 2LL * f + f + c, da * g * sg);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Loss over the 256-bin head: one warp per scored row.  z fp32 [rows][256] logits in, dz T out.
+// Per-CTA partial sums {surrogate, clipped count, ratio} go to part[blockIdx][3].
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+loss_rows_kernel(const float* __restrict__ z, const uint8_t* __restrict__ tgt, const float* __restrict__ lpo,
+                 const float* __restrict__ adv_c, float eps_low, float eps_high, float loss_scale,
+                 T* __restrict__ dz, float* __restrict__ logp_out, float* __restrict__ part, long long rows,
+                 int fwd_only) {
+  __shared__ float red[8][3];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long r = (long long)blockIdx.x * 8 + warp;
+  float my_s = 0.f, my_clip = 0.f, my_ratio = 0.f;
+  if (r < rows) {
+    float v[8];
+    const float4 a = *reinterpret_cast<const float4*>(z + r * NB + lane * 8);
+    const float4 b = *reinterpret_cast<const float4*>(z + r * NB + lane * 8 + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    float mx = v[0];
+#pragma unroll
+    for (int e = 1; e < 8; ++e) mx = fmaxf(mx, v[e]);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    float se = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) se += expf(v[e] - mx);
+    se = warp_sum(se);
+    const float lse = mx + logf(se);
+    const int t = tgt[r];
+    float mine = v[0];                                    // this lane's value at sub-index t & 7
+#pragma unroll
+    for (int e = 1; e < 8; ++e) mine = ((t & 7) == e) ? v[e] : mine;
+    const float zt = __shfl_sync(0xffffffffu, mine, t >> 3);
+    const float logp = zt - lse;
+    const float A = adv_c[r / ACT];
+    const float ratio = expf(logp - lpo[r]);
+    const float lo = 1.f - eps_low, hi = 1.f + eps_high;
+    const float clipped = fminf(fmaxf(ratio, lo), hi);
+    const float surr = fminf(ratio * A, clipped * A);
+    const bool active = (A >= 0.f && ratio <= hi) || (A < 0.f && ratio >= lo);
+    const float dlogp = active ? -loss_scale * A * ratio : 0.f;
+    if (lane == 0) {
+      if (logp_out) logp_out[r] = logp;
+      my_s = surr; my_clip = active ? 0.f : 1.f; my_ratio = ratio;
+    }
+    if (!fwd_only) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int col = lane * 8 + e;
+        const float p = expf(v[e] - lse);
+        stf(dz + r * NB + col, dlogp * ((col == t ? 1.f : 0.f) - p));
+      }
+    }
+  }
+  if (lane == 0) { red[warp][0] = my_s; red[warp][1] = my_clip; red[warp][2] = my_ratio; }
+  __syncthreads();
+  if (threadIdx.x < 3) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += red[w][threadIdx.x];
+    part[(size_t)blockIdx.x * 3 + threadIdx.x] = s;
+  }
+}
+
+// acc[0..2] += ordered sums of part; loss[0] = -loss_scale * acc[0]   (single CTA, fixed order)
+__global__ void loss_reduce_kernel(const float* __restrict__ part, int nblk, float loss_scale,
+                                   float* __restrict__ acc, float* __restrict__ loss) {
+  __shared__ double sh[256][3];
+  double s[3] = {0, 0, 0};
+  for (int b = threadIdx.x; b < nblk; b += blockDim.x)
+    for (int e = 0; e < 3; ++e) s[e] += (double)part[(size_t)b * 3 + e];
+  for (int e = 0; e < 3; ++e) sh[threadIdx.x][e] = s[e];
+  __syncthreads();
+  for (int off = 128; off; off >>= 1) {
+    if (threadIdx.x < off)
+      for (int e = 0; e < 3; ++e) sh[threadIdx.x][e] += sh[threadIdx.x + off][e];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    for (int e = 0; e < 3; ++e) acc[e] += (float)sh[0][e];
+    loss[0] = -loss_scale * acc[0];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Embedding gradient: dE[v][:] += sum over action positions whose token is v of dx[row][:],
+// visited in ascending row order (deterministic).  grid = (256 tokens, column tiles of 256).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+embed_grad_kernel(const float* __restrict__ dx, const uint8_t* __restrict__ tgt, int n_chunks, int S, int P, int d,
+                  float* __restrict__ dE) {
+  const int v = blockIdx.x;
+  const int c = blockIdx.y * 256 + threadIdx.x;
+  __shared__ int hits[256];
+  __shared__ int wcount[8];
+  __shared__ int n_hits;
+  float acc = 0.f;
+  const int total = n_chunks * ACT;
+  for (int base = 0; base < total; base += 256) {
+    const int idx = base + threadIdx.x;
+    const bool hit = idx < total && tgt[idx] == v;
+    // ordered compaction: warp ballots, then warp offsets in warp order
+    const unsigned m = __ballot_sync(0xffffffffu, hit);
+    if ((threadIdx.x & 31) == 0) wcount[threadIdx.x >> 5] = __popc(m);
+    __syncthreads();
+    int off = 0;
+    for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) off += wcount[w];
+    if (hit) hits[off + __popc(m & ((1u << (threadIdx.x & 31)) - 1u))] = idx;
+    if (threadIdx.x == 255) n_hits = off + __popc(m);
+    __syncthreads();
+    if (c < d) {
+      for (int k = 0; k < n_hits; ++k) {
+        const int id = hits[k];
+        const int j = id / ACT, t = id - j * ACT;
+        acc += dx[((long long)j * S + P + t) * d + c];
+      }
+    }
+    __syncthreads();
+  }
+  if (c < d) dE[(long long)v * d + c] += acc;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Arena {
+  unsigned char* base;
+  size_t off;
+  void* take(size_t bytes) {
+    void* p = base ? base + off : nullptr;
+    off += align_up(bytes, 256);
+    return p;
+  }
+};
+
+struct LayerActs {
+  void* h1; void* qkv; void* attn; float* lse; float* rstd1; float* x_mid; float* rstd2; void* h2; void* gu; void* act;
+};
+
+struct Workspace {
+  float2* rope_tab;
+  float* x[129];                 // residual stream, x[0..L]
+  LayerActs la[128];
+  void* hs; float* rstdf; float* z; void* dz; float* loss_part; float* loss_acc;
+  float* dx; void* dx_t; void* dact; void* dgu; float* dh; void* dattn; void* dqkv; float* dsum;
+  float* norm_part; float* dhs;
+  size_t bytes;
+};
+
+static void carve(Workspace& w, unsigned char* base, const grpo_model_cfg& c, int mb, bool fwd_only) {
+  Arena a{base, 0};
+  const size_t es = c.dtype == GRPO_BF16 ? 2 : 4;
+  const int S = c.prefix_len + ACT, d = c.d, H = c.n_heads, L = c.n_layers;
+  const size_t M = (size_t)mb * S, R = (size_t)mb * ACT;
+  w.rope_tab = (float2*)a.take((size_t)S * (d / H / 2) * sizeof(float2));
+  // with backward every layer keeps its activations; forward-only reuses one layer's worth
+  const int kept_layers = fwd_only ? 1 : L;
+  for (int l = 0; l <= (fwd_only ? 1 : L); ++l) w.x[l] = (float*)a.take(M * d * 4);
+  for (int l = 0; l < kept_layers; ++l) {
+    LayerActs& la = w.la[l];
+    la.h1 = a.take(M * d * es); la.qkv = a.take(M * 3 * d * es); la.attn = a.take(M * d * es);
+    la.lse = (float*)a.take((size_t)mb * H * S * 4); la.rstd1 = (float*)a.take(M * 4);
+    la.x_mid = (float*)a.take(M * d * 4); la.rstd2 = (float*)a.take(M * 4); la.h2 = a.take(M * d * es);
+    la.gu = a.take(M * 8 * d * es); la.act = a.take(M * 4 * d * es);
+  }
+  if (fwd_only) {
+    for (int l = 1; l < L; ++l) w.la[l] = w.la[0];
+    for (int l = 2; l <= L; ++l) w.x[l] = w.x[l & 1];
+  }
+  w.hs = a.take(R * d * es); w.rstdf = (float*)a.take(R * 4); w.z = (float*)a.take(R * NB * 4);
+  w.dz = a.take(R * NB * es);
+  w.loss_part = (float*)a.take(((R + 7) / 8) * 3 * 4); w.loss_acc = (float*)a.take(256);
+  if (!fwd_only) {
+    w.dx = (float*)a.take(M * d * 4); w.dx_t = a.take(M * d * es); w.dact = a.take(M * 4 * d * es);
+    w.dgu = a.take(M * 8 * d * es); w.dh = (float*)a.take(M * d * 4); w.dattn = a.take(M * d * es);
+    w.dqkv = a.take(M * 3 * d * es); w.dsum = (float*)a.take((size_t)mb * H * S * 4);
+    w.norm_part = (float*)a.take((size_t)NORM_BWD_BLOCKS * d * 4); w.dhs = (float*)a.take(R * d * 4);
+  }
+  w.bytes = a.off;
+}
+
+static int check_cfg(const grpo_model_cfg* c) {
+  if (!c) return PCM_ERR_ARG;
+  if (c->dtype != GRPO_F32 && c->dtype != GRPO_BF16) return PCM_ERR_ARG;
+  if (c->d < 8 || c->n_layers < 1 || c->n_layers > 128 || c->n_heads < 1 || c->prefix_len < 1) return PCM_ERR_ARG;
+  if (c->d % c->n_heads) return PCM_ERR_SHAPE;
+  const int dh = c->d / c->n_heads;
+  if (dh != 32 && dh != 64 && dh != 128) return PCM_ERR_SHAPE;
+  if (c->d % 8) return PCM_ERR_SHAPE;
+  if (c->prefix_len + ACT > 384) return PCM_ERR_SHAPE;
+  return PCM_OK;
+}
+
+template <typename T>
+static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* lc, grpo_grads* gr, float* loss,
+               float* logp, grpo_stats* stats, void* workspace, size_t workspace_bytes, cudaStream_t s) {
+  const grpo_model_cfg& c = m->cfg;
+  const int d = c.d, L = c.n_layers, H = c.n_heads, dh = d / H, P = c.prefix_len, S = P + ACT;
+  const int dt = c.dtype == GRPO_BF16 ? DT_BF16 : DT_F32;
+  const bool fwd_only = lc->flags & GRPO_FWD_ONLY;
+  const int n = pk->n_kept;
+  const int mb_max = lc->mb_chunks < n ? lc->mb_chunks : (n > 0 ? n : 1);
+  const float loss_scale = lc->loss_scale > 0.f ? lc->loss_scale : 1.0f / ((float)ACT * (float)(n > 0 ? n : 1));
+  const long long launches0 = g_launches.load();
+
+  Workspace w;
+  memset(&w, 0, sizeof(w));
+  carve(w, (unsigned char*)workspace, c, mb_max, fwd_only);
+  if (w.bytes > workspace_bytes) return PCM_ERR_WORKSPACE;
+
+  const T* w_qkv = (const T*)m->w_qkv; const T* w_o = (const T*)m->w_o; const T* w_gu = (const T*)m->w_gu;
+  const T* w_d = (const T*)m->w_d; const T* g1 = (const T*)m->g1; const T* g2 = (const T*)m->g2;
+  const T* gf = (const T*)m->gf; const T* w_h = (const T*)m->w_h;
+
+  // gradients start from zero unless the caller accumulates
+  if (!fwd_only && !(lc->flags & GRPO_ACCUMULATE)) {
+    const size_t dd = (size_t)d * d;
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_qkv, 0, (size_t)L * 3 * dd * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_o, 0, (size_t)L * dd * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_gu, 0, (size_t)L * 8 * dd * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_d, 0, (size_t)L * 4 * dd * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->g1, 0, (size_t)L * d * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->g2, 0, (size_t)L * d * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->gf, 0, (size_t)d * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_h, 0, (size_t)NB * d * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(gr->e_act, 0, (size_t)NB * d * 4, s));
+  }
+  PCM_CUDA_TRY(cudaMemsetAsync(w.loss_acc, 0, 256, s));
+  PCM_CUDA_TRY(cudaMemsetAsync(loss, 0, sizeof(float), s));
+  rope_table_kernel<<<ceil_div((long long)S * dh / 2, 256), 256, 0, s>>>(w.rope_tab, S, dh);
+  PCM_LAUNCH_CHECK();
+
+  auto G = [&](int M_, int N_, int K_, const void* A, long long lda, bool ak, const void* B, long long ldb, bool bk,
+               int abdt, void* C, long long ldc, int cdt, const float* R, long long ldr) -> int {
+    GemmArgs g{M_, N_, K_, A, lda, ak, B, ldb, bk, abdt, C, ldc, cdt, R, ldr};
+    return gemm(g, s);
+  };
+#define TRY(expr) do { int rc__ = (expr); if (rc__ != PCM_OK) return rc__; } while (0)
+
+  for (int c0 = 0; c0 < n; c0 += mb_max) {
+    const int mb = (n - c0) < mb_max ? (n - c0) : mb_max;
+    const long long M = (long long)mb * S, R = (long long)mb * ACT;
+    const int Mi = (int)M, Ri = (int)R;
+    const T* Xmb = (const T*)pk->X + (long long)c0 * S * d;
+    const uint8_t* tgt = pk->tgt + (long long)c0 * ACT;
+    const float* lpo = pk->lpo + (long long)c0 * ACT;
+    const float* advc = pk->adv_c + c0;
+
+    // ---------------- forward ----------------
+    to_residual_kernel<T><<<ceil_div(M * d, 1024), 256, 0, s>>>(Xmb, w.x[0], M * d);
+    PCM_LAUNCH_CHECK();
+    for (int l = 0; l < L; ++l) {
+      LayerActs& la = w.la[l];
+      const float* x_in = w.x[l];
+      float* x_out = w.x[l + 1];
+      rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(x_in, g1 + (size_t)l * d, (T*)la.h1, la.rstd1, M, d, 0, 0);
+      PCM_LAUNCH_CHECK();
+      TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0));
+      rope_kernel<T><<<ceil_div(M * H * dh, 256), 256, 0, s>>>((T*)la.qkv, w.rope_tab, M, S, H, dh, 1.f);
+      PCM_LAUNCH_CHECK();
+      TRY(attention_fwd(dt, la.qkv, la.attn, la.lse, mb, S, H, dh, s));
+      TRY(G(Mi, d, d, la.attn, d, true, w_o + (size_t)l * d * d, d, true, dt, la.x_mid, d, DT_F32, x_in, d));
+      rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(la.x_mid, g2 + (size_t)l * d, (T*)la.h2, la.rstd2, M, d, 0, 0);
+      PCM_LAUNCH_CHECK();
+      TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0));
+      swiglu_fwd_kernel<T><<<ceil_div(M * 4 * d, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, M, 4 * d);
+      PCM_LAUNCH_CHECK();
+      TRY(G(Mi, d, 4 * d, la.act, 4 * d, true, w_d + (size_t)l * 4 * d * d, 4 * d, true, dt, x_out, d, DT_F32, la.x_mid, d));
+    }
+    // head on the scored rows only
+    rmsnorm_fwd_kernel<T><<<ceil_div(R, 8), 256, 0, s>>>(w.x[L], gf, (T*)w.hs, w.rstdf, R, d, S, P);
+    PCM_LAUNCH_CHECK();
+    TRY(G(Ri, NB, d, w.hs, d, true, w_h, d, true, dt, w.z, NB, DT_F32, nullptr, 0));
+    const int loss_blocks = ceil_div(R, 8);
+    loss_rows_kernel<T><<<loss_blocks, 256, 0, s>>>(w.z, tgt, lpo, advc, lc->eps_low, lc->eps_high, loss_scale,
+                                                  (T*)w.dz, logp ? logp + (long long)c0 * ACT : nullptr, w.loss_part,
+                                                  R, fwd_only ? 1 : 0);
+    PCM_LAUNCH_CHECK();
+    loss_reduce_kernel<<<1, 256, 0, s>>>(w.loss_part, loss_blocks, loss_scale, w.loss_acc, loss);
+    PCM_LAUNCH_CHECK();
+    if (fwd_only) continue;
+
+    // ---------------- backward ----------------
+    // head: dW_h += dz^T hs ; dhs = dz W_h ; final norm backward scatters into dx
+    TRY(G(NB, d, Ri, w.dz, NB, false, w.hs, d, false, dt, gr->w_h, d, DT_F32, gr->w_h, d));
+    TRY(G(Ri, d, NB, w.dz, NB, true, w_h, d, false, dt, w.dhs, d, DT_F32, nullptr, 0));
+    PCM_CUDA_TRY(cudaMemsetAsync(w.dx, 0, (size_t)M * d * 4, s));
+    PCM_CUDA_TRY(cudaMemsetAsync(w.dx_t, 0, (size_t)M * d * sizeof(T), s));
+    const size_t nb_smem = (size_t)8 * d * sizeof(float);
+    if (nb_smem > 48 * 1024)
+      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
+    auto norm_bwd = [&](const float* dy, const float* x, const float* rstd, const T* gamma, const float* dx_in,
+                        long long rows, int mS, int mP, float* dgamma) -> int {
+      const int blocks = (int)(rows / 8 + 1 < NORM_BWD_BLOCKS ? rows / 8 + 1 : NORM_BWD_BLOCKS);
+      rmsnorm_bwd_kernel<T><<<blocks, 256, nb_smem, s>>>(dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t, w.norm_part, rows,
+                                                       d, mS, mP);
+      PCM_LAUNCH_CHECK();
+      colsum_accumulate_kernel<<<ceil_div(d, 256), 256, 0, s>>>(w.norm_part, blocks, d, dgamma);
+      PCM_LAUNCH_CHECK();
+      return PCM_OK;
+    };
+    TRY(norm_bwd(w.dhs, w.x[L], w.rstdf, gf, nullptr, R, S, P, gr->gf));
+
+    for (int l = L - 1; l >= 0; --l) {
+      LayerActs& la = w.la[l];
+      const size_t dd = (size_t)d * d;
+      // MLP: x_out = x_mid + act W_d^T
+      TRY(G(d, 4 * d, Mi, w.dx_t, d, false, la.act, 4 * d, false, dt, gr->w_d + l * 4 * dd, 4 * d, DT_F32,
+            gr->w_d + l * 4 * dd, 4 * d));
+      TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dact, 4 * d, dt, nullptr, 0));
+      swiglu_bwd_kernel<T><<<ceil_div(M * 4 * d, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, M, 4 * d);
+      PCM_LAUNCH_CHECK();
+      TRY(G(8 * d, d, Mi, w.dgu, 8 * d, false, la.h2, d, false, dt, gr->w_gu + l * 8 * dd, d, DT_F32,
+            gr->w_gu + l * 8 * dd, d));
+      TRY(G(Mi, d, 8 * d, w.dgu, 8 * d, true, w_gu + l * 8 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
+      TRY(norm_bwd(w.dh, la.x_mid, la.rstd2, g2 + (size_t)l * d, w.dx, M, 0, 0, gr->g2 + (size_t)l * d));
+      // attention block: x_mid = x_in + attn W_o^T
+      TRY(G(d, d, Mi, w.dx_t, d, false, la.attn, d, false, dt, gr->w_o + l * dd, d, DT_F32, gr->w_o + l * dd, d));
+      TRY(G(Mi, d, d, w.dx_t, d, true, w_o + l * dd, d, false, dt, w.dattn, d, dt, nullptr, 0));
+      TRY(attention_bwd(dt, la.qkv, la.attn, w.dattn, la.lse, w.dsum, w.dqkv, mb, S, H, dh, s));
+      rope_kernel<T><<<ceil_div(M * H * dh, 256), 256, 0, s>>>((T*)w.dqkv, w.rope_tab, M, S, H, dh, -1.f);
+      PCM_LAUNCH_CHECK();
+      TRY(G(3 * d, d, Mi, w.dqkv, 3 * d, false, la.h1, d, false, dt, gr->w_qkv + l * 3 * dd, d, DT_F32,
+            gr->w_qkv + l * 3 * dd, d));
+      TRY(G(Mi, d, 3 * d, w.dqkv, 3 * d, true, w_qkv + l * 3 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
+      TRY(norm_bwd(w.dh, w.x[l], la.rstd1, g1 + (size_t)l * d, w.dx, M, 0, 0, gr->g1 + (size_t)l * d));
+    }
+    embed_grad_kernel<<<dim3(NB, ceil_div(d, 256)), 256, 0, s>>>(w.dx, tgt, mb, S, P, d, gr->e_act);
+    PCM_LAUNCH_CHECK();
+  }
+#undef TRY
+
+  if (stats) {
+    float acc[3] = {0, 0, 0}, l = 0;
+    PCM_CUDA_TRY(cudaMemcpyAsync(acc, w.loss_acc, sizeof(acc), cudaMemcpyDeviceToHost, s));
+    PCM_CUDA_TRY(cudaMemcpyAsync(&l, loss, sizeof(float), cudaMemcpyDeviceToHost, s));
+    PCM_CUDA_TRY(cudaStreamSynchronize(s));
+    const float tokens = (float)n * ACT;
+    stats->loss = l;
+    stats->clip_frac = tokens > 0 ? acc[1] / tokens : 0.f;
+    stats->mean_ratio = tokens > 0 ? acc[2] / tokens : 0.f;
+    stats->n_launches = (int32_t)(g_launches.load() - launches0);
+    stats->workspace_high_water = w.bytes;
+    const int tcs = tcgen05_poll_status();
+    if (tcs != PCM_OK) return tcs;
+  }
+  return PCM_OK;
+}
+
+static GemmBackend backend_from_env() {
+  const char* e = getenv("PCM_GEMM_BACKEND");
+  if (e && !strcmp(e, "simt")) return GEMM_SIMT;
+  if (e && !strcmp(e, "tcgen05")) return GEMM_TCGEN05;
+  return GEMM_AUTO;
+}
+
+int gemm(const GemmArgs& g, cudaStream_t s, GemmBackend backend) {
+  if (backend == GEMM_AUTO) backend = backend_from_env();
+  if (backend == GEMM_TCGEN05) {
+    if (!gemm_tcgen05_supported(g)) return PCM_ERR_SHAPE;
+    return gemm_tcgen05(g, s);
+  }
+  if (backend == GEMM_AUTO && gemm_tcgen05_supported(g)) return gemm_tcgen05(g, s);
+  return gemm_simt(g, s);
+}
+
+}  // namespace pcm
+
+using namespace pcm;
+
+extern "C" size_t grpo_workspace_bytes(const grpo_model_cfg* cfg, int32_t mb_chunks, uint32_t flags) {
+  if (check_cfg(cfg) != PCM_OK || mb_chunks < 1) return 0;
+  Workspace w;
+  memset(&w, 0, sizeof(w));
+  carve(w, nullptr, *cfg, mb_chunks, flags & GRPO_FWD_ONLY);
+  return w.bytes;
+}
+
+extern "C" int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* batch, const grpo_loss_cfg* lc,
+                                  grpo_grads* grads, float* loss, float* logp, grpo_stats* stats, void* workspace,
+                                  size_t workspace_bytes, pcm_stream stream) {
+  if (!model || !batch || !lc || !loss || !workspace) return PCM_ERR_ARG;
+  int rc = check_cfg(&model->cfg);
+  if (rc) return rc;
+  if (!model->w_qkv || !model->w_o || !model->w_gu || !model->w_d || !model->g1 || !model->g2 || !model->gf ||
+      !model->w_h || !model->e_act)
+    return PCM_ERR_ARG;
+  if (batch->n_kept < 0 || lc->mb_chunks < 1 || !(lc->eps_low >= 0.f) || !(lc->eps_high >= 0.f)) return PCM_ERR_ARG;
+  if (batch->n_kept > 0 && (!batch->X || !batch->tgt || !batch->lpo || !batch->adv_c)) return PCM_ERR_ARG;
+  const bool fwd_only = lc->flags & GRPO_FWD_ONLY;
+  if (!fwd_only) {
+    if (!grads || !grads->w_qkv || !grads->w_o || !grads->w_gu || !grads->w_d || !grads->g1 || !grads->g2 ||
+        !grads->gf || !grads->w_h || !grads->e_act)
+      return PCM_ERR_ARG;
+  }
+  if (((uintptr_t)workspace) & 255) return PCM_ERR_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (model->cfg.dtype == GRPO_BF16)
+    return run<__nv_bfloat16>(model, batch, lc, grads, loss, logp, stats, workspace, workspace_bytes, s);
+  return run<float>(model, batch, lc, grads, loss, logp, stats, workspace, workspace_bytes, s);
+}
+
+extern "C" int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_kmajor, const void* B,
+                         int64_t ldb, int32_t b_kmajor, int32_t ab_dtype, void* C, int64_t ldc, int32_t c_dtype,
+                         const float* R, int64_t ldr, int32_t backend, pcm_stream stream) {
+  if (!A || !B || !C || M < 1 || N < 1 || K < 1 || backend < 0 || backend > 2) return PCM_ERR_ARG;
+  if ((ab_dtype != GRPO_F32 && ab_dtype != GRPO_BF16) || (c_dtype != GRPO_F32 && c_dtype != GRPO_BF16)) return PCM_ERR_ARG;
+  GemmArgs g{M, N, K, A, lda, a_kmajor != 0, B, ldb, b_kmajor != 0, ab_dtype == GRPO_BF16 ? DT_BF16 : DT_F32,
+             C, ldc, c_dtype == GRPO_BF16 ? DT_BF16 : DT_F32, R, ldr};
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc = gemm(g, s, backend == 1 ? GEMM_SIMT : backend == 2 ? GEMM_TCGEN05 : GEMM_AUTO);
+  if (rc != PCM_OK) return rc;
+  PCM_CUDA_TRY(cudaStreamSynchronize(s));
+  return tcgen05_poll_status();
+}
+
+extern "C" int grpo_attention(int32_t dtype, const void* qkv, void* out, float* lse, const void* dout, void* dqkv,
+                              float* scratch, int32_t n_seq, int32_t S, int32_t n_heads, int32_t head_dim,
+                              pcm_stream stream) {
+  if (!qkv || !out || !lse || n_seq < 1 || S < 1 || n_heads < 1) return PCM_ERR_ARG;
+  if (dtype != GRPO_F32 && dtype != GRPO_BF16) return PCM_ERR_ARG;
+  if (dout && (!dqkv || !scratch)) return PCM_ERR_ARG;
+  const int dt = dtype == GRPO_BF16 ? DT_BF16 : DT_F32;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc = attention_fwd(dt, qkv, out, lse, n_seq, S, n_heads, head_dim, s);
+  if (rc != PCM_OK) return rc;
+  if (dout) {
+    rc = attention_bwd(dt, qkv, out, dout, lse, scratch, dqkv, n_seq, S, n_heads, head_dim, s);
+    if (rc != PCM_OK) return rc;
+  }
+  PCM_CUDA_TRY(cudaStreamSynchronize(s));
+  return PCM_OK;
+}
