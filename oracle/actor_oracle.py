@@ -71,6 +71,27 @@ def silu(x):
     return x / (1.0 + np.exp(-x))
 
 
+def causal_attention(q, k, v):
+    """softmax(q k^T / sqrt(dh) + causal mask) v for q, k, v of shape [n, H, S, dh]; returns (o, p)."""
+    S, dh = q.shape[-2], q.shape[-1]
+    causal = np.triu(np.ones((S, S), dtype=bool), k=1)       # True where key position > query position
+    s = (q @ k.transpose(0, 1, 3, 2)) / np.sqrt(dh)          # [n, H, S(query), S(key)]
+    s = np.where(causal[None, None], -np.inf, s)
+    s = s - s.max(axis=-1, keepdims=True)
+    p = np.exp(s)
+    p = p / p.sum(axis=-1, keepdims=True)
+    return p @ v, p
+
+
+def causal_attention_bwd(do, q, k, v, p):
+    """Gradients of causal_attention w.r.t. q, k, v given do = dL/do (all [n, H, S, dh])."""
+    dh = q.shape[-1]
+    dv = p.transpose(0, 1, 3, 2) @ do
+    dp = do @ v.transpose(0, 1, 3, 2)
+    ds = p * (dp - np.sum(dp * p, axis=-1, keepdims=True)) / np.sqrt(dh)
+    return ds @ k, ds.transpose(0, 1, 3, 2) @ q, dv
+
+
 def forward(weights: Dict[str, np.ndarray], X, H: int, P: int, keep_cache: bool = True):
     """X [n, S, d] -> (z [n, 56, V] logits at the scored positions, cache)."""
     Wt = {k: _f64(v) for k, v in weights.items()}
@@ -79,7 +100,6 @@ def forward(weights: Dict[str, np.ndarray], X, H: int, P: int, keep_cache: bool 
     L = Wt["w_qkv"].shape[0]
     dh = d // H
     cos, sin = rope_tables(S, dh)
-    causal = np.triu(np.ones((S, S), dtype=bool), k=1)       # True where key position > query position
     layers = []
     for l in range(L):
         x_in = x
@@ -89,12 +109,8 @@ def forward(weights: Dict[str, np.ndarray], X, H: int, P: int, keep_cache: bool 
         q = rope(qkv[..., :d].reshape(n, S, H, dh), cos, sin).transpose(0, 2, 1, 3)
         k = rope(qkv[..., d:2 * d].reshape(n, S, H, dh), cos, sin).transpose(0, 2, 1, 3)
         v = qkv[..., 2 * d:].reshape(n, S, H, dh).transpose(0, 2, 1, 3)
-        s = (q @ k.transpose(0, 1, 3, 2)) / np.sqrt(dh)                    # [n, H, S(query), S(key)]
-        s = np.where(causal[None, None], -np.inf, s)
-        s = s - s.max(axis=-1, keepdims=True)
-        p = np.exp(s)
-        p = p / p.sum(axis=-1, keepdims=True)
-        o = (p @ v).transpose(0, 2, 1, 3).reshape(n, S, d)
+        o, p = causal_attention(q, k, v)
+        o = o.transpose(0, 2, 1, 3).reshape(n, S, d)
         x_mid = x_in + o @ Wt["w_o"][l].T
         h2, rstd2 = rmsnorm(x_mid, Wt["g2"][l])
         gu = h2 @ Wt["w_gu"][l].T
@@ -190,12 +206,9 @@ def fwd_bwd(weights, X, tgt, logp_old, adv_c, H, P, eps_low=0.2, eps_high=0.2, l
         # x_mid = x_in + o @ W_o^T
         grads["w_o"][l] = dx_mid.reshape(n * S, d).T @ c["o"].reshape(n * S, d)
         do = (dx_mid @ Wt["w_o"][l]).reshape(n, S, H, dh).transpose(0, 2, 1, 3)   # [n, H, S, dh]
-        p = c["p"]
-        dv = p.transpose(0, 1, 3, 2) @ do
-        dp = do @ c["v"].transpose(0, 1, 3, 2)
-        ds = p * (dp - np.sum(dp * p, axis=-1, keepdims=True)) / np.sqrt(dh)
-        dq = rope_bwd((ds @ c["k"]).transpose(0, 2, 1, 3), cos, sin)               # [n, S, H, dh]
-        dk = rope_bwd((ds.transpose(0, 1, 3, 2) @ c["q"]).transpose(0, 2, 1, 3), cos, sin)
+        dq, dk, dv = causal_attention_bwd(do, c["q"], c["k"], c["v"], c["p"])
+        dq = rope_bwd(dq.transpose(0, 2, 1, 3), cos, sin)                           # [n, S, H, dh]
+        dk = rope_bwd(dk.transpose(0, 2, 1, 3), cos, sin)
         dv = dv.transpose(0, 2, 1, 3)
         dqkv = np.concatenate([dq.reshape(n, S, d), dk.reshape(n, S, d), dv.reshape(n, S, d)], axis=-1)
         grads["w_qkv"][l] = dqkv.reshape(n * S, 3 * d).T @ c["h1"].reshape(n * S, d)

@@ -1,0 +1,48 @@
+"""The shared library loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "pcm_b200.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b((?:pcm|grpo)_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    from paper_2605_16154_b200 import build
+    lib = ctypes.CDLL(build.build())
+    names = _declared()
+    assert {"pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
+            "grpo_actor_fwd_bwd"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_binding_struct_sizes_match_the_header_layout():
+    from paper_2605_16154_b200 import binding as B
+    assert ctypes.sizeof(B.pcm_config) == 40
+    assert ctypes.sizeof(B.pcm_batch) == 16 + 6 * 8
+    assert ctypes.sizeof(B.grpo_model_cfg) == 24
+    assert ctypes.sizeof(B.grpo_model) == 24 + 9 * 8
+    assert ctypes.sizeof(B.grpo_packed) == 8 + 5 * 8
+    assert ctypes.sizeof(B.grpo_loss_cfg) == 24
+    assert ctypes.sizeof(B.grpo_stats) == 24
+    assert set(B.EXPORTED) == set(_declared())
+
+
+def test_host_side_argument_checks_need_no_gpu():
+    from paper_2605_16154_b200 import binding as B
+    cfg = B.grpo_model_cfg(100, 2, 3, 4, 1, 0)          # d not divisible by heads
+    assert B._lib.grpo_workspace_bytes(ctypes.byref(cfg), 4, 0) == 0
+    cfg = B.grpo_model_cfg(1024, 8, 16, 256, 1, 0)
+    full = B._lib.grpo_workspace_bytes(ctypes.byref(cfg), 64, 0)
+    fwd = B._lib.grpo_workspace_bytes(ctypes.byref(cfg), 64, B.GRPO_FWD_ONLY)
+    assert 0 < fwd < full
+    # activations kept per token per layer: 18 d bf16 + 2 d fp32 (+ small terms)
+    per_token = full / (64 * 312)
+    assert 8 * 44 * 1024 < per_token < 8 * 44 * 1024 * 1.3
+    assert B._lib.pcm_create(None, None, 0) == -1

@@ -1,0 +1,191 @@
+"""CUDA path vs oracle for the PCM control plane and the pack step: bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pcm_oracle as po
+from paper_2605_16154_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _mods():
+    from paper_2605_16154_b200 import binding as B, pipeline as PL
+    return B, PL
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+@pytest.mark.parametrize("name", ["C0", "C1", "C3", "C4"])
+def test_score_update_sample_bit_exact(name):
+    B, PL = _mods()
+    w = synth.WORKLOADS[name]
+    rb = synth.make_rollouts(w)
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=1234 + w.seed, max_traj=w.n_traj)
+    batch = PL.upload_rollouts(w, rb)
+    adv, Cc, valid, p, q, kept_idx, kept_off, per_phase = PL.select(ctx, batch, it=7)
+    assert B.pcm_poll_status(ctx) == 0
+    C_o, valid_o, nvalid_o, _, _ = po.score_phases(rb["traj_off"], rb["tok"], rb["phase"], rb["reward"], w.G, w.n_phases)
+    assert np.array_equal(_np(Cc).view(np.uint64), C_o.view(np.uint64))            # bit-exact fp64
+    assert np.array_equal(_np(valid), valid_o)
+    adv_o = po.advantages(rb["reward"], w.G, 1e-6).astype(np.float32)
+    assert np.array_equal(_np(adv).view(np.uint32), adv_o.view(np.uint32))
+    st = po.KeepProbState(w.n_phases, w.p_min, w.t_rc)
+    p_o, q_o, _ = po.update_keep_probs(st, C_o, valid_o)
+    assert np.array_equal(_np(q).astype(np.int64), q_o)
+    assert np.array_equal(_np(p), p_o.astype(np.float32))
+    k_o, off_o, pp_o = po.sample_chunks(rb["traj_off"], rb["phase"], q_o, w.budget, 1234 + w.seed, 7)
+    n_kept = int(off_o[-1])
+    assert np.array_equal(_np(kept_off), off_o)
+    assert np.array_equal(_np(kept_idx)[:n_kept], k_o)
+    assert np.array_equal(_np(per_phase), pp_o)
+    ctx.close()
+
+
+def test_online_chain_50_iterations_ragged():
+    """C4: rollouts resampled every iteration, keep-probability state carried across iterations."""
+    B, PL = _mods()
+    w = synth.WORKLOADS["C4"]
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=99, max_traj=w.n_traj)
+    st = po.KeepProbState(w.n_phases, w.p_min, w.t_rc)
+    refreshes = []
+    for it in range(50):
+        rb = synth.make_rollouts(w, seed=it)
+        batch = PL.upload_rollouts(w, rb)
+        adv, Cc, valid, p, q, kept_idx, kept_off, per_phase = PL.select(ctx, batch, it)
+        C_o, valid_o, _, _, _ = po.score_phases(rb["traj_off"], rb["tok"], rb["phase"], rb["reward"], w.G, w.n_phases)
+        p_o, q_o, refreshed = po.update_keep_probs(st, C_o, valid_o)
+        if refreshed:
+            refreshes.append(it)
+        k_o, off_o, pp_o = po.sample_chunks(rb["traj_off"], rb["phase"], q_o, w.budget, 99, it)
+        assert np.array_equal(_np(Cc).view(np.uint64), C_o.view(np.uint64)), it
+        assert np.array_equal(_np(q).astype(np.int64), q_o), it
+        assert np.array_equal(_np(kept_off), off_o), it
+        assert np.array_equal(_np(kept_idx)[: int(off_o[-1])], k_o), it
+        assert np.array_equal(_np(per_phase), pp_o), it
+        if it == 22:      # stop and resume from an exported state blob
+            blob = B.pcm_state_export(ctx)
+            ctx.close()
+            ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=99, max_traj=w.n_traj)
+            B.pcm_state_import(ctx, blob)
+    assert refreshes == list(range(0, 50, 5))
+    assert B.pcm_poll_status(ctx) == 0
+    ctx.close()
+
+
+def test_sampler_edge_cases():
+    """Budget above every length (keep all), lengths below the budget, single-chunk and empty
+    trajectories, arbitrary (non-contiguous) phase labels, more than one tile of 32 chunks."""
+    B, PL = _mods()
+    rng = np.random.default_rng(0)
+    lengths = np.array([1, 0, 5, 33, 64, 2, 100, 31, 32, 7, 257, 3], dtype=np.int64)
+    traj_off = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    total = int(traj_off[-1])
+    Kc = 6
+    rb = {"traj_off": traj_off, "tok": rng.integers(0, 256, (total, 56), dtype=np.uint8),
+          "phase": rng.integers(0, Kc, total).astype(np.uint8), "reward": np.array([1, 0] * 6, dtype=np.uint8)}
+    w = synth.WORKLOADS["C0"].with_(n_phases=Kc, G=4)
+    for budget in (1, 6, 40, 500):
+        ctx = B.Context(Kc, budget, 4, 5, 0.1, 1e-6, seed=(1 << 40) + 17, max_traj=12)
+        batch = PL.upload_rollouts(w, rb)
+        q_np = np.array([1 << 24, 1677722, 5000000, 1, 9999999, 1 << 23], dtype=np.int64)
+        q = torch.from_numpy(q_np.astype(np.int32)).cuda()
+        it = (3 << 32) + 5
+        kept_idx, kept_off, per_phase = B.pcm_sample_chunks(ctx, batch, q, it)
+        k_o, off_o, pp_o = po.sample_chunks(traj_off, rb["phase"], q_np, budget, (1 << 40) + 17, it)
+        assert np.array_equal(_np(kept_off), off_o)
+        assert np.array_equal(_np(kept_idx)[: int(off_o[-1])], k_o)
+        assert np.array_equal(_np(per_phase), pp_o)
+        assert B.pcm_poll_status(ctx) == 0
+        ctx.close()
+
+
+def test_score_edge_cases_and_status_word():
+    B, PL = _mods()
+    rng = np.random.default_rng(1)
+    # long runs inside one phase (> 256 chunks between flushes), uniform groups, a missing phase
+    lengths = np.array([700, 3, 1, 650, 10, 10, 10, 10], dtype=np.int64)
+    traj_off = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    total = int(traj_off[-1])
+    phase = np.zeros(total, dtype=np.uint8)
+    phase[traj_off[3]: traj_off[3] + 600] = 1
+    phase[traj_off[4]:] = rng.integers(0, 3, total - traj_off[4]).astype(np.uint8)
+    rb = {"traj_off": traj_off, "tok": np.full((total, 56), 255, dtype=np.uint8), "phase": phase,
+          "reward": np.array([1, 0, 0, 0, 1, 1, 1, 1], dtype=np.uint8)}
+    rb["tok"][traj_off[3]:] = rng.integers(0, 256, (total - traj_off[3], 56), dtype=np.uint8)
+    w = synth.WORKLOADS["C0"].with_(n_phases=3, G=4)
+    ctx = B.Context(3, 2, 4, 5, 0.1, 1e-6, seed=0, max_traj=8)
+    batch = PL.upload_rollouts(w, rb)
+    Cc, valid, n_valid, adv = B.pcm_score_phases(ctx, batch)
+    C_o, valid_o, nv_o, _, _ = po.score_phases(traj_off, rb["tok"], phase, rb["reward"], 4, 3)
+    assert np.array_equal(_np(Cc).view(np.uint64), C_o.view(np.uint64))
+    assert np.array_equal(_np(valid), valid_o) and np.array_equal(_np(n_valid), nv_o)
+    assert B.pcm_poll_status(ctx) == 0
+    # a phase label beyond n_phases is reported through the status word, not by a fault
+    bad = dict(rb)
+    bad["phase"] = phase.copy()
+    bad["phase"][5] = 9
+    B.pcm_score_phases(ctx, PL.upload_rollouts(w, bad))
+    assert B.pcm_poll_status(ctx) == -7
+    assert B.pcm_poll_status(ctx) == 0
+    ctx.close()
+
+
+def test_host_argument_errors():
+    B, PL = _mods()
+    with pytest.raises(B.PcmError):
+        B.Context(0, 3, 8)                      # no phases
+    with pytest.raises(B.PcmError):
+        B.Context(4, 3, 8, p_min=0.0)           # floor must be positive
+    ctx = B.Context(4, 3, 8, max_traj=8)
+    w = synth.WORKLOADS["C0"]
+    rb = synth.make_rollouts(w)
+    batch = PL.upload_rollouts(w, rb)
+    batch.n_traj = 7                             # not a multiple of the group size
+    with pytest.raises(B.PcmError):
+        B.pcm_score_phases(ctx, batch)
+    with pytest.raises(B.PcmError):
+        B.pcm_state_import(ctx, b"\0" * 10)
+    ctx.close()
+
+
+@pytest.mark.parametrize("case", ["C0", "bf16_wide", "bf16_ragged"])
+def test_pack_bit_exact(case):
+    B, PL = _mods()
+    if case == "C0":
+        w = synth.WORKLOADS["C0"]
+    elif case == "bf16_wide":
+        w = synth.WORKLOADS["C1"].with_(n_tasks=1, G=4, T=9, budget=4)          # 512 KB prefixes, 2 KB rows
+    else:
+        w = synth.WORKLOADS["C4"].with_(n_tasks=1, G=4, d=2048, P=37, len_lo=3, len_hi_succ=9, len_hi_fail=12,
+                                        n_phases=3, budget=5)
+    rb = synth.make_rollouts(w, seed=3)
+    total = int(rb["traj_off"][-1])
+    e_act = synth.round_to_dtype(np.random.default_rng(2).standard_normal((256, w.d)).astype(np.float32), w.dtype)
+    obs = synth.obs_all(w, 5, total)
+    lpo = np.random.default_rng(3).standard_normal((total, 56)).astype(np.float32)
+    adv = po.advantages(rb["reward"], w.G).astype(np.float32)
+    q = [1 << 24] * w.n_phases
+    kept, off, _ = po.sample_chunks(rb["traj_off"], rb["phase"], q, w.budget, 5, 0)
+    X_o, tgt_o, lpo_o, advc_o, src_o = po.pack_chunks(lambda c: obs[c], rb["tok"], lpo, adv, rb["traj_off"], kept, e_act)
+
+    td = PL.torch_dtype(w)
+    ctx = B.Context(w.n_phases, w.budget, w.G, max_traj=w.n_traj)
+    batch = PL.upload_rollouts(w, rb, obs=PL.dev(obs, td), logp_old=PL.dev(lpo))
+
+    class _M:      # only what pack needs from a model
+        cfg = B.grpo_model_cfg(w.d, w.L, w.H, w.P, PL.model_dtype(w), 0)
+        weights = {"e_act": PL.dev(e_act, td)}
+        S = w.S
+    out = B.Packed(_M, len(kept))
+    out.X.fill_(7.0)
+    B.grpo_pack_chunks(ctx, batch, _M, PL.dev(kept), PL.dev(off), PL.dev(adv), out)
+    assert B.pcm_poll_status(ctx) == 0
+    assert np.array_equal(_np(out.X.float()), X_o.astype(np.float32))      # values exact in the dtype => bit-exact
+    assert np.array_equal(_np(out.tgt), tgt_o)
+    assert np.array_equal(_np(out.lpo), lpo_o)
+    assert np.array_equal(_np(out.adv_c), advc_o)
+    assert np.array_equal(_np(out.src), src_o)
+    ctx.close()
