@@ -1,0 +1,189 @@
+"""CUDA actor update vs the fp64 oracle: per-kernel (GEMM, attention) and end to end.
+
+Tolerances: fp32 mode 1e-5 relative (loss, log-probs, per-tensor Frobenius of gradients);
+bf16 inputs / fp32 accumulate: gradients 2e-2 relative Frobenius per tensor, loss 1e-3 absolute."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import actor_oracle as ao
+from paper_2605_16154_b200 import synth
+from tests.gpu_helpers import device_packed, grads_to_numpy, host_problem, oracle_update, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+F32_TOL = 1e-5
+BF16_GRAD_TOL = 2e-2
+BF16_LOSS_TOL = 1e-3
+
+
+def _mods():
+    from paper_2605_16154_b200 import binding as B, pipeline as PL
+    return B, PL
+
+
+# ------------------------------------------------------------------ GEMM (SIMT: fp32 mode and fallback)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("a_k,b_k", [(True, True), (True, False), (False, True), (False, False)])
+def test_gemm_simt_all_layouts(dtype, a_k, b_k):
+    B, PL = _mods()
+    rng = np.random.default_rng(3)
+    M, N, K = 150, 77, 93                      # several 64-tiles and ragged tails
+    A = synth.round_to_dtype(rng.standard_normal((M, K)).astype(np.float32), dtype)
+    Bm = synth.round_to_dtype(rng.standard_normal((N, K)).astype(np.float32), dtype)
+    R = rng.standard_normal((M, N)).astype(np.float32)
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    At = PL.dev(A if a_k else A.T.copy(), td)
+    Bt = PL.dev(Bm if b_k else Bm.T.copy(), td)
+    out = B.grpo_gemm(At, a_k, Bt, b_k, M, N, K, torch.float32, R=PL.dev(R), backend=1)
+    expect = A.astype(np.float64) @ Bm.astype(np.float64).T + R
+    assert rel_fro(out.cpu().numpy(), expect) < 2e-6
+    acc = PL.dev(R.copy())
+    B.grpo_gemm(At, a_k, Bt, b_k, M, N, K, R=acc, backend=1, C_out=acc)      # accumulate in place
+    assert rel_fro(acc.cpu().numpy(), expect) < 2e-6
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("dtype,dh,S,H,n_seq", [("f32", 32, 88, 4, 3), ("f32", 64, 45, 2, 2), ("bf16", 64, 312, 3, 2),
+                                                ("bf16", 128, 100, 2, 2), ("bf16", 32, 33, 2, 1)])
+def test_attention_fwd_bwd(dtype, dh, S, H, n_seq):
+    B, PL = _mods()
+    rng = np.random.default_rng(5)
+    d = H * dh
+    qkv = synth.round_to_dtype(rng.standard_normal((n_seq * S, 3 * d)).astype(np.float32), dtype)
+    do = synth.round_to_dtype(rng.standard_normal((n_seq * S, d)).astype(np.float32), dtype)
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    out, lse, dqkv = B.grpo_attention(PL.dev(qkv, td), n_seq, S, H, dh, dout=PL.dev(do, td))
+
+    def heads(x):
+        return x.astype(np.float64).reshape(n_seq, S, H, dh).transpose(0, 2, 1, 3)
+    q, k, v = heads(qkv[:, :d]), heads(qkv[:, d:2 * d]), heads(qkv[:, 2 * d:])
+    o, p = ao.causal_attention(q, k, v)
+    dq, dk, dv = ao.causal_attention_bwd(heads(do), q, k, v, p)
+    back = lambda x: x.transpose(0, 2, 1, 3).reshape(n_seq * S, d)
+    tol = 2e-6 if dtype == "f32" else 6e-3
+    assert rel_fro(out.float().cpu().numpy(), back(o)) < tol
+    got = dqkv.float().cpu().numpy()
+    assert rel_fro(got[:, :d], back(dq)) < tol * 2
+    assert rel_fro(got[:, d:2 * d], back(dk)) < tol * 2
+    assert rel_fro(got[:, 2 * d:], back(dv)) < tol * 2
+
+
+# ------------------------------------------------------------------ end to end
+def _compare(B, PL, hp, tol_grad, tol_loss_rel=None, tol_loss_abs=None, mb=64, eps=(0.2, 0.2), loss_scale=None):
+    w = hp["w"]
+    model = PL.upload_model(w, hp["weights"])
+    pk = device_packed(B, PL, model, hp)
+    loss_o, logp_o, grads_o, stats_o = oracle_update(hp, eps[0], eps[1], loss_scale)
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, pk, eps[0], eps[1], loss_scale or 0.0, mb_chunks=mb)
+    loss = float(loss.item())
+    if tol_loss_rel is not None:
+        assert abs(loss - loss_o) <= tol_loss_rel * abs(loss_o) + 1e-9
+    if tol_loss_abs is not None:
+        assert abs(loss - loss_o) <= tol_loss_abs
+    g = grads_to_numpy(grads)
+    errs = {k: rel_fro(g[k], grads_o[k]) for k in grads_o}
+    assert max(errs.values()) < tol_grad, errs
+    assert abs(stats.clip_frac - stats_o["clip_frac"]) < 0.02
+    assert stats.n_launches > 0
+    return model, pk, (loss, logp, g, stats), (loss_o, logp_o, grads_o, stats_o), errs
+
+
+def test_c0_fp32_end_to_end():
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"].with_(gamma_std=0.1)
+    hp = host_problem(w)
+    assert len(hp["kept"]) == 24
+    model, pk, got, ref, errs = _compare(B, PL, hp, F32_TOL, tol_loss_rel=F32_TOL)
+    assert np.max(np.abs(got[1].cpu().numpy() - ref[1])) < 1e-5 * np.max(np.abs(ref[1]))
+    assert 0.0 < ref[3]["clip_frac"] < 0.5
+    # micro-batching only changes the rounding order
+    _, _, g2, _ = B.grpo_actor_fwd_bwd(model, pk, mb_chunks=7)
+    for k, v in grads_to_numpy(g2).items():
+        assert rel_fro(v, ref[2][k]) < F32_TOL, k
+    # forward-only gives the same log-probs and touches no gradient
+    before = {k: v.clone() for k, v in model.grads.items()}
+    _, logp_f, none_g, _ = B.grpo_actor_fwd_bwd(model, pk, flags=B.GRPO_FWD_ONLY)
+    assert none_g is None and torch.equal(logp_f, got[1])
+    assert all(torch.equal(before[k], model.grads[k]) for k in before)
+    # accumulate doubles the gradient
+    B.grpo_actor_fwd_bwd(model, pk, mb_chunks=7, flags=B.GRPO_ACCUMULATE)
+    for k, v in grads_to_numpy(model.grads).items():
+        assert rel_fro(v, 2 * ref[2][k]) < F32_TOL, k
+
+
+def test_c0_fp32_paper_clip_and_heavy_clipping():
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"].with_(gamma_std=0.1)
+    hp = host_problem(w, seed=4, sigma=0.3, lpo_mode="uniform")
+    _, _, got, ref, _ = _compare(B, PL, hp, F32_TOL, tol_loss_rel=F32_TOL, eps=(0.2, 0.4), loss_scale=1.0 / w.n_traj)
+    assert ref[3]["clip_frac"] > 0.1
+
+
+def test_c0_full_pipeline_through_the_c_abi():
+    """score -> update -> sample -> pack -> actor, every step on the device, against the oracle chain."""
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"].with_(gamma_std=0.1)
+    hp = host_problem(w)
+    model = PL.upload_model(w, hp["weights"])
+    total = int(hp["rb"]["traj_off"][-1])
+    obs = synth.obs_all(w, w.seed, total)
+    lpo_all = np.zeros((total, 56), dtype=np.float32)
+    lpo_all[hp["kept"]] = hp["lpo"]
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=7 + w.seed, max_traj=w.n_traj)
+    batch = PL.upload_rollouts(w, hp["rb"], obs=PL.dev(obs), logp_old=PL.dev(lpo_all))
+    adv, Cc, valid, p, q, kept_idx, kept_off, _ = PL.select(ctx, batch, 0)
+    n_kept = PL.n_kept_of(w.budget, hp["rb"]["traj_off"])
+    assert np.array_equal(kept_idx.cpu().numpy()[:n_kept], hp["kept"])
+    pk = B.grpo_pack_chunks(ctx, batch, model, kept_idx, kept_off, adv, B.Packed(model, n_kept))
+    assert B.pcm_poll_status(ctx) == 0
+    assert np.array_equal(pk.X.cpu().numpy(), hp["X"].astype(np.float32))
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, pk)
+    loss_o, _, grads_o, _ = oracle_update(hp)
+    assert abs(float(loss.item()) - loss_o) <= F32_TOL * abs(loss_o)
+    for k, v in grads_to_numpy(grads).items():
+        assert rel_fro(v, grads_o[k]) < F32_TOL, k
+    ctx.close()
+
+
+BF16_CASES = {
+    # several 128-row tiles with a ragged tail (5 * 96 = 480 tokens), two layers
+    "small": dict(n_tasks=1, G=4, T=8, n_phases=4, budget=2, P=40, d=256, L=2, H=4, max_kept=5),
+    # one layer of the medium model at its real width and sequence length (3 * 312 = 936 tokens)
+    "c1_layer": dict(n_tasks=1, G=4, T=8, n_phases=4, budget=1, P=256, d=1024, L=1, H=16, max_kept=3),
+    # head dim 128 as in the large model
+    "dh128": dict(n_tasks=1, G=4, T=8, n_phases=4, budget=1, P=72, d=256, L=2, H=2, max_kept=4),
+}
+
+
+@pytest.mark.parametrize("case", list(BF16_CASES))
+@pytest.mark.parametrize("backend", ["simt", "auto"])
+def test_bf16_end_to_end(case, backend, monkeypatch):
+    B, PL = _mods()
+    kw = dict(BF16_CASES[case])
+    max_kept = kw.pop("max_kept")
+    w = synth.WORKLOADS["C1"].with_(gamma_std=0.1, force_mixed=True, p_succ=0.5, **kw)
+    hp = host_problem(w, seed=2, max_kept=max_kept)
+    if backend == "simt":
+        monkeypatch.setenv("PCM_GEMM_BACKEND", "simt")
+    else:
+        monkeypatch.delenv("PCM_GEMM_BACKEND", raising=False)
+    _, _, got, ref, errs = _compare(B, PL, hp, BF16_GRAD_TOL, tol_loss_abs=BF16_LOSS_TOL, mb=2)
+    assert np.max(np.abs(got[1].cpu().numpy() - ref[1])) < 0.05
+
+
+def test_argument_errors():
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"]
+    hp = host_problem(w)
+    model = PL.upload_model(w, hp["weights"])
+    pk = device_packed(B, PL, model, hp)
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.PcmError) as e:
+        B.grpo_actor_fwd_bwd(model, pk, workspace=small)
+    assert e.value.code == -3
+    bad = B.Model(w.d, w.L, 3, w.P, B.GRPO_F32, model.weights)          # d not divisible by heads
+    with pytest.raises(B.PcmError):
+        B.grpo_actor_fwd_bwd(bad, pk)
