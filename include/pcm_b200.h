@@ -243,6 +243,22 @@ int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32
 int grpo_attention(int32_t dtype, const void* qkv, void* out, float* lse, const void* dout, void* dqkv,
                    float* scratch, int32_t n_seq, int32_t S, int32_t n_heads, int32_t head_dim, pcm_stream stream);
 
+/* Per-kernel-class timing.  While enabled, every launch of the classes below is bracketed by a
+ * pair of CUDA events on its stream; pcm_profile_read() synchronises the device, adds up elapsed
+ * milliseconds, the algorithmic flops / bytes of the launches and their count since the last read,
+ * and clears the records.  Classes: 0 GEMM (all linear layers, head), 1 attention, 2 RMSNorm,
+ * 3 element-wise (rotary, SwiGLU, residual cast), 4 loss rows, 5 embedding gradient, 6 pack,
+ * 7 PCM control plane (score, update, sample). */
+#define PCM_PROFILE_CLASSES 8
+typedef struct {
+  double ms[PCM_PROFILE_CLASSES];
+  double flops[PCM_PROFILE_CLASSES];
+  double bytes[PCM_PROFILE_CLASSES];
+  int64_t launches[PCM_PROFILE_CLASSES];
+} pcm_profile;
+int pcm_profile_enable(int32_t on);
+int pcm_profile_read(pcm_profile* out);
+
 /* Number of kernels this library has launched in the calling process (for accounting). */
 int64_t pcm_launch_count(void);
 

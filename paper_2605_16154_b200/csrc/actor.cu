@@ -445,9 +445,13 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
   auto G = [&](int M_, int N_, int K_, const void* A, long long lda, bool ak, const void* B, long long ldb, bool bk,
                int abdt, void* C, long long ldc, int cdt, const float* R, long long ldr) -> int {
     GemmArgs g{M_, N_, K_, A, lda, ak, B, ldb, bk, abdt, C, ldc, cdt, R, ldr};
-    return gemm(g, s);
+    prof_begin(PC_GEMM, s);
+    const int rc = gemm(g, s);
+    prof_end(s, 2.0 * M_ * (double)N_ * K_, 0.0);
+    return rc;
   };
 #define TRY(expr) do { int rc__ = (expr); if (rc__ != PCM_OK) return rc__; } while (0)
+  const double es = (double)sizeof(T);
 
   for (int c0 = 0; c0 < n; c0 += mb_max) {
     const int mb = (n - c0) < mb_max ? (n - c0) : mb_max;
@@ -459,35 +463,51 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     const float* advc = pk->adv_c + c0;
 
     // ---------------- forward ----------------
+    prof_begin(PC_ELEM, s);
     to_residual_kernel<T><<<ceil_div(M * d, 1024), 256, 0, s>>>(Xmb, w.x[0], M * d);
     PCM_LAUNCH_CHECK();
+    prof_end(s, 0.0, (double)M * d * (es + 4.0));
     for (int l = 0; l < L; ++l) {
       LayerActs& la = w.la[l];
       const float* x_in = w.x[l];
       float* x_out = w.x[l + 1];
+      prof_begin(PC_NORM, s);
       rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(x_in, g1 + (size_t)l * d, (T*)la.h1, la.rstd1, M, d, 0, 0);
       PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)M * d * (es + 4.0));
       TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0));
+      prof_begin(PC_ELEM, s);
       rope_kernel<T><<<ceil_div(M * H * dh, 256), 256, 0, s>>>((T*)la.qkv, w.rope_tab, M, S, H, dh, 1.f);
       PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
+      prof_begin(PC_ATTN, s);
       TRY(attention_fwd(dt, la.qkv, la.attn, la.lse, mb, S, H, dh, s));
+      prof_end(s, 2.0 * S * (double)S * d * mb, (double)M * 4 * d * es);
       TRY(G(Mi, d, d, la.attn, d, true, w_o + (size_t)l * d * d, d, true, dt, la.x_mid, d, DT_F32, x_in, d));
+      prof_begin(PC_NORM, s);
       rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(la.x_mid, g2 + (size_t)l * d, (T*)la.h2, la.rstd2, M, d, 0, 0);
       PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)M * d * (es + 4.0));
       TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0));
+      prof_begin(PC_ELEM, s);
       swiglu_fwd_kernel<T><<<ceil_div(M * 4 * d, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, M, 4 * d);
       PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)M * 4 * d * es * 3.0);
       TRY(G(Mi, d, 4 * d, la.act, 4 * d, true, w_d + (size_t)l * 4 * d * d, 4 * d, true, dt, x_out, d, DT_F32, la.x_mid, d));
     }
     // head on the scored rows only
+    prof_begin(PC_NORM, s);
     rmsnorm_fwd_kernel<T><<<ceil_div(R, 8), 256, 0, s>>>(w.x[L], gf, (T*)w.hs, w.rstdf, R, d, S, P);
     PCM_LAUNCH_CHECK();
+    prof_end(s, 0.0, (double)R * d * (es + 4.0));
     TRY(G(Ri, NB, d, w.hs, d, true, w_h, d, true, dt, w.z, NB, DT_F32, nullptr, 0));
     const int loss_blocks = ceil_div(R, 8);
+    prof_begin(PC_LOSS, s);
     loss_rows_kernel<T><<<loss_blocks, 256, 0, s>>>(w.z, tgt, lpo, advc, lc->eps_low, lc->eps_high, loss_scale,
                                                   (T*)w.dz, logp ? logp + (long long)c0 * ACT : nullptr, w.loss_part,
                                                   R, fwd_only ? 1 : 0);
     PCM_LAUNCH_CHECK();
+    prof_end(s, 0.0, (double)R * NB * (4.0 + (fwd_only ? 0.0 : es)));
     loss_reduce_kernel<<<1, 256, 0, s>>>(w.loss_part, loss_blocks, loss_scale, w.loss_acc, loss);
     PCM_LAUNCH_CHECK();
     if (fwd_only) continue;
@@ -504,9 +524,11 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     auto norm_bwd = [&](const float* dy, const float* x, const float* rstd, const T* gamma, const float* dx_in,
                         long long rows, int mS, int mP, float* dgamma) -> int {
       const int blocks = (int)(rows / 8 + 1 < NORM_BWD_BLOCKS ? rows / 8 + 1 : NORM_BWD_BLOCKS);
+      prof_begin(PC_NORM, s);
       rmsnorm_bwd_kernel<T><<<blocks, 256, nb_smem, s>>>(dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t, w.norm_part, rows,
                                                        d, mS, mP);
       PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)rows * d * ((dx_in ? 16.0 : 12.0) + es));
       colsum_accumulate_kernel<<<ceil_div(d, 256), 256, 0, s>>>(w.norm_part, blocks, d, dgamma);
       PCM_LAUNCH_CHECK();
       return PCM_OK;
@@ -520,8 +542,10 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       TRY(G(d, 4 * d, Mi, w.dx_t, d, false, la.act, 4 * d, false, dt, gr->w_d + l * 4 * dd, 4 * d, DT_F32,
             gr->w_d + l * 4 * dd, 4 * d));
       TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dact, 4 * d, dt, nullptr, 0));
+      prof_begin(PC_ELEM, s);
       swiglu_bwd_kernel<T><<<ceil_div(M * 4 * d, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, M, 4 * d);
       PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)M * 4 * d * es * 5.0);
       TRY(G(8 * d, d, Mi, w.dgu, 8 * d, false, la.h2, d, false, dt, gr->w_gu + l * 8 * dd, d, DT_F32,
             gr->w_gu + l * 8 * dd, d));
       TRY(G(Mi, d, 8 * d, w.dgu, 8 * d, true, w_gu + l * 8 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
@@ -529,16 +553,22 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       // attention block: x_mid = x_in + attn W_o^T
       TRY(G(d, d, Mi, w.dx_t, d, false, la.attn, d, false, dt, gr->w_o + l * dd, d, DT_F32, gr->w_o + l * dd, d));
       TRY(G(Mi, d, d, w.dx_t, d, true, w_o + l * dd, d, false, dt, w.dattn, d, dt, nullptr, 0));
+      prof_begin(PC_ATTN, s);
       TRY(attention_bwd(dt, la.qkv, la.attn, w.dattn, la.lse, w.dsum, w.dqkv, mb, S, H, dh, s));
+      prof_end(s, 5.0 * S * (double)S * d * mb, (double)M * 8 * d * es);
+      prof_begin(PC_ELEM, s);
       rope_kernel<T><<<ceil_div(M * H * dh, 256), 256, 0, s>>>((T*)w.dqkv, w.rope_tab, M, S, H, dh, -1.f);
       PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
       TRY(G(3 * d, d, Mi, w.dqkv, 3 * d, false, la.h1, d, false, dt, gr->w_qkv + l * 3 * dd, d, DT_F32,
             gr->w_qkv + l * 3 * dd, d));
       TRY(G(Mi, d, 3 * d, w.dqkv, 3 * d, true, w_qkv + l * 3 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
       TRY(norm_bwd(w.dh, w.x[l], la.rstd1, g1 + (size_t)l * d, w.dx, M, 0, 0, gr->g1 + (size_t)l * d));
     }
+    prof_begin(PC_EMBED, s);
     embed_grad_kernel<<<dim3(NB, ceil_div(d, 256)), 256, 0, s>>>(w.dx, tgt, mb, S, P, d, gr->e_act);
     PCM_LAUNCH_CHECK();
+    prof_end(s, 0.0, (double)mb * ACT * d * 4.0);
   }
 #undef TRY
 

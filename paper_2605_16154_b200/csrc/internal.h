@@ -36,4 +36,10 @@ int attention_fwd(int dtype, const void* qkv, void* out, float* lse, int n_seq, 
 int attention_bwd(int dtype, const void* qkv, const void* out, const void* dout, const float* lse, float* dsum,
                   void* dqkv, int n_seq, int S, int H, int dh, cudaStream_t s);
 
+// Event-pair profiling (profile.cu).  prof_begin/prof_end nest like a stack and cost nothing when off.
+enum { PC_GEMM = 0, PC_ATTN = 1, PC_NORM = 2, PC_ELEM = 3, PC_LOSS = 4, PC_EMBED = 5, PC_PACK = 6, PC_PCM = 7 };
+bool prof_enabled();
+void prof_begin(int cls, cudaStream_t s);
+void prof_end(cudaStream_t s, double flops, double bytes);
+
 }  // namespace pcm

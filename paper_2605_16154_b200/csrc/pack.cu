@@ -1,7 +1,7 @@
 // Physical shrinking (Sec. 4.5): gather the kept chunks into a dense batch with bulk asynchronous
 // copies (global -> shared -> global through the TMA engine); no thread touches the payload.
 #include "async_ptx.cuh"
-#include "common.cuh"
+#include "internal.h"
 
 struct pcm_ctx;   // opaque here; only the status word is needed
 namespace pcm { unsigned* ctx_status(pcm_ctx*); }
@@ -145,10 +145,12 @@ extern "C" int grpo_pack_chunks(pcm_ctx* ctx, const pcm_batch* b, const grpo_mod
     attr_set = true;
   }
   dim3 grid(pieces + 1, out->n_kept);
+  prof_begin(PC_PACK, (cudaStream_t)stream);
   pack_chunks_kernel<<<grid, 64, smem, (cudaStream_t)stream>>>(
       (const uint8_t*)b->obs, (const uint8_t*)e_act, b->tok, b->logp_old, adv, kept_idx, kept_off, b->n_traj,
       b->n_chunks, out->n_kept, prefix_bytes, (int)row_bytes, pieces, (uint8_t*)out->X, out->tgt, out->lpo,
       out->adv_c, out->src, ctx_status(ctx));
   PCM_LAUNCH_CHECK();
+  prof_end((cudaStream_t)stream, 0.0, (double)out->n_kept * (2.0 * prefix_bytes + 2.0 * PCM_ACT_DIM * row_bytes));
   return PCM_OK;
 }

@@ -4,7 +4,7 @@
 #include <cstring>
 #include <new>
 
-#include "common.cuh"
+#include "internal.h"
 
 namespace pcm {
 std::atomic<long long> g_launches{0};
@@ -448,9 +448,11 @@ int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* b, double* C, uint8_t* valid
   cudaStream_t s = (cudaStream_t)stream;
   const int G = ctx->cfg.group_size, Kc = ctx->cfg.n_phases, ng = b->n_traj / G;
   const size_t smem = (size_t)Kc * 2 * (ACT + 1) * sizeof(unsigned);
+  prof_begin(PC_PCM, s);
   score_groups_kernel<<<ng, 256, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, G, Kc, ctx->c_group,
                                              ctx->valid_group, ctx->status);
   PCM_LAUNCH_CHECK();
+  prof_end(s, 0.0, (double)b->n_chunks * (ACT + 1));
   const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
   score_finalize_kernel<<<1 + adv_blocks, 128, 0, s>>>(ctx->c_group, ctx->valid_group, ng, Kc, C, valid,
                                                        n_valid_groups, b->reward, G, ctx->cfg.adv_eps, adv);
@@ -481,11 +483,13 @@ int pcm_sample_chunks(pcm_ctx* ctx, const pcm_batch* b, const uint32_t* q, uint6
   const size_t smem = (size_t)warps * b->max_len * sizeof(unsigned);
   if (smem > 48 * 1024)
     PCM_CUDA_TRY(cudaFuncSetAttribute(sample_chunks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  prof_begin(PC_PCM, s);
   sample_chunks_kernel<<<ceil_div(b->n_traj, warps), warps * 32, smem, s>>>(
       b->traj_off, b->phase, q, b->n_traj, ctx->cfg.n_phases, ctx->cfg.budget, b->max_len,
       (uint32_t)(ctx->cfg.seed & 0xFFFFFFFFu), (uint32_t)(ctx->cfg.seed >> 32), (uint32_t)(iter & 0xFFFFFFFFu),
       (uint32_t)(iter >> 32), kept_off, kept_idx, kept_per_phase, ctx->status);
   PCM_LAUNCH_CHECK();
+  prof_end(s, 0.0, (double)b->n_chunks + 4.0 * b->n_traj * ctx->cfg.budget);
   return PCM_OK;
 }
 

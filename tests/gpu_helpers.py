@@ -15,8 +15,14 @@ def rel_fro(a, b):
     return float(np.linalg.norm(a - b) / den) if den > 0 else float(np.linalg.norm(a - b))
 
 
-def host_problem(w, seed=None, budget=None, sigma=0.1, lpo_mode="oracle", max_kept=None):
-    """Rollouts -> oracle selection -> oracle pack; logp_old = oracle log-probs + seeded noise."""
+def host_problem(w, seed=None, budget=None, sigma=0.1, lpo_mode="oracle", max_kept=None, clip_margin=0.0,
+                 eps=(0.2, 0.2)):
+    """Rollouts -> oracle selection -> oracle pack; logp_old = oracle log-probs + seeded noise.
+
+    The clipped surrogate's gradient switches off discontinuously at ratio = 1 +- eps, so a token whose
+    ratio sits on a boundary is decided by rounding.  With clip_margin > 0 the noise is moved so that
+    no oracle ratio lies within that margin (in log space) of either boundary: the comparison then
+    covers what is uniquely defined."""
     seed = w.seed if seed is None else seed
     budget = w.budget if budget is None else budget
     rb = synth.make_rollouts(w, seed)
@@ -33,7 +39,14 @@ def host_problem(w, seed=None, budget=None, sigma=0.1, lpo_mode="oracle", max_ke
     X, tgt, _, adv_c, src = po.pack_chunks(lambda c: obs[c], rb["tok"], lpo_all, adv, rb["traj_off"], kept, weights["e_act"])
     if lpo_mode == "oracle":
         lp = ao.logp_only(weights, X, tgt, w.H, w.P)
-        lpo = (lp + synth.logp_noise(seed, len(kept), sigma)).astype(np.float32)
+        noise = synth.logp_noise(seed, len(kept), sigma).astype(np.float64)
+        if clip_margin > 0.0:
+            log_r = -noise                                   # log ratio seen by the oracle
+            hi, lo = np.log(1.0 + eps[1]), np.log(1.0 - eps[0])
+            log_r = np.where(np.abs(log_r - hi) < clip_margin, hi + 2 * clip_margin * np.sign(log_r - hi + 1e-30), log_r)
+            log_r = np.where(np.abs(log_r - lo) < clip_margin, lo + 2 * clip_margin * np.sign(log_r - lo + 1e-30), log_r)
+            noise = -log_r
+        lpo = (lp + noise).astype(np.float32)
     else:   # constant near-uniform behaviour policy: heavy clipping
         lpo = (-np.log(256.0) + synth.logp_noise(seed, len(kept), sigma)).astype(np.float32)
     return dict(w=w, rb=rb, weights=weights, adv=adv, kept=kept, off=off, X=X, tgt=tgt, lpo=lpo, adv_c=adv_c, src=src,

@@ -165,13 +165,14 @@ def test_bf16_end_to_end(case, backend, monkeypatch):
     kw = dict(BF16_CASES[case])
     max_kept = kw.pop("max_kept")
     w = synth.WORKLOADS["C1"].with_(gamma_std=0.1, force_mixed=True, p_succ=0.5, **kw)
-    hp = host_problem(w, seed=2, max_kept=max_kept)
+    hp = host_problem(w, seed=2, max_kept=max_kept, clip_margin=0.05)
     if backend == "simt":
         monkeypatch.setenv("PCM_GEMM_BACKEND", "simt")
     else:
         monkeypatch.delenv("PCM_GEMM_BACKEND", raising=False)
     _, _, got, ref, errs = _compare(B, PL, hp, BF16_GRAD_TOL, tol_loss_abs=BF16_LOSS_TOL, mb=2)
-    assert np.max(np.abs(got[1].cpu().numpy() - ref[1])) < 0.05
+    assert np.max(np.abs(got[1].cpu().numpy() - ref[1])) < 0.04          # well inside the clip margin
+    assert got[3].clip_frac == pytest.approx(ref[3]["clip_frac"], abs=1e-6)   # same clip decisions
 
 
 def test_argument_errors():

@@ -24,7 +24,7 @@ def _operands(rng, M, N, K, a_k, b_k, PL):
 
 
 @pytest.mark.parametrize("a_k,b_k", [(True, True), (True, False), (False, True), (False, False)])
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 768, 200), (936, 1024, 1024), (200, 96, 72)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (304, 768, 200), (936, 1024, 1024), (200, 96, 72)])
 def test_tcgen05_gemm_layouts_and_tails(a_k, b_k, M, N, K):
     B, PL = _mods()
     rng = np.random.default_rng(11)
