@@ -76,6 +76,14 @@ class grpo_stats(C.Structure):
                 ("workspace_high_water", C.c_uint64)]
 
 
+PROFILE_CLASSES = ("gemm", "attention", "rmsnorm", "elementwise", "loss", "embed_grad", "pack", "pcm")
+
+
+class pcm_profile(C.Structure):
+    _fields_ = [("ms", C.c_double * 8), ("flops", C.c_double * 8), ("bytes", C.c_double * 8),
+                ("launches", C.c_int64 * 8)]
+
+
 _P = C.c_void_p
 _lib.pcm_create.argtypes = [C.POINTER(_P), C.POINTER(pcm_config), C.c_int32]
 _lib.pcm_destroy.argtypes = [_P]
@@ -95,14 +103,17 @@ _lib.grpo_gemm.argtypes = [C.c_int32, C.c_int32, C.c_int32, _P, C.c_int64, C.c_i
                            C.c_int32, _P, C.c_int64, C.c_int32, _P, C.c_int64, C.c_int32, _P]
 _lib.grpo_attention.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P]
 _lib.pcm_launch_count.restype = C.c_int64
+_lib.pcm_profile_enable.argtypes = [C.c_int32]
+_lib.pcm_profile_read.argtypes = [C.POINTER(pcm_profile)]
 for _name in ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", "pcm_state_import",
               "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
-              "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention"):
+              "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_profile_enable", "pcm_profile_read"):
     getattr(_lib, _name).restype = C.c_int
 
 EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", "pcm_state_import",
             "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
-            "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count")
+            "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
+            "pcm_profile_enable", "pcm_profile_read")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -321,3 +332,15 @@ def grpo_attention(qkv: torch.Tensor, n_seq: int, S: int, H: int, dh: int, dout:
 
 def pcm_launch_count() -> int:
     return int(_lib.pcm_launch_count())
+
+
+def pcm_profile_enable(on: bool) -> None:
+    _check("pcm_profile_enable", _lib.pcm_profile_enable(int(on)))
+
+
+def pcm_profile_read() -> Dict[str, Dict[str, float]]:
+    """Per kernel class since the last read: elapsed ms, algorithmic flops and bytes, launches."""
+    prof = pcm_profile()
+    _check("pcm_profile_read", _lib.pcm_profile_read(C.byref(prof)))
+    return {name: {"ms": prof.ms[i], "flops": prof.flops[i], "bytes": prof.bytes[i], "launches": int(prof.launches[i])}
+            for i, name in enumerate(PROFILE_CLASSES)}
