@@ -109,6 +109,31 @@ int pcm_state_import(pcm_ctx* ctx, const void* host_buf, size_t bytes);
 int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* batch, double* C, uint8_t* valid,
                      int32_t* n_valid_groups, float* adv, pcm_stream stream);
 
+/* ---- allocation-free variant of pcm_score_phases (the paper has no counterpart) -----------------
+ * Same computation and outputs as pcm_score_phases, for callers that are not allowed to allocate
+ * device memory: code that runs inside a region where the allocator is off limits (a serving or
+ * training loop with a frozen memory plan, a real-time control thread next to the robot, a plugin
+ * that only gets pointers from its host program), where a cudaMalloc would synchronise the device,
+ * fragment the plan or simply be forbidden.  It needs no pcm_ctx (pcm_create allocates): the
+ * per-group scratch (C_{c,g} and its validity flag) lives in a fixed array inside the library,
+ * PCM_STATIC_SCRATCH_BYTES of device memory that every GPU which loads the library holds until the
+ * process exits.  Limits: n_traj / group_size <= PCM_STATIC_MAX_GROUPS; larger batches are rejected
+ * with PCM_ERR_SHAPE before anything is launched.
+ * The first call on each device looks up the array's device address (no allocation, but a
+ * synchronous runtime query): make that first call before any stream capture.
+ * All calls share the one array, which keeps whatever the previous call left in it; every entry a
+ * call reads is rewritten by that call first, and the status word is cleared at the start of each
+ * call.  Two calls whose kernels overlap on the GPU (different streams, no dependency) race on the
+ * array: order them.
+ * device_status (device [1], may be NULL) receives 0, or a non-zero bit mask when a phase label
+ * >= n_phases was met (that chunk is ignored), once the stream reaches that point.
+ * Calls no cudaMalloc / cudaFree and no allocating library routine. */
+#define PCM_STATIC_MAX_GROUPS 4096
+#define PCM_STATIC_SCRATCH_BYTES (PCM_STATIC_MAX_GROUPS * PCM_MAX_PHASES * 9 + 256)
+int pcm_score_phases_static(int32_t n_phases, int32_t group_size, double adv_eps, const pcm_batch* batch,
+                            double* C, uint8_t* valid, int32_t* n_valid_groups, float* adv,
+                            uint32_t* device_status, pcm_stream stream);
+
 /* ---- Eq. 7-9, Algorithm 1 ---------------------------------------------------------------------
  * Appends C (0 where valid[c] == 0) to the phase buffers.  On the first call, or when the buffers
  * hold t_rc entries: S_c = sum of buffer, rho_c = S_c / sum S, rho~_c = rho_c / max rho,

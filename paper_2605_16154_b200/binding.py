@@ -102,6 +102,8 @@ _lib.grpo_actor_fwd_bwd.argtypes = [C.POINTER(grpo_model), C.POINTER(grpo_packed
 _lib.grpo_gemm.argtypes = [C.c_int32, C.c_int32, C.c_int32, _P, C.c_int64, C.c_int32, _P, C.c_int64, C.c_int32,
                            C.c_int32, _P, C.c_int64, C.c_int32, _P, C.c_int64, C.c_int32, _P]
 _lib.grpo_attention.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P]
+_lib.pcm_score_phases_static.argtypes = [C.c_int32, C.c_int32, C.c_double, C.POINTER(pcm_batch), _P, _P, _P, _P, _P, _P]
+_lib.pcm_score_phases_static.restype = C.c_int
 _lib.pcm_launch_count.restype = C.c_int64
 _lib.pcm_profile_enable.argtypes = [C.c_int32]
 _lib.pcm_profile_read.argtypes = [C.POINTER(pcm_profile)]
@@ -113,7 +115,7 @@ for _name in ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export"
 EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", "pcm_state_import",
             "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
-            "pcm_profile_enable", "pcm_profile_read")
+            "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -194,6 +196,20 @@ def pcm_score_phases(ctx: Context, batch: pcm_batch, want_adv: bool = True):
     _check("pcm_score_phases", _lib.pcm_score_phases(ctx.handle, C.byref(batch), _ptr(Cc), _ptr(valid), _ptr(n_valid),
                                                      _ptr(adv), _stream()))
     return Cc, valid, n_valid, adv
+
+
+STATIC_MAX_GROUPS = 4096
+
+
+def pcm_score_phases_static(n_phases: int, group_size: int, adv_eps: float, batch: pcm_batch, out: Dict[str, torch.Tensor]):
+    """Allocation-free variant of pcm_score_phases: every output tensor, including the one-word
+    `status`, is passed in by the caller (keys C, valid, n_valid, adv, status); this wrapper creates
+    no tensor, so that the call stays free of device allocations end to end."""
+    _check("pcm_score_phases_static",
+           _lib.pcm_score_phases_static(n_phases, group_size, adv_eps, C.byref(batch), _ptr(out["C"]), _ptr(out["valid"]),
+                                        _ptr(out.get("n_valid")), _ptr(out.get("adv")), _ptr(out.get("status")),
+                                        _stream()))
+    return out
 
 
 def pcm_update_keep_probs(ctx: Context, Cc: torch.Tensor, valid: torch.Tensor):

@@ -2,6 +2,7 @@
 // update (Eq. 7-9), fixed-budget weighted sampling on a Philox stream (Eq. 10), and the context that
 // holds the persistent state.
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "internal.h"
@@ -496,3 +497,70 @@ int pcm_sample_chunks(pcm_ctx* ctx, const pcm_batch* b, const uint32_t* q, uint6
 int64_t pcm_launch_count(void) { return (int64_t)g_launches.load(); }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free scoring: the per-group scratch is a fixed device array owned by the library.
+// ------------------------------------------------------------------------------------------------
+namespace pcm {
+
+constexpr size_t NA_CGROUP_BYTES = (size_t)PCM_STATIC_MAX_GROUPS * PCM_MAX_PHASES * sizeof(double);
+constexpr size_t NA_VALID_BYTES = (size_t)PCM_STATIC_MAX_GROUPS * PCM_MAX_PHASES;
+static_assert(NA_CGROUP_BYTES + NA_VALID_BYTES + 256 == PCM_STATIC_SCRATCH_BYTES, "scratch layout and header disagree");
+
+// [C_{c,g} as fp64][validity bytes][status word]; held by every device that loads the library.
+static __device__ __align__(256) unsigned char g_static_scratch[PCM_STATIC_SCRATCH_BYTES];
+
+// In host code the symbol above is only a handle, not a device address: the address a kernel can use
+// is looked up once per device (with that device current) and cached here.
+constexpr int NA_MAX_DEVICES = 64;
+static std::mutex g_na_mu;
+static unsigned char* g_na_addr[NA_MAX_DEVICES] = {};
+
+static int static_scratch_address(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return PCM_ERR_CUDA;
+  if (dev < 0 || dev >= NA_MAX_DEVICES) return PCM_ERR_ARG;
+  std::lock_guard<std::mutex> lk(g_na_mu);
+  if (!g_na_addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return PCM_ERR_CUDA;
+    }
+    g_na_addr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_na_addr[dev];
+  return PCM_OK;
+}
+
+}  // namespace pcm
+
+extern "C" int pcm_score_phases_static(int32_t n_phases, int32_t group_size, double adv_eps, const pcm_batch* b,
+                                       double* C, uint8_t* valid, int32_t* n_valid_groups, float* adv,
+                                       uint32_t* device_status, pcm_stream stream) {
+  if (!b || !b->traj_off || !b->phase || !b->tok || !b->reward || !C || !valid) return PCM_ERR_ARG;
+  if (n_phases < 1 || n_phases > PCM_MAX_PHASES || group_size < 1 || !(adv_eps >= 0.0)) return PCM_ERR_ARG;
+  if (b->n_traj <= 0 || b->n_traj % group_size || b->n_chunks < 0) return PCM_ERR_ARG;
+  if (((uintptr_t)b->tok) & 3) return PCM_ERR_ARG;
+  const int ng = b->n_traj / group_size;
+  if (ng > PCM_STATIC_MAX_GROUPS) return PCM_ERR_SHAPE;          // beyond the fixed scratch: refuse, do not truncate
+  unsigned char* base = nullptr;
+  const int rc = static_scratch_address(&base);
+  if (rc != PCM_OK) return rc;
+  double* c_group = reinterpret_cast<double*>(base);
+  uint8_t* valid_group = base + NA_CGROUP_BYTES;
+  unsigned* status = reinterpret_cast<unsigned*>(base + NA_CGROUP_BYTES + NA_VALID_BYTES);
+  cudaStream_t s = (cudaStream_t)stream;
+  PCM_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(unsigned), s));   // the only part that must start at zero
+  const size_t smem = (size_t)n_phases * 2 * (ACT + 1) * sizeof(unsigned);
+  score_groups_kernel<<<ng, 256, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, group_size, n_phases, c_group,
+                                             valid_group, status);
+  PCM_LAUNCH_CHECK();
+  const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
+  score_finalize_kernel<<<1 + adv_blocks, 128, 0, s>>>(c_group, valid_group, ng, n_phases, C, valid, n_valid_groups,
+                                                       b->reward, group_size, adv_eps, adv);
+  PCM_LAUNCH_CHECK();
+  if (device_status)
+    PCM_CUDA_TRY(cudaMemcpyAsync(device_status, status, sizeof(unsigned), cudaMemcpyDeviceToDevice, s));
+  return PCM_OK;
+}
