@@ -27,6 +27,32 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// four consecutive elements of T <-> floats (8- or 16-byte accesses)
+template <typename T>
+__device__ __forceinline__ void load4(const T* p, float (&v)[4]) {
+  if constexpr (sizeof(T) == 2) {
+    const uint2 raw = *reinterpret_cast<const uint2*>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+  } else {
+    const float4 f = *reinterpret_cast<const float4*>(p);
+    v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+  }
+}
+template <typename T>
+__device__ __forceinline__ void store4(T* p, float a, float b, float c, float d) {
+  if constexpr (sizeof(T) == 2) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 raw;
+    raw.x = *reinterpret_cast<uint32_t*>(&lo);
+    raw.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = raw;
+  } else {
+    *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+  }
+}
+
 // Row r of a [rows][d] tensor that holds only the scored positions maps to token row
 // (r / 56) * S + P - 1 + r % 56 of the full activation; map_S == 0 means identity.
 __device__ __forceinline__ long long map_row(long long r, int map_S, int map_P) {
@@ -42,9 +68,9 @@ template <typename T>
 __global__ void to_residual_kernel(const T* __restrict__ x, float* __restrict__ y, long long n) {
   const long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i + 3 < n) {
-    float4 o;
-    o.x = ldf(x + i); o.y = ldf(x + i + 1); o.z = ldf(x + i + 2); o.w = ldf(x + i + 3);
-    *reinterpret_cast<float4*>(y + i) = o;
+    float v[4];
+    load4<T>(x + i, v);
+    *reinterpret_cast<float4*>(y + i) = make_float4(v[0], v[1], v[2], v[3]);
   } else {
     for (long long k = i; k < n; ++k) y[k] = ldf(x + k);
   }
@@ -72,10 +98,9 @@ rmsnorm_fwd_kernel(const float* __restrict__ x, const T* __restrict__ gamma, T* 
   T* hr = h + r * d;
   for (int c = lane * 4; c < d; c += 128) {
     const float4 v = *reinterpret_cast<const float4*>(xr + c);
-    stf(hr + c, v.x * rs * ldf(gamma + c));
-    stf(hr + c + 1, v.y * rs * ldf(gamma + c + 1));
-    stf(hr + c + 2, v.z * rs * ldf(gamma + c + 2));
-    stf(hr + c + 3, v.w * rs * ldf(gamma + c + 3));
+    float gm[4];
+    load4<T>(gamma + c, gm);
+    store4<T>(hr + c, v.x * rs * gm[0], v.y * rs * gm[1], v.z * rs * gm[2], v.w * rs * gm[3]);
   }
 }
 
@@ -103,8 +128,9 @@ rmsnorm_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ x, co
     for (int c = lane * 4; c < d; c += 128) {
       const float4 xv = *reinterpret_cast<const float4*>(xr + c);
       const float4 gv = *reinterpret_cast<const float4*>(dyr + c);
-      dot += gv.x * ldf(gamma + c) * xv.x + gv.y * ldf(gamma + c + 1) * xv.y + gv.z * ldf(gamma + c + 2) * xv.z +
-             gv.w * ldf(gamma + c + 3) * xv.w;
+      float gm[4];
+      load4<T>(gamma + c, gm);
+      dot += gv.x * gm[0] * xv.x + gv.y * gm[1] * xv.y + gv.z * gm[2] * xv.z + gv.w * gm[3] * xv.w;
     }
     dot = warp_sum(dot);
     const float coef = dot * rs * rs * rs / (float)d;    // mean(dn * n) * rstd, with n = x * rstd
@@ -113,10 +139,11 @@ rmsnorm_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ x, co
       const float4 gv = *reinterpret_cast<const float4*>(dyr + c);
       const float xa[4] = {xv.x, xv.y, xv.z, xv.w};
       const float ga[4] = {gv.x, gv.y, gv.z, gv.w};
-      float o[4];
+      float o[4], gm[4];
+      load4<T>(gamma + c, gm);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        o[e] = rs * ga[e] * ldf(gamma + c + e) - coef * xa[e];
+        o[e] = rs * ga[e] * gm[e] - coef * xa[e];
         mine[c + e] += ga[e] * xa[e] * rs;
       }
       if (dx_in) {
@@ -124,8 +151,7 @@ rmsnorm_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ x, co
         o[0] += pv.x; o[1] += pv.y; o[2] += pv.z; o[3] += pv.w;
       }
       *reinterpret_cast<float4*>(dx_out + xr_i * d + c) = make_float4(o[0], o[1], o[2], o[3]);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) stf(dx_out_t + xr_i * d + c + e, o[e]);
+      store4<T>(dx_out_t + xr_i * d + c, o[0], o[1], o[2], o[3]);
     }
   }
   __syncthreads();
@@ -160,51 +186,105 @@ __global__ void rope_table_kernel(float2* __restrict__ tab, int S, int dh) {
   tab[idx] = make_float2((float)cos(ang), (float)sin(ang));
 }
 
+// 16-byte vectors of T: 8 bf16 or 4 fp32
+template <typename T> struct Vec16 { static constexpr int N = 16 / sizeof(T); };
+template <typename T>
+__device__ __forceinline__ void load_vec(const T* p, float (&v)[Vec16<T>::N]) {
+  const uint4 raw = *reinterpret_cast<const uint4*>(p);
+  if constexpr (sizeof(T) == 2) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { const float2 f = __bfloat1622float2(h[e]); v[2 * e] = f.x; v[2 * e + 1] = f.y; }
+  } else {
+    v[0] = __uint_as_float(raw.x); v[1] = __uint_as_float(raw.y); v[2] = __uint_as_float(raw.z); v[3] = __uint_as_float(raw.w);
+  }
+}
+template <typename T>
+__device__ __forceinline__ void store_vec(T* p, const float (&v)[Vec16<T>::N]) {
+  uint4 raw;
+  if constexpr (sizeof(T) == 2) {
+    __nv_bfloat162 h[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+    raw = *reinterpret_cast<uint4*>(h);
+  } else {
+    raw = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+  }
+  *reinterpret_cast<uint4*>(p) = raw;
+}
+
+// One thread rotates VEC consecutive pairs (i, i + dh/2) of one head of q or k.
 template <typename T>
 __global__ void rope_kernel(T* __restrict__ qkv, const float2* __restrict__ tab, long long rows, int S, int H,
                             int dh, float sign) {
-  const int half = dh / 2, d = H * dh;
-  const long long per_row = 2LL * H * half;              // q and k pairs
+  constexpr int VEC = Vec16<T>::N;
+  const int half = dh / 2, d = H * dh, per_head = half / VEC;
+  const long long per_row = 2LL * H * per_head;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= rows * per_row) return;
   const long long r = idx / per_row;
   const int rem = (int)(idx - r * per_row);
-  const int which = rem / (H * half);                    // 0 = q, 1 = k
-  const int hh = (rem - which * H * half) / half;
-  const int i = rem % half;
+  const int which = rem / (H * per_head);                // 0 = q, 1 = k
+  const int hh = (rem - which * H * per_head) / per_head;
+  const int i0 = (rem % per_head) * VEC;
   const int pos = (int)(r % S);
-  const float2 cs = tab[pos * half + i];
-  T* p = qkv + r * 3LL * d + (long long)which * d + (long long)hh * dh + i;
-  const float a = ldf(p), b = ldf(p + half);
-  const float sn = cs.y * sign;
-  stf(p, a * cs.x - b * sn);
-  stf(p + half, b * cs.x + a * sn);
+  T* p = qkv + r * 3LL * d + (long long)which * d + (long long)hh * dh + i0;
+  float a[VEC], b[VEC];
+  load_vec<T>(p, a);
+  load_vec<T>(p + half, b);
+  const float2* cs = tab + pos * half + i0;
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    const float2 t = cs[e];
+    const float sn = t.y * sign, x = a[e], y = b[e];
+    a[e] = x * t.x - y * sn;
+    b[e] = y * t.x + x * sn;
+  }
+  store_vec<T>(p, a);
+  store_vec<T>(p + half, b);
 }
 
 // ------------------------------------------------------------------------------------------------
-// SwiGLU: gu [rows][8d] = gate | up
+// SwiGLU: gu [rows][8d] = gate | up; one thread handles one 16-byte vector of the hidden dimension
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void swiglu_fwd_kernel(const T* __restrict__ gu, T* __restrict__ act, long long rows, int f) {
+  constexpr int VEC = Vec16<T>::N;
+  const int fv = f / VEC;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * f) return;
-  const long long r = idx / f;
-  const int c = (int)(idx - r * f);
-  const float g = ldf(gu + r * 2LL * f + c), u = ldf(gu + r * 2LL * f + f + c);
-  stf(act + idx, g / (1.f + __expf(-g)) * u);
+  if (idx >= rows * fv) return;
+  const long long r = idx / fv;
+  const int c = (int)(idx - r * fv) * VEC;
+  float g[VEC], u[VEC];
+  load_vec<T>(gu + r * 2LL * f + c, g);
+  load_vec<T>(gu + r * 2LL * f + f + c, u);
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+  store_vec<T>(act + r * (long long)f + c, g);
 }
 
 template <typename T>
 __global__ void swiglu_bwd_kernel(const T* __restrict__ gu, const T* __restrict__ dact, T* __restrict__ dgu,
                                   long long rows, int f) {
+  constexpr int VEC = Vec16<T>::N;
+  const int fv = f / VEC;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * f) return;
-  const long long r = idx / f;
-  const int c = (int)(idx - r * f);
-  const float g = ldf(gu + r * 2LL * f + c), u = ldf(gu + r * 2LL * f + f + c), da = ldf(dact + idx);
-  const float sg = 1.f / (1.f + __expf(-g));
-  stf(dgu + r * 2LL * f + c, da * u * sg * (1.f + g * (1.f - sg)));
-  stf(dgu + r * 2LL * f + f + c, da * g * sg);
+  if (idx >= rows * fv) return;
+  const long long r = idx / fv;
+  const int c = (int)(idx - r * fv) * VEC;
+  float g[VEC], u[VEC], da[VEC];
+  load_vec<T>(gu + r * 2LL * f + c, g);
+  load_vec<T>(gu + r * 2LL * f + f + c, u);
+  load_vec<T>(dact + r * (long long)f + c, da);
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    const float sg = 1.f / (1.f + __expf(-g[e]));
+    const float dg = da[e] * u[e] * sg * (1.f + g[e] * (1.f - sg));
+    u[e] = da[e] * g[e] * sg;
+    g[e] = dg;
+  }
+  store_vec<T>(dgu + r * 2LL * f + c, g);
+  store_vec<T>(dgu + r * 2LL * f + f + c, u);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -477,7 +557,7 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       prof_end(s, 0.0, (double)M * d * (es + 4.0));
       TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0));
       prof_begin(PC_ELEM, s);
-      rope_kernel<T><<<ceil_div(M * H * dh, 256), 256, 0, s>>>((T*)la.qkv, w.rope_tab, M, S, H, dh, 1.f);
+      rope_kernel<T><<<ceil_div(M * H * dh / Vec16<T>::N, 256), 256, 0, s>>>((T*)la.qkv, w.rope_tab, M, S, H, dh, 1.f);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
       prof_begin(PC_ATTN, s);
@@ -490,7 +570,7 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       prof_end(s, 0.0, (double)M * d * (es + 4.0));
       TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0));
       prof_begin(PC_ELEM, s);
-      swiglu_fwd_kernel<T><<<ceil_div(M * 4 * d, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, M, 4 * d);
+      swiglu_fwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, M, 4 * d);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)M * 4 * d * es * 3.0);
       TRY(G(Mi, d, 4 * d, la.act, 4 * d, true, w_d + (size_t)l * 4 * d * d, 4 * d, true, dt, x_out, d, DT_F32, la.x_mid, d));
@@ -543,7 +623,7 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
             gr->w_d + l * 4 * dd, 4 * d));
       TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dact, 4 * d, dt, nullptr, 0));
       prof_begin(PC_ELEM, s);
-      swiglu_bwd_kernel<T><<<ceil_div(M * 4 * d, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, M, 4 * d);
+      swiglu_bwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, M, 4 * d);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)M * 4 * d * es * 5.0);
       TRY(G(8 * d, d, Mi, w.dgu, 8 * d, false, la.h2, d, false, dt, gr->w_gu + l * 8 * dd, d, DT_F32,
@@ -557,7 +637,7 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       TRY(attention_bwd(dt, la.qkv, la.attn, w.dattn, la.lse, w.dsum, w.dqkv, mb, S, H, dh, s));
       prof_end(s, 5.0 * S * (double)S * d * mb, (double)M * 8 * d * es);
       prof_begin(PC_ELEM, s);
-      rope_kernel<T><<<ceil_div(M * H * dh, 256), 256, 0, s>>>((T*)w.dqkv, w.rope_tab, M, S, H, dh, -1.f);
+      rope_kernel<T><<<ceil_div(M * H * dh / Vec16<T>::N, 256), 256, 0, s>>>((T*)w.dqkv, w.rope_tab, M, S, H, dh, -1.f);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
       TRY(G(3 * d, d, Mi, w.dqkv, 3 * d, false, la.h1, d, false, dt, gr->w_qkv + l * 3 * dd, d, DT_F32,

@@ -1,4 +1,5 @@
-// Dispatch of the attention entry points on the activation dtype.
+// Dispatch of the attention entry points on the activation dtype: fp32 runs the SIMT kernels
+// (attention_f32.cu), bf16 the tensor-core kernels (attention_mma.cu).
 #include "internal.h"
 
 namespace pcm {

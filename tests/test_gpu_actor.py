@@ -63,7 +63,7 @@ def test_attention_fwd_bwd(dtype, dh, S, H, n_seq):
     o, p = ao.causal_attention(q, k, v)
     dq, dk, dv = ao.causal_attention_bwd(heads(do), q, k, v, p)
     back = lambda x: x.transpose(0, 2, 1, 3).reshape(n_seq * S, d)
-    tol = 2e-6 if dtype == "f32" else 6e-3
+    tol = 2e-6 if dtype == "f32" else 1e-2
     assert rel_fro(out.float().cpu().numpy(), back(o)) < tol
     got = dqkv.float().cpu().numpy()
     assert rel_fro(got[:, :d], back(dq)) < tol * 2
