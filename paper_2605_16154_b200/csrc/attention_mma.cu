@@ -39,17 +39,25 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros without touching global memory
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 // rows [row0, row0 + nrows) of a [.][DH] matrix (global row stride ld elements) -> shared rows
-// [0, nrows) with stride DH + 8; rows at or beyond row_limit are zero.
+// [0, nrows) with stride DH + 8; rows at or beyond row_limit are zero.  All copies of a thread are
+// in flight together; the caller waits with cp_async_wait_all() + __syncthreads().
 template <int DH>
 __device__ __forceinline__ void stage_rows(bf16* dst, const bf16* __restrict__ src, long long ld, int row0, int nrows,
                                            int row_limit) {
   constexpr int RS = DH + 8, VEC = DH / 8;                 // 8 bf16 per 16-byte vector
   for (int idx = threadIdx.x; idx < nrows * VEC; idx += blockDim.x) {
     const int r = idx / VEC, v = idx - r * VEC;
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if (row0 + r < row_limit) val = *reinterpret_cast<const uint4*>(src + (long long)(row0 + r) * ld + v * 8);
-    *reinterpret_cast<uint4*>(dst + r * RS + v * 8) = val;
+    const bool ok = row0 + r < row_limit;
+    const bf16* g = ok ? src + (long long)(row0 + r) * ld + v * 8 : src;
+    cp_async16(dst + r * RS + v * 8, g, ok ? 16 : 0);
   }
 }
 
@@ -100,6 +108,7 @@ fa_fwd_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __res
   stage_rows<DH>(Qs, base, ld, q0, FA_ROWS, S);
   stage_rows<DH>(Ks, base + d, ld, 0, key_rows, n_keys);
   stage_rows<DH>(Vs, base + 2 * d, ld, 0, key_rows, n_keys);
+  cp_async_wait_all();
   __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -233,6 +242,7 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
   stage_rows<DH>(Gs, dout + (long long)seq * S * d + (long long)h * DH, d, q0, FA_ROWS, S);
   stage_rows<DH>(Ks, base + d, ld, 0, key_rows, n_keys);
   stage_rows<DH>(Vs, base + 2 * d, ld, 0, key_rows, n_keys);
+  cp_async_wait_all();
   __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -336,6 +346,7 @@ fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, c
     Ls[i] = ok ? lse[sbase + q_lo + i] * LOG2E : 0.f;
     Ds[i] = ok ? dsum[sbase + q_lo + i] : 0.f;
   }
+  cp_async_wait_all();
   __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;

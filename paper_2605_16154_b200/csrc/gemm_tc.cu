@@ -10,6 +10,9 @@
 // one bit of the instruction descriptor, so forward, input-gradient and weight-gradient GEMMs
 // are the same kernel.
 //
+// Persistent: one CTA per SM walks a static list of output tiles; the shared-memory ring keeps
+// flowing across tile boundaries and the accumulator is double-buffered in tensor memory, so the
+// epilogue of one tile overlaps the MMAs of the next.
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = tensor-memory allocation + MMA issue,
 // warps 2..5 = epilogue.  Every mbarrier wait is bounded; when one runs out the CTA sets a status
 // flag, all roles leave their loops, tensor memory is released and the kernel returns.
@@ -30,7 +33,8 @@ __device__ unsigned g_tc_status = 0;          // bit 0: a bounded wait expired
 
 struct TcParams {
   int M, N, K;
-  int kb_per_split;                           // k-blocks of 64 handled by one blockIdx.z
+  int kb_per_split;                           // k-blocks of 64 handled by one split of the contraction
+  int tiles_m, tiles_n, splits;
   void* C; long long ldc; int c_dtype;        // DT_BF16 / DT_F32
   const float* R; long long ldr;
   int reduce;                                 // 1: fp32 reduction into C
@@ -73,57 +77,63 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + TC_STAGES * SM::STAGE_BYTES);
   uint64_t* full = bars;                      // [TC_STAGES] producer -> MMA
   uint64_t* empty = bars + TC_STAGES;         // [TC_STAGES] MMA -> producer
-  uint64_t* acc_full = bars + 2 * TC_STAGES;  // MMA -> epilogue
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * TC_STAGES + 1);
+  uint64_t* acc_full = bars + 2 * TC_STAGES;  // [2] MMA -> epilogue, one per accumulator buffer
+  uint64_t* acc_empty = acc_full + 2;         // [2] epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * TC_BM;
   const int num_kb_total = (p.K + TC_BK - 1) / TC_BK;
-  const int kb_lo = blockIdx.z * p.kb_per_split;
-  const int kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
-  const int num_kb = kb_hi - kb_lo;           // >= 1 by construction of the grid
+  const int tiles_mn = p.tiles_m * p.tiles_n;
+  const int total_tiles = tiles_mn * p.splits;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(acc_full, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, 2 * BN);            // two accumulator buffers: the epilogue of one tile overlaps the next tile's MMAs
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_acc = *tmem_slot;
+  const uint32_t tmem_base = *tmem_slot;
 
+  // Tiles are walked in the same order by every role: tile -> (split, m, n) with n fastest, so that
+  // CTAs running at the same time share A row-tiles and the whole B operand stays in L2.
   if (warp == 0) {
     if (lane == 0) {
       // ------------------------------ TMA producer ------------------------------
-      for (int i = 0; i < num_kb; ++i) {
-        const int st = i % TC_STAGES;
-        const unsigned ph = (unsigned)(i / TC_STAGES) & 1u;
-        if (*abort_flag) break;
-        if (!mbar_wait_bounded(&empty[st], ph ^ 1u, TC_WAIT_LIMIT_NS)) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); break; }
-        uint8_t* sa = tiles + st * SM::STAGE_BYTES;
-        uint8_t* sb = sa + SM::A_BYTES;
-        mbar_expect_tx(&full[st], SM::STAGE_BYTES);
-        const int k0 = (kb_lo + i) * TC_BK;
-        if (p.a_kmajor) {
-          tma_load_2d(sa, &tmA, k0, m0, &full[st]);                     // box {64 k, 128 m}
-        } else {
+      unsigned it = 0;                        // k-blocks issued so far, across tiles
+      for (int tile = blockIdx.x; tile < total_tiles && !*abort_flag; tile += gridDim.x) {
+        const int split = tile / tiles_mn, mn = tile - split * tiles_mn;
+        const int m0 = (mn / p.tiles_n) * TC_BM, n0 = (mn % p.tiles_n) * BN;
+        const int kb_lo = split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+          const int st = it % TC_STAGES;
+          const unsigned ph = (it / TC_STAGES) & 1u;
+          if (!mbar_wait_bounded(&empty[st], ph ^ 1u, TC_WAIT_LIMIT_NS)) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); break; }
+          uint8_t* sa = tiles + st * SM::STAGE_BYTES;
+          uint8_t* sb = sa + SM::A_BYTES;
+          mbar_expect_tx(&full[st], SM::STAGE_BYTES);
+          const int k0 = kb * TC_BK;
+          if (p.a_kmajor) {
+            tma_load_2d(sa, &tmA, k0, m0, &full[st]);                     // box {64 k, 128 m}
+          } else {
 #pragma unroll
-          for (int b = 0; b < TC_BM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, m0 + b * 64, k0, &full[st]);  // box {64 m, 64 k}
-        }
-        if (p.b_kmajor) {
-          tma_load_2d(sb, &tmB, k0, n0, &full[st]);                     // box {64 k, BN n}
-        } else {
+            for (int b = 0; b < TC_BM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, m0 + b * 64, k0, &full[st]);  // box {64 m, 64 k}
+          }
+          if (p.b_kmajor) {
+            tma_load_2d(sb, &tmB, k0, n0, &full[st]);                     // box {64 k, BN n}
+          } else {
 #pragma unroll
-          for (int b = 0; b < BN / 64; ++b) tma_load_2d(sb + b * 8192, &tmB, n0 + b * 64, k0, &full[st]);
+            for (int b = 0; b < BN / 64; ++b) tma_load_2d(sb + b * 8192, &tmB, n0 + b * 64, k0, &full[st]);
+          }
         }
       }
     }
@@ -136,44 +146,60 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       //                a k-step of 16 rows is 2048 B.
       const uint32_t a_lbo = p.a_kmajor ? 16u : 8192u, b_lbo = p.b_kmajor ? 16u : 8192u;
       const uint32_t a_step = p.a_kmajor ? 32u : 2048u, b_step = p.b_kmajor ? 32u : 2048u;
+      unsigned it = 0, tcount = 0;
       bool ok = true;
-      for (int i = 0; i < num_kb && ok; ++i) {
-        const int st = i % TC_STAGES;
-        const unsigned ph = (unsigned)(i / TC_STAGES) & 1u;
-        if (*abort_flag) { ok = false; break; }
-        if (!mbar_wait_bounded(&full[st], ph, TC_WAIT_LIMIT_NS)) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); ok = false; break; }
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
+        const int split = tile / tiles_mn;
+        const int kb_lo = split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
+        const unsigned ab = tcount & 1u, aph = (tcount >> 1) & 1u;
+        if (*abort_flag || !mbar_wait_bounded(&acc_empty[ab], aph ^ 1u, TC_WAIT_LIMIT_NS)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t sa = smem_u32(tiles + st * SM::STAGE_BYTES);
-        const uint32_t sb = sa + SM::A_BYTES;
+        const uint32_t tmem_acc = tmem_base + ab * BN;
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+          const int st = it % TC_STAGES;
+          const unsigned ph = (it / TC_STAGES) & 1u;
+          if (*abort_flag || !mbar_wait_bounded(&full[st], ph, TC_WAIT_LIMIT_NS)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(tiles + st * SM::STAGE_BYTES);
+          const uint32_t sb = sa + SM::A_BYTES;
 #pragma unroll
-        for (int k = 0; k < TC_BK / 16; ++k) {
-          const uint64_t da = make_smem_desc(sa + k * a_step, a_lbo, 1024u);
-          const uint64_t db = make_smem_desc(sb + k * b_step, b_lbo, 1024u);
-          umma_bf16(tmem_acc, da, db, idesc, (i | k) ? 1u : 0u);
+          for (int k = 0; k < TC_BK / 16; ++k) {
+            const uint64_t da = make_smem_desc(sa + k * a_step, a_lbo, 1024u);
+            const uint64_t db = make_smem_desc(sb + k * b_step, b_lbo, 1024u);
+            umma_bf16(tmem_acc, da, db, idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
+          }
+          umma_commit(&empty[st]);            // frees the stage once the MMAs above have read it
         }
-        umma_commit(&empty[st]);              // frees the stage once the MMAs above have read it
+        if (ok) umma_commit(&acc_full[ab]);
       }
-      if (ok) umma_commit(acc_full);
+      if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
     }
   } else {
     // ------------------------------ epilogue: warps 2..5 ------------------------------
     const int quad = warp & 3;                // tensor-memory lane quadrant this warp may access
-    const int row = m0 + quad * 32 + lane;
-    int ok = 1;
-    if (lane == 0) {
-      ok = (mbar_wait_bounded(acc_full, 0u, TC_WAIT_LIMIT_NS * 2ull) && !*abort_flag) ? 1 : 0;
-      if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
-    }
-    ok = __shfl_sync(0xffffffffu, ok, 0);
-    if (ok) {
+    unsigned tcount = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
+      const int split = tile / tiles_mn, mn = tile - split * tiles_mn;
+      const int m0 = (mn / p.tiles_n) * TC_BM, n0 = (mn % p.tiles_n) * BN;
+      const int row = m0 + quad * 32 + lane;
+      const unsigned ab = tcount & 1u, aph = (tcount >> 1) & 1u;
+      int ok = 1;
+      if (lane == 0) {
+        ok = (!*abort_flag && mbar_wait_bounded(&acc_full[ab], aph, TC_WAIT_LIMIT_NS * 2ull)) ? 1 : 0;
+        if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
       tc_fence_after();
+      const uint32_t tmem_acc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld_32x32(tmem_acc + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, r);
-        tmem_ld_wait();
         const int col = n0 + c0;
-        if (row < p.M && col < p.N) {        // N is a multiple of 32 on this path
+        if (col >= p.N) break;                // warp-uniform: N is a multiple of 32 on this path
+        uint32_t r[32];
+        tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
+        tmem_ld_wait();
+        if (row < p.M) {
           if (p.reduce) {
             float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
 #pragma unroll
@@ -213,6 +239,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       }
+      // hand the accumulator buffer back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[ab]);
     }
   }
 
@@ -225,7 +255,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_acc, BN);
+    tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 
@@ -274,8 +304,17 @@ bool gemm_tcgen05_supported(const GemmArgs& g) {
   if (g.c_dtype == DT_F32 && (g.ldc % 4)) return false;
   if (g.R && (((uintptr_t)g.R & 15) || (g.ldr % 4))) return false;
   if (g.R && (const void*)g.R == (const void*)g.C && g.c_dtype != DT_F32) return false;
-  if ((g.M + TC_BM - 1) / TC_BM > 65535) return false;
-  return encode_fn() != nullptr;
+    return encode_fn() != nullptr;
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      n = 148;
+  }
+  return n;
 }
 
 template <int BN>
@@ -311,7 +350,9 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
     PCM_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<BN>::TOTAL));
     attr_done = true;
   }
-  dim3 grid(tiles_n, tiles_m, splits);
+  p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits;
+  const long long total = (long long)tiles_m * tiles_n * splits;
+  const int grid = (int)(total < sm_count() ? total : sm_count());      // persistent: one CTA per SM walks the tile list
   gemm_tc_kernel<BN><<<grid, TC_THREADS, TcSmem<BN>::TOTAL, s>>>(tmA, tmB, p);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
