@@ -256,7 +256,8 @@ int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* batch, const 
  * a_kmajor != 0: A is stored [M][K] with row stride lda, else [K][M]; likewise B ([N][K] / [K][N]).
  * ab_dtype / c_dtype are grpo_dtype values; R (fp32, may be NULL) may alias C to accumulate (C fp32).
  * backend: 0 = automatic, 1 = SIMT kernel, 2 = tcgen05 kernel (PCM_ERR_SHAPE when it cannot take the
- * problem).  Synchronises `stream`; returns PCM_ERR_DEVICE_TIMEOUT when a bounded wait expired. */
+ * problem); adding 4 skips the synchronisation.  Otherwise synchronises `stream` and returns
+ * PCM_ERR_DEVICE_TIMEOUT when a bounded wait expired. */
 int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_kmajor, const void* B,
               int64_t ldb, int32_t b_kmajor, int32_t ab_dtype, void* C, int64_t ldc, int32_t c_dtype,
               const float* R, int64_t ldr, int32_t backend, pcm_stream stream);

@@ -725,13 +725,15 @@ extern "C" int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* ba
 extern "C" int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_kmajor, const void* B,
                          int64_t ldb, int32_t b_kmajor, int32_t ab_dtype, void* C, int64_t ldc, int32_t c_dtype,
                          const float* R, int64_t ldr, int32_t backend, pcm_stream stream) {
-  if (!A || !B || !C || M < 1 || N < 1 || K < 1 || backend < 0 || backend > 2) return PCM_ERR_ARG;
+  const bool no_sync = (backend & 4) != 0;
+  backend &= 3;
+  if (!A || !B || !C || M < 1 || N < 1 || K < 1 || backend > 2) return PCM_ERR_ARG;
   if ((ab_dtype != GRPO_F32 && ab_dtype != GRPO_BF16) || (c_dtype != GRPO_F32 && c_dtype != GRPO_BF16)) return PCM_ERR_ARG;
   GemmArgs g{M, N, K, A, lda, a_kmajor != 0, B, ldb, b_kmajor != 0, ab_dtype == GRPO_BF16 ? DT_BF16 : DT_F32,
              C, ldc, c_dtype == GRPO_BF16 ? DT_BF16 : DT_F32, R, ldr};
   cudaStream_t s = (cudaStream_t)stream;
   int rc = gemm(g, s, backend == 1 ? GEMM_SIMT : backend == 2 ? GEMM_TCGEN05 : GEMM_AUTO);
-  if (rc != PCM_OK) return rc;
+  if (rc != PCM_OK || no_sync) return rc;
   PCM_CUDA_TRY(cudaStreamSynchronize(s));
   return tcgen05_poll_status();
 }
