@@ -88,11 +88,12 @@ score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restr
       acc_lo = acc_hi = run = 0;
     };
     if (sub < 2) {
-      for (int ch0 = a + sub; ch0 < b; ch0 += 8) {       // four chunk pairs per iteration
-        uint32_t wv[4];
-        int ph[4];
+      constexpr int UNROLL = 8;                          // chunk pairs in flight per iteration
+      for (int ch0 = a + sub; ch0 < b; ch0 += 2 * UNROLL) {
+        uint32_t wv[UNROLL];
+        int ph[UNROLL];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
           const int ch = ch0 + 2 * u;
           if (ch < b) {
             wv[u] = __ldg(tokw + (size_t)ch * WORDS + word);
@@ -103,7 +104,7 @@ score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restr
           }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
           if (ph[u] < 0) continue;
           if (ph[u] >= n_phases) {
             atomicOr(status, STATUS_BAD_PHASE);
@@ -146,24 +147,31 @@ score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restr
   }
 }
 
-// Block 0: mean of C_{c,g} over valid groups in ascending g (one thread per phase).
-// Blocks 1..: Eq. 1 advantages, one thread per group.
+// Blocks 0 .. n_phases-1: mean of C_{c,g} over valid groups.  One warp per phase loads 32 groups at a
+// time in parallel and adds them in ascending g (every lane runs the same chain, so the order of the
+// fp64 additions is exactly the sequential one).
+// Blocks n_phases ..: Eq. 1 advantages, one thread per group.
 __global__ void score_finalize_kernel(const double* __restrict__ c_group,
                                       const uint8_t* __restrict__ valid_group, int n_groups, int n_phases,
                                       double* __restrict__ C, uint8_t* __restrict__ valid,
                                       int32_t* __restrict__ n_valid, const uint8_t* __restrict__ reward,
                                       int G, double eps, float* __restrict__ adv) {
-  if (blockIdx.x == 0) {
-    const int c = threadIdx.x;
-    if (c < n_phases) {
-      double s = 0.0;
-      int k = 0;
-      for (int g = 0; g < n_groups; ++g) {
-        if (valid_group[(size_t)g * n_phases + c]) {
-          s = __dadd_rn(s, c_group[(size_t)g * n_phases + c]);
-          ++k;
-        }
+  if ((int)blockIdx.x < n_phases) {
+    if (threadIdx.x >= 32) return;
+    const int c = blockIdx.x, lane = threadIdx.x;
+    double s = 0.0;
+    int k = 0;
+    for (int g0 = 0; g0 < n_groups; g0 += 32) {
+      const int g = g0 + lane;
+      const bool ok = g < n_groups && valid_group[(size_t)g * n_phases + c];
+      const double x = ok ? c_group[(size_t)g * n_phases + c] : 0.0;
+      const unsigned m = __ballot_sync(0xffffffffu, ok);
+      for (int l = 0; l < 32; ++l) {
+        const double xl = __shfl_sync(0xffffffffu, x, l);
+        if (m & (1u << l)) { s = __dadd_rn(s, xl); ++k; }
       }
+    }
+    if (lane == 0) {
       C[c] = k ? __ddiv_rn(s, (double)k) : 0.0;
       valid[c] = k ? 1 : 0;
       if (n_valid) n_valid[c] = k;
@@ -171,7 +179,7 @@ __global__ void score_finalize_kernel(const double* __restrict__ c_group,
     return;
   }
   if (!adv) return;
-  const int g = (blockIdx.x - 1) * blockDim.x + threadIdx.x;
+  const int g = (blockIdx.x - n_phases) * blockDim.x + threadIdx.x;
   if (g >= n_groups) return;
   double s = 0.0;
   for (int j = 0; j < G; ++j) s = __dadd_rn(s, reward[g * G + j] ? 1.0 : 0.0);
@@ -455,7 +463,7 @@ int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* b, double* C, uint8_t* valid
   PCM_LAUNCH_CHECK();
   prof_end(s, 0.0, (double)b->n_chunks * (ACT + 1));
   const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
-  score_finalize_kernel<<<1 + adv_blocks, 128, 0, s>>>(ctx->c_group, ctx->valid_group, ng, Kc, C, valid,
+  score_finalize_kernel<<<Kc + adv_blocks, 128, 0, s>>>(ctx->c_group, ctx->valid_group, ng, Kc, C, valid,
                                                        n_valid_groups, b->reward, G, ctx->cfg.adv_eps, adv);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
@@ -557,7 +565,7 @@ extern "C" int pcm_score_phases_static(int32_t n_phases, int32_t group_size, dou
                                              valid_group, status);
   PCM_LAUNCH_CHECK();
   const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
-  score_finalize_kernel<<<1 + adv_blocks, 128, 0, s>>>(c_group, valid_group, ng, n_phases, C, valid, n_valid_groups,
+  score_finalize_kernel<<<n_phases + adv_blocks, 128, 0, s>>>(c_group, valid_group, ng, n_phases, C, valid, n_valid_groups,
                                                        b->reward, group_size, adv_eps, adv);
   PCM_LAUNCH_CHECK();
   if (device_status)

@@ -1,0 +1,115 @@
+"""Parity at the full size of the medium workload (C1), in the launch configuration bench.py times
+(whole batch of 384 kept chunks in one micro-batch): selection and packed rows bit-exact against the
+oracle, sampled outputs the oracle can compute one by one, and properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import actor_oracle as ao
+from oracle import pcm_oracle as po
+from paper_2605_16154_b200 import synth
+from tests.gpu_helpers import grads_to_numpy, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def c1():
+    from paper_2605_16154_b200 import binding as B, pipeline as PL
+    w = synth.WORKLOADS["C1"]
+    rb = synth.make_rollouts(w)
+    weights = synth.make_weights(w)
+    total = int(rb["traj_off"][-1])
+    obs = synth.obs_all(w, w.seed, total)
+    lpo_all = (-np.log(256.0) + synth.logp_noise(w.seed, total, 0.3)).astype(np.float32)
+    model = PL.upload_model(w, weights)
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=5, max_traj=w.n_traj)
+    batch = PL.upload_rollouts(w, rb, obs=PL.dev(obs, torch.bfloat16), logp_old=PL.dev(lpo_all))
+    adv, Cc, valid, p, q, kept_idx, kept_off, per_phase = PL.select(ctx, batch, 0)
+    n_kept = PL.n_kept_of(w.budget, rb["traj_off"])
+    pk = B.grpo_pack_chunks(ctx, batch, model, kept_idx, kept_off, adv, B.Packed(model, n_kept))
+    assert B.pcm_poll_status(ctx) == 0
+    return dict(B=B, PL=PL, w=w, rb=rb, weights=weights, obs=obs, lpo_all=lpo_all, model=model, ctx=ctx, batch=batch,
+                adv=adv, q=q, kept_idx=kept_idx, kept_off=kept_off, pk=pk, n_kept=n_kept)
+
+
+def test_selection_and_pack_bit_exact_at_full_size(c1):
+    w, rb = c1["w"], c1["rb"]
+    C_o, valid_o, _, _, _ = po.score_phases(rb["traj_off"], rb["tok"], rb["phase"], rb["reward"], w.G, w.n_phases)
+    _, q_o, _ = po.update_keep_probs(po.KeepProbState(w.n_phases, w.p_min, w.t_rc), C_o, valid_o)
+    kept_o, off_o, _ = po.sample_chunks(rb["traj_off"], rb["phase"], q_o, w.budget, 5, 0)
+    assert c1["n_kept"] == 384 == len(kept_o)
+    assert np.array_equal(c1["kept_idx"].cpu().numpy()[:384], kept_o)
+    assert np.array_equal(c1["kept_off"].cpu().numpy(), off_o)
+    pk = c1["pk"]
+    X = pk.X.float().cpu().numpy()
+    e_act = c1["weights"]["e_act"]
+    for j in (0, 57, 200, 383):                                   # sampled packed rows against their sources
+        c = int(kept_o[j])
+        assert np.array_equal(X[j, :w.P], c1["obs"][c])
+        assert np.array_equal(X[j, w.P:], e_act[rb["tok"][c].astype(int)])
+        assert np.array_equal(pk.tgt[j].cpu().numpy(), rb["tok"][c])
+        assert np.array_equal(pk.lpo[j].cpu().numpy(), c1["lpo_all"][c])
+    adv_o = po.advantages(rb["reward"], w.G, 1e-6).astype(np.float32)
+    owner = np.searchsorted(rb["traj_off"], kept_o, side="right") - 1
+    assert np.array_equal(pk.adv_c.cpu().numpy(), adv_o[owner])
+
+
+def test_sampled_log_probs_and_batch_properties_at_full_size(c1):
+    B, w, model, pk = c1["B"], c1["w"], c1["model"], c1["pk"]
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, pk, mb_chunks=384)
+    g_full = {k: v.clone() for k, v in grads.items()}
+    loss_full = float(loss.item())
+    assert np.isfinite(loss_full) and stats.n_launches > 0
+    # sampled chunks: the oracle's forward pass on one chunk at a time
+    X = pk.X.float().cpu().numpy()
+    tgt = pk.tgt.cpu().numpy()
+    for j in (3, 311):
+        lp_o = ao.logp_only(c1["weights"], X[j:j + 1], tgt[j:j + 1], w.H, w.P)
+        assert np.max(np.abs(logp[j].cpu().numpy() - lp_o[0])) < 0.04
+    # micro-batching changes only the fp32 accumulation order
+    loss_mb, logp_mb, grads_mb, _ = B.grpo_actor_fwd_bwd(model, pk, mb_chunks=100)
+    assert torch.equal(logp_mb, logp)
+    assert abs(float(loss_mb.item()) - loss_full) < 1e-6
+    for k in g_full:
+        assert rel_fro(grads_mb[k].cpu().numpy(), g_full[k].cpu().numpy()) < 2e-3, k
+    # the masked objective is a sum over kept chunks: two halves with the same scale add up to the whole
+    scale = 1.0 / (56 * 384)
+    halves = {k: torch.zeros_like(v) for k, v in g_full.items()}
+    loss_sum = 0.0
+    for lo, hi in ((0, 192), (192, 384)):
+        sub = B.Packed(model, hi - lo)
+        sub.X.copy_(pk.X[lo:hi]); sub.tgt.copy_(pk.tgt[lo:hi]); sub.lpo.copy_(pk.lpo[lo:hi])
+        sub.adv_c.copy_(pk.adv_c[lo:hi]); sub.src.copy_(pk.src[lo:hi])
+        l, _, g, _ = B.grpo_actor_fwd_bwd(model, sub, loss_scale=scale, mb_chunks=192)
+        loss_sum += float(l.item())
+        for k in halves:
+            halves[k] += g[k]
+    assert abs(loss_sum - loss_full) < 1e-6
+    for k in g_full:
+        assert rel_fro(halves[k].cpu().numpy(), g_full[k].cpu().numpy()) < 2e-3, k
+
+
+def test_two_chunk_update_of_the_full_model_against_the_oracle(c1):
+    """Every kernel at the medium model's real width, depth and sequence length (8 layers, d = 1024,
+    S = 312), on a batch small enough for the fp64 oracle."""
+    B, PL, w, model, pk = c1["B"], c1["PL"], c1["w"], c1["model"], c1["pk"]
+    sel = [5, 250]
+    X = pk.X[sel].float().cpu().numpy()
+    tgt = pk.tgt[sel].cpu().numpy()
+    adv_c = np.array([0.8, -1.2], dtype=np.float32)               # both signs, whatever the sampled rewards were
+    lp_o = ao.logp_only(c1["weights"], X, tgt, w.H, w.P)
+    noise = synth.logp_noise(11, 2, 0.1).astype(np.float64)
+    hi, lo, m = np.log(1.2), np.log(0.8), 0.05
+    log_r = -noise
+    log_r = np.where(np.abs(log_r - hi) < m, hi + 2 * m * np.sign(log_r - hi + 1e-30), log_r)
+    log_r = np.where(np.abs(log_r - lo) < m, lo + 2 * m * np.sign(log_r - lo + 1e-30), log_r)
+    lpo = (lp_o - log_r).astype(np.float32)
+    loss_o, _, grads_o, stats_o = ao.fwd_bwd(c1["weights"], X, tgt, lpo, adv_c, w.H, w.P, 0.2, 0.2)
+    sub = B.Packed(model, 2)
+    sub.X.copy_(pk.X[sel]); sub.tgt.copy_(pk.tgt[sel]); sub.lpo.copy_(PL.dev(lpo)); sub.adv_c.copy_(PL.dev(adv_c))
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, sub)
+    assert abs(float(loss.item()) - loss_o) < 1e-3
+    assert stats.clip_frac == pytest.approx(stats_o["clip_frac"], abs=1e-6)
+    errs = {k: rel_fro(v, grads_o[k]) for k, v in grads_to_numpy(grads).items()}
+    assert max(errs.values()) < 2e-2, errs
