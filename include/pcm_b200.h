@@ -274,8 +274,8 @@ int grpo_attention(int32_t dtype, const void* qkv, void* out, float* lse, const 
  * milliseconds, the algorithmic flops / bytes of the launches and their count since the last read,
  * and clears the records.  Classes: 0 GEMM (all linear layers, head), 1 attention, 2 RMSNorm,
  * 3 element-wise (rotary, SwiGLU, residual cast), 4 loss rows, 5 embedding gradient, 6 pack,
- * 7 PCM control plane (score, update, sample). */
-#define PCM_PROFILE_CLASSES 8
+ * 7 phase-score reduction (the per-group kernel of pcm_score_phases), 8 chunk sampling. */
+#define PCM_PROFILE_CLASSES 9
 typedef struct {
   double ms[PCM_PROFILE_CLASSES];
   double flops[PCM_PROFILE_CLASSES];

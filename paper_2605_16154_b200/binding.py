@@ -76,12 +76,12 @@ class grpo_stats(C.Structure):
                 ("workspace_high_water", C.c_uint64)]
 
 
-PROFILE_CLASSES = ("gemm", "attention", "rmsnorm", "elementwise", "loss", "embed_grad", "pack", "pcm")
+PROFILE_CLASSES = ("gemm", "attention", "rmsnorm", "elementwise", "loss", "embed_grad", "pack", "pcm_score", "pcm_sample")
 
 
 class pcm_profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 8), ("flops", C.c_double * 8), ("bytes", C.c_double * 8),
-                ("launches", C.c_int64 * 8)]
+    _fields_ = [("ms", C.c_double * 9), ("flops", C.c_double * 9), ("bytes", C.c_double * 9),
+                ("launches", C.c_int64 * 9)]
 
 
 _P = C.c_void_p

@@ -483,6 +483,8 @@ static int check_cfg(const grpo_model_cfg* c) {
   return PCM_OK;
 }
 
+static GemmBackend backend_from_env();
+
 template <typename T>
 static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* lc, grpo_grads* gr, float* loss,
                float* logp, grpo_stats* stats, void* workspace, size_t workspace_bytes, cudaStream_t s) {
@@ -523,8 +525,9 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
   PCM_LAUNCH_CHECK();
 
   auto G = [&](int M_, int N_, int K_, const void* A, long long lda, bool ak, const void* B, long long ldb, bool bk,
-               int abdt, void* C, long long ldc, int cdt, const float* R, long long ldr) -> int {
-    GemmArgs g{M_, N_, K_, A, lda, ak, B, ldb, bk, abdt, C, ldc, cdt, R, ldr};
+               int abdt, void* C, long long ldc, int cdt, const float* R, long long ldr,
+               const GemmEpilogue& epi = GemmEpilogue()) -> int {
+    GemmArgs g{M_, N_, K_, A, lda, ak, B, ldb, bk, abdt, C, ldc, cdt, R, ldr, epi};
     prof_begin(PC_GEMM, s);
     const int rc = gemm(g, s);
     prof_end(s, 2.0 * M_ * (double)N_ * K_, 0.0);
@@ -532,6 +535,16 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
   };
 #define TRY(expr) do { int rc__ = (expr); if (rc__ != PCM_OK) return rc__; } while (0)
   const double es = (double)sizeof(T);
+  // bf16 on the tensor-core path: SwiGLU and the rotary embedding run inside GEMM / attention epilogues
+  bool fuse_swiglu = false, fuse_rope = false;
+  if (dt == DT_BF16 && backend_from_env() != GEMM_SIMT) {
+    GemmArgs probe{128, 8 * d, d, w.la[0].h2, d, true, w_gu, d, true, dt, w.la[0].gu, 8 * d, dt, nullptr, 0};
+    probe.epi.kind = EPI_SWIGLU_FWD; probe.epi.out2 = w.la[0].act; probe.epi.ld_out2 = 4 * d;
+    fuse_swiglu = gemm_epilogue_supported(probe);
+    GemmArgs probe2{128, 3 * d, d, w.la[0].h1, d, true, w_qkv, d, true, dt, w.la[0].qkv, 3 * d, dt, nullptr, 0};
+    probe2.epi.kind = EPI_ROPE; probe2.epi.rope_tab = w.rope_tab; probe2.epi.S = S; probe2.epi.dh = dh; probe2.epi.d = d;
+    fuse_rope = gemm_epilogue_supported(probe2);
+  }
 
   for (int c0 = 0; c0 < n; c0 += mb_max) {
     const int mb = (n - c0) < mb_max ? (n - c0) : mb_max;
@@ -555,11 +568,17 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(x_in, g1 + (size_t)l * d, (T*)la.h1, la.rstd1, M, d, 0, 0);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)M * d * (es + 4.0));
-      TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0));
-      prof_begin(PC_ELEM, s);
-      rope_kernel<T><<<ceil_div(M * H * dh / Vec16<T>::N, 256), 256, 0, s>>>((T*)la.qkv, w.rope_tab, M, S, H, dh, 1.f);
-      PCM_LAUNCH_CHECK();
-      prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
+      if (fuse_rope) {
+        GemmEpilogue e;
+        e.kind = EPI_ROPE; e.rope_tab = w.rope_tab; e.S = S; e.dh = dh; e.d = d;
+        TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0, e));
+      } else {
+        TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0));
+        prof_begin(PC_ELEM, s);
+        rope_kernel<T><<<ceil_div(M * H * dh / Vec16<T>::N, 256), 256, 0, s>>>((T*)la.qkv, w.rope_tab, M, S, H, dh, 1.f);
+        PCM_LAUNCH_CHECK();
+        prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
+      }
       prof_begin(PC_ATTN, s);
       TRY(attention_fwd(dt, la.qkv, la.attn, la.lse, mb, S, H, dh, s));
       prof_end(s, 2.0 * S * (double)S * d * mb, (double)M * 4 * d * es);
@@ -568,11 +587,17 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(la.x_mid, g2 + (size_t)l * d, (T*)la.h2, la.rstd2, M, d, 0, 0);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)M * d * (es + 4.0));
-      TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0));
-      prof_begin(PC_ELEM, s);
-      swiglu_fwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, M, 4 * d);
-      PCM_LAUNCH_CHECK();
-      prof_end(s, 0.0, (double)M * 4 * d * es * 3.0);
+      if (fuse_swiglu) {
+        GemmEpilogue e;
+        e.kind = EPI_SWIGLU_FWD; e.out2 = la.act; e.ld_out2 = 4 * d;
+        TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0, e));
+      } else {
+        TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0));
+        prof_begin(PC_ELEM, s);
+        swiglu_fwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, M, 4 * d);
+        PCM_LAUNCH_CHECK();
+        prof_end(s, 0.0, (double)M * 4 * d * es * 3.0);
+      }
       TRY(G(Mi, d, 4 * d, la.act, 4 * d, true, w_d + (size_t)l * 4 * d * d, 4 * d, true, dt, x_out, d, DT_F32, la.x_mid, d));
     }
     // head on the scored rows only
@@ -621,11 +646,17 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       // MLP: x_out = x_mid + act W_d^T
       TRY(G(d, 4 * d, Mi, w.dx_t, d, false, la.act, 4 * d, false, dt, gr->w_d + l * 4 * dd, 4 * d, DT_F32,
             gr->w_d + l * 4 * dd, 4 * d));
-      TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dact, 4 * d, dt, nullptr, 0));
-      prof_begin(PC_ELEM, s);
-      swiglu_bwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, M, 4 * d);
-      PCM_LAUNCH_CHECK();
-      prof_end(s, 0.0, (double)M * 4 * d * es * 5.0);
+      if (fuse_swiglu) {
+        GemmEpilogue e;
+        e.kind = EPI_SWIGLU_BWD; e.aux = la.gu; e.ld_aux = 8 * d;
+        TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dgu, 8 * d, dt, nullptr, 0, e));
+      } else {
+        TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dact, 4 * d, dt, nullptr, 0));
+        prof_begin(PC_ELEM, s);
+        swiglu_bwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, M, 4 * d);
+        PCM_LAUNCH_CHECK();
+        prof_end(s, 0.0, (double)M * 4 * d * es * 5.0);
+      }
       TRY(G(8 * d, d, Mi, w.dgu, 8 * d, false, la.h2, d, false, dt, gr->w_gu + l * 8 * dd, d, DT_F32,
             gr->w_gu + l * 8 * dd, d));
       TRY(G(Mi, d, 8 * d, w.dgu, 8 * d, true, w_gu + l * 8 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
@@ -634,12 +665,15 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       TRY(G(d, d, Mi, w.dx_t, d, false, la.attn, d, false, dt, gr->w_o + l * dd, d, DT_F32, gr->w_o + l * dd, d));
       TRY(G(Mi, d, d, w.dx_t, d, true, w_o + l * dd, d, false, dt, w.dattn, d, dt, nullptr, 0));
       prof_begin(PC_ATTN, s);
-      TRY(attention_bwd(dt, la.qkv, la.attn, w.dattn, la.lse, w.dsum, w.dqkv, mb, S, H, dh, s));
+      TRY(attention_bwd(dt, la.qkv, la.attn, w.dattn, la.lse, w.dsum, w.dqkv, mb, S, H, dh, s,
+                        fuse_rope ? w.rope_tab : nullptr));
       prof_end(s, 5.0 * S * (double)S * d * mb, (double)M * 8 * d * es);
-      prof_begin(PC_ELEM, s);
-      rope_kernel<T><<<ceil_div(M * H * dh / Vec16<T>::N, 256), 256, 0, s>>>((T*)w.dqkv, w.rope_tab, M, S, H, dh, -1.f);
-      PCM_LAUNCH_CHECK();
-      prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
+      if (!fuse_rope) {
+        prof_begin(PC_ELEM, s);
+        rope_kernel<T><<<ceil_div(M * H * dh / Vec16<T>::N, 256), 256, 0, s>>>((T*)w.dqkv, w.rope_tab, M, S, H, dh, -1.f);
+        PCM_LAUNCH_CHECK();
+        prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
+      }
       TRY(G(3 * d, d, Mi, w.dqkv, 3 * d, false, la.h1, d, false, dt, gr->w_qkv + l * 3 * dd, d, DT_F32,
             gr->w_qkv + l * 3 * dd, d));
       TRY(G(Mi, d, 3 * d, w.dqkv, 3 * d, true, w_qkv + l * 3 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
@@ -683,6 +717,7 @@ int gemm(const GemmArgs& g, cudaStream_t s, GemmBackend backend) {
     return gemm_tcgen05(g, s);
   }
   if (backend == GEMM_AUTO && gemm_tcgen05_supported(g)) return gemm_tcgen05(g, s);
+  if (g.epi.kind != EPI_NONE) return PCM_ERR_SHAPE;        // fused epilogues exist on the tensor-core path only
   return gemm_simt(g, s);
 }
 

@@ -219,13 +219,37 @@ __global__ void fa_dsum_kernel(const bf16* __restrict__ out, const bf16* __restr
   }
 }
 
+// Transpose of the rotary embedding applied to an accumulator tile of 16 rows x DH columns: pairs
+// (c, c + DH/2) sit in n-tiles i and i + DH/16 of the same thread.  Rows a / b are positions in the sequence.
+template <int DH>
+__device__ __forceinline__ void unrotate(float (&acc)[DH / 8][4], const float2* __restrict__ tab, int row_a, int row_b,
+                                         int S, int t) {
+  constexpr int HALF = DH / 2;
+  const int pa = min(row_a, S - 1), pb = min(row_b, S - 1);      // rows past the end are never stored
+#pragma unroll
+  for (int i = 0; i < DH / 16; ++i) {
+    const int c = i * 8 + 2 * t;
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const float2 ta = tab[pa * HALF + c + e], tb = tab[pb * HALF + c + e];
+      const float la = acc[i][e], ha = acc[i + DH / 16][e];
+      acc[i][e] = la * ta.x + ha * ta.y;
+      acc[i + DH / 16][e] = ha * ta.x - la * ta.y;
+      const float lb = acc[i][2 + e], hb = acc[i + DH / 16][2 + e];
+      acc[i][2 + e] = lb * tb.x + hb * tb.y;
+      acc[i + DH / 16][2 + e] = hb * tb.x - lb * tb.y;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // dQ: same tiling as the forward pass
 // ------------------------------------------------------------------------------------------------
 template <int DH>
 __global__ void __launch_bounds__(FA_THREADS)
 fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, const float* __restrict__ lse,
-                 const float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H, float scale) {
+                 const float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H, float scale,
+                 const float2* __restrict__ rope_tab) {
   extern __shared__ __align__(16) unsigned char smraw[];
   constexpr int RS = DH + 8;
   const int qt = blockIdx.x, h = blockIdx.y, seq = blockIdx.z, d = H * DH;
@@ -303,6 +327,7 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
       }
     }
   }
+  if (rope_tab) unrotate<DH>(dq, rope_tab, row_a, row_b, S, t);   // gradient w.r.t. q before the rotary embedding
   if (row_a < S) {
     bf16* p = dqkv + ((long long)seq * S + row_a) * ld + (long long)h * DH;
 #pragma unroll
@@ -321,7 +346,8 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
 template <int DH>
 __global__ void __launch_bounds__(FA_THREADS)
 fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, const float* __restrict__ lse,
-                  const float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H, float scale) {
+                  const float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H, float scale,
+                  const float2* __restrict__ rope_tab) {
   extern __shared__ __align__(16) unsigned char smraw[];
   constexpr int RS = DH + 8;
   const int kt = blockIdx.x, h = blockIdx.y, seq = blockIdx.z, d = H * DH;
@@ -419,6 +445,7 @@ fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, c
       }
     }
   }
+  if (rope_tab) unrotate<DH>(dk, rope_tab, key_a, key_b, S, t);   // gradient w.r.t. k before the rotary embedding
   if (key_a < S) {
     bf16* pk = dqkv + ((long long)seq * S + key_a) * ld + d + (long long)h * DH;
 #pragma unroll
@@ -454,7 +481,7 @@ static int fa_fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int 
 
 template <int DH>
 static int fa_bwd_launch(const void* qkv, const void* out, const void* dout, const float* lse, float* dsum, void* dqkv,
-                         int n_seq, int S, int H, cudaStream_t s) {
+                         int n_seq, int S, int H, const float2* rope_tab, cudaStream_t s) {
   const int tiles = (S + FA_ROWS - 1) / FA_ROWS;
   const size_t smem_dq = (size_t)(2 * FA_ROWS + 2 * tiles * FA_BLK) * (DH + 8) * sizeof(bf16);
   const size_t smem_dkv = smem_dq + (size_t)2 * tiles * FA_BLK * sizeof(float);
@@ -465,11 +492,11 @@ static int fa_bwd_launch(const void* qkv, const void* out, const void* dout, con
   PCM_LAUNCH_CHECK();
   PCM_CUDA_TRY(cudaFuncSetAttribute(fa_bwd_dq_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq));
   fa_bwd_dq_kernel<DH><<<dim3(tiles, H, n_seq), FA_THREADS, smem_dq, s>>>((const bf16*)qkv, (const bf16*)dout, lse, dsum,
-                                                                         (bf16*)dqkv, S, H, scale);
+                                                                         (bf16*)dqkv, S, H, scale, rope_tab);
   PCM_LAUNCH_CHECK();
   PCM_CUDA_TRY(cudaFuncSetAttribute(fa_bwd_dkv_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dkv));
   fa_bwd_dkv_kernel<DH><<<dim3(tiles, H, n_seq), FA_THREADS, smem_dkv, s>>>((const bf16*)qkv, (const bf16*)dout, lse,
-                                                                           dsum, (bf16*)dqkv, S, H, scale);
+                                                                           dsum, (bf16*)dqkv, S, H, scale, rope_tab);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
 }
@@ -483,11 +510,11 @@ int attention_fwd_bf16(const void* qkv, void* out, float* lse, int n_seq, int S,
 }
 
 int attention_bwd_bf16(const void* qkv, const void* out, const void* dout, const float* lse, float* dsum, void* dqkv,
-                       int n_seq, int S, int H, int dh, cudaStream_t s) {
+                       int n_seq, int S, int H, int dh, const float2* rope_tab, cudaStream_t s) {
   if (n_seq > 65535 || H > 65535) return PCM_ERR_SHAPE;
-  if (dh == 32) return fa_bwd_launch<32>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, s);
-  if (dh == 64) return fa_bwd_launch<64>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, s);
-  if (dh == 128) return fa_bwd_launch<128>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, s);
+  if (dh == 32) return fa_bwd_launch<32>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s);
+  if (dh == 64) return fa_bwd_launch<64>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s);
+  if (dh == 128) return fa_bwd_launch<128>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s);
   return PCM_ERR_SHAPE;
 }
 

@@ -39,7 +39,40 @@ struct TcParams {
   const float* R; long long ldr;
   int reduce;                                 // 1: fp32 reduction into C
   int a_kmajor, b_kmajor;
+  // fused epilogues (see GemmEpilogue)
+  const __nv_bfloat16* aux; long long ld_aux;
+  __nv_bfloat16* out2; long long ld_out2;
+  const float2* rope_tab; int S, dh, d;
+  int up_row0;                                // EPI_SWIGLU_FWD: first "up" row of B (= F)
 };
+
+__device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(v[8 * e], v[8 * e + 1]);
+    __nv_bfloat162 h1 = __floats2bfloat162_rn(v[8 * e + 2], v[8 * e + 3]);
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * e + 4], v[8 * e + 5]);
+    __nv_bfloat162 h3 = __floats2bfloat162_rn(v[8 * e + 6], v[8 * e + 7]);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+    o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+    d4[e] = o;
+  }
+}
+__device__ __forceinline__ void load_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const uint4 raw = s4[e];
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(h[j]);
+      v[8 * e + 2 * j] = f.x; v[8 * e + 2 * j + 1] = f.y;
+    }
+  }
+}
 
 // Shared-memory matrix descriptor (tcgen05): start address, leading / stride byte offsets in
 // 16-byte units, descriptor version 1, 128-byte swizzle.
@@ -67,7 +100,7 @@ struct TcSmem {
   static constexpr int TOTAL = TC_STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
 
-template <int BN>
+template <int BN, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -128,7 +161,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
             for (int b = 0; b < TC_BM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, m0 + b * 64, k0, &full[st]);  // box {64 m, 64 k}
           }
-          if (p.b_kmajor) {
+          if (EPI == EPI_SWIGLU_FWD) {
+            // n0 counts accumulator columns (256 per tile = 128 hidden units): gate rows, then the matching up rows
+            tma_load_2d(sb, &tmB, k0, n0 / 2, &full[st]);                 // box {64 k, 128 n}
+            tma_load_2d(sb + 128 * 128, &tmB, k0, p.up_row0 + n0 / 2, &full[st]);
+          } else if (p.b_kmajor) {
             tma_load_2d(sb, &tmB, k0, n0, &full[st]);                     // box {64 k, BN n}
           } else {
 #pragma unroll
@@ -192,6 +229,62 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       tc_fence_after();
       const uint32_t tmem_acc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
+      if constexpr (EPI == EPI_SWIGLU_FWD) {
+        // accumulator columns [0,128) = gate, [128,256) = up, for hidden units hid0 .. hid0+127
+        const int hid0 = n0 / 2, F = p.up_row0;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          if (hid0 + c0 >= F) break;
+          uint32_t rg[32], ru[32];
+          tmem_ld_32x32(tmem_acc + (uint32_t)c0, rg);
+          tmem_ld_32x32(tmem_acc + (uint32_t)(128 + c0), ru);
+          tmem_ld_wait();
+          if (row < p.M) {
+            float g[32], u[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) { g[e] = __uint_as_float(rg[e]); u[e] = __uint_as_float(ru[e]); }
+            __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + hid0 + c0;
+            store_bf16x32(gu, g);
+            store_bf16x32(gu + F, u);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+            store_bf16x32(p.out2 + (long long)row * p.ld_out2 + hid0 + c0, g);
+          }
+        }
+      } else if constexpr (EPI == EPI_ROPE) {
+        const int half = p.dh / 2;
+        const int pos = row % p.S;
+#pragma unroll 1
+        for (int h0 = 0; h0 < BN; h0 += p.dh) {          // heads inside the tile
+          if (n0 + h0 >= p.N) break;
+          const bool rotate = n0 + h0 < 2 * p.d;          // q and k regions; v passes through
+#pragma unroll 1
+          for (int ic = 0; ic < half; ic += 32) {
+            uint32_t rl[32], rh[32];
+            tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + ic), rl);
+            tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + half + ic), rh);
+            tmem_ld_wait();
+            if (row < p.M) {
+              float lo[32], hi[32];
+#pragma unroll
+              for (int e = 0; e < 32; ++e) { lo[e] = __uint_as_float(rl[e]); hi[e] = __uint_as_float(rh[e]); }
+              if (rotate) {
+                const float2* cs = p.rope_tab + (long long)pos * half + ic;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                  const float2 t = cs[e];
+                  const float x = lo[e], y = hi[e];
+                  lo[e] = x * t.x - y * t.y;
+                  hi[e] = y * t.x + x * t.y;
+                }
+              }
+              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + n0 + h0 + ic;
+              store_bf16x32(dst, lo);
+              store_bf16x32(dst + half, hi);
+            }
+          }
+        }
+      } else {
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         const int col = n0 + c0;
@@ -200,7 +293,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
         tmem_ld_wait();
         if (row < p.M) {
-          if (p.reduce) {
+          if constexpr (EPI == EPI_SWIGLU_BWD) {
+            // r = d(act) in fp32; gate | up come from aux; d(gate) | d(up) go to C
+            const int F = p.N;
+            float g[32], u[32];
+            const __nv_bfloat16* gu = p.aux + (long long)row * p.ld_aux + col;
+            load_bf16x32(gu, g);
+            load_bf16x32(gu + F, u);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float da = __uint_as_float(r[e]);
+              const float sg = 1.f / (1.f + __expf(-g[e]));
+              const float dg = da * u[e] * sg * (1.f + g[e] * (1.f - sg));
+              u[e] = da * g[e] * sg;
+              g[e] = dg;
+            }
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col;
+            store_bf16x32(dst, g);
+            store_bf16x32(dst + F, u);
+          } else if (p.reduce) {
             float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
 #pragma unroll
             for (int e = 0; e < 32; e += 4)
@@ -223,21 +334,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
               for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
             } else {
-              uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col);
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                __nv_bfloat162 h0 = __floats2bfloat162_rn(v[8 * e], v[8 * e + 1]);
-                __nv_bfloat162 h1 = __floats2bfloat162_rn(v[8 * e + 2], v[8 * e + 3]);
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * e + 4], v[8 * e + 5]);
-                __nv_bfloat162 h3 = __floats2bfloat162_rn(v[8 * e + 6], v[8 * e + 7]);
-                uint4 o;
-                o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
-                o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
-                dst[e] = o;
-              }
+              store_bf16x32(reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v);
             }
           }
         }
+      }
       }
       // hand the accumulator buffer back to the MMA issuer
       tc_fence_before();
@@ -317,13 +418,14 @@ static int sm_count() {
   return n;
 }
 
-template <int BN>
+template <int BN, int EPI>
 static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   CUtensorMap tmA, tmB;
+  constexpr int B_BOX_ROWS = (EPI == EPI_SWIGLU_FWD) ? 128 : BN;
   // K-major operand: tensor [MN][K] -> box {64 k, rows}.  MN-major operand: tensor [K][MN] -> box {64 mn, 64 k}.
   const bool okA = g.a_kmajor ? make_tmap(&tmA, g.A, g.M, g.K, g.lda, TC_BK, TC_BM)
                               : make_tmap(&tmA, g.A, g.K, g.M, g.lda, 64, TC_BK);
-  const bool okB = g.b_kmajor ? make_tmap(&tmB, g.B, g.N, g.K, g.ldb, TC_BK, BN)
+  const bool okB = g.b_kmajor ? make_tmap(&tmB, g.B, g.N, g.K, g.ldb, TC_BK, B_BOX_ROWS)
                               : make_tmap(&tmB, g.B, g.K, g.N, g.ldb, 64, TC_BK);
   if (!okA || !okB) return PCM_ERR_CUDA;
   TcParams p;
@@ -332,6 +434,10 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   p.reduce = (g.R && (const void*)g.R == (const void*)g.C) ? 1 : 0;
   p.R = p.reduce ? nullptr : g.R; p.ldr = g.ldr;
   p.a_kmajor = g.a_kmajor; p.b_kmajor = g.b_kmajor;
+  p.aux = (const __nv_bfloat16*)g.epi.aux; p.ld_aux = g.epi.ld_aux;
+  p.out2 = (__nv_bfloat16*)g.epi.out2; p.ld_out2 = g.epi.ld_out2;
+  p.rope_tab = g.epi.rope_tab; p.S = g.epi.S; p.dh = g.epi.dh; p.d = g.epi.d;
+  p.up_row0 = g.N / 2;
   const int tiles_m = (g.M + TC_BM - 1) / TC_BM, tiles_n = (g.N + BN - 1) / BN;
   const int num_kb = (g.K + TC_BK - 1) / TC_BK;
   int splits = 1;
@@ -347,20 +453,41 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;          // no empty split
   static bool attr_done = false;
   if (!attr_done) {
-    PCM_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<BN>::TOTAL));
+    PCM_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<BN>::TOTAL));
     attr_done = true;
   }
   p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits;
   const long long total = (long long)tiles_m * tiles_n * splits;
   const int grid = (int)(total < sm_count() ? total : sm_count());      // persistent: one CTA per SM walks the tile list
-  gemm_tc_kernel<BN><<<grid, TC_THREADS, TcSmem<BN>::TOTAL, s>>>(tmA, tmB, p);
+  gemm_tc_kernel<BN, EPI><<<grid, TC_THREADS, TcSmem<BN>::TOTAL, s>>>(tmA, tmB, p);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
 }
 
+bool gemm_epilogue_supported(const GemmArgs& g) {
+  if (!gemm_tcgen05_supported(g) || g.c_dtype != DT_BF16 || g.R) return false;
+  const GemmEpilogue& e = g.epi;
+  switch (e.kind) {
+    case EPI_NONE: return true;
+    case EPI_SWIGLU_FWD:   // N = 2F accumulator columns; tiles of 128 hidden units
+      return g.b_kmajor && (g.N % 256 == 0) && e.out2 && (e.ld_out2 % 8 == 0) && !(((uintptr_t)e.out2) & 15);
+    case EPI_SWIGLU_BWD:   // N = F
+      return e.aux && (e.ld_aux % 8 == 0) && !(((uintptr_t)e.aux) & 15) && (g.N % 32 == 0);
+    case EPI_ROPE:
+      return e.rope_tab && (e.dh == 64 || e.dh == 128) && e.S > 0 && e.d > 0 && (e.d % 256 == 0) && g.N == 3 * e.d;
+  }
+  return false;
+}
+
 int gemm_tcgen05(const GemmArgs& g, cudaStream_t s) {
-  if (g.N % 256 == 0 || g.N > 256) return launch_tc<256>(g, s);
-  return launch_tc<128>(g, s);
+  switch (g.epi.kind) {
+    case EPI_SWIGLU_FWD: return gemm_epilogue_supported(g) ? launch_tc<256, EPI_SWIGLU_FWD>(g, s) : PCM_ERR_SHAPE;
+    case EPI_SWIGLU_BWD: return gemm_epilogue_supported(g) ? launch_tc<256, EPI_SWIGLU_BWD>(g, s) : PCM_ERR_SHAPE;
+    case EPI_ROPE: return gemm_epilogue_supported(g) ? launch_tc<256, EPI_ROPE>(g, s) : PCM_ERR_SHAPE;
+    default: break;
+  }
+  if (g.N % 256 == 0 || g.N > 256) return launch_tc<256, EPI_NONE>(g, s);
+  return launch_tc<128, EPI_NONE>(g, s);
 }
 
 int tcgen05_poll_status() {

@@ -10,6 +10,22 @@ enum { DT_F32 = 0, DT_BF16 = 1 };
 // An operand is "K-major" when its contraction index is contiguous in memory:
 //   a_kmajor: A stored [M][K] with row stride lda;   otherwise A stored [K][M] with row stride lda.
 //   b_kmajor: B stored [N][K] with row stride ldb;   otherwise B stored [K][N] with row stride ldb.
+// Work fused into the tensor-core GEMM's epilogue (ignored by the SIMT kernel: callers use it only
+// when gemm_tcgen05_supported() holds).
+enum { EPI_NONE = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2, EPI_ROPE = 3 };
+struct GemmEpilogue {
+  int kind = EPI_NONE;
+  // EPI_SWIGLU_FWD: B is [2F][K] (gate rows, then up rows); C receives gate | up as [M][2F] and
+  //                 out2 [M][F] receives silu(gate) * up, both from the fp32 accumulators.
+  // EPI_SWIGLU_BWD: the product is d(act) [M][F]; aux = gate | up [M][2F]; C [M][2F] receives
+  //                 d(gate) | d(up); d(act) itself is never stored.
+  // EPI_ROPE:       C = q | k | v [M][3d]; columns below 2d are rotated (pairs (i, i + dh/2) of each
+  //                 head, position = row % S) with the (cos, sin) table before the bf16 store.
+  const void* aux = nullptr; long long ld_aux = 0;
+  void* out2 = nullptr; long long ld_out2 = 0;
+  const float2* rope_tab = nullptr; int S = 0, dh = 0, d = 0;
+};
+
 struct GemmArgs {
   int M, N, K;
   const void* A; long long lda; bool a_kmajor;
@@ -17,6 +33,7 @@ struct GemmArgs {
   int ab_dtype;                 // DT_F32 or DT_BF16 (both operands)
   void* C; long long ldc; int c_dtype;
   const float* R; long long ldr;
+  GemmEpilogue epi;
 };
 
 enum GemmBackend { GEMM_AUTO = 0, GEMM_SIMT = 1, GEMM_TCGEN05 = 2 };
@@ -25,6 +42,8 @@ int gemm(const GemmArgs& g, cudaStream_t s, GemmBackend backend = GEMM_AUTO);
 int gemm_simt(const GemmArgs& g, cudaStream_t s);
 int gemm_tcgen05(const GemmArgs& g, cudaStream_t s);
 bool gemm_tcgen05_supported(const GemmArgs& g);
+// True when the tensor-core kernel can run g including its fused epilogue.
+bool gemm_epilogue_supported(const GemmArgs& g);
 // Reads and clears the tensor-core kernels' device status word (synchronous copy).
 int tcgen05_poll_status();
 
@@ -32,12 +51,14 @@ int tcgen05_poll_status();
 // inside each), out [n_seq*S][d], lse [n_seq][H][S].
 int attention_fwd(int dtype, const void* qkv, void* out, float* lse, int n_seq, int S, int H, int dh,
                   cudaStream_t s);
-// dqkv [n_seq*S][3d] receives dq | dk | dv.  dsum [n_seq][H][S] is scratch.
+// dqkv [n_seq*S][3d] receives dq | dk | dv.  dsum [n_seq][H][S] is scratch.  With rope_tab (bf16 only:
+// the [S][dh/2] table of (cos, sin)) dq and dk are rotated back, i.e. they are the gradients with
+// respect to q and k before the rotary embedding.
 int attention_bwd(int dtype, const void* qkv, const void* out, const void* dout, const float* lse, float* dsum,
-                  void* dqkv, int n_seq, int S, int H, int dh, cudaStream_t s);
+                  void* dqkv, int n_seq, int S, int H, int dh, cudaStream_t s, const float2* rope_tab = nullptr);
 
 // Event-pair profiling (profile.cu).  prof_begin/prof_end nest like a stack and cost nothing when off.
-enum { PC_GEMM = 0, PC_ATTN = 1, PC_NORM = 2, PC_ELEM = 3, PC_LOSS = 4, PC_EMBED = 5, PC_PACK = 6, PC_PCM = 7 };
+enum { PC_GEMM = 0, PC_ATTN = 1, PC_NORM = 2, PC_ELEM = 3, PC_LOSS = 4, PC_EMBED = 5, PC_PACK = 6, PC_SCORE = 7, PC_SAMPLE = 8 };
 bool prof_enabled();
 void prof_begin(int cls, cudaStream_t s);
 void prof_end(cudaStream_t s, double flops, double bytes);

@@ -457,7 +457,7 @@ int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* b, double* C, uint8_t* valid
   cudaStream_t s = (cudaStream_t)stream;
   const int G = ctx->cfg.group_size, Kc = ctx->cfg.n_phases, ng = b->n_traj / G;
   const size_t smem = (size_t)Kc * 2 * (ACT + 1) * sizeof(unsigned);
-  prof_begin(PC_PCM, s);
+  prof_begin(PC_SCORE, s);
   score_groups_kernel<<<ng, 256, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, G, Kc, ctx->c_group,
                                              ctx->valid_group, ctx->status);
   PCM_LAUNCH_CHECK();
@@ -492,7 +492,7 @@ int pcm_sample_chunks(pcm_ctx* ctx, const pcm_batch* b, const uint32_t* q, uint6
   const size_t smem = (size_t)warps * b->max_len * sizeof(unsigned);
   if (smem > 48 * 1024)
     PCM_CUDA_TRY(cudaFuncSetAttribute(sample_chunks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  prof_begin(PC_PCM, s);
+  prof_begin(PC_SAMPLE, s);
   sample_chunks_kernel<<<ceil_div(b->n_traj, warps), warps * 32, smem, s>>>(
       b->traj_off, b->phase, q, b->n_traj, ctx->cfg.n_phases, ctx->cfg.budget, b->max_len,
       (uint32_t)(ctx->cfg.seed & 0xFFFFFFFFu), (uint32_t)(ctx->cfg.seed >> 32), (uint32_t)(iter & 0xFFFFFFFFu),

@@ -84,13 +84,16 @@ def bench_pcm(a):
         if it == 2:
             B.pcm_profile_read()          # drop the warm-up iterations
     B.pcm_profile_enable(False)
-    prof = B.pcm_profile_read()["pcm"]
+    prof_all = B.pcm_profile_read()
+    prof, prof_s = prof_all["pcm_score"], prof_all["pcm_sample"]
     ms_score = _time(lambda: B.pcm_score_phases(ctx, batch), a.iters)
     ms_sample = _time(lambda: B.pcm_sample_chunks(ctx, batch, q, 1, out=out), a.iters)
     print(json.dumps({"kernel": "pcm", "n_traj": n_traj, "chunks": total, "input_bytes": total * 57,
                       "score_ms": ms_score, "score_gbs": total * 57 / (ms_score * 1e6),
                       "sample_ms": ms_sample, "sample_gbs": (total + 4 * n_traj * a.budget) / (ms_sample * 1e6),
-                      "event_pairs_gbs": prof["bytes"] / (prof["ms"] * 1e6) if prof["ms"] > 0 else None,
+                      "score_groups_kernel_ms": prof["ms"] / max(1, prof["launches"]),
+                      "score_groups_kernel_gbs": prof["bytes"] / (prof["ms"] * 1e6) if prof["ms"] > 0 else None,
+                      "sample_kernel_ms": prof_s["ms"] / max(1, prof_s["launches"]),
                       "status": B.pcm_poll_status(ctx)}))
     ctx.close()
 
