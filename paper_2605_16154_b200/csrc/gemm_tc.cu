@@ -13,8 +13,8 @@
 // Persistent: one CTA per SM walks a static list of output tiles; the shared-memory ring keeps
 // flowing across tile boundaries and the accumulator is double-buffered in tensor memory, so the
 // epilogue of one tile overlaps the MMAs of the next.
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = tensor-memory allocation + MMA issue,
-// warps 2..5 = epilogue.  Every mbarrier wait is bounded; when one runs out the CTA sets a status
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = tensor-memory allocation + MMA issue,
+// warps 2..9 = epilogue (two per tensor-memory lane quadrant, splitting the tile's columns).  Every mbarrier wait is bounded; when one runs out the CTA sets a status
 // flag, all roles leave their loops, tensor memory is released and the kernel returns.
 #include <cuda.h>
 
@@ -26,7 +26,8 @@ namespace pcm {
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                     // 64 bf16 = one 128-byte swizzle row
 constexpr int TC_STAGES = 4;
-constexpr int TC_THREADS = 192;
+constexpr int TC_EPI_WARPS = 8;                // two per tensor-memory lane quadrant, each takes half of the columns
+constexpr int TC_THREADS = 320;               // producer warp, MMA warp, 8 epilogue warps
 constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per mbarrier wait
 
 __device__ unsigned g_tc_status = 0;          // bit 0: a bounded wait expired
@@ -58,6 +59,22 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&
     o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
     o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
     d4[e] = o;
+  }
+}
+__device__ __forceinline__ void fetch_bf16x32(const __nv_bfloat16* src, uint4 (&raw)[4]) {
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) raw[e] = s4[e];
+}
+__device__ __forceinline__ void unpack_bf16x32(const uint4 (&raw)[4], float (&v)[32]) {
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw[e]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(h[j]);
+      v[8 * e + 2 * j] = f.x; v[8 * e + 2 * j + 1] = f.y;
+    }
   }
 }
 __device__ __forceinline__ void load_bf16x32(const __nv_bfloat16* src, float (&v)[32]) {
@@ -122,7 +139,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], TC_EPI_WARPS); }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmA);
@@ -212,14 +229,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
     }
   } else {
-    // ------------------------------ epilogue: warps 2..5 ------------------------------
+    // ------------------------------ epilogue: warps 2..9 ------------------------------
     const int quad = warp & 3;                // tensor-memory lane quadrant this warp may access
+    const int chalf = (warp - 2) >> 2;        // which half of the tile's columns this warp handles
     unsigned tcount = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
       const int split = tile / tiles_mn, mn = tile - split * tiles_mn;
       const int m0 = (mn / p.tiles_n) * TC_BM, n0 = (mn % p.tiles_n) * BN;
       const int row = m0 + quad * 32 + lane;
       const unsigned ab = tcount & 1u, aph = (tcount >> 1) & 1u;
+      uint4 pre_g[4], pre_u[4];               // EPI_SWIGLU_BWD: gate / up of the next 32 columns, fetched ahead of use
+      if constexpr (EPI == EPI_SWIGLU_BWD) {
+        const int col0 = n0 + chalf * (BN / 2);
+        if (row < p.M && col0 < p.N) {
+          const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col0;
+          fetch_bf16x32(nx, pre_g);           // issued before waiting for the accumulator
+          fetch_bf16x32(nx + p.N, pre_u);
+        }
+      }
+      float4 pre_r[8];                        // residual of the next 32 columns, fetched ahead of use
+      if constexpr (EPI == EPI_NONE) {
+        const int col0 = n0 + chalf * (BN / 2);
+        if (p.R && row < p.M && col0 < p.N) {
+          const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col0);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) pre_r[e] = rp[e];
+        }
+      }
       int ok = 1;
       if (lane == 0) {
         ok = (!*abort_flag && mbar_wait_bounded(&acc_full[ab], aph, TC_WAIT_LIMIT_NS * 2ull)) ? 1 : 0;
@@ -233,7 +269,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // accumulator columns [0,128) = gate, [128,256) = up, for hidden units hid0 .. hid0+127
         const int hid0 = n0 / 2, F = p.up_row0;
 #pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
+        for (int c0 = chalf * 64; c0 < chalf * 64 + 64; c0 += 32) {
           if (hid0 + c0 >= F) break;
           uint32_t rg[32], ru[32];
           tmem_ld_32x32(tmem_acc + (uint32_t)c0, rg);
@@ -252,14 +288,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       } else if constexpr (EPI == EPI_ROPE) {
+        // every head of a row uses the same (cos, sin) values: load them once per 32-pair slice and
+        // reuse them for all heads of this warp's half of the tile
         const int half = p.dh / 2;
         const int pos = row % p.S;
 #pragma unroll 1
-        for (int h0 = 0; h0 < BN; h0 += p.dh) {          // heads inside the tile
-          if (n0 + h0 >= p.N) break;
-          const bool rotate = n0 + h0 < 2 * p.d;          // q and k regions; v passes through
+        for (int ic = 0; ic < half; ic += 32) {
+          float2 cs[32];
+          {
+            const float4* tp = reinterpret_cast<const float4*>(p.rope_tab + (long long)pos * half + ic);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float4 t4 = tp[e];
+              cs[2 * e] = make_float2(t4.x, t4.y);
+              cs[2 * e + 1] = make_float2(t4.z, t4.w);
+            }
+          }
 #pragma unroll 1
-          for (int ic = 0; ic < half; ic += 32) {
+          for (int h0 = chalf * (BN / 2); h0 < (chalf + 1) * (BN / 2); h0 += p.dh) {   // heads inside this warp's half
+            if (n0 + h0 >= p.N) break;
+            const bool rotate = n0 + h0 < 2 * p.d;        // q and k regions; v passes through
             uint32_t rl[32], rh[32];
             tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + ic), rl);
             tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + half + ic), rh);
@@ -269,13 +317,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
               for (int e = 0; e < 32; ++e) { lo[e] = __uint_as_float(rl[e]); hi[e] = __uint_as_float(rh[e]); }
               if (rotate) {
-                const float2* cs = p.rope_tab + (long long)pos * half + ic;
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                  const float2 t = cs[e];
                   const float x = lo[e], y = hi[e];
-                  lo[e] = x * t.x - y * t.y;
-                  hi[e] = y * t.x + x * t.y;
+                  lo[e] = x * cs[e].x - y * cs[e].y;
+                  hi[e] = y * cs[e].x + x * cs[e].y;
                 }
               }
               __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + n0 + h0 + ic;
@@ -286,7 +332,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       } else {
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
         const int col = n0 + c0;
         if (col >= p.N) break;                // warp-uniform: N is a multiple of 32 on this path
         uint32_t r[32];
@@ -294,12 +340,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_ld_wait();
         if (row < p.M) {
           if constexpr (EPI == EPI_SWIGLU_BWD) {
-            // r = d(act) in fp32; gate | up come from aux; d(gate) | d(up) go to C
+            // r = d(act) in fp32; gate | up come from aux (fetched one chunk ahead); d(gate) | d(up) go to C
             const int F = p.N;
             float g[32], u[32];
-            const __nv_bfloat16* gu = p.aux + (long long)row * p.ld_aux + col;
-            load_bf16x32(gu, g);
-            load_bf16x32(gu + F, u);
+            unpack_bf16x32(pre_g, g);
+            unpack_bf16x32(pre_u, u);
+            if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
+              const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col + 32;
+              fetch_bf16x32(nx, pre_g);
+              fetch_bf16x32(nx + F, pre_u);
+            }
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
               const float da = __uint_as_float(r[e]);
@@ -322,11 +372,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
             for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
             if (p.R) {
-              const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col);
 #pragma unroll
               for (int e = 0; e < 8; ++e) {
-                const float4 t = rp[e];
-                v[4 * e] += t.x; v[4 * e + 1] += t.y; v[4 * e + 2] += t.z; v[4 * e + 3] += t.w;
+                v[4 * e] += pre_r[e].x; v[4 * e + 1] += pre_r[e].y; v[4 * e + 2] += pre_r[e].z; v[4 * e + 3] += pre_r[e].w;
+              }
+              if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
+                const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col + 32);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) pre_r[e] = rp[e];
               }
             }
             if (p.c_dtype == DT_F32) {

@@ -90,26 +90,26 @@ def test_sampled_log_probs_and_batch_properties_at_full_size(c1):
         assert rel_fro(halves[k].cpu().numpy(), g_full[k].cpu().numpy()) < 2e-3, k
 
 
-def test_two_chunk_update_of_the_full_model_against_the_oracle(c1):
+def test_eight_chunk_update_of_the_full_model_against_the_oracle(c1):
     """Every kernel at the medium model's real width, depth and sequence length (8 layers, d = 1024,
     S = 312), on a batch small enough for the fp64 oracle."""
     B, PL, w, model, pk = c1["B"], c1["PL"], c1["w"], c1["model"], c1["pk"]
-    sel = [5, 250]
+    sel = [5, 60, 111, 170, 250, 300, 340, 380]
     X = pk.X[sel].float().cpu().numpy()
     tgt = pk.tgt[sel].cpu().numpy()
-    adv_c = np.array([0.8, -1.2], dtype=np.float32)               # both signs, whatever the sampled rewards were
+    adv_c = np.array([1.0, -1.0] * 4, dtype=np.float32)           # zero-mean like a rollout group's advantages
     lp_o = ao.logp_only(c1["weights"], X, tgt, w.H, w.P)
-    noise = synth.logp_noise(11, 2, 0.1).astype(np.float64)
+    noise = synth.logp_noise(11, len(sel), 0.1).astype(np.float64)
     hi, lo, m = np.log(1.2), np.log(0.8), 0.05
     log_r = -noise
     log_r = np.where(np.abs(log_r - hi) < m, hi + 2 * m * np.sign(log_r - hi + 1e-30), log_r)
     log_r = np.where(np.abs(log_r - lo) < m, lo + 2 * m * np.sign(log_r - lo + 1e-30), log_r)
     lpo = (lp_o - log_r).astype(np.float32)
     loss_o, _, grads_o, stats_o = ao.fwd_bwd(c1["weights"], X, tgt, lpo, adv_c, w.H, w.P, 0.2, 0.2)
-    sub = B.Packed(model, 2)
+    sub = B.Packed(model, len(sel))
     sub.X.copy_(pk.X[sel]); sub.tgt.copy_(pk.tgt[sel]); sub.lpo.copy_(PL.dev(lpo)); sub.adv_c.copy_(PL.dev(adv_c))
     loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, sub)
+    errs = {k: rel_fro(v, grads_o[k]) for k, v in grads_to_numpy(grads).items()}
+    assert max(errs.values()) < 2e-2, (errs, float(loss.item()), loss_o)
     assert abs(float(loss.item()) - loss_o) < 1e-3
     assert stats.clip_frac == pytest.approx(stats_o["clip_frac"], abs=1e-6)
-    errs = {k: rel_fro(v, grads_o[k]) for k, v in grads_to_numpy(grads).items()}
-    assert max(errs.values()) < 2e-2, errs
