@@ -18,6 +18,8 @@
 // flag, all roles leave their loops, tensor memory is released and the kernel returns.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "async_ptx.cuh"
 #include "internal.h"
 
@@ -116,6 +118,166 @@ struct TcSmem {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TOTAL = TC_STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
+
+// Operands of the epilogue that are fetched one 32-column slice ahead of their use.
+struct EpiRegs {
+  uint4 g[4], u[4];                           // EPI_SWIGLU_BWD: gate / up
+  float4 r[8];                                // fp32 residual
+};
+
+// Issued before the wait for the accumulator, so that the first slice's loads overlap it.
+template <int BN, int EPI>
+__device__ __forceinline__ void epi_prefetch(const TcParams& p, int row, int n0, int chalf, EpiRegs& pre) {
+      if constexpr (EPI == EPI_SWIGLU_BWD) {
+        const int col0 = n0 + chalf * (BN / 2);
+        if (row < p.M && col0 < p.N) {
+          const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col0;
+          fetch_bf16x32(nx, pre.g);           // issued before waiting for the accumulator
+          fetch_bf16x32(nx + p.N, pre.u);
+        }
+      }
+      if constexpr (EPI == EPI_NONE) {
+        const int col0 = n0 + chalf * (BN / 2);
+        if (p.R && row < p.M && col0 < p.N) {
+          const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col0);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) pre.r[e] = rp[e];
+        }
+      }
+}
+
+// One epilogue warp's share of a tile: rows = this warp's 32 tensor-memory lanes, columns = its half of the tile.
+template <int BN, int EPI>
+__device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, int row, int n0, int chalf, EpiRegs& pre) {
+      if constexpr (EPI == EPI_SWIGLU_FWD) {
+        // accumulator columns [0,128) = gate, [128,256) = up, for hidden units hid0 .. hid0+127
+        const int hid0 = n0 / 2, F = p.up_row0;
+#pragma unroll 1
+        for (int c0 = chalf * 64; c0 < chalf * 64 + 64; c0 += 32) {
+          if (hid0 + c0 >= F) break;
+          uint32_t rg[32], ru[32];
+          tmem_ld_32x32(tmem_acc + (uint32_t)c0, rg);
+          tmem_ld_32x32(tmem_acc + (uint32_t)(128 + c0), ru);
+          tmem_ld_wait();
+          if (row < p.M) {
+            float g[32], u[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) { g[e] = __uint_as_float(rg[e]); u[e] = __uint_as_float(ru[e]); }
+            __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + hid0 + c0;
+            store_bf16x32(gu, g);
+            store_bf16x32(gu + F, u);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
+            store_bf16x32(p.out2 + (long long)row * p.ld_out2 + hid0 + c0, g);
+          }
+        }
+      } else if constexpr (EPI == EPI_ROPE) {
+        // every head of a row uses the same (cos, sin) values: load them once per 32-pair slice and
+        // reuse them for all heads of this warp's half of the tile
+        const int half = p.dh / 2;
+        const int pos = row % p.S;
+#pragma unroll 1
+        for (int ic = 0; ic < half; ic += 32) {
+          float2 cs[32];
+          {
+            const float4* tp = reinterpret_cast<const float4*>(p.rope_tab + (long long)pos * half + ic);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float4 t4 = tp[e];
+              cs[2 * e] = make_float2(t4.x, t4.y);
+              cs[2 * e + 1] = make_float2(t4.z, t4.w);
+            }
+          }
+#pragma unroll 1
+          for (int h0 = chalf * (BN / 2); h0 < (chalf + 1) * (BN / 2); h0 += p.dh) {   // heads inside this warp's half
+            if (n0 + h0 >= p.N) break;
+            const bool rotate = n0 + h0 < 2 * p.d;        // q and k regions; v passes through
+            uint32_t rl[32], rh[32];
+            tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + ic), rl);
+            tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + half + ic), rh);
+            tmem_ld_wait();
+            if (row < p.M) {
+              float lo[32], hi[32];
+#pragma unroll
+              for (int e = 0; e < 32; ++e) { lo[e] = __uint_as_float(rl[e]); hi[e] = __uint_as_float(rh[e]); }
+              if (rotate) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                  const float x = lo[e], y = hi[e];
+                  lo[e] = x * cs[e].x - y * cs[e].y;
+                  hi[e] = y * cs[e].x + x * cs[e].y;
+                }
+              }
+              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + n0 + h0 + ic;
+              store_bf16x32(dst, lo);
+              store_bf16x32(dst + half, hi);
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+      for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
+        const int col = n0 + c0;
+        if (col >= p.N) break;                // warp-uniform: N is a multiple of 32 on this path
+        uint32_t r[32];
+        tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
+        tmem_ld_wait();
+        if (row < p.M) {
+          if constexpr (EPI == EPI_SWIGLU_BWD) {
+            // r = d(act) in fp32; gate | up come from aux (fetched one chunk ahead); d(gate) | d(up) go to C
+            const int F = p.N;
+            float g[32], u[32];
+            unpack_bf16x32(pre.g, g);
+            unpack_bf16x32(pre.u, u);
+            if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
+              const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col + 32;
+              fetch_bf16x32(nx, pre.g);
+              fetch_bf16x32(nx + F, pre.u);
+            }
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float da = __uint_as_float(r[e]);
+              const float sg = 1.f / (1.f + __expf(-g[e]));
+              const float dg = da * u[e] * sg * (1.f + g[e] * (1.f - sg));
+              u[e] = da * g[e] * sg;
+              g[e] = dg;
+            }
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col;
+            store_bf16x32(dst, g);
+            store_bf16x32(dst + F, u);
+          } else if (p.reduce) {
+            float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              red_add_v4(dst + e, __uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
+                         __uint_as_float(r[e + 3]));
+          } else {
+            float v[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
+            if (p.R) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                v[4 * e] += pre.r[e].x; v[4 * e + 1] += pre.r[e].y; v[4 * e + 2] += pre.r[e].z; v[4 * e + 3] += pre.r[e].w;
+              }
+              if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
+                const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col + 32);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) pre.r[e] = rp[e];
+              }
+            }
+            if (p.c_dtype == DT_F32) {
+              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+            } else {
+              store_bf16x32(reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v);
+            }
+          }
+        }
+      }
+      }
+}
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -238,24 +400,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int m0 = (mn / p.tiles_n) * TC_BM, n0 = (mn % p.tiles_n) * BN;
       const int row = m0 + quad * 32 + lane;
       const unsigned ab = tcount & 1u, aph = (tcount >> 1) & 1u;
-      uint4 pre_g[4], pre_u[4];               // EPI_SWIGLU_BWD: gate / up of the next 32 columns, fetched ahead of use
-      if constexpr (EPI == EPI_SWIGLU_BWD) {
-        const int col0 = n0 + chalf * (BN / 2);
-        if (row < p.M && col0 < p.N) {
-          const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col0;
-          fetch_bf16x32(nx, pre_g);           // issued before waiting for the accumulator
-          fetch_bf16x32(nx + p.N, pre_u);
-        }
-      }
-      float4 pre_r[8];                        // residual of the next 32 columns, fetched ahead of use
-      if constexpr (EPI == EPI_NONE) {
-        const int col0 = n0 + chalf * (BN / 2);
-        if (p.R && row < p.M && col0 < p.N) {
-          const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col0);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) pre_r[e] = rp[e];
-        }
-      }
+      EpiRegs pre;
+      epi_prefetch<BN, EPI>(p, row, n0, chalf, pre);
       int ok = 1;
       if (lane == 0) {
         ok = (!*abort_flag && mbar_wait_bounded(&acc_full[ab], aph, TC_WAIT_LIMIT_NS * 2ull)) ? 1 : 0;
@@ -265,134 +411,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       tc_fence_after();
       const uint32_t tmem_acc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
-      if constexpr (EPI == EPI_SWIGLU_FWD) {
-        // accumulator columns [0,128) = gate, [128,256) = up, for hidden units hid0 .. hid0+127
-        const int hid0 = n0 / 2, F = p.up_row0;
-#pragma unroll 1
-        for (int c0 = chalf * 64; c0 < chalf * 64 + 64; c0 += 32) {
-          if (hid0 + c0 >= F) break;
-          uint32_t rg[32], ru[32];
-          tmem_ld_32x32(tmem_acc + (uint32_t)c0, rg);
-          tmem_ld_32x32(tmem_acc + (uint32_t)(128 + c0), ru);
-          tmem_ld_wait();
-          if (row < p.M) {
-            float g[32], u[32];
-#pragma unroll
-            for (int e = 0; e < 32; ++e) { g[e] = __uint_as_float(rg[e]); u[e] = __uint_as_float(ru[e]); }
-            __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + hid0 + c0;
-            store_bf16x32(gu, g);
-            store_bf16x32(gu + F, u);
-#pragma unroll
-            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
-            store_bf16x32(p.out2 + (long long)row * p.ld_out2 + hid0 + c0, g);
-          }
-        }
-      } else if constexpr (EPI == EPI_ROPE) {
-        // every head of a row uses the same (cos, sin) values: load them once per 32-pair slice and
-        // reuse them for all heads of this warp's half of the tile
-        const int half = p.dh / 2;
-        const int pos = row % p.S;
-#pragma unroll 1
-        for (int ic = 0; ic < half; ic += 32) {
-          float2 cs[32];
-          {
-            const float4* tp = reinterpret_cast<const float4*>(p.rope_tab + (long long)pos * half + ic);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float4 t4 = tp[e];
-              cs[2 * e] = make_float2(t4.x, t4.y);
-              cs[2 * e + 1] = make_float2(t4.z, t4.w);
-            }
-          }
-#pragma unroll 1
-          for (int h0 = chalf * (BN / 2); h0 < (chalf + 1) * (BN / 2); h0 += p.dh) {   // heads inside this warp's half
-            if (n0 + h0 >= p.N) break;
-            const bool rotate = n0 + h0 < 2 * p.d;        // q and k regions; v passes through
-            uint32_t rl[32], rh[32];
-            tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + ic), rl);
-            tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + half + ic), rh);
-            tmem_ld_wait();
-            if (row < p.M) {
-              float lo[32], hi[32];
-#pragma unroll
-              for (int e = 0; e < 32; ++e) { lo[e] = __uint_as_float(rl[e]); hi[e] = __uint_as_float(rh[e]); }
-              if (rotate) {
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                  const float x = lo[e], y = hi[e];
-                  lo[e] = x * cs[e].x - y * cs[e].y;
-                  hi[e] = y * cs[e].x + x * cs[e].y;
-                }
-              }
-              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + n0 + h0 + ic;
-              store_bf16x32(dst, lo);
-              store_bf16x32(dst + half, hi);
-            }
-          }
-        }
-      } else {
-#pragma unroll 1
-      for (int c0 = chalf * (BN / 2); c0 < (chalf + 1) * (BN / 2); c0 += 32) {
-        const int col = n0 + c0;
-        if (col >= p.N) break;                // warp-uniform: N is a multiple of 32 on this path
-        uint32_t r[32];
-        tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
-        tmem_ld_wait();
-        if (row < p.M) {
-          if constexpr (EPI == EPI_SWIGLU_BWD) {
-            // r = d(act) in fp32; gate | up come from aux (fetched one chunk ahead); d(gate) | d(up) go to C
-            const int F = p.N;
-            float g[32], u[32];
-            unpack_bf16x32(pre_g, g);
-            unpack_bf16x32(pre_u, u);
-            if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
-              const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col + 32;
-              fetch_bf16x32(nx, pre_g);
-              fetch_bf16x32(nx + F, pre_u);
-            }
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const float da = __uint_as_float(r[e]);
-              const float sg = 1.f / (1.f + __expf(-g[e]));
-              const float dg = da * u[e] * sg * (1.f + g[e] * (1.f - sg));
-              u[e] = da * g[e] * sg;
-              g[e] = dg;
-            }
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col;
-            store_bf16x32(dst, g);
-            store_bf16x32(dst + F, u);
-          } else if (p.reduce) {
-            float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
-#pragma unroll
-            for (int e = 0; e < 32; e += 4)
-              red_add_v4(dst + e, __uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
-                         __uint_as_float(r[e + 3]));
-          } else {
-            float v[32];
-#pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
-            if (p.R) {
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                v[4 * e] += pre_r[e].x; v[4 * e + 1] += pre_r[e].y; v[4 * e + 2] += pre_r[e].z; v[4 * e + 3] += pre_r[e].w;
-              }
-              if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
-                const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col + 32);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) pre_r[e] = rp[e];
-              }
-            }
-            if (p.c_dtype == DT_F32) {
-              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-            } else {
-              store_bf16x32(reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v);
-            }
-          }
-        }
-      }
-      }
+      epi_tile<BN, EPI>(p, tmem_acc, row, n0, chalf, pre);
       // hand the accumulator buffer back to the MMA issuer
       tc_fence_before();
       __syncwarp();
@@ -410,6 +429,180 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// CTA-pair variant: two CTAs of a cluster share one 256 x 256 output tile.  Each CTA stages its own
+// 128 rows of A and one half (128 of the 256 columns) of B, so every byte of B is read into shared
+// memory once per pair instead of once per CTA; the leader CTA issues tcgen05.mma.cta_group::2 and
+// each CTA's tensor memory receives the accumulator rows of its half of the tile.
+//   full[s]      (leader)  <- both producers' TMA bytes + the leader producer's arrival
+//   empty[s]     (each)    <- multicast commit from the leader's MMA thread
+//   acc_full[b]  (each)    <- multicast commit from the leader's MMA thread
+//   acc_empty[b] (leader)  <- the epilogue warps of both CTAs
+// ------------------------------------------------------------------------------------------------
+constexpr int T2_BN = 256;
+constexpr int T2_STAGES = 6;
+constexpr int T2_A_BYTES = TC_BM * TC_BK * 2;          // 16 KB: this CTA's 128 rows of A
+constexpr int T2_B_BYTES = (T2_BN / 2) * TC_BK * 2;    // 16 KB: this CTA's 128 columns of B
+constexpr int T2_STAGE_BYTES = T2_A_BYTES + T2_B_BYTES;
+constexpr int T2_SMEM_TOTAL = T2_STAGES * T2_STAGE_BYTES + 1024 + 256;
+
+template <int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int BN = T2_BN;
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t* tiles = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + T2_STAGES * T2_STAGE_BYTES);
+  uint64_t* full = bars;                       // [T2_STAGES]
+  uint64_t* empty = bars + T2_STAGES;          // [T2_STAGES]
+  uint64_t* acc_full = bars + 2 * T2_STAGES;   // [2]
+  uint64_t* acc_empty = acc_full + 2;          // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int num_kb_total = (p.K + TC_BK - 1) / TC_BK;
+  const int tiles_mn = p.tiles_m * p.tiles_n;  // tiles of 256 x 256
+  const int total_tiles = tiles_mn * p.splits;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < T2_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 2 * TC_EPI_WARPS); }
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, 2 * BN);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                          // the peer's barriers exist before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------ TMA producer (both CTAs) ------------------------------
+      unsigned it = 0;
+      for (int tile = pair; tile < total_tiles && !*abort_flag; tile += n_pairs) {
+        const int split = tile / tiles_mn, mn = tile - split * tiles_mn;
+        const int m0 = (mn / p.tiles_n) * (2 * TC_BM) + (int)rank * TC_BM;      // this CTA's rows
+        const int n0 = (mn % p.tiles_n) * BN;
+        const int nb0 = n0 + (int)rank * (BN / 2);                              // this CTA's columns of B
+        const int kb_lo = split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+          const int st = it % T2_STAGES;
+          const unsigned ph = (it / T2_STAGES) & 1u;
+          if (!mbar_wait_bounded(&empty[st], ph ^ 1u, TC_WAIT_LIMIT_NS)) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); break; }
+          uint8_t* sa = tiles + st * T2_STAGE_BYTES;
+          uint8_t* sb = sa + T2_A_BYTES;
+          const uint32_t bar = mapa_shared(smem_u32(&full[st]), 0);             // the leader's barrier counts both CTAs' bytes
+          if (leader) mbar_expect_tx(&full[st], 2 * T2_STAGE_BYTES);
+          const int k0 = kb * TC_BK;
+          if (p.a_kmajor) {
+            tma_load_2d_pair(sa, &tmA, k0, m0, bar);                            // box {64 k, 128 m}
+          } else {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sa + b * 8192, &tmA, m0 + b * 64, k0, bar);   // box {64 m, 64 k}
+          }
+          if (EPI == EPI_SWIGLU_FWD) {
+            // accumulator columns [0,128) = gate (leader's half of B), [128,256) = up (the peer's half)
+            tma_load_2d_pair(sb, &tmB, k0, (leader ? 0 : p.up_row0) + n0 / 2, bar);                 // box {64 k, 128 n}
+          } else if (p.b_kmajor) {
+            tma_load_2d_pair(sb, &tmB, k0, nb0, bar);                           // box {64 k, 128 n}
+          } else {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sb + b * 8192, &tmB, nb0 + b * 64, k0, bar);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && leader) {
+      // ------------------------------ MMA issuer (leader CTA only) ------------------------------
+      constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                                      ((uint32_t)((2 * TC_BM) >> 4) << 24);
+      const uint32_t idesc = idesc_base | ((p.a_kmajor ? 0u : 1u) << 15) | ((p.b_kmajor ? 0u : 1u) << 16);
+      const uint32_t a_lbo = p.a_kmajor ? 16u : 8192u, b_lbo = p.b_kmajor ? 16u : 8192u;
+      const uint32_t a_step = p.a_kmajor ? 32u : 2048u, b_step = p.b_kmajor ? 32u : 2048u;
+      unsigned it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++tcount) {
+        const int split = tile / tiles_mn;
+        const int kb_lo = split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
+        const unsigned ab = tcount & 1u, aph = (tcount >> 1) & 1u;
+        if (*abort_flag || !mbar_wait_bounded(&acc_empty[ab], aph ^ 1u, TC_WAIT_LIMIT_NS)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_acc = tmem_base + ab * BN;
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+          const int st = it % T2_STAGES;
+          const unsigned ph = (it / T2_STAGES) & 1u;
+          if (*abort_flag || !mbar_wait_bounded(&full[st], ph, TC_WAIT_LIMIT_NS)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(tiles + st * T2_STAGE_BYTES);
+          const uint32_t sb = sa + T2_A_BYTES;
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k) {
+            const uint64_t da = make_smem_desc(sa + k * a_step, a_lbo, 1024u);
+            const uint64_t db = make_smem_desc(sb + k * b_step, b_lbo, 1024u);
+            umma_bf16_pair(tmem_acc, da, db, idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
+          }
+          umma_commit_pair(&empty[st], 3);     // both CTAs may refill the stage
+        }
+        if (ok) umma_commit_pair(&acc_full[ab], 3);
+      }
+      if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
+    }
+  } else {
+    // ------------------------------ epilogue: warps 2..9 of both CTAs ------------------------------
+    const int quad = warp & 3;
+    const int chalf = (warp - 2) >> 2;
+    unsigned tcount = 0;
+    for (int tile = pair; tile < total_tiles; tile += n_pairs, ++tcount) {
+      const int split = tile / tiles_mn, mn = tile - split * tiles_mn;
+      const int m0 = (mn / p.tiles_n) * (2 * TC_BM) + (int)rank * TC_BM, n0 = (mn % p.tiles_n) * BN;
+      const int row = m0 + quad * 32 + lane;
+      const unsigned ab = tcount & 1u, aph = (tcount >> 1) & 1u;
+      EpiRegs pre;
+      epi_prefetch<BN, EPI>(p, row, n0, chalf, pre);
+      int ok = 1;
+      if (lane == 0) {
+        ok = (!*abort_flag && mbar_wait_bounded(&acc_full[ab], aph, TC_WAIT_LIMIT_NS * 2ull)) ? 1 : 0;
+        if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t tmem_acc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
+      epi_tile<BN, EPI>(p, tmem_acc, row, n0, chalf, pre);
+      // hand the accumulator buffer back to the leader's MMA thread
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&acc_empty[ab]), 0));
+    }
+  }
+
+  // teardown: neither CTA may leave while its peer can still touch its shared memory or barriers
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 2 * BN);
   }
 }
 
@@ -461,6 +654,19 @@ bool gemm_tcgen05_supported(const GemmArgs& g) {
     return encode_fn() != nullptr;
 }
 
+static void fill_params(TcParams& p, const GemmArgs& g) {
+  p.M = g.M; p.N = g.N; p.K = g.K;
+  p.C = g.C; p.ldc = g.ldc; p.c_dtype = g.c_dtype;
+  p.reduce = (g.R && (const void*)g.R == (const void*)g.C) ? 1 : 0;
+  p.R = p.reduce ? nullptr : g.R; p.ldr = g.ldr;
+  p.a_kmajor = g.a_kmajor; p.b_kmajor = g.b_kmajor;
+  p.aux = (const __nv_bfloat16*)g.epi.aux; p.ld_aux = g.epi.ld_aux;
+  p.out2 = (__nv_bfloat16*)g.epi.out2; p.ld_out2 = g.epi.ld_out2;
+  p.rope_tab = g.epi.rope_tab; p.S = g.epi.S; p.dh = g.epi.dh; p.d = g.epi.d;
+  p.up_row0 = g.N / 2;
+  p.kb_per_split = 1; p.tiles_m = p.tiles_n = p.splits = 1;
+}
+
 static int sm_count() {
   static int n = 0;
   if (!n) {
@@ -482,15 +688,7 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
                               : make_tmap(&tmB, g.B, g.K, g.N, g.ldb, 64, TC_BK);
   if (!okA || !okB) return PCM_ERR_CUDA;
   TcParams p;
-  p.M = g.M; p.N = g.N; p.K = g.K;
-  p.C = g.C; p.ldc = g.ldc; p.c_dtype = g.c_dtype;
-  p.reduce = (g.R && (const void*)g.R == (const void*)g.C) ? 1 : 0;
-  p.R = p.reduce ? nullptr : g.R; p.ldr = g.ldr;
-  p.a_kmajor = g.a_kmajor; p.b_kmajor = g.b_kmajor;
-  p.aux = (const __nv_bfloat16*)g.epi.aux; p.ld_aux = g.epi.ld_aux;
-  p.out2 = (__nv_bfloat16*)g.epi.out2; p.ld_out2 = g.epi.ld_out2;
-  p.rope_tab = g.epi.rope_tab; p.S = g.epi.S; p.dh = g.epi.dh; p.d = g.epi.d;
-  p.up_row0 = g.N / 2;
+  fill_params(p, g);
   const int tiles_m = (g.M + TC_BM - 1) / TC_BM, tiles_n = (g.N + BN - 1) / BN;
   const int num_kb = (g.K + TC_BK - 1) / TC_BK;
   int splits = 1;
@@ -517,6 +715,65 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   return PCM_OK;
 }
 
+static bool pair_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("PCM_GEMM_PAIR");
+    v = (e && e[0] == '0') ? 0 : 1;
+  }
+  return v == 1;
+}
+
+// CTA-pair launch: 256 x 256 tiles, clusters of two CTAs, one pair per two SMs.
+template <int EPI>
+static int launch_tc2(const GemmArgs& g, cudaStream_t s) {
+  CUtensorMap tmA, tmB;
+  const bool okA = g.a_kmajor ? make_tmap(&tmA, g.A, g.M, g.K, g.lda, TC_BK, TC_BM)
+                              : make_tmap(&tmA, g.A, g.K, g.M, g.lda, 64, TC_BK);
+  const bool okB = g.b_kmajor ? make_tmap(&tmB, g.B, g.N, g.K, g.ldb, TC_BK, T2_BN / 2)
+                              : make_tmap(&tmB, g.B, g.K, g.N, g.ldb, 64, TC_BK);
+  if (!okA || !okB) return PCM_ERR_CUDA;
+  TcParams p;
+  fill_params(p, g);
+  const int tiles_m = (g.M + 2 * TC_BM - 1) / (2 * TC_BM), tiles_n = (g.N + T2_BN - 1) / T2_BN;
+  const int num_kb = (g.K + TC_BK - 1) / TC_BK;
+  const int n_pairs_max = sm_count() / 2;
+  int splits = 1;
+  if (p.reduce) {
+    const long long tiles = (long long)tiles_m * tiles_n;
+    long long want = (2 * n_pairs_max + tiles - 1) / tiles;
+    long long cap = num_kb / 8 > 0 ? num_kb / 8 : 1;
+    splits = (int)(want < cap ? want : cap);
+    if (splits < 1) splits = 1;
+  }
+  p.kb_per_split = (num_kb + splits - 1) / splits;
+  splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;
+  p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits;
+  static bool attr_done = false;
+  if (!attr_done) {
+    PCM_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, T2_SMEM_TOTAL));
+    attr_done = true;
+  }
+  const long long total = (long long)tiles_m * tiles_n * splits;
+  const int pairs = (int)(total < n_pairs_max ? total : n_pairs_max);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = T2_SMEM_TOTAL;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, tmA, tmB, p) != cudaSuccess) {
+    cudaGetLastError();
+    return PCM_ERR_CUDA;
+  }
+  pcm::g_launches.fetch_add(1, std::memory_order_relaxed);
+  return PCM_OK;
+}
+
 bool gemm_epilogue_supported(const GemmArgs& g) {
   if (!gemm_tcgen05_supported(g) || g.c_dtype != DT_BF16 || g.R) return false;
   const GemmEpilogue& e = g.epi;
@@ -533,12 +790,21 @@ bool gemm_epilogue_supported(const GemmArgs& g) {
 }
 
 int gemm_tcgen05(const GemmArgs& g, cudaStream_t s) {
+  // CTA pairs whenever the output is at least one 256-wide tile; single CTAs otherwise (or with PCM_GEMM_PAIR=0)
+  const bool pair = pair_enabled() && g.N >= 256 && g.M > TC_BM;
   switch (g.epi.kind) {
-    case EPI_SWIGLU_FWD: return gemm_epilogue_supported(g) ? launch_tc<256, EPI_SWIGLU_FWD>(g, s) : PCM_ERR_SHAPE;
-    case EPI_SWIGLU_BWD: return gemm_epilogue_supported(g) ? launch_tc<256, EPI_SWIGLU_BWD>(g, s) : PCM_ERR_SHAPE;
-    case EPI_ROPE: return gemm_epilogue_supported(g) ? launch_tc<256, EPI_ROPE>(g, s) : PCM_ERR_SHAPE;
+    case EPI_SWIGLU_FWD:
+      if (!gemm_epilogue_supported(g)) return PCM_ERR_SHAPE;
+      return pair ? launch_tc2<EPI_SWIGLU_FWD>(g, s) : launch_tc<256, EPI_SWIGLU_FWD>(g, s);
+    case EPI_SWIGLU_BWD:
+      if (!gemm_epilogue_supported(g)) return PCM_ERR_SHAPE;
+      return pair ? launch_tc2<EPI_SWIGLU_BWD>(g, s) : launch_tc<256, EPI_SWIGLU_BWD>(g, s);
+    case EPI_ROPE:
+      if (!gemm_epilogue_supported(g)) return PCM_ERR_SHAPE;
+      return pair ? launch_tc2<EPI_ROPE>(g, s) : launch_tc<256, EPI_ROPE>(g, s);
     default: break;
   }
+  if (pair) return launch_tc2<EPI_NONE>(g, s);
   if (g.N % 256 == 0 || g.N > 256) return launch_tc<256, EPI_NONE>(g, s);
   return launch_tc<128, EPI_NONE>(g, s);
 }
