@@ -2,18 +2,22 @@
 // (mma.sync m16n8k16, fp32 accumulate), flash style: probabilities live in registers only, the
 // backward pass rebuilds them from the saved row log-sum-exp.
 //
-// Sequences are short (S <= 384), so a CTA stages every key/value row it needs in shared memory once
-// and then runs without further synchronisation:
-//   forward / dQ : CTA = 64 query rows of one (sequence, head); 4 warps x 16 rows; loop over 64-key blocks
-//   dK / dV      : CTA = 64 key rows; 4 warps x 16 keys; loop over 64-query blocks at or below the diagonal
+// The operand a CTA sweeps over (keys/values, or queries/dO in the dK/dV pass) streams through two
+// shared-memory stages of 64 rows filled with cp.async while the other stage is being consumed:
+//   forward / dQ : CTA = 128 (head dim <= 64) or 64 query rows of one (sequence, head); a warp per 16 rows;
+//                  loop over 64-key blocks
+//   dK / dV      : CTA = 128 or 64 key rows; a warp per 16 keys; loop over 64-query blocks at or below the diagonal
 // Shared-memory rows are padded by 16 bytes so that ldmatrix reads are bank-conflict free.
 #include "internal.h"
 
 namespace pcm {
 
-constexpr int FA_ROWS = 64;                  // rows per CTA
+// rows per CTA (16 per warp); equal to the inner block so that every warp of a CTA walks the same blocks
+template <int DH> struct FaCfg {
+  static constexpr int ROWS = 64;
+  static constexpr int THREADS = ROWS * 2;
+};
 constexpr int FA_BLK = 64;                   // columns per inner block
-constexpr int FA_THREADS = 128;
 constexpr float LOG2E = 1.4426950408889634f;
 
 typedef __nv_bfloat16 bf16;
@@ -44,11 +48,13 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int
   const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(src_bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // rows [row0, row0 + nrows) of a [.][DH] matrix (global row stride ld elements) -> shared rows
 // [0, nrows) with stride DH + 8; rows at or beyond row_limit are zero.  All copies of a thread are
-// in flight together; the caller waits with cp_async_wait_all() + __syncthreads().
+// in flight together; the caller commits the group and waits with cp_async_wait_group + __syncthreads().
 template <int DH>
 __device__ __forceinline__ void stage_rows(bf16* dst, const bf16* __restrict__ src, long long ld, int row0, int nrows,
                                            int row_limit) {
@@ -92,30 +98,30 @@ __device__ __forceinline__ float quad_sum(float v) {
 // forward
 // ------------------------------------------------------------------------------------------------
 template <int DH>
-__global__ void __launch_bounds__(FA_THREADS)
+__global__ void __launch_bounds__(FaCfg<DH>::THREADS)
 fa_fwd_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __restrict__ lse, int S, int H, float scale) {
   extern __shared__ __align__(16) unsigned char smraw[];
   constexpr int RS = DH + 8;
   const int qt = blockIdx.x, h = blockIdx.y, seq = blockIdx.z, d = H * DH;
   const long long ld = 3LL * d;
   const bf16* base = qkv + (long long)seq * S * ld + (long long)h * DH;
-  const int q0 = qt * FA_ROWS;
-  const int n_keys = min(S, q0 + FA_ROWS);                  // causal: keys beyond the tile's last row are never used
-  const int key_rows = (n_keys + FA_BLK - 1) / FA_BLK * FA_BLK;
+  const int q0 = qt * FaCfg<DH>::ROWS;
+  const int n_keys = min(S, q0 + FaCfg<DH>::ROWS);                  // causal: keys beyond the tile's last row are never used
+  constexpr int STAGE = 2 * FA_BLK * RS;                            // one 64-key block of K followed by the same block of V
   bf16* Qs = reinterpret_cast<bf16*>(smraw);
-  bf16* Ks = Qs + FA_ROWS * RS;
-  bf16* Vs = Ks + key_rows * RS;
-  stage_rows<DH>(Qs, base, ld, q0, FA_ROWS, S);
-  stage_rows<DH>(Ks, base + d, ld, 0, key_rows, n_keys);
-  stage_rows<DH>(Vs, base + 2 * d, ld, 0, key_rows, n_keys);
-  cp_async_wait_all();
-  __syncthreads();
+  bf16* KV = Qs + FaCfg<DH>::ROWS * RS;                              // two stages, refilled while the other one is in use
+  auto load_kv = [&](int kb) {
+    bf16* st = KV + (kb & 1) * STAGE;
+    stage_rows<DH>(st, base + d, ld, kb * FA_BLK, FA_BLK, n_keys);
+    stage_rows<DH>(st + FA_BLK * RS, base + 2 * d, ld, kb * FA_BLK, FA_BLK, n_keys);
+    cp_async_commit();
+  };
+  stage_rows<DH>(Qs, base, ld, q0, FaCfg<DH>::ROWS, S);
+  load_kv(0);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int wrow0 = warp * 16;                               // first row of this warp inside the tile
   uint32_t qf[DH / 16][4];
-#pragma unroll
-  for (int kk = 0; kk < DH / 16; ++kk) load_a<RS>(qf[kk], Qs, wrow0, kk * 16, lane);
 
   float o[DH / 8][4];
 #pragma unroll
@@ -123,9 +129,17 @@ fa_fwd_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __res
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // rows g and g + 8, log2 domain
   const int row_a = q0 + wrow0 + g, row_b = row_a + 8;
   const float c = scale * LOG2E;
-  const int last_blk = min((q0 + wrow0 + 15) / FA_BLK, (n_keys - 1) / FA_BLK);
+  const int last_blk = (n_keys - 1) / FA_BLK;                 // the same for every warp of the CTA
 
   for (int kb = 0; kb <= last_blk; ++kb) {
+    if (kb < last_blk) { load_kv(kb + 1); cp_async_wait_group<1>(); } else { cp_async_wait_group<0>(); }
+    __syncthreads();                                           // block kb has landed for every thread
+    if (kb == 0) {
+#pragma unroll
+      for (int kk = 0; kk < DH / 16; ++kk) load_a<RS>(qf[kk], Qs, wrow0, kk * 16, lane);
+    }
+    const bf16* Ks = KV + (kb & 1) * STAGE;
+    const bf16* Vs = Ks + FA_BLK * RS;
     float s[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
@@ -134,7 +148,7 @@ fa_fwd_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __res
 #pragma unroll
       for (int np = 0; np < 4; ++np) {
         uint32_t b[4];
-        load_b_nk<RS>(b, Ks, kb * FA_BLK + np * 16, kk * 16, lane);
+        load_b_nk<RS>(b, Ks, np * 16, kk * 16, lane);
         mma_bf16(s[2 * np], qf[kk], b[0], b[1]);
         mma_bf16(s[2 * np + 1], qf[kk], b[2], b[3]);
       }
@@ -173,11 +187,12 @@ fa_fwd_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __res
 #pragma unroll
       for (int dp = 0; dp < DH / 16; ++dp) {
         uint32_t b[4];
-        load_b_kn<RS>(b, Vs, kb * FA_BLK + k2 * 16, dp * 16, lane);
+        load_b_kn<RS>(b, Vs, k2 * 16, dp * 16, lane);
         mma_bf16(o[2 * dp], pa, b[0], b[1]);
         mma_bf16(o[2 * dp + 1], pa, b[2], b[3]);
       }
     }
+    __syncthreads();                                           // everyone is done with this stage before it is refilled
   }
   const float inv0 = 1.f / l0, inv1 = 1.f / l1;
   if (row_a < S) {
@@ -246,7 +261,7 @@ __device__ __forceinline__ void unrotate(float (&acc)[DH / 8][4], const float2* 
 // dQ: same tiling as the forward pass
 // ------------------------------------------------------------------------------------------------
 template <int DH>
-__global__ void __launch_bounds__(FA_THREADS)
+__global__ void __launch_bounds__(FaCfg<DH>::THREADS)
 fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, const float* __restrict__ lse,
                  const float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H, float scale,
                  const float2* __restrict__ rope_tab) {
@@ -255,19 +270,21 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
   const int qt = blockIdx.x, h = blockIdx.y, seq = blockIdx.z, d = H * DH;
   const long long ld = 3LL * d;
   const bf16* base = qkv + (long long)seq * S * ld + (long long)h * DH;
-  const int q0 = qt * FA_ROWS;
-  const int n_keys = min(S, q0 + FA_ROWS);
-  const int key_rows = (n_keys + FA_BLK - 1) / FA_BLK * FA_BLK;
+  const int q0 = qt * FaCfg<DH>::ROWS;
+  const int n_keys = min(S, q0 + FaCfg<DH>::ROWS);
+  constexpr int STAGE = 2 * FA_BLK * RS;
   bf16* Qs = reinterpret_cast<bf16*>(smraw);
-  bf16* Gs = Qs + FA_ROWS * RS;                              // dO rows of the tile
-  bf16* Ks = Gs + FA_ROWS * RS;
-  bf16* Vs = Ks + key_rows * RS;
-  stage_rows<DH>(Qs, base, ld, q0, FA_ROWS, S);
-  stage_rows<DH>(Gs, dout + (long long)seq * S * d + (long long)h * DH, d, q0, FA_ROWS, S);
-  stage_rows<DH>(Ks, base + d, ld, 0, key_rows, n_keys);
-  stage_rows<DH>(Vs, base + 2 * d, ld, 0, key_rows, n_keys);
-  cp_async_wait_all();
-  __syncthreads();
+  bf16* Gs = Qs + FaCfg<DH>::ROWS * RS;                              // dO rows of the tile
+  bf16* KV = Gs + FaCfg<DH>::ROWS * RS;                              // two stages of (K block, V block)
+  auto load_kv = [&](int kb) {
+    bf16* st = KV + (kb & 1) * STAGE;
+    stage_rows<DH>(st, base + d, ld, kb * FA_BLK, FA_BLK, n_keys);
+    stage_rows<DH>(st + FA_BLK * RS, base + 2 * d, ld, kb * FA_BLK, FA_BLK, n_keys);
+    cp_async_commit();
+  };
+  stage_rows<DH>(Qs, base, ld, q0, FaCfg<DH>::ROWS, S);
+  stage_rows<DH>(Gs, dout + (long long)seq * S * d + (long long)h * DH, d, q0, FaCfg<DH>::ROWS, S);
+  load_kv(0);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int wrow0 = warp * 16;
@@ -280,9 +297,13 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
   float dq[DH / 8][4];
 #pragma unroll
   for (int i = 0; i < DH / 8; ++i) { dq[i][0] = dq[i][1] = dq[i][2] = dq[i][3] = 0.f; }
-  const int last_blk = min((q0 + wrow0 + 15) / FA_BLK, (n_keys - 1) / FA_BLK);
+  const int last_blk = (n_keys - 1) / FA_BLK;
 
   for (int kb = 0; kb <= last_blk; ++kb) {
+    if (kb < last_blk) { load_kv(kb + 1); cp_async_wait_group<1>(); } else { cp_async_wait_group<0>(); }
+    __syncthreads();
+    const bf16* Ks = KV + (kb & 1) * STAGE;
+    const bf16* Vs = Ks + FA_BLK * RS;
     float s[8][4], dp[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -297,10 +318,10 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
 #pragma unroll
       for (int np = 0; np < 4; ++np) {
         uint32_t b[4];
-        load_b_nk<RS>(b, Ks, kb * FA_BLK + np * 16, kk * 16, lane);
+        load_b_nk<RS>(b, Ks, np * 16, kk * 16, lane);
         mma_bf16(s[2 * np], qa, b[0], b[1]);
         mma_bf16(s[2 * np + 1], qa, b[2], b[3]);
-        load_b_nk<RS>(b, Vs, kb * FA_BLK + np * 16, kk * 16, lane);
+        load_b_nk<RS>(b, Vs, np * 16, kk * 16, lane);
         mma_bf16(dp[2 * np], ga, b[0], b[1]);
         mma_bf16(dp[2 * np + 1], ga, b[2], b[3]);
       }
@@ -321,11 +342,12 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
 #pragma unroll
       for (int dpi = 0; dpi < DH / 16; ++dpi) {
         uint32_t b[4];
-        load_b_kn<RS>(b, Ks, kb * FA_BLK + k2 * 16, dpi * 16, lane);
+        load_b_kn<RS>(b, Ks, k2 * 16, dpi * 16, lane);
         mma_bf16(dq[2 * dpi], sa, b[0], b[1]);
         mma_bf16(dq[2 * dpi + 1], sa, b[2], b[3]);
       }
     }
+    __syncthreads();
   }
   if (rope_tab) unrotate<DH>(dq, rope_tab, row_a, row_b, S, t);   // gradient w.r.t. q before the rotary embedding
   if (row_a < S) {
@@ -344,7 +366,7 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
 // dK, dV: CTA = 64 key rows; transposed score tiles (rows = keys, columns = queries)
 // ------------------------------------------------------------------------------------------------
 template <int DH>
-__global__ void __launch_bounds__(FA_THREADS)
+__global__ void __launch_bounds__(FaCfg<DH>::THREADS)
 fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, const float* __restrict__ lse,
                   const float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H, float scale,
                   const float2* __restrict__ rope_tab) {
@@ -353,27 +375,31 @@ fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, c
   const int kt = blockIdx.x, h = blockIdx.y, seq = blockIdx.z, d = H * DH;
   const long long ld = 3LL * d;
   const bf16* base = qkv + (long long)seq * S * ld + (long long)h * DH;
-  const int k0 = kt * FA_ROWS;                               // first key of the tile
+  const int k0 = kt * FaCfg<DH>::ROWS;                               // first key of the tile
   const int q_lo = k0;                                       // queries below the tile's first key never see it
   const int q_rows = (S - q_lo + FA_BLK - 1) / FA_BLK * FA_BLK;
+  constexpr int STAGE = 2 * FA_BLK * RS;                      // one 64-query block of Q followed by the same block of dO
   bf16* Ks = reinterpret_cast<bf16*>(smraw);
-  bf16* Vs = Ks + FA_ROWS * RS;
-  bf16* Qs = Vs + FA_ROWS * RS;                              // rows = queries q_lo ..
-  bf16* Gs = Qs + q_rows * RS;
-  float* Ls = reinterpret_cast<float*>(Gs + q_rows * RS);    // lse * log2(e), indexed like Qs
+  bf16* Vs = Ks + FaCfg<DH>::ROWS * RS;
+  bf16* QG = Vs + FaCfg<DH>::ROWS * RS;                       // two stages of (Q block, dO block)
+  float* Ls = reinterpret_cast<float*>(QG + 2 * STAGE);      // lse * log2(e) for queries q_lo ..
   float* Ds = Ls + q_rows;
-  stage_rows<DH>(Ks, base + d, ld, k0, FA_ROWS, S);
-  stage_rows<DH>(Vs, base + 2 * d, ld, k0, FA_ROWS, S);
-  stage_rows<DH>(Qs, base, ld, q_lo, q_rows, S);
-  stage_rows<DH>(Gs, dout + (long long)seq * S * d + (long long)h * DH, d, q_lo, q_rows, S);
+  const bf16* gbase = dout + (long long)seq * S * d + (long long)h * DH;
+  auto load_qg = [&](int qb) {
+    bf16* st = QG + (qb & 1) * STAGE;
+    stage_rows<DH>(st, base, ld, q_lo + qb * FA_BLK, FA_BLK, S);
+    stage_rows<DH>(st + FA_BLK * RS, gbase, d, q_lo + qb * FA_BLK, FA_BLK, S);
+    cp_async_commit();
+  };
+  stage_rows<DH>(Ks, base + d, ld, k0, FaCfg<DH>::ROWS, S);
+  stage_rows<DH>(Vs, base + 2 * d, ld, k0, FaCfg<DH>::ROWS, S);
+  load_qg(0);
   const long long sbase = ((long long)seq * H + h) * S;
   for (int i = threadIdx.x; i < q_rows; i += blockDim.x) {
     const bool ok = q_lo + i < S;
     Ls[i] = ok ? lse[sbase + q_lo + i] * LOG2E : 0.f;
     Ds[i] = ok ? dsum[sbase + q_lo + i] : 0.f;
   }
-  cp_async_wait_all();
-  __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int wrow0 = warp * 16;
@@ -386,8 +412,11 @@ fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, c
     dv[i][0] = dv[i][1] = dv[i][2] = dv[i][3] = 0.f;
   }
   const int n_blk = q_rows / FA_BLK;
-  const int first_blk = wrow0 / FA_BLK;                      // always 0 (64-row tile); kept for clarity
-  for (int qb = first_blk; qb < n_blk; ++qb) {
+  for (int qb = 0; qb < n_blk; ++qb) {
+    if (qb + 1 < n_blk) { load_qg(qb + 1); cp_async_wait_group<1>(); } else { cp_async_wait_group<0>(); }
+    __syncthreads();                                           // also publishes Ls / Ds on the first pass
+    const bf16* Qs = QG + (qb & 1) * STAGE;
+    const bf16* Gs = Qs + FA_BLK * RS;
     float st[8][4], dpt[8][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -402,10 +431,10 @@ fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, c
 #pragma unroll
       for (int np = 0; np < 4; ++np) {
         uint32_t b[4];
-        load_b_nk<RS>(b, Qs, qb * FA_BLK + np * 16, kk * 16, lane);
+        load_b_nk<RS>(b, Qs, np * 16, kk * 16, lane);
         mma_bf16(st[2 * np], ka, b[0], b[1]);
         mma_bf16(st[2 * np + 1], ka, b[2], b[3]);
-        load_b_nk<RS>(b, Gs, qb * FA_BLK + np * 16, kk * 16, lane);
+        load_b_nk<RS>(b, Gs, np * 16, kk * 16, lane);
         mma_bf16(dpt[2 * np], va, b[0], b[1]);
         mma_bf16(dpt[2 * np + 1], va, b[2], b[3]);
       }
@@ -436,14 +465,15 @@ fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, c
 #pragma unroll
       for (int dpi = 0; dpi < DH / 16; ++dpi) {
         uint32_t b[4];
-        load_b_kn<RS>(b, Gs, qb * FA_BLK + k2 * 16, dpi * 16, lane);
+        load_b_kn<RS>(b, Gs, k2 * 16, dpi * 16, lane);
         mma_bf16(dv[2 * dpi], pa, b[0], b[1]);
         mma_bf16(dv[2 * dpi + 1], pa, b[2], b[3]);
-        load_b_kn<RS>(b, Qs, qb * FA_BLK + k2 * 16, dpi * 16, lane);
+        load_b_kn<RS>(b, Qs, k2 * 16, dpi * 16, lane);
         mma_bf16(dk[2 * dpi], sa, b[0], b[1]);
         mma_bf16(dk[2 * dpi + 1], sa, b[2], b[3]);
       }
     }
+    __syncthreads();
   }
   if (rope_tab) unrotate<DH>(dk, rope_tab, key_a, key_b, S, t);   // gradient w.r.t. k before the rotary embedding
   if (key_a < S) {
@@ -469,11 +499,11 @@ fa_bwd_dkv_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, c
 // ------------------------------------------------------------------------------------------------
 template <int DH>
 static int fa_fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int S, int H, cudaStream_t s) {
-  const int tiles = (S + FA_ROWS - 1) / FA_ROWS;
-  const size_t smem = (size_t)(FA_ROWS + 2 * tiles * FA_BLK) * (DH + 8) * sizeof(bf16);
+  const int tiles = (S + FaCfg<DH>::ROWS - 1) / FaCfg<DH>::ROWS;
+  const size_t smem = (size_t)(FaCfg<DH>::ROWS + 4 * FA_BLK) * (DH + 8) * sizeof(bf16);     // Q tile + 2 stages of (K, V)
   if (smem > 227 * 1024) return PCM_ERR_SHAPE;
   PCM_CUDA_TRY(cudaFuncSetAttribute(fa_fwd_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  fa_fwd_kernel<DH><<<dim3(tiles, H, n_seq), FA_THREADS, smem, s>>>((const bf16*)qkv, (bf16*)out, lse, S, H,
+  fa_fwd_kernel<DH><<<dim3(tiles, H, n_seq), FaCfg<DH>::THREADS, smem, s>>>((const bf16*)qkv, (bf16*)out, lse, S, H,
                                                                     1.0f / sqrtf((float)DH));
   PCM_LAUNCH_CHECK();
   return PCM_OK;
@@ -482,20 +512,21 @@ static int fa_fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int 
 template <int DH>
 static int fa_bwd_launch(const void* qkv, const void* out, const void* dout, const float* lse, float* dsum, void* dqkv,
                          int n_seq, int S, int H, const float2* rope_tab, cudaStream_t s) {
-  const int tiles = (S + FA_ROWS - 1) / FA_ROWS;
-  const size_t smem_dq = (size_t)(2 * FA_ROWS + 2 * tiles * FA_BLK) * (DH + 8) * sizeof(bf16);
-  const size_t smem_dkv = smem_dq + (size_t)2 * tiles * FA_BLK * sizeof(float);
+  const int tiles = (S + FaCfg<DH>::ROWS - 1) / FaCfg<DH>::ROWS;
+  const int key_rows = (S + FA_BLK - 1) / FA_BLK * FA_BLK;
+  const size_t smem_dq = (size_t)(2 * FaCfg<DH>::ROWS + 4 * FA_BLK) * (DH + 8) * sizeof(bf16);   // 2 tiles + 2 stages of 2 blocks
+  const size_t smem_dkv = smem_dq + (size_t)2 * key_rows * sizeof(float);
   if (smem_dkv > 227 * 1024) return PCM_ERR_SHAPE;
   const float scale = 1.0f / sqrtf((float)DH);
   const long long rows = (long long)n_seq * S * H;
   fa_dsum_kernel<DH><<<ceil_div(rows, 8), 256, 0, s>>>((const bf16*)out, (const bf16*)dout, dsum, n_seq, S, H);
   PCM_LAUNCH_CHECK();
   PCM_CUDA_TRY(cudaFuncSetAttribute(fa_bwd_dq_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq));
-  fa_bwd_dq_kernel<DH><<<dim3(tiles, H, n_seq), FA_THREADS, smem_dq, s>>>((const bf16*)qkv, (const bf16*)dout, lse, dsum,
+  fa_bwd_dq_kernel<DH><<<dim3(tiles, H, n_seq), FaCfg<DH>::THREADS, smem_dq, s>>>((const bf16*)qkv, (const bf16*)dout, lse, dsum,
                                                                          (bf16*)dqkv, S, H, scale, rope_tab);
   PCM_LAUNCH_CHECK();
   PCM_CUDA_TRY(cudaFuncSetAttribute(fa_bwd_dkv_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dkv));
-  fa_bwd_dkv_kernel<DH><<<dim3(tiles, H, n_seq), FA_THREADS, smem_dkv, s>>>((const bf16*)qkv, (const bf16*)dout, lse,
+  fa_bwd_dkv_kernel<DH><<<dim3(tiles, H, n_seq), FaCfg<DH>::THREADS, smem_dkv, s>>>((const bf16*)qkv, (const bf16*)dout, lse,
                                                                            dsum, (bf16*)dqkv, S, H, scale, rope_tab);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
