@@ -27,8 +27,11 @@ namespace pcm {
 
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                     // 64 bf16 = one 128-byte swizzle row
-constexpr int TC_STAGES = 4;
+constexpr int TC_STAGES = 3;
 constexpr int TC_EPI_WARPS = 8;                // two per tensor-memory lane quadrant, each takes half of the columns
+constexpr int EPI_STAGE_STRIDE = 36;            // floats per staged epilogue row (32 + 4 of padding: conflict free)
+constexpr int EPI_STAGE_FLOATS = 32 * EPI_STAGE_STRIDE;   // per epilogue warp
+constexpr int EPI_STAGE_BYTES = TC_EPI_WARPS * EPI_STAGE_FLOATS * 4;
 constexpr int TC_THREADS = 320;               // producer warp, MMA warp, 8 epilogue warps
 constexpr unsigned long long TC_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per mbarrier wait
 
@@ -116,8 +119,85 @@ struct TcSmem {
   static constexpr int A_BYTES = TC_BM * TC_BK * 2;           // 16 KB
   static constexpr int B_BYTES = BN * TC_BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int TOTAL = TC_STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+  static constexpr int TOTAL = TC_STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + EPI_STAGE_BYTES;
 };
+
+// The plain epilogue stores through a per-warp shared-memory buffer: tcgen05.ld hands every thread one row
+// of 32 columns, the buffer turns that into "a quarter warp per row" so that each global access of a warp
+// covers whole 128-byte (fp32) or 64-byte (bf16) row segments instead of 32 scattered rows.
+
+// fp32 output: pass i covers rows 4i .. 4i+3, lane -> (row 4i + lane/8, columns 4 (lane%8) ..)
+// bf16 output: pass i covers rows 8i .. 8i+7, lane -> (row 8i + lane/4, columns 8 (lane%4) ..)
+__device__ __forceinline__ void fetch_residual(const TcParams& p, int row_base, int col, int lane, float4 (&r)[8]) {
+  if (p.c_dtype == DT_F32) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int gr = row_base + i * 4 + (lane >> 3);
+      if (gr < p.M) r[i] = *reinterpret_cast<const float4*>(p.R + (long long)gr * p.ldr + col + (lane & 7) * 4);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int gr = row_base + i * 8 + (lane >> 2);
+      if (gr < p.M) {
+        const float4* q = reinterpret_cast<const float4*>(p.R + (long long)gr * p.ldr + col + (lane & 3) * 8);
+        r[2 * i] = q[0];
+        r[2 * i + 1] = q[1];
+      }
+    }
+  }
+}
+
+// Row layout (thread = row, 32 fp32 columns) -> bf16 rows in global memory, an eighth of a warp per row.
+__device__ __forceinline__ void staged_store_bf16(float* stage, int lane, const float (&v)[32], __nv_bfloat16* C,
+                                                  long long ldc, int row_base, int M, int col) {
+  float* srow = stage + lane * EPI_STAGE_STRIDE;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) *reinterpret_cast<float4*>(srow + 4 * e) = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 8 + (lane >> 2), gr = row_base + r;
+    const float* sp = stage + r * EPI_STAGE_STRIDE + (lane & 3) * 8;
+    const float4 a = *reinterpret_cast<const float4*>(sp), b = *reinterpret_cast<const float4*>(sp + 4);
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w);
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(b.x, b.y), h3 = __floats2bfloat162_rn(b.z, b.w);
+    uint4 o;
+    o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+    o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+    if (gr < M) *reinterpret_cast<uint4*>(C + (long long)gr * ldc + col + (lane & 3) * 8) = o;
+  }
+  __syncwarp();
+}
+// 32 rows x 32 bf16 columns fetched with an eighth of a warp per row (kept in that layout until used)
+__device__ __forceinline__ void fetch_bf16_rows(const __nv_bfloat16* A, long long ld, int row_base, int M, int col, int lane,
+                                                uint4 (&o)[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int gr = row_base + i * 8 + (lane >> 2);
+    o[i] = gr < M ? *reinterpret_cast<const uint4*>(A + (long long)gr * ld + col + (lane & 3) * 8) : make_uint4(0, 0, 0, 0);
+  }
+}
+// ... and turned into the row layout (thread = row) through the staging buffer
+__device__ __forceinline__ void unstage_bf16_rows(float* stage, int lane, const uint4 (&o)[4], float (&v)[32]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float* sp = stage + (i * 8 + (lane >> 2)) * EPI_STAGE_STRIDE + (lane & 3) * 8;
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&o[i]);
+    const float2 f0 = __bfloat1622float2(h[0]), f1 = __bfloat1622float2(h[1]);
+    const float2 f2 = __bfloat1622float2(h[2]), f3 = __bfloat1622float2(h[3]);
+    *reinterpret_cast<float4*>(sp) = make_float4(f0.x, f0.y, f1.x, f1.y);
+    *reinterpret_cast<float4*>(sp + 4) = make_float4(f2.x, f2.y, f3.x, f3.y);
+  }
+  __syncwarp();
+  const float* srow = stage + lane * EPI_STAGE_STRIDE;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const float4 t = *reinterpret_cast<const float4*>(srow + 4 * e);
+    v[4 * e] = t.x; v[4 * e + 1] = t.y; v[4 * e + 2] = t.z; v[4 * e + 3] = t.w;
+  }
+  __syncwarp();
+}
 
 // Operands of the epilogue that are fetched one 32-column slice ahead of their use.
 struct EpiRegs {
@@ -128,27 +208,25 @@ struct EpiRegs {
 // Issued before the wait for the accumulator, so that the first slice's loads overlap it.
 template <int BN, int EPI>
 __device__ __forceinline__ void epi_prefetch(const TcParams& p, int row, int n0, int chalf, EpiRegs& pre) {
+  const int lane_ = threadIdx.x & 31;
       if constexpr (EPI == EPI_SWIGLU_BWD) {
         const int col0 = n0 + chalf * (BN / 2);
-        if (row < p.M && col0 < p.N) {
-          const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col0;
-          fetch_bf16x32(nx, pre.g);           // issued before waiting for the accumulator
-          fetch_bf16x32(nx + p.N, pre.u);
+        if (col0 < p.N) {                     // issued before waiting for the accumulator
+          fetch_bf16_rows(p.aux, p.ld_aux, row - lane_, p.M, col0, lane_, pre.g);
+          fetch_bf16_rows(p.aux + p.N, p.ld_aux, row - lane_, p.M, col0, lane_, pre.u);
         }
       }
       if constexpr (EPI == EPI_NONE) {
         const int col0 = n0 + chalf * (BN / 2);
-        if (p.R && row < p.M && col0 < p.N) {
-          const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col0);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) pre.r[e] = rp[e];
-        }
+        if (p.R && !p.reduce && col0 < p.N) fetch_residual(p, row - lane_, col0, lane_, pre.r);
       }
 }
 
 // One epilogue warp's share of a tile: rows = this warp's 32 tensor-memory lanes, columns = its half of the tile.
 template <int BN, int EPI>
-__device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, int row, int n0, int chalf, EpiRegs& pre) {
+__device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, int row, int n0, int chalf, EpiRegs& pre,
+                                         float* stage) {
+  const int lane_ = threadIdx.x & 31;
       if constexpr (EPI == EPI_SWIGLU_FWD) {
         // accumulator columns [0,128) = gate, [128,256) = up, for hidden units hid0 .. hid0+127
         const int hid0 = n0 / 2, F = p.up_row0;
@@ -159,16 +237,17 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
           tmem_ld_32x32(tmem_acc + (uint32_t)c0, rg);
           tmem_ld_32x32(tmem_acc + (uint32_t)(128 + c0), ru);
           tmem_ld_wait();
-          if (row < p.M) {
+          {
             float g[32], u[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) { g[e] = __uint_as_float(rg[e]); u[e] = __uint_as_float(ru[e]); }
-            __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + hid0 + c0;
-            store_bf16x32(gu, g);
-            store_bf16x32(gu + F, u);
+            const int row_base = row - lane_;
+            __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(p.C);
+            staged_store_bf16(stage, lane_, g, gu, p.ldc, row_base, p.M, hid0 + c0);
+            staged_store_bf16(stage, lane_, u, gu + F, p.ldc, row_base, p.M, hid0 + c0);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) g[e] = g[e] / (1.f + __expf(-g[e])) * u[e];
-            store_bf16x32(p.out2 + (long long)row * p.ld_out2 + hid0 + c0, g);
+            for (int e = 0; e < 32; ++e) g[e] = __fdividef(g[e], 1.f + __expf(-g[e])) * u[e];
+            staged_store_bf16(stage, lane_, g, p.out2, p.ld_out2, row_base, p.M, hid0 + c0);
           }
         }
       } else if constexpr (EPI == EPI_ROPE) {
@@ -196,7 +275,7 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
             tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + ic), rl);
             tmem_ld_32x32(tmem_acc + (uint32_t)(h0 + half + ic), rh);
             tmem_ld_wait();
-            if (row < p.M) {
+            {
               float lo[32], hi[32];
 #pragma unroll
               for (int e = 0; e < 32; ++e) { lo[e] = __uint_as_float(rl[e]); hi[e] = __uint_as_float(rh[e]); }
@@ -208,9 +287,9 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
                   hi[e] = y * cs[e].x + x * cs[e].y;
                 }
               }
-              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + n0 + h0 + ic;
-              store_bf16x32(dst, lo);
-              store_bf16x32(dst + half, hi);
+              __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
+              staged_store_bf16(stage, lane_, lo, Cb, p.ldc, row - lane_, p.M, n0 + h0 + ic);
+              staged_store_bf16(stage, lane_, hi, Cb, p.ldc, row - lane_, p.M, n0 + h0 + ic + half);
             }
           }
         }
@@ -222,58 +301,82 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
         uint32_t r[32];
         tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
         tmem_ld_wait();
-        if (row < p.M) {
-          if constexpr (EPI == EPI_SWIGLU_BWD) {
-            // r = d(act) in fp32; gate | up come from aux (fetched one chunk ahead); d(gate) | d(up) go to C
-            const int F = p.N;
-            float g[32], u[32];
-            unpack_bf16x32(pre.g, g);
-            unpack_bf16x32(pre.u, u);
-            if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
-              const __nv_bfloat16* nx = p.aux + (long long)row * p.ld_aux + col + 32;
-              fetch_bf16x32(nx, pre.g);
-              fetch_bf16x32(nx + F, pre.u);
-            }
+        if constexpr (EPI == EPI_SWIGLU_BWD) {
+          // r = d(act) in fp32; gate | up come from aux (fetched one slice ahead); d(gate) | d(up) go to C
+          const int F = p.N, row_base = row - lane_;
+          float g[32], u[32];
+          unstage_bf16_rows(stage, lane_, pre.g, g);
+          unstage_bf16_rows(stage, lane_, pre.u, u);
+          if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
+            fetch_bf16_rows(p.aux, p.ld_aux, row_base, p.M, col + 32, lane_, pre.g);
+            fetch_bf16_rows(p.aux + F, p.ld_aux, row_base, p.M, col + 32, lane_, pre.u);
+          }
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const float da = __uint_as_float(r[e]);
-              const float sg = 1.f / (1.f + __expf(-g[e]));
-              const float dg = da * u[e] * sg * (1.f + g[e] * (1.f - sg));
-              u[e] = da * g[e] * sg;
-              g[e] = dg;
-            }
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col;
-            store_bf16x32(dst, g);
-            store_bf16x32(dst + F, u);
-          } else if (p.reduce) {
+          for (int e = 0; e < 32; ++e) {
+            const float da = __uint_as_float(r[e]);
+            const float sg = __fdividef(1.f, 1.f + __expf(-g[e]));
+            const float dg = da * u[e] * sg * (1.f + g[e] * (1.f - sg));
+            u[e] = da * g[e] * sg;
+            g[e] = dg;
+          }
+          __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
+          staged_store_bf16(stage, lane_, g, Cb, p.ldc, row_base, p.M, col);
+          staged_store_bf16(stage, lane_, u, Cb + F, p.ldc, row_base, p.M, col);
+        } else if (p.reduce) {
+          if (row < p.M) {
             float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
 #pragma unroll
             for (int e = 0; e < 32; e += 4)
               red_add_v4(dst + e, __uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
                          __uint_as_float(r[e + 3]));
-          } else {
-            float v[32];
+          }
+        } else {
+          // stage the 32 x 32 slice (thread = row), then store it with a quarter (or eighth) warp per row
+          float* srow = stage + lane_ * EPI_STAGE_STRIDE;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
-            if (p.R) {
+          for (int e = 0; e < 8; ++e)
+            *reinterpret_cast<uint4*>(srow + 4 * e) = make_uint4(r[4 * e], r[4 * e + 1], r[4 * e + 2], r[4 * e + 3]);
+          __syncwarp();
+          const int row_base = row - lane_;
+          const bool more = c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N;
+          if (p.c_dtype == DT_F32) {
+            float4 v[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                v[4 * e] += pre.r[e].x; v[4 * e + 1] += pre.r[e].y; v[4 * e + 2] += pre.r[e].z; v[4 * e + 3] += pre.r[e].w;
-              }
-              if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
-                const float4* rp = reinterpret_cast<const float4*>(p.R + (long long)row * p.ldr + col + 32);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) pre.r[e] = rp[e];
-              }
+            for (int i = 0; i < 8; ++i) {
+              v[i] = *reinterpret_cast<const float4*>(stage + (i * 4 + (lane_ >> 3)) * EPI_STAGE_STRIDE + (lane_ & 7) * 4);
+              if (p.R) { v[i].x += pre.r[i].x; v[i].y += pre.r[i].y; v[i].z += pre.r[i].z; v[i].w += pre.r[i].w; }
             }
-            if (p.c_dtype == DT_F32) {
-              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col);
+            if (p.R && more) fetch_residual(p, row_base, col + 32, lane_, pre.r);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-            } else {
-              store_bf16x32(reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)row * p.ldc + col, v);
+            for (int i = 0; i < 8; ++i) {
+              const int gr = row_base + i * 4 + (lane_ >> 3);
+              if (gr < p.M)
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.C) + (long long)gr * p.ldc + col + (lane_ & 7) * 4) = v[i];
+            }
+          } else {
+            uint4 o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float* sp = stage + (i * 8 + (lane_ >> 2)) * EPI_STAGE_STRIDE + (lane_ & 3) * 8;
+              float4 a = *reinterpret_cast<const float4*>(sp), b = *reinterpret_cast<const float4*>(sp + 4);
+              if (p.R) {
+                a.x += pre.r[2 * i].x; a.y += pre.r[2 * i].y; a.z += pre.r[2 * i].z; a.w += pre.r[2 * i].w;
+                b.x += pre.r[2 * i + 1].x; b.y += pre.r[2 * i + 1].y; b.z += pre.r[2 * i + 1].z; b.w += pre.r[2 * i + 1].w;
+              }
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w);
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(b.x, b.y), h3 = __floats2bfloat162_rn(b.z, b.w);
+              o[i].x = *reinterpret_cast<uint32_t*>(&h0); o[i].y = *reinterpret_cast<uint32_t*>(&h1);
+              o[i].z = *reinterpret_cast<uint32_t*>(&h2); o[i].w = *reinterpret_cast<uint32_t*>(&h3);
+            }
+            if (p.R && more) fetch_residual(p, row_base, col + 32, lane_, pre.r);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int gr = row_base + i * 8 + (lane_ >> 2);
+              if (gr < p.M)
+                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.C) + (long long)gr * p.ldc + col + (lane_ & 3) * 8) = o[i];
             }
           }
+          __syncwarp();                       // the buffer is free again for the next slice
         }
       }
       }
@@ -293,6 +396,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint64_t* acc_empty = acc_full + 2;         // [2] epilogue -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* epi_stage = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb_total = (p.K + TC_BK - 1) / TC_BK;
@@ -411,7 +515,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!ok) break;
       tc_fence_after();
       const uint32_t tmem_acc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
-      epi_tile<BN, EPI>(p, tmem_acc, row, n0, chalf, pre);
+      epi_tile<BN, EPI>(p, tmem_acc, row, n0, chalf, pre, epi_stage + (warp - 2) * EPI_STAGE_FLOATS);
       // hand the accumulator buffer back to the MMA issuer
       tc_fence_before();
       __syncwarp();
@@ -443,11 +547,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 //   acc_empty[b] (leader)  <- the epilogue warps of both CTAs
 // ------------------------------------------------------------------------------------------------
 constexpr int T2_BN = 256;
-constexpr int T2_STAGES = 6;
+constexpr int T2_STAGES = 5;
 constexpr int T2_A_BYTES = TC_BM * TC_BK * 2;          // 16 KB: this CTA's 128 rows of A
 constexpr int T2_B_BYTES = (T2_BN / 2) * TC_BK * 2;    // 16 KB: this CTA's 128 columns of B
 constexpr int T2_STAGE_BYTES = T2_A_BYTES + T2_B_BYTES;
-constexpr int T2_SMEM_TOTAL = T2_STAGES * T2_STAGE_BYTES + 1024 + 256;
+constexpr int T2_SMEM_TOTAL = T2_STAGES * T2_STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES;   // ring + slack + barriers + epilogue staging
 
 template <int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -463,6 +567,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   uint64_t* acc_empty = acc_full + 2;          // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* epi_stage = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -584,7 +689,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       const uint32_t tmem_acc = tmem_base + ab * BN + ((uint32_t)(quad * 32) << 16);
-      epi_tile<BN, EPI>(p, tmem_acc, row, n0, chalf, pre);
+      epi_tile<BN, EPI>(p, tmem_acc, row, n0, chalf, pre, epi_stage + (warp - 2) * EPI_STAGE_FLOATS);
       // hand the accumulator buffer back to the leader's MMA thread
       tc_fence_before();
       __syncwarp();
