@@ -240,16 +240,31 @@ def run_cuda(args):
         B.grpo_actor_fwd_bwd(model, packed, w.eps_low, w.eps_high, 0.0, mb_chunks=mb, workspace=ws, want_stats=False,
                              logp=logp, loss=loss)
 
+    kept_host = torch.empty(w.n_traj * w.budget, dtype=torch.int32).pin_memory()
+
     def step_e2e(it):
+        """Host buffers in, loss out.  The mask is applied before the big transfer: the control plane runs on
+        the small arrays first, the kept chunk ids come back (a few KB), and only the kept chunks'
+        observation prefixes cross the bus."""
         for k in ("traj_off", "tok", "phase", "reward"):
             d_in[k].copy_(h[k], non_blocking=True)
-        d_obs.copy_(h_obs, non_blocking=True)
         d_lpo.copy_(h_lpo, non_blocking=True)
-        step(it, batch)
+        Cc, valid, _, adv = B.pcm_score_phases(ctx, batch)
+        _, q = B.pcm_update_keep_probs(ctx, Cc, valid)
+        kept_idx, kept_off, _ = B.pcm_sample_chunks(ctx, batch, q, it, out=samp)
+        kept_host.copy_(kept_idx, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        for c in kept_host[:n_kept].tolist():
+            d_obs[c].copy_(h_obs[c], non_blocking=True)
+        B.grpo_pack_chunks(ctx, batch, model, kept_idx, kept_off, adv, packed)
+        B.grpo_actor_fwd_bwd(model, packed, w.eps_low, w.eps_high, 0.0, mb_chunks=mb, workspace=ws, want_stats=False,
+                             logp=logp, loss=loss)
         return float(loss.item())                  # device -> host read of the step's result
 
-    h2d = sum(v.numel() * v.element_size() for v in h.values()) + h_obs.numel() * h_obs.element_size() + \
-        h_lpo.numel() * h_lpo.element_size()
+    chunk_bytes = w.P * w.d * h_obs.element_size()
+    h2d = sum(v.numel() * v.element_size() for v in h.values()) + h_lpo.numel() * h_lpo.element_size() + \
+        n_kept * chunk_bytes
+    d2h = 4 + 4 * w.n_traj * w.budget
 
     def barrier():
         if world > 1:
@@ -332,7 +347,7 @@ def run_cuda(args):
                          "flops_per_launch": g["flops"] / max(1, g["launches"]),
                          "step_tflops": step_tflops, "step_frac": step_tflops / peak},
             "kernel_classes": classes,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": 4,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": int(launches),
             "clocks": clocks,
