@@ -67,7 +67,7 @@ typedef struct {
   int32_t max_len;             /* upper bound on chunks per trajectory (sizes shared memory)      */
   int32_t reserved;
   const int32_t* traj_off;     /* device [n_traj+1]                                               */
-  const uint8_t* tok;          /* device [n_chunks][56], 4-byte aligned                           */
+  const uint8_t* tok;          /* device [n_chunks][56], 16-byte aligned                          */
   const uint8_t* phase;        /* device [n_chunks], labels < n_phases, any order                 */
   const uint8_t* reward;       /* device [n_traj], 0 or 1                                         */
   const void* obs;             /* device [n_chunks][P][d] in the model dtype; pack only           */

@@ -211,29 +211,6 @@ fa_fwd_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __res
   }
 }
 
-// D_i = sum_c dO_i[c] * O_i[c]; one warp per (token row, head)
-template <int DH>
-__global__ void fa_dsum_kernel(const bf16* __restrict__ out, const bf16* __restrict__ dout, float* __restrict__ dsum,
-                               int n_seq, int S, int H) {
-  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= (long long)n_seq * S * H) return;
-  const long long tok = row / H;
-  const int h = (int)(row - tok * H);
-  const bf16* o = out + tok * (long long)(H * DH) + (long long)h * DH;
-  const bf16* gr = dout + tok * (long long)(H * DH) + (long long)h * DH;
-  float s = 0.f;
-#pragma unroll
-  for (int e = 0; e < DH / 32; ++e)
-    s = fmaf(__bfloat162float(o[lane + 32 * e]), __bfloat162float(gr[lane + 32 * e]), s);
-#pragma unroll
-  for (int off = 16; off; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-  if (lane == 0) {
-    const long long seq = tok / S;
-    dsum[(seq * H + h) * S + (tok - seq * S)] = s;
-  }
-}
-
 // Transpose of the rotary embedding applied to an accumulator tile of 16 rows x DH columns: pairs
 // (c, c + DH/2) sit in n-tiles i and i + DH/16 of the same thread.  Rows a / b are positions in the sequence.
 template <int DH>
@@ -262,9 +239,9 @@ __device__ __forceinline__ void unrotate(float (&acc)[DH / 8][4], const float2* 
 // ------------------------------------------------------------------------------------------------
 template <int DH>
 __global__ void __launch_bounds__(FaCfg<DH>::THREADS)
-fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, const float* __restrict__ lse,
-                 const float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H, float scale,
-                 const float2* __restrict__ rope_tab) {
+fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out, const bf16* __restrict__ dout,
+                 const float* __restrict__ lse, float* __restrict__ dsum, bf16* __restrict__ dqkv, int S, int H,
+                 float scale, const float2* __restrict__ rope_tab) {
   extern __shared__ __align__(16) unsigned char smraw[];
   constexpr int RS = DH + 8;
   const int qt = blockIdx.x, h = blockIdx.y, seq = blockIdx.z, d = H * DH;
@@ -292,7 +269,7 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
   const long long sbase = ((long long)seq * H + h) * S;
   const float c = scale * LOG2E;
   const float la = row_a < S ? lse[sbase + row_a] * LOG2E : 0.f, lb = row_b < S ? lse[sbase + row_b] * LOG2E : 0.f;
-  const float da = row_a < S ? dsum[sbase + row_a] : 0.f, db = row_b < S ? dsum[sbase + row_b] : 0.f;
+  float da = 0.f, db = 0.f;                                  // D = rowsum(dO * O) of rows a and b, computed below
 
   float dq[DH / 8][4];
 #pragma unroll
@@ -302,6 +279,32 @@ fa_bwd_dq_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ dout, co
   for (int kb = 0; kb <= last_blk; ++kb) {
     if (kb < last_blk) { load_kv(kb + 1); cp_async_wait_group<1>(); } else { cp_async_wait_group<0>(); }
     __syncthreads();
+    if (kb == 0) {
+      // D_i = sum_c dO_i[c] O_i[c] for this warp's 16 rows: two lanes per row, half of the head dimension each.
+      // It is also written out for the dK / dV pass.
+      const int r = wrow0 + (lane >> 1), hf = lane & 1, grow = q0 + r;
+      float acc = 0.f;
+      if (grow < S) {
+        const bf16* op = out + ((long long)seq * S + grow) * d + (long long)h * DH + hf * (DH / 2);
+        const bf16* gp = Gs + r * RS + hf * (DH / 2);
+#pragma unroll
+        for (int v = 0; v < DH / 16; ++v) {
+          const uint4 ov = *reinterpret_cast<const uint4*>(op + v * 8);
+          const uint4 gv = *reinterpret_cast<const uint4*>(gp + v * 8);
+          const __nv_bfloat162* oh = reinterpret_cast<const __nv_bfloat162*>(&ov);
+          const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&gv);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 a = __bfloat1622float2(oh[e]), b = __bfloat1622float2(gh[e]);
+            acc = fmaf(a.x, b.x, fmaf(a.y, b.y, acc));
+          }
+        }
+      }
+      acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+      if (hf == 0 && grow < S) dsum[sbase + grow] = acc;
+      da = __shfl_sync(0xffffffffu, acc, 2 * g);
+      db = __shfl_sync(0xffffffffu, acc, 2 * (g + 8));
+    }
     const bf16* Ks = KV + (kb & 1) * STAGE;
     const bf16* Vs = Ks + FA_BLK * RS;
     float s[8][4], dp[8][4];
@@ -518,11 +521,8 @@ static int fa_bwd_launch(const void* qkv, const void* out, const void* dout, con
   const size_t smem_dkv = smem_dq + (size_t)2 * key_rows * sizeof(float);
   if (smem_dkv > 227 * 1024) return PCM_ERR_SHAPE;
   const float scale = 1.0f / sqrtf((float)DH);
-  const long long rows = (long long)n_seq * S * H;
-  fa_dsum_kernel<DH><<<ceil_div(rows, 8), 256, 0, s>>>((const bf16*)out, (const bf16*)dout, dsum, n_seq, S, H);
-  PCM_LAUNCH_CHECK();
   PCM_CUDA_TRY(cudaFuncSetAttribute(fa_bwd_dq_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dq));
-  fa_bwd_dq_kernel<DH><<<dim3(tiles, H, n_seq), FaCfg<DH>::THREADS, smem_dq, s>>>((const bf16*)qkv, (const bf16*)dout, lse, dsum,
+  fa_bwd_dq_kernel<DH><<<dim3(tiles, H, n_seq), FaCfg<DH>::THREADS, smem_dq, s>>>((const bf16*)qkv, (const bf16*)out, (const bf16*)dout, lse, dsum,
                                                                          (bf16*)dqkv, S, H, scale, rope_tab);
   PCM_LAUNCH_CHECK();
   PCM_CUDA_TRY(cudaFuncSetAttribute(fa_bwd_dkv_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dkv));

@@ -49,11 +49,13 @@ unsigned* ctx_status(pcm_ctx* c) { return c->status; }
 // ------------------------------------------------------------------------------------------------
 // Eq. 5, per group: integer token sums per (phase, outcome), then C_{c,g}
 // ------------------------------------------------------------------------------------------------
-// One CTA per group.  A warp walks whole trajectories; lanes 0..27 cover two chunks per step (14
-// words each).  Four tokens travel in one 32-bit word and are accumulated as two words of two 16-bit
-// lanes; a run ends when the phase changes or after 256 chunks (255 * 257 < 2^16), and is then
-// flushed to 32-bit shared-memory counters.  Integer sums are exact, so any order gives the same
-// result.
+// One CTA per group.  A warp walks whole trajectories.  Two consecutive chunks are 112 bytes = seven
+// 16-byte vectors, so lanes 0..27 load four chunk pairs per step (one per group of seven lanes); each lane owns the
+// same two 8-byte halves of every pair, i.e. the same 8 + 8 action dimensions of the pair's first or second
+// chunk.  Bytes are accumulated as packed 16-bit lanes; a run ends when the phase changes or after 256
+// chunks (255 * 257 < 2^16) and is flushed to 32-bit shared-memory counters.  Integer sums are exact, so
+// any order gives the same result.  A chunk at an odd index at either end of a trajectory (the vectors must
+// be 16-byte aligned) goes through a scalar path.
 __global__ void __launch_bounds__(256)
 score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restrict__ tok,
                     const uint8_t* __restrict__ phase, const uint8_t* __restrict__ reward, int G,
@@ -67,83 +69,133 @@ score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restr
   __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  const int sub = lane / WORDS;                          // 0, 1 active; 2 idle
-  const int word = lane - sub * WORDS;
+  const int slot = lane / 7, vec = lane - slot * 7;      // slot 0..3 active (4 = idle lanes 28..31)
   const uint32_t* tokw = reinterpret_cast<const uint32_t*>(tok);
 
   for (int i = g * G + warp; i < (g + 1) * G; i += nwarps) {
     const int o = reward[i] ? 1 : 0;
     const int a = traj_off[i], b = traj_off[i + 1];
-    unsigned acc_lo = 0, acc_hi = 0, run = 0;
-    int cur = -1;
-    auto flush = [&]() {
-      if (run) {
-        unsigned* s = sums + (cur * 2 + o) * ACT + word * 4;
-        atomicAdd(s + 0, acc_lo & 0xFFFFu);
-        atomicAdd(s + 1, acc_hi & 0xFFFFu);
-        atomicAdd(s + 2, acc_lo >> 16);
-        atomicAdd(s + 3, acc_hi >> 16);
-        if (word == 0) atomicAdd(cnt + cur * 2 + o, run);
+    // scalar path for one chunk: 14 lanes x 4 tokens
+    auto single = [&](int ch) {
+      if (lane < WORDS) {
+        const int ph = phase[ch];
+        if (ph >= n_phases) {
+          atomicOr(status, STATUS_BAD_PHASE);
+        } else {
+          const uint32_t wv = __ldg(tokw + (size_t)ch * WORDS + lane);
+          unsigned* sp = sums + (ph * 2 + o) * ACT + lane * 4;
+          atomicAdd(sp + 0, wv & 0xFFu);
+          atomicAdd(sp + 1, (wv >> 8) & 0xFFu);
+          atomicAdd(sp + 2, (wv >> 16) & 0xFFu);
+          atomicAdd(sp + 3, wv >> 24);
+          if (lane == 0) atomicAdd(cnt + ph * 2 + o, 1u);
+        }
       }
-      acc_lo = acc_hi = run = 0;
     };
-    if (sub < 2) {
-      constexpr int UNROLL = 8;                          // chunk pairs in flight per iteration
-      for (int ch0 = a + sub; ch0 < b; ch0 += 2 * UNROLL) {
-        uint32_t wv[UNROLL];
-        int ph[UNROLL];
+    int lo = a;
+    if ((lo & 1) && lo < b) { single(lo); ++lo; }        // pairs start at an even chunk index (16-byte alignment)
+    const int n_pairs = (b - lo) >> 1;
+    if (((b - lo) & 1) && lo < b) single(b - 1);
+
+    if (slot < 4) {
+      // this lane's two 8-byte halves of a pair: which chunk of the pair they belong to and their first dimension
+      const int bo0 = 16 * vec, bo1 = 16 * vec + 8;
+      const int sel[2] = {bo0 >= ACT ? 1 : 0, bo1 >= ACT ? 1 : 0};
+      const int dim0[2] = {bo0 >= ACT ? bo0 - ACT : bo0, bo1 >= ACT ? bo1 - ACT : bo1};
+      const bool counts[2] = {vec == 0, vec == 6};        // one half per chunk also counts the chunk
+      unsigned acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+      unsigned run[2] = {0, 0};
+      int cur[2] = {-1, -1};
+      auto flush = [&](int hf) {
+        if (run[hf]) {
+          unsigned* sp = sums + (cur[hf] * 2 + o) * ACT + dim0[hf];
+          atomicAdd(sp + 0, acc[hf][0] & 0xFFFFu); atomicAdd(sp + 2, acc[hf][0] >> 16);
+          atomicAdd(sp + 1, acc[hf][1] & 0xFFFFu); atomicAdd(sp + 3, acc[hf][1] >> 16);
+          atomicAdd(sp + 4, acc[hf][2] & 0xFFFFu); atomicAdd(sp + 6, acc[hf][2] >> 16);
+          atomicAdd(sp + 5, acc[hf][3] & 0xFFFFu); atomicAdd(sp + 7, acc[hf][3] >> 16);
+          if (counts[hf]) atomicAdd(cnt + cur[hf] * 2 + o, run[hf]);
+        }
+        acc[hf][0] = acc[hf][1] = acc[hf][2] = acc[hf][3] = 0;
+        run[hf] = 0;
+      };
+      constexpr int UNROLL = 4;                          // pair groups in flight per iteration
+      const uint4* tok16 = reinterpret_cast<const uint4*>(tok + (size_t)lo * ACT);
+      // each of the four lane groups walks its own contiguous quarter of the pairs: runs of equal phase stay long
+      const int per = (n_pairs + 3) >> 2;
+      const int p_end = min(n_pairs, (slot + 1) * per);
+      for (int p0 = slot * per; p0 < p_end; p0 += UNROLL) {
+        uint4 wv[UNROLL];
+        int ph[UNROLL][2];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-          const int ch = ch0 + 2 * u;
-          if (ch < b) {
-            wv[u] = __ldg(tokw + (size_t)ch * WORDS + word);
-            ph[u] = __ldg(phase + ch);
+          const int p = p0 + u;
+          if (p < p_end) {
+            wv[u] = __ldg(tok16 + (size_t)p * 7 + vec);
+            ph[u][0] = __ldg(phase + lo + 2 * p + sel[0]);
+            ph[u][1] = __ldg(phase + lo + 2 * p + sel[1]);
           } else {
-            wv[u] = 0;
-            ph[u] = -1;
+            wv[u] = make_uint4(0, 0, 0, 0);
+            ph[u][0] = ph[u][1] = -1;
           }
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-          if (ph[u] < 0) continue;
-          if (ph[u] >= n_phases) {
-            atomicOr(status, STATUS_BAD_PHASE);
-            continue;
+          const unsigned w4[4] = {wv[u].x, wv[u].y, wv[u].z, wv[u].w};
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            const int pv = ph[u][hf];
+            if (pv < 0) continue;
+            if (pv >= n_phases) {
+              atomicOr(status, STATUS_BAD_PHASE);
+              continue;
+            }
+            if (pv != cur[hf] || run[hf] == 256) {
+              flush(hf);
+              cur[hf] = pv;
+            }
+            acc[hf][0] += w4[2 * hf] & 0x00FF00FFu;
+            acc[hf][1] += (w4[2 * hf] >> 8) & 0x00FF00FFu;
+            acc[hf][2] += w4[2 * hf + 1] & 0x00FF00FFu;
+            acc[hf][3] += (w4[2 * hf + 1] >> 8) & 0x00FF00FFu;
+            ++run[hf];
           }
-          if (ph[u] != cur || run == 256) {
-            flush();
-            cur = ph[u];
-          }
-          acc_lo += wv[u] & 0x00FF00FFu;
-          acc_hi += (wv[u] >> 8) & 0x00FF00FFu;
-          ++run;
         }
       }
-      flush();
+      flush(0);
+      flush(1);
     }
   }
   __syncthreads();
 
-  // C_{c,g}: individually rounded fp64 operations in ascending-dimension order
-  for (int c = threadIdx.x; c < n_phases; c += blockDim.x) {
+  // C_{c,g}: individually rounded fp64 operations.  A warp per phase: the 56 squared differences are formed
+  // in parallel (two dimensions per lane), then lane 0 adds them in ascending-dimension order, which is the
+  // order the result is defined with.
+  __shared__ double sq[8][ACT];
+  for (int c = warp; c < n_phases; c += nwarps) {
     const unsigned n_succ = cnt[c * 2 + 1], n_fail = cnt[c * 2 + 0];
-    double val = 0.0;
-    uint8_t ok = 0;
-    if (n_succ && n_fail) {
-      double acc = 0.0;
+    const bool both = n_succ && n_fail;
+    if (both) {
       const unsigned* s1 = sums + (c * 2 + 1) * ACT;
       const unsigned* s0 = sums + (c * 2 + 0) * ACT;
-      for (int dim = 0; dim < ACT; ++dim) {
+      for (int dim = lane; dim < ACT; dim += 32) {
         const double m1 = __ddiv_rn((double)s1[dim], (double)n_succ);
         const double m0 = __ddiv_rn((double)s0[dim], (double)n_fail);
         const double diff = __dsub_rn(m1, m0);
-        acc = __dadd_rn(acc, __dmul_rn(diff, diff));
+        sq[warp][dim] = __dmul_rn(diff, diff);
       }
-      val = __dmul_rn(__dsqrt_rn(acc), 2.0 / 256.0);
-      ok = 1;
     }
-    c_group[(size_t)g * n_phases + c] = val;
-    valid_group[(size_t)g * n_phases + c] = ok;
+    __syncwarp();
+    if (lane == 0) {
+      double val = 0.0;
+      if (both) {
+        double acc = 0.0;
+        for (int dim = 0; dim < ACT; ++dim) acc = __dadd_rn(acc, sq[warp][dim]);
+        val = __dmul_rn(__dsqrt_rn(acc), 2.0 / 256.0);
+      }
+      c_group[(size_t)g * n_phases + c] = val;
+      valid_group[(size_t)g * n_phases + c] = both ? 1 : 0;
+    }
+    __syncwarp();
   }
 }
 
@@ -453,7 +505,7 @@ int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* b, double* C, uint8_t* valid
   int rc = check_batch(ctx, b);
   if (rc) return rc;
   if (!b->tok || !b->reward || !C || !valid) return PCM_ERR_ARG;
-  if (((uintptr_t)b->tok) & 3) return PCM_ERR_ARG;
+  if (((uintptr_t)b->tok) & 15) return PCM_ERR_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   const int G = ctx->cfg.group_size, Kc = ctx->cfg.n_phases, ng = b->n_traj / G;
   const size_t smem = (size_t)Kc * 2 * (ACT + 1) * sizeof(unsigned);
@@ -549,7 +601,7 @@ extern "C" int pcm_score_phases_static(int32_t n_phases, int32_t group_size, dou
   if (!b || !b->traj_off || !b->phase || !b->tok || !b->reward || !C || !valid) return PCM_ERR_ARG;
   if (n_phases < 1 || n_phases > PCM_MAX_PHASES || group_size < 1 || !(adv_eps >= 0.0)) return PCM_ERR_ARG;
   if (b->n_traj <= 0 || b->n_traj % group_size || b->n_chunks < 0) return PCM_ERR_ARG;
-  if (((uintptr_t)b->tok) & 3) return PCM_ERR_ARG;
+  if (((uintptr_t)b->tok) & 15) return PCM_ERR_ARG;
   const int ng = b->n_traj / group_size;
   if (ng > PCM_STATIC_MAX_GROUPS) return PCM_ERR_SHAPE;          // beyond the fixed scratch: refuse, do not truncate
   unsigned char* base = nullptr;
