@@ -199,6 +199,35 @@ __device__ __forceinline__ void unstage_bf16_rows(float* stage, int lane, const 
   __syncwarp();
 }
 
+// Row layout (thread = row, 32 fp32 columns, raw tcgen05.ld registers) into the staging buffer ...
+__device__ __forceinline__ void stage_put_rows(float* stage, int lane, const uint32_t (&r)[32]) {
+  float* srow = stage + lane * EPI_STAGE_STRIDE;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) *reinterpret_cast<uint4*>(srow + 4 * e) = make_uint4(r[4 * e], r[4 * e + 1], r[4 * e + 2], r[4 * e + 3]);
+}
+// ... and back out as 8 consecutive columns of row 8 i + lane / 4 (the layout of fetch_bf16_rows / bf16 stores)
+__device__ __forceinline__ void stage_get8(const float* stage, int lane, int i, float (&v)[8]) {
+  const float* sp = stage + (i * 8 + (lane >> 2)) * EPI_STAGE_STRIDE + (lane & 3) * 8;
+  const float4 a = *reinterpret_cast<const float4*>(sp), b = *reinterpret_cast<const float4*>(sp + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ uint4 pack8_bf16(const float (&v)[8]) {
+  __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 h2 = __floats2bfloat162_rn(v[4], v[5]), h3 = __floats2bfloat162_rn(v[6], v[7]);
+  uint4 o;
+  o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+  o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+  return o;
+}
+__device__ __forceinline__ void unpack8_bf16(const uint4& raw, float (&v)[8]) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = __bfloat1622float2(h[j]);
+    v[2 * j] = f.x; v[2 * j + 1] = f.y;
+  }
+}
+
 // Operands of the epilogue that are fetched one 32-column slice ahead of their use.
 struct EpiRegs {
   uint4 g[4], u[4];                           // EPI_SWIGLU_BWD: gate / up
@@ -238,16 +267,34 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
           tmem_ld_32x32(tmem_acc + (uint32_t)(128 + c0), ru);
           tmem_ld_wait();
           {
-            float g[32], u[32];
-#pragma unroll
-            for (int e = 0; e < 32; ++e) { g[e] = __uint_as_float(rg[e]); u[e] = __uint_as_float(ru[e]); }
+            // gate and up go through the staging buffer one after the other; the activation is formed and all
+            // three tensors are stored in the "eighth of a warp per row" layout
             const int row_base = row - lane_;
-            __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(p.C);
-            staged_store_bf16(stage, lane_, g, gu, p.ldc, row_base, p.M, hid0 + c0);
-            staged_store_bf16(stage, lane_, u, gu + F, p.ldc, row_base, p.M, hid0 + c0);
+            float gq[4][8];
+            stage_put_rows(stage, lane_, rg);
+            __syncwarp();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) g[e] = __fdividef(g[e], 1.f + __expf(-g[e])) * u[e];
-            staged_store_bf16(stage, lane_, g, p.out2, p.ld_out2, row_base, p.M, hid0 + c0);
+            for (int i = 0; i < 4; ++i) stage_get8(stage, lane_, i, gq[i]);
+            __syncwarp();
+            stage_put_rows(stage, lane_, ru);
+            __syncwarp();
+            __nv_bfloat16* gu = reinterpret_cast<__nv_bfloat16*>(p.C);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float u[8];
+              stage_get8(stage, lane_, i, u);
+              const int gr = row_base + i * 8 + (lane_ >> 2);
+              const uint4 pg = pack8_bf16(gq[i]), pu = pack8_bf16(u);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) u[e] = __fdividef(gq[i][e], 1.f + __expf(-gq[i][e])) * u[e];
+              if (gr < p.M) {
+                __nv_bfloat16* dst = gu + (long long)gr * p.ldc + hid0 + c0 + (lane_ & 3) * 8;
+                *reinterpret_cast<uint4*>(dst) = pg;
+                *reinterpret_cast<uint4*>(dst + F) = pu;
+                *reinterpret_cast<uint4*>(p.out2 + (long long)gr * p.ld_out2 + hid0 + c0 + (lane_ & 3) * 8) = pack8_bf16(u);
+              }
+            }
+            __syncwarp();
           }
         }
       } else if constexpr (EPI == EPI_ROPE) {
@@ -302,26 +349,43 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
         tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
         tmem_ld_wait();
         if constexpr (EPI == EPI_SWIGLU_BWD) {
-          // r = d(act) in fp32; gate | up come from aux (fetched one slice ahead); d(gate) | d(up) go to C
+          // r = d(act) in fp32 goes through the staging buffer into the "eighth of a warp per row" layout, where
+          // gate | up (fetched one slice ahead in that layout) are combined with it and d(gate) | d(up) are stored
           const int F = p.N, row_base = row - lane_;
-          float g[32], u[32];
-          unstage_bf16_rows(stage, lane_, pre.g, g);
-          unstage_bf16_rows(stage, lane_, pre.u, u);
+          stage_put_rows(stage, lane_, r);
+          __syncwarp();
+          uint4 og[4], ou[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float da[8], g[8], u[8];
+            stage_get8(stage, lane_, i, da);
+            unpack8_bf16(pre.g[i], g);
+            unpack8_bf16(pre.u[i], u);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float sg = __fdividef(1.f, 1.f + __expf(-g[e]));
+              const float dg = da[e] * u[e] * sg * (1.f + g[e] * (1.f - sg));
+              u[e] = da[e] * g[e] * sg;
+              g[e] = dg;
+            }
+            og[i] = pack8_bf16(g);
+            ou[i] = pack8_bf16(u);
+          }
+          __syncwarp();
           if (c0 + 32 < (chalf + 1) * (BN / 2) && col + 32 < p.N) {
             fetch_bf16_rows(p.aux, p.ld_aux, row_base, p.M, col + 32, lane_, pre.g);
             fetch_bf16_rows(p.aux + F, p.ld_aux, row_base, p.M, col + 32, lane_, pre.u);
           }
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const float da = __uint_as_float(r[e]);
-            const float sg = __fdividef(1.f, 1.f + __expf(-g[e]));
-            const float dg = da * u[e] * sg * (1.f + g[e] * (1.f - sg));
-            u[e] = da * g[e] * sg;
-            g[e] = dg;
-          }
           __nv_bfloat16* Cb = reinterpret_cast<__nv_bfloat16*>(p.C);
-          staged_store_bf16(stage, lane_, g, Cb, p.ldc, row_base, p.M, col);
-          staged_store_bf16(stage, lane_, u, Cb + F, p.ldc, row_base, p.M, col);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int gr = row_base + i * 8 + (lane_ >> 2);
+            if (gr < p.M) {
+              __nv_bfloat16* dst = Cb + (long long)gr * p.ldc + col + (lane_ & 3) * 8;
+              *reinterpret_cast<uint4*>(dst) = og[i];
+              *reinterpret_cast<uint4*>(dst + F) = ou[i];
+            }
+          }
         } else if (p.reduce) {
           if (row < p.M) {
             float* dst = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
