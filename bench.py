@@ -23,6 +23,11 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
+# DRAM traffic of the dominant kernel from one ncu capture (profiles/gemm_tc2_kernel_M19968_N3072_K1024_ncu.md):
+# dram__bytes_read.sum + dram__bytes_write.sum = 120.1 MB for the QKV-shaped launch at M = 19968 rows against
+# 169.9 MB of algorithmic bytes; traffic grows in proportion to the rows for a fixed weight matrix.
+GEMM_TRAFFIC_CAPTURE = {"rows": 19968, "n": 3072, "k": 1024, "dram_bytes": 120.1e6, "algorithmic_bytes": 169.9e6}
+
 METRIC = "kept_chunks_per_s_actor_fwd_bwd"
 UNIT = "chunks/s"
 ACT = 56
@@ -341,7 +346,10 @@ def run_cuda(args):
                        "tokens_per_step": n_kept * w.S, "mb_chunks": mb, "l2": "inputs_larger_than_l2",
                        "multi_gpu": "independent replicas, no collective"},
             "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak,
-                         "unit": "TFLOP/s", "frac": achieved / peak if peak else None, "traffic": None,
+                         "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
+                         "traffic": GEMM_TRAFFIC_CAPTURE["dram_bytes"] * (n_kept * w.S) / GEMM_TRAFFIC_CAPTURE["rows"]
+                         if (w.d == 1024 and mb >= n_kept) else None,
+                         "traffic_of": "QKV-shaped launch [tokens x 3072 x 1024], ncu capture at 19968 rows scaled by rows",
                          "peak_source": peaks["source"] + " bf16_tflops_sustained",
                          "launches_per_step": g["launches"] / args.steps,
                          "flops_per_launch": g["flops"] / max(1, g["launches"]),

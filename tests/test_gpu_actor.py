@@ -155,6 +155,8 @@ BF16_CASES = {
     "c1_layer": dict(n_tasks=1, G=4, T=8, n_phases=4, budget=1, P=256, d=1024, L=1, H=16, max_kept=3),
     # head dim 128 as in the large model
     "dh128": dict(n_tasks=1, G=4, T=8, n_phases=4, budget=1, P=72, d=256, L=2, H=2, max_kept=4),
+    # one layer of the large model at its real width, head dim and sequence length (2 * 312 tokens)
+    "c3_layer": dict(n_tasks=1, G=4, T=8, n_phases=4, budget=1, P=256, d=2048, L=1, H=16, max_kept=2),
 }
 
 
