@@ -176,7 +176,7 @@ def run_cuda(args):
 
     from paper_2605_16154_b200 import build as _build
     _build.build()
-    from paper_2605_16154_b200 import binding as B, pipeline as PL, synth
+    from paper_2605_16154_b200 import binding as B, dist_util, pipeline as PL, synth
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -187,7 +187,7 @@ def run_cuda(args):
 
     w = synth.WORKLOADS[args.workload]
     td = PL.torch_dtype(w)
-    seed = w.seed + 1000 * rank                    # every rank works on its own batch (replicas, no exchange)
+    seed = dist_util.replica_seed(w.seed, rank)    # every rank works on its own batch (replicas, no exchange)
     rb = synth.make_rollouts(w, seed)
     weights = synth.make_weights(w)
     lengths = np.diff(rb["traj_off"])
@@ -284,12 +284,7 @@ def run_cuda(args):
             fn(it0 + i)
         ev1.record()
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return dist_util.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
 
     it = 0
     for _ in range(max(args.warmup, 3)):
@@ -322,8 +317,8 @@ def run_cuda(args):
     if rank == 0:
         peaks = measured_peaks()
         ms_step = ms_total / args.steps
-        value = world * n_kept * args.steps / (ms_total / 1e3)
-        e2e_value = world * n_kept * args.steps / (ms_e2e / 1e3)
+        value = dist_util.aggregate_throughput(n_kept, args.steps, ms_total, world)
+        e2e_value = dist_util.aggregate_throughput(n_kept, args.steps, ms_e2e, world)
         g = prof["gemm"]
         achieved = g["flops"] / (g["ms"] * 1e9) if g["ms"] > 0 else 0.0
         peak = peaks["bf16_tflops_sustained"]

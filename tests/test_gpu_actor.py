@@ -190,3 +190,61 @@ def test_argument_errors():
     bad = B.Model(w.d, w.L, 3, w.P, B.GRPO_F32, model.weights)          # d not divisible by heads
     with pytest.raises(B.PcmError):
         B.grpo_actor_fwd_bwd(bad, pk)
+
+
+def test_empty_batch_and_shape_limits():
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"]
+    hp = host_problem(w)
+    model = PL.upload_model(w, hp["weights"])
+    empty = B.Packed(model, 0)
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, empty)
+    assert float(loss.item()) == 0.0 and logp.shape[0] == 0
+    assert all(float(g.abs().max()) == 0.0 for g in grads.values())
+    # longest supported sequence is 384 tokens; one more is refused on the host
+    ok = B.Model(w.d, w.L, w.H, 384 - 56, B.GRPO_F32, model.weights)
+    assert B.grpo_workspace_bytes(ok, 1) > 0
+    too_long = B.Model(w.d, w.L, w.H, 384 - 56 + 1, B.GRPO_F32, model.weights)
+    assert B.grpo_workspace_bytes(too_long, 1) == 0
+    with pytest.raises(B.PcmError) as e:
+        B.grpo_actor_fwd_bwd(too_long, B.Packed(too_long, 1))
+    assert e.value.code == -2
+
+
+def test_longest_sequence_bf16_and_ragged_micro_batches():
+    """S = 384 (six full 64-row attention tiles), 7 kept chunks in micro-batches of 3, 3, 1."""
+    B, PL = _mods()
+    w = synth.WORKLOADS["C1"].with_(n_tasks=1, G=4, T=8, n_phases=4, budget=2, P=328, d=256, L=1, H=4,
+                                    gamma_std=0.1, force_mixed=True, p_succ=0.5)
+    hp = host_problem(w, seed=5, max_kept=7, clip_margin=0.05)
+    _compare(B, PL, hp, BF16_GRAD_TOL, tol_loss_abs=BF16_LOSS_TOL, mb=3)
+
+
+def test_ragged_rollouts_through_the_whole_c_abi_chain_bf16():
+    """C4-shaped batch (lengths 3..12, some below the budget, random phase cuts) on a small bf16 model:
+    selection and pack bit-exact, update within the bf16 tolerances."""
+    B, PL = _mods()
+    w = synth.WORKLOADS["C4"].with_(n_tasks=2, G=4, d=256, L=2, H=4, P=40, len_lo=3, len_hi_succ=9, len_hi_fail=12,
+                                    n_phases=3, budget=5, gamma_std=0.1, force_mixed=True, p_succ=0.5)
+    hp = host_problem(w, seed=8, clip_margin=0.05)
+    lengths = np.diff(hp["rb"]["traj_off"])
+    assert lengths.min() < w.budget < lengths.max()
+    model = PL.upload_model(w, hp["weights"])
+    total = int(hp["rb"]["traj_off"][-1])
+    obs = synth.obs_all(w, 8, total)
+    lpo_all = np.zeros((total, 56), dtype=np.float32)
+    lpo_all[hp["kept"]] = hp["lpo"]
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=7 + 8, max_traj=w.n_traj)
+    batch = PL.upload_rollouts(w, hp["rb"], obs=PL.dev(obs, torch.bfloat16), logp_old=PL.dev(lpo_all))
+    adv, Cc, valid, p, q, kept_idx, kept_off, _ = PL.select(ctx, batch, 0)
+    n_kept = PL.n_kept_of(w.budget, hp["rb"]["traj_off"])
+    assert n_kept == len(hp["kept"]) and np.array_equal(kept_idx.cpu().numpy()[:n_kept], hp["kept"])
+    pk = B.grpo_pack_chunks(ctx, batch, model, kept_idx, kept_off, adv, B.Packed(model, n_kept))
+    assert B.pcm_poll_status(ctx) == 0
+    assert np.array_equal(pk.X.float().cpu().numpy(), hp["X"].astype(np.float32))
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, pk, mb_chunks=16)
+    loss_o, _, grads_o, stats_o = oracle_update(hp)
+    assert abs(float(loss.item()) - loss_o) < BF16_LOSS_TOL
+    errs = {k: rel_fro(v, grads_o[k]) for k, v in grads_to_numpy(grads).items()}
+    assert max(errs.values()) < BF16_GRAD_TOL, errs
+    ctx.close()
