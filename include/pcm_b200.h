@@ -251,6 +251,24 @@ int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* batch, const 
                        grpo_grads* grads, float* loss, float* logp, grpo_stats* stats,
                        void* workspace, size_t workspace_bytes, pcm_stream stream);
 
+/* ---- optimizer step (App. E: AdamW, lr 1e-5, betas (0.9, 0.999), weight decay 0, clipping at 2.0) -----
+ * The step that follows grpo_actor_fwd_bwd.  Global L2 norm of all gradients (fp64 partial sums in a fixed
+ * order), clip coefficient min(1, max_grad_norm / (norm + 1e-6)) (max_grad_norm = 0: no clipping), then per
+ * parameter, with g the clipped gradient and t = step (counted from 1):
+ *     m = beta1 m + (1 - beta1) g;  v = beta2 v + (1 - beta2) g^2;
+ *     w = w - lr * ( (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps) + weight_decay * w )
+ * on fp32 master weights; the weights of `model` (cfg.dtype, device, WRITTEN by this call) receive the
+ * rounded masters.  master, m, v, grads: fp32 tensors with the shapes of grpo_model.  grad_norm (device
+ * [1], may be NULL) receives the norm before clipping.  scratch: device, 256-byte aligned,
+ * >= grpo_adamw_scratch_bytes(). */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay, max_grad_norm;
+} grpo_adamw_cfg;
+size_t grpo_adamw_scratch_bytes(void);
+int grpo_adamw_step(const grpo_model_cfg* cfg, const grpo_adamw_cfg* opt, int64_t step, grpo_model* model,
+                    grpo_grads* master, const grpo_grads* grads, grpo_grads* m, grpo_grads* v, float* grad_norm,
+                    void* scratch, size_t scratch_bytes, pcm_stream stream);
+
 /* ---- diagnostic entry points (per-kernel tests and measurements; not part of Algorithm 1) -------
  * grpo_gemm: C[m][n] = sum_k A(m,k) B(n,k) (+ R[m][n]) with the GEMM kernels the actor update uses.
  * a_kmajor != 0: A is stored [M][K] with row stride lda, else [K][M]; likewise B ([N][K] / [K][N]).

@@ -76,6 +76,11 @@ class grpo_stats(C.Structure):
                 ("workspace_high_water", C.c_uint64)]
 
 
+class grpo_adamw_cfg(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("max_grad_norm", C.c_float)]
+
+
 PROFILE_CLASSES = ("gemm", "attention", "rmsnorm", "elementwise", "loss", "embed_grad", "pack", "pcm_score", "pcm_sample")
 
 
@@ -104,6 +109,11 @@ _lib.grpo_gemm.argtypes = [C.c_int32, C.c_int32, C.c_int32, _P, C.c_int64, C.c_i
 _lib.grpo_attention.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P]
 _lib.pcm_score_phases_static.argtypes = [C.c_int32, C.c_int32, C.c_double, C.POINTER(pcm_batch), _P, _P, _P, _P, _P, _P]
 _lib.pcm_score_phases_static.restype = C.c_int
+_lib.grpo_adamw_scratch_bytes.restype = C.c_size_t
+_lib.grpo_adamw_step.argtypes = [C.POINTER(grpo_model_cfg), C.POINTER(grpo_adamw_cfg), C.c_int64, C.POINTER(grpo_model),
+                                 C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.POINTER(grpo_grads),
+                                 _P, _P, C.c_size_t, _P]
+_lib.grpo_adamw_step.restype = C.c_int
 _lib.pcm_launch_count.restype = C.c_int64
 _lib.pcm_profile_enable.argtypes = [C.c_int32]
 _lib.pcm_profile_read.argtypes = [C.POINTER(pcm_profile)]
@@ -115,7 +125,8 @@ for _name in ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export"
 EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", "pcm_state_import",
             "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
-            "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static")
+            "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static",
+            "grpo_adamw_scratch_bytes", "grpo_adamw_step")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -360,3 +371,33 @@ def pcm_profile_read() -> Dict[str, Dict[str, float]]:
     _check("pcm_profile_read", _lib.pcm_profile_read(C.byref(prof)))
     return {name: {"ms": prof.ms[i], "flops": prof.flops[i], "bytes": prof.bytes[i], "launches": int(prof.launches[i])}
             for i, name in enumerate(PROFILE_CLASSES)}
+
+
+class AdamW:
+    """fp32 master weights and moments for a Model, stepped by grpo_adamw_step."""
+
+    def __init__(self, model: Model, lr: float = 1e-5, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                 weight_decay: float = 0.0, max_grad_norm: float = 2.0):
+        self.model = model
+        self.cfg = grpo_adamw_cfg(lr, beta1, beta2, eps, weight_decay, max_grad_norm)
+        self.master = {k: v.float().contiguous() for k, v in model.weights.items()}
+        self.m = {k: torch.zeros_like(v) for k, v in self.master.items()}
+        self.v = {k: torch.zeros_like(v) for k, v in self.master.items()}
+        self.c_master = grpo_grads(*[_ptr(self.master[k]) for k in _WEIGHTS])
+        self.c_m = grpo_grads(*[_ptr(self.m[k]) for k in _WEIGHTS])
+        self.c_v = grpo_grads(*[_ptr(self.v[k]) for k in _WEIGHTS])
+        n = int(_lib.grpo_adamw_scratch_bytes())
+        self.scratch = torch.empty(n + 256, dtype=torch.uint8, device="cuda")
+        self.grad_norm = torch.zeros(1, dtype=torch.float32, device="cuda")
+        self.step_count = 0
+
+    def step(self) -> torch.Tensor:
+        """Applies the model's current gradients; returns the (device) gradient norm before clipping."""
+        assert self.model.c_grads is not None, "run grpo_actor_fwd_bwd first"
+        self.step_count += 1
+        off = (-self.scratch.data_ptr()) % 256
+        _check("grpo_adamw_step",
+               _lib.grpo_adamw_step(C.byref(self.model.cfg), C.byref(self.cfg), self.step_count, C.byref(self.model.c_model),
+                                    C.byref(self.c_master), C.byref(self.model.c_grads), C.byref(self.c_m), C.byref(self.c_v),
+                                    _ptr(self.grad_norm), self.scratch.data_ptr() + off, self.scratch.numel() - off, _stream()))
+        return self.grad_norm
