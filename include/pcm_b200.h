@@ -134,6 +134,21 @@ int pcm_score_phases_static(int32_t n_phases, int32_t group_size, double adv_eps
                             double* C, uint8_t* valid, int32_t* n_valid_groups, float* adv,
                             uint32_t* device_status, pcm_stream stream);
 
+/* ---- phase labelling (Sec. 5.1 "Phase Labeling", App. E.2; Algorithm 1, the step before scoring) -------
+ * Labels every chunk with one of five phases from the per-timestep gripper-close command:
+ * 0 approach, 1 pre-grasp, 2 active-grip, 3 release-ramp, 4 tail.  g_f = fraction of the chunk's timesteps
+ * with the command active (the last chunk of a trajectory may be shorter than chunk_len).  A sustained-close
+ * interval is a maximal run of chunks with g_f >= 0.75.  active-grip: g_f >= 0.5.  pre-grasp: the three chunk
+ * positions before a sustained interval, where 0.1 <= g_f < 0.5.  release-ramp: the three positions after
+ * it, where g_f < 0.5.  Overlaps resolve by active-grip > pre-grasp > release-ramp > approach > tail.  Chunks
+ * left over: approach when a sustained interval starts later; tail when after the last one with g_f < 0.1;
+ * approach otherwise.  Fractions are compared through integer counts.
+ * Inputs (device): traj_off[n_traj+1] in chunks, step_off[n_traj+1] in timesteps with
+ * N_i = ceil(T_i / chunk_len) (a mismatch is latched in the status word), grip_close[total timesteps]
+ * (non-zero = close).  Output: device phase[n_chunks]. */
+int pcm_label_phases(pcm_ctx* ctx, int32_t n_traj, const int32_t* traj_off, const int32_t* step_off,
+                     const uint8_t* grip_close, int32_t chunk_len, uint8_t* phase, pcm_stream stream);
+
 /* ---- Eq. 7-9, Algorithm 1 ---------------------------------------------------------------------
  * Appends C (0 where valid[c] == 0) to the phase buffers.  On the first call, or when the buffers
  * hold t_rc entries: S_c = sum of buffer, rho_c = S_c / sum S, rho~_c = rho_c / max rho,

@@ -109,6 +109,8 @@ _lib.grpo_gemm.argtypes = [C.c_int32, C.c_int32, C.c_int32, _P, C.c_int64, C.c_i
 _lib.grpo_attention.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P]
 _lib.pcm_score_phases_static.argtypes = [C.c_int32, C.c_int32, C.c_double, C.POINTER(pcm_batch), _P, _P, _P, _P, _P, _P]
 _lib.pcm_score_phases_static.restype = C.c_int
+_lib.pcm_label_phases.argtypes = [_P, C.c_int32, _P, _P, _P, C.c_int32, _P, _P]
+_lib.pcm_label_phases.restype = C.c_int
 _lib.grpo_adamw_scratch_bytes.restype = C.c_size_t
 _lib.grpo_adamw_step.argtypes = [C.POINTER(grpo_model_cfg), C.POINTER(grpo_adamw_cfg), C.c_int64, C.POINTER(grpo_model),
                                  C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.POINTER(grpo_grads),
@@ -126,7 +128,7 @@ EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", 
             "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
             "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static",
-            "grpo_adamw_scratch_bytes", "grpo_adamw_step")
+            "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -221,6 +223,16 @@ def pcm_score_phases_static(n_phases: int, group_size: int, adv_eps: float, batc
                                         _ptr(out.get("n_valid")), _ptr(out.get("adv")), _ptr(out.get("status")),
                                         _stream()))
     return out
+
+
+def pcm_label_phases(ctx: Context, traj_off: torch.Tensor, step_off: torch.Tensor, grip_close: torch.Tensor,
+                     chunk_len: int = 8, phase: Optional[torch.Tensor] = None) -> torch.Tensor:
+    n_traj = traj_off.numel() - 1
+    if phase is None:
+        phase = torch.empty(int(traj_off[-1].item()), dtype=torch.uint8, device=traj_off.device)
+    _check("pcm_label_phases", _lib.pcm_label_phases(ctx.handle, n_traj, _ptr(traj_off), _ptr(step_off), _ptr(grip_close),
+                                                     chunk_len, _ptr(phase), _stream()))
+    return phase
 
 
 def pcm_update_keep_probs(ctx: Context, Cc: torch.Tensor, valid: torch.Tensor):
