@@ -59,7 +59,15 @@ typedef struct {
   double p_min;                /* keep-probability floor, in (0, 1]                               */
   double adv_eps;              /* epsilon of Eq. 1                                                */
   uint64_t seed;               /* Philox key of the sampler                                       */
+  int32_t mode;                /* pcm_mask_mode: how keep-probabilities are formed                */
+  int32_t reserved;
 } pcm_config;
+
+/* PCM_MASK_PCM: Eq. 8-9.  The other two are the ablations of RQ4: PCM_MASK_RANDOM keeps every phase at
+ * weight 1 (B chunks uniformly at random per trajectory); PCM_MASK_FULL gives weight 1 to the single
+ * highest-S_c phase (first one on ties) and 0 to all others, so only chunks of that phase are kept and a
+ * trajectory keeps min(B, its chunks in that phase). */
+typedef enum { PCM_MASK_PCM = 0, PCM_MASK_RANDOM = 1, PCM_MASK_FULL = 2 } pcm_mask_mode;
 
 typedef struct {
   int32_t n_traj;              /* multiple of group_size                                          */
@@ -161,11 +169,12 @@ int pcm_update_keep_probs(pcm_ctx* ctx, const double* C, const uint8_t* valid, f
 
 /* ---- Eq. 10 -----------------------------------------------------------------------------------
  * For every trajectory draws m_i = min(budget, N_i) chunks by successive sampling without
- * replacement (Plackett-Luce) with integer weights w_ik = q[phase(i,k)].  Draw r of trajectory i
+ * replacement (Plackett-Luce) with integer weights w_ik = q[phase(i,k)]; chunks of weight 0 (only with
+ * PCM_MASK_FULL) are never kept and N_i then counts the chunks of positive weight.  Draw r of trajectory i
  * takes 64 bits from Philox4x32-10 with key (seed lo, seed hi) and counter (iter lo, i, r, iter hi),
  * maps them to x = floor(bits * W_remaining / 2^64) and selects the first remaining chunk, in index
  * order, whose running weight sum exceeds x.  When m_i = N_i every chunk is kept and no random
- * numbers are consumed.  max_len <= 12000.
+ * numbers are consumed.  max_len <= 12000.  Uses n_traj ints of context scratch.
  * Outputs: device kept_idx[sum m_i] i32 global chunk ids, trajectory-major and ascending within a
  * trajectory (capacity n_traj*budget is always enough); kept_off[n_traj+1] i32;
  * kept_per_phase[n_phases] i32 (may be NULL). */

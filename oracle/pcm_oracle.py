@@ -120,7 +120,8 @@ def score_phases(traj_off, tok, phase, reward, G: int, n_phases: int):
 class KeepProbState:
     """Phase-score buffers B_c, the step counter and the current keep-probabilities p_c."""
 
-    def __init__(self, n_phases: int, p_min: float = 0.1, t_rc: int = 5):
+    def __init__(self, n_phases: int, p_min: float = 0.1, t_rc: int = 5, mode: int = 0):
+        self.mode = int(mode)              # 0 PCM (Eq. 8-9); 1 random masking; 2 full masking (ablations of RQ4)
         self.n_phases = n_phases
         self.p_min = float(p_min)
         self.t_rc = int(t_rc)
@@ -154,15 +155,22 @@ def update_keep_probs(state: KeepProbState, C: Sequence[float], valid: Sequence[
         s_tot = 0.0
         for c in range(K):
             s_tot = s_tot + S[c]
-        if s_tot > 0.0:
+        if state.mode == 1:
+            pass                                     # random masking: every phase keeps weight 1 (uniform sampling)
+        elif s_tot > 0.0:
             rho = [S[c] / s_tot for c in range(K)]
             rho_max = 0.0
+            c_max = 0
             for c in range(K):
                 if rho[c] > rho_max:
                     rho_max = rho[c]
+                    c_max = c
             for c in range(K):
-                rho_t = rho[c] / rho_max
-                state.p[c] = rho_t if rho_t > state.p_min else state.p_min
+                if state.mode == 2:                  # full masking: only the single highest-C_c phase survives
+                    state.p[c] = 1.0 if c == c_max else 0.0
+                else:
+                    rho_t = rho[c] / rho_max
+                    state.p[c] = rho_t if rho_t > state.p_min else state.p_min
         for c in range(K):
             state.buf[c] = []
         refreshed = True
@@ -209,7 +217,8 @@ def draw_bits(seed: int, it: int, traj: int, draw: int) -> int:
 # ----------------------------------------------------------------------------------------------
 def sample_one_trajectory(weights: Sequence[int], m: int, bits: Sequence[int]) -> List[int]:
     """Successive (Plackett-Luce) sampling: m times, pick a remaining chunk with probability
-    proportional to its integer weight and remove it.  Draw r maps its 64 random bits to
+    proportional to its integer weight and remove it (chunks of weight 0 are never picked; the caller
+    passes m <= number of positive weights).  Draw r maps its 64 random bits to
     x = floor(bits * W_remaining / 2^64) and selects the first remaining chunk, in index order,
     whose running weight sum exceeds x.  Returns the kept chunk positions in ascending order."""
     w = [int(v) for v in weights]
@@ -244,8 +253,8 @@ def sample_chunks(traj_off, phase, q, budget: int, seed: int, it: int):
     kept_per_phase = np.zeros(len(q), dtype=np.int32)
     for i in range(n_traj):
         a, b = int(traj_off[i]), int(traj_off[i + 1])
-        m = min(budget, b - a)
         weights = [int(q[int(phase[ch])]) for ch in range(a, b)]
+        m = min(budget, sum(1 for wk in weights if wk > 0))      # |K_i| = min(B, N_i) over the chunks that can be kept
         bits = [draw_bits(seed, it, i, r) for r in range(m)]
         for k in sample_one_trajectory(weights, m, bits):
             kept_idx.append(a + k)

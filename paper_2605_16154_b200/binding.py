@@ -23,6 +23,7 @@ ACT_DIM = 56
 N_BINS = 256
 GRPO_F32, GRPO_BF16 = 0, 1
 GRPO_FWD_ONLY, GRPO_ACCUMULATE = 1, 2
+MASK_PCM, MASK_RANDOM, MASK_FULL = 0, 1, 2
 
 STATUS_NAMES = {0: "PCM_OK", -1: "PCM_ERR_ARG", -2: "PCM_ERR_SHAPE", -3: "PCM_ERR_WORKSPACE", -4: "PCM_ERR_CUDA",
                 -5: "PCM_ERR_DEVICE_TIMEOUT", -6: "PCM_ERR_STATE", -7: "PCM_ERR_DEVICE_DATA"}
@@ -36,7 +37,8 @@ class PcmError(RuntimeError):
 
 class pcm_config(C.Structure):
     _fields_ = [("n_phases", C.c_int32), ("budget", C.c_int32), ("group_size", C.c_int32), ("t_rc", C.c_int32),
-                ("p_min", C.c_double), ("adv_eps", C.c_double), ("seed", C.c_uint64)]
+                ("p_min", C.c_double), ("adv_eps", C.c_double), ("seed", C.c_uint64), ("mode", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class pcm_batch(C.Structure):
@@ -156,9 +158,9 @@ class Context:
     """Owns a pcm_ctx (configuration + persistent keep-probability state on the device)."""
 
     def __init__(self, n_phases: int, budget: int, group_size: int, t_rc: int = 5, p_min: float = 0.1,
-                 adv_eps: float = 1e-6, seed: int = 0, max_traj: int = 1024):
+                 adv_eps: float = 1e-6, seed: int = 0, max_traj: int = 1024, mode: int = 0):
         self.handle = _P()
-        self.cfg = pcm_config(n_phases, budget, group_size, t_rc, p_min, adv_eps, seed)
+        self.cfg = pcm_config(n_phases, budget, group_size, t_rc, p_min, adv_eps, seed, mode, 0)
         _check("pcm_create", _lib.pcm_create(C.byref(self.handle), C.byref(self.cfg), max_traj))
 
     def close(self):

@@ -40,6 +40,7 @@ struct pcm_ctx {
   unsigned* status;            // device status word
   double* c_group;             // device [max_groups][n_phases]
   uint8_t* valid_group;        // device [max_groups][n_phases]
+  int32_t* n_pos;              // device [max_traj]: chunks of positive weight per trajectory (sampler scratch)
 };
 
 namespace pcm {
@@ -251,7 +252,8 @@ __global__ void score_finalize_kernel(const double* __restrict__ c_group,
 // ------------------------------------------------------------------------------------------------
 __global__ void update_keep_probs_kernel(KeepState* st, const double* __restrict__ C,
                                          const uint8_t* __restrict__ valid, int n_phases, int t_rc,
-                                         double p_min, float* __restrict__ p_out, uint32_t* __restrict__ q_out) {
+                                         double p_min, int mode, float* __restrict__ p_out,
+                                         uint32_t* __restrict__ q_out) {
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
   for (int c = 0; c < n_phases; ++c) st->buf[c][st->count] = valid[c] ? C[c] : 0.0;
   st->count += 1;
@@ -264,15 +266,20 @@ __global__ void update_keep_probs_kernel(KeepState* st, const double* __restrict
       S[c] = s;
     }
     for (int c = 0; c < n_phases; ++c) tot = __dadd_rn(tot, S[c]);
-    if (tot > 0.0) {
+    if (mode != PCM_MASK_RANDOM && tot > 0.0) {
       double rho_max = 0.0;
+      int c_max = 0;
       for (int c = 0; c < n_phases; ++c) {
         S[c] = __ddiv_rn(S[c], tot);                      // share rho_c
-        if (S[c] > rho_max) rho_max = S[c];
+        if (S[c] > rho_max) { rho_max = S[c]; c_max = c; }
       }
       for (int c = 0; c < n_phases; ++c) {
-        const double r = __ddiv_rn(S[c], rho_max);        // rho~_c
-        st->p[c] = r > p_min ? r : p_min;
+        if (mode == PCM_MASK_FULL) {
+          st->p[c] = c == c_max ? 1.0 : 0.0;              // only the highest-S_c phase survives
+        } else {
+          const double r = __ddiv_rn(S[c], rho_max);      // rho~_c
+          st->p[c] = r > p_min ? r : p_min;
+        }
       }
     }
     st->count = 0;
@@ -301,15 +308,32 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
   o0 = c0; o1 = c1;
 }
 
-// kept_off = exclusive prefix sum of min(budget, N_i); single block.
-__global__ void kept_offsets_kernel(const int32_t* __restrict__ traj_off, int n_traj, int budget,
+// n_pos[i] = chunks of trajectory i whose phase has a positive weight; one warp per trajectory
+__global__ void count_positive_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restrict__ phase,
+                                      const uint32_t* __restrict__ q, int n_traj, int n_phases,
+                                      int32_t* __restrict__ n_pos) {
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (i >= n_traj) return;
+  const int a = traj_off[i], b = traj_off[i + 1];
+  int c = 0;
+  for (int k = a + lane; k < b; k += 32) {
+    const int ph = phase[k];
+    c += (ph < n_phases && q[ph] != 0) ? 1 : 0;
+  }
+#pragma unroll
+  for (int off = 16; off; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+  if (lane == 0) n_pos[i] = c;
+}
+
+// kept_off = exclusive prefix sum of min(budget, n_pos[i]); single block.
+__global__ void kept_offsets_kernel(const int32_t* __restrict__ n_pos, int n_traj, int budget,
                                     int32_t* __restrict__ kept_off) {
   __shared__ int part[1024];
   const int t = threadIdx.x, nt = blockDim.x;
   const int per = (n_traj + nt - 1) / nt;
   const int lo = min(t * per, n_traj), hi = min(lo + per, n_traj);
   int s = 0;
-  for (int i = lo; i < hi; ++i) s += min(budget, traj_off[i + 1] - traj_off[i]);
+  for (int i = lo; i < hi; ++i) s += min(budget, n_pos[i]);
   part[t] = s;
   __syncthreads();
   for (int off = 1; off < nt; off <<= 1) {               // Hillis-Steele inclusive scan
@@ -321,7 +345,7 @@ __global__ void kept_offsets_kernel(const int32_t* __restrict__ traj_off, int n_
   int run = part[t] - s;
   for (int i = lo; i < hi; ++i) {
     kept_off[i] = run;
-    run += min(budget, traj_off[i + 1] - traj_off[i]);
+    run += min(budget, n_pos[i]);
   }
   if (t == nt - 1) kept_off[n_traj] = part[nt - 1];
 }
@@ -343,20 +367,25 @@ sample_chunks_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __rest
     if (lane == 0) atomicOr(status, STATUS_TOO_LONG);
     return;
   }
-  const int m = min(budget, N);
   unsigned long long W = 0;
+  int n_pos = 0;                                          // chunks that can be kept at all (weight > 0)
   for (int k = lane; k < N; k += 32) {
     const int ph = phase[a + k];
     unsigned wk = 0;
     if (ph < n_phases) wk = q[ph]; else atomicOr(status, STATUS_BAD_PHASE);
     w[k] = wk;
     W += wk;
+    n_pos += wk ? 1 : 0;
   }
 #pragma unroll
-  for (int off = 16; off; off >>= 1) W += __shfl_xor_sync(0xffffffffu, W, off);
+  for (int off = 16; off; off >>= 1) {
+    W += __shfl_xor_sync(0xffffffffu, W, off);
+    n_pos += __shfl_xor_sync(0xffffffffu, n_pos, off);
+  }
   __syncwarp();
+  const int m = min(budget, n_pos);
 
-  if (m < N) {
+  if (m < n_pos) {
     for (int r = 0; r < m; ++r) {
       uint32_t b0, b1;
       philox4x32_10(it_lo, (uint32_t)i, (uint32_t)r, it_hi, seed_lo, seed_hi, b0, b1);
@@ -392,7 +421,8 @@ sample_chunks_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __rest
       __syncwarp();
     }
   } else {
-    for (int k = lane; k < N; k += 32) w[k] = 0x80000000u;
+    for (int k = lane; k < N; k += 32)
+      if (w[k]) w[k] = 0x80000000u;                       // every chunk of positive weight is kept
     __syncwarp();
   }
 
@@ -427,19 +457,20 @@ int pcm_create(pcm_ctx** out, const pcm_config* cfg, int32_t max_traj) {
   if (!out || !cfg) return PCM_ERR_ARG;
   if (cfg->n_phases < 1 || cfg->n_phases > PCM_MAX_PHASES || cfg->budget < 1 || cfg->group_size < 1 ||
       cfg->t_rc < 1 || cfg->t_rc > PCM_MAX_TRC || !(cfg->p_min > 0.0) || cfg->p_min > 1.0 ||
-      !(cfg->adv_eps >= 0.0) || max_traj < cfg->group_size)
+      !(cfg->adv_eps >= 0.0) || max_traj < cfg->group_size || cfg->mode < PCM_MASK_PCM || cfg->mode > PCM_MASK_FULL)
     return PCM_ERR_ARG;
   pcm_ctx* c = new (std::nothrow) pcm_ctx();
   if (!c) return PCM_ERR_ARG;
   c->cfg = *cfg;
   c->max_traj = max_traj;
-  c->state = nullptr; c->status = nullptr; c->c_group = nullptr; c->valid_group = nullptr;
+  c->state = nullptr; c->status = nullptr; c->c_group = nullptr; c->valid_group = nullptr; c->n_pos = nullptr;
   const size_t ng = (size_t)max_traj / cfg->group_size;
   bool ok = cudaGetDevice(&c->device) == cudaSuccess &&
             cudaMalloc(&c->state, sizeof(KeepState)) == cudaSuccess &&
             cudaMalloc(&c->status, 256) == cudaSuccess &&
             cudaMalloc(&c->c_group, ng * cfg->n_phases * sizeof(double)) == cudaSuccess &&
-            cudaMalloc(&c->valid_group, ng * cfg->n_phases) == cudaSuccess;
+            cudaMalloc(&c->valid_group, ng * cfg->n_phases) == cudaSuccess &&
+            cudaMalloc(&c->n_pos, (size_t)max_traj * sizeof(int32_t)) == cudaSuccess;
   if (ok) {
     KeepState init;
     memset(&init, 0, sizeof(init));
@@ -457,7 +488,7 @@ int pcm_create(pcm_ctx** out, const pcm_config* cfg, int32_t max_traj) {
 
 int pcm_destroy(pcm_ctx* c) {
   if (!c) return PCM_ERR_ARG;
-  cudaFree(c->state); cudaFree(c->status); cudaFree(c->c_group); cudaFree(c->valid_group);
+  cudaFree(c->state); cudaFree(c->status); cudaFree(c->c_group); cudaFree(c->valid_group); cudaFree(c->n_pos);
   delete c;
   return PCM_OK;
 }
@@ -525,7 +556,7 @@ int pcm_update_keep_probs(pcm_ctx* ctx, const double* C, const uint8_t* valid, f
                           pcm_stream stream) {
   if (!ctx || !C || !valid || !p || !q) return PCM_ERR_ARG;
   update_keep_probs_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->state, C, valid, ctx->cfg.n_phases,
-                                                               ctx->cfg.t_rc, ctx->cfg.p_min, p, q);
+                                                               ctx->cfg.t_rc, ctx->cfg.p_min, ctx->cfg.mode, p, q);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
 }
@@ -537,7 +568,10 @@ int pcm_sample_chunks(pcm_ctx* ctx, const pcm_batch* b, const uint32_t* q, uint6
   if (!q || !kept_idx || !kept_off) return PCM_ERR_ARG;
   if (b->max_len < 1 || b->max_len > 12000) return PCM_ERR_SHAPE;     // 4 warps x max_len x 4 B <= 192 KB
   cudaStream_t s = (cudaStream_t)stream;
-  kept_offsets_kernel<<<1, 1024, 0, s>>>(b->traj_off, b->n_traj, ctx->cfg.budget, kept_off);
+  count_positive_kernel<<<ceil_div(b->n_traj, 8), 256, 0, s>>>(b->traj_off, b->phase, q, b->n_traj, ctx->cfg.n_phases,
+                                                               ctx->n_pos);
+  PCM_LAUNCH_CHECK();
+  kept_offsets_kernel<<<1, 1024, 0, s>>>(ctx->n_pos, b->n_traj, ctx->cfg.budget, kept_off);
   PCM_LAUNCH_CHECK();
   if (kept_per_phase) PCM_CUDA_TRY(cudaMemsetAsync(kept_per_phase, 0, ctx->cfg.n_phases * sizeof(int32_t), s));
   const int warps = 4;

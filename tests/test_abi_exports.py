@@ -24,7 +24,7 @@ def test_library_loads_and_exports_every_declared_symbol():
 
 def test_binding_struct_sizes_match_the_header_layout():
     from paper_2605_16154_b200 import binding as B
-    assert ctypes.sizeof(B.pcm_config) == 40
+    assert ctypes.sizeof(B.pcm_config) == 48
     assert ctypes.sizeof(B.pcm_batch) == 16 + 6 * 8
     assert ctypes.sizeof(B.grpo_model_cfg) == 24
     assert ctypes.sizeof(B.grpo_model) == 24 + 9 * 8

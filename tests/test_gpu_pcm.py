@@ -189,3 +189,39 @@ def test_pack_bit_exact(case):
     assert np.array_equal(_np(out.adv_c), advc_o)
     assert np.array_equal(_np(out.src), src_o)
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("name", ["C0", "C4"])
+def test_ablation_samplers_bit_exact(name, mode):
+    """Random masking and full masking (RQ4): keep-probabilities, offsets and kept ids against the oracle
+    over a chain of iterations; full masking keeps chunks of one phase only."""
+    B, PL = _mods()
+    w = synth.WORKLOADS[name]
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=5, max_traj=w.n_traj, mode=mode)
+    st = po.KeepProbState(w.n_phases, w.p_min, w.t_rc, mode=mode)
+    for it in range(7):
+        rb = synth.make_rollouts(w, seed=100 + it)
+        batch = PL.upload_rollouts(w, rb)
+        adv, Cc, valid, p, q, kept_idx, kept_off, per_phase = PL.select(ctx, batch, it)
+        C_o, valid_o, _, _, _ = po.score_phases(rb["traj_off"], rb["tok"], rb["phase"], rb["reward"], w.G, w.n_phases)
+        p_o, q_o, _ = po.update_keep_probs(st, C_o, valid_o)
+        k_o, off_o, pp_o = po.sample_chunks(rb["traj_off"], rb["phase"], q_o, w.budget, 5, it)
+        assert np.array_equal(_np(q).astype(np.int64), q_o), it
+        assert np.array_equal(_np(p), p_o.astype(np.float32)), it
+        assert np.array_equal(_np(kept_off), off_o), it
+        assert np.array_equal(_np(kept_idx)[: int(off_o[-1])], k_o), it
+        assert np.array_equal(_np(per_phase), pp_o), it
+        if mode == 2:
+            assert np.count_nonzero(_np(per_phase)) == 1 and int(np.count_nonzero(q_o)) == 1
+        else:
+            lens = np.diff(rb["traj_off"])
+            assert np.array_equal(np.diff(off_o), np.minimum(lens, w.budget))
+    assert B.pcm_poll_status(ctx) == 0
+    ctx.close()
+
+
+def test_bad_mask_mode_is_rejected():
+    B, _ = _mods()
+    with pytest.raises(RuntimeError):
+        B.Context(4, 4, 4, mode=3)

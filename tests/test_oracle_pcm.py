@@ -273,3 +273,65 @@ def test_pack_round_trip():
             assert np.array_equal(X[j, P + t], e_act[tok[c, t]])
         assert np.array_equal(tgt[j], tok[c]) and np.array_equal(l2[j], lpo[c])
     assert list(adv_c) == [0.5, 0.5, -2.0, -2.0] and list(src) == list(kept)
+
+
+# ---- ablation samplers of RQ4 (random masking, full masking) ------------------------------------
+def test_random_masking_keeps_unit_weights_whatever_the_scores():
+    st = po.KeepProbState(4, p_min=0.1, t_rc=2, mode=1)
+    for C in ([5.0, 1.0, 0.0, 0.25], [0.0, 9.0, 1.0, 1.0], [1.0, 1.0, 1.0, 1.0]):
+        p, q, _ = po.update_keep_probs(st, C, [1, 1, 1, 1])
+        assert p.tolist() == [1.0] * 4 and q.tolist() == [1 << 24] * 4
+
+
+def test_random_masking_is_uniform_over_chunks():
+    """Inclusion frequency B/N for every chunk, independent of its phase (binomial 5-sigma band)."""
+    N, Bk, n_seeds = 9, 3, 20000
+    phase = np.array([0, 0, 0, 1, 1, 2, 2, 2, 2], dtype=np.uint8)
+    traj_off = np.array([0, N], dtype=np.int32)
+    q = np.full(3, 1 << 24, dtype=np.int64)
+    cnt = np.zeros(N)
+    for s in range(n_seeds):
+        k, off, _ = po.sample_chunks(traj_off, phase, q, Bk, s, 0)
+        assert off[-1] == Bk
+        cnt[k] += 1
+    f, sd = Bk / N, math.sqrt(Bk / N * (1 - Bk / N) / n_seeds)
+    assert np.all(np.abs(cnt / n_seeds - f) < 5 * sd)
+
+
+def test_full_masking_keeps_only_the_highest_scoring_phase():
+    st = po.KeepProbState(4, p_min=0.1, t_rc=2, mode=2)
+    p, q, _ = po.update_keep_probs(st, [0.5, 3.0, 3.0, 1.0], [1, 1, 1, 1])      # tie: the first arg-max wins
+    assert p.tolist() == [0.0, 1.0, 0.0, 0.0] and q.tolist() == [0, 1 << 24, 0, 0]
+    # trajectories with 5, 2 and 0 chunks in phase 1; budget 3
+    phase = np.array([0, 1, 1, 2, 1, 1, 1, 3,   1, 0, 1,   0, 2, 3], dtype=np.uint8)
+    traj_off = np.array([0, 8, 11, 14], dtype=np.int32)
+    for it in range(50):
+        k, off, per_phase = po.sample_chunks(traj_off, phase, q, 3, 77, it)
+        assert off.tolist() == [0, 3, 5, 5]                                    # min(B, chunks of that phase)
+        assert np.all(phase[k] == 1) and per_phase.tolist() == [0, 5, 0, 0]
+        assert k[3:].tolist() == [8, 10]                                       # below the budget: all of them
+        assert set(k[:3].tolist()) <= {1, 2, 4, 5, 6} and len(set(k[:3].tolist())) == 3
+    # all five candidates of the first trajectory get drawn over the iterations
+    seen = set()
+    for it in range(200):
+        seen |= set(po.sample_chunks(traj_off, phase, q, 3, 77, it)[0][:3].tolist())
+    assert seen == {1, 2, 4, 5, 6}
+
+
+def test_full_masking_follows_the_buffered_sum_not_the_last_step():
+    st = po.KeepProbState(3, p_min=0.1, t_rc=2, mode=2)
+    po.update_keep_probs(st, [1.0, 0.0, 0.0], [1, 1, 1])                        # step 0 refreshes: phase 0
+    po.update_keep_probs(st, [0.0, 5.0, 0.0], [1, 1, 1])                        # buffered, p unchanged
+    assert st.p == [1.0, 0.0, 0.0]
+    p, _, refreshed = po.update_keep_probs(st, [0.0, 0.0, 4.0], [1, 1, 1])      # S = (0, 5, 4)
+    assert refreshed and p.tolist() == [0.0, 1.0, 0.0]
+
+
+def test_default_mode_unchanged_by_the_ablation_switch():
+    a, b = po.KeepProbState(5, 0.1, 3), po.KeepProbState(5, 0.1, 3, mode=0)
+    rng = np.random.default_rng(3)
+    for _ in range(10):
+        C = rng.random(5)
+        pa, qa, _ = po.update_keep_probs(a, C, [1] * 5)
+        pb, qb, _ = po.update_keep_probs(b, C, [1] * 5)
+        assert np.array_equal(pa, pb) and np.array_equal(qa, qb) and np.all(qa >= round(0.1 * (1 << 24)))
