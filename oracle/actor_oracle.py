@@ -8,7 +8,9 @@ CPU-baseline leg may call it.
 Parity status: the gradient is pinned by central finite differences of `loss_only` on a 2-layer d=16
 model; the pieces are pinned by textbook definitions (softmax attention as a double loop, RMSNorm,
 single-row log-softmax); Eq. 11 -> Eq. 2 (mask keeps every chunk), the per-phase decomposition Eq. 3,
-and the zero-gradient cases are checked as invariants.
+and the zero-gradient cases are checked as invariants.  The entropy bonus and the chunk-level ratio are
+pinned by finite differences, by autograd of a library model, by H = log 256 for a zero head, and by the
+on-policy identity (chunk-level and token-level gradients coincide at r = 1 for equal scales).
 
 Model (every kept chunk is its own sequence of S = P + 56 tokens): pre-norm decoder, RMSNorm,
 rotary position embedding on q and k (base 10000, pairs (i, i + dh/2)), causal softmax attention
@@ -150,39 +152,79 @@ def surrogate(logp, logp_old, adv_c, eps_low, eps_high, loss_scale):
     return loss, dlogp, r, active
 
 
+def surrogate_chunk(logp, logp_old, adv_c, eps_low, eps_high, loss_scale):
+    """Chunk-level clipped surrogate: the chunk's action is the joint of its 56 tokens, so
+    log pi(a_ik | s_ik) = sum_j logp_j (the quantity Eq. 2 / Eq. 11 write) and one ratio per chunk,
+    r = exp(sum_j logp_j - sum_j logp_old_j), goes through the same clip.
+    loss = -loss_scale * sum_chunks min(r A, clip(r) A).  Returns (loss, dloss/dlogp [n,56], r [n], active [n])."""
+    A = _f64(adv_c)
+    r = np.exp(logp.sum(axis=-1) - _f64(logp_old).sum(axis=-1))
+    s = np.minimum(r * A, np.clip(r, 1.0 - eps_low, 1.0 + eps_high) * A)
+    loss = -loss_scale * float(np.sum(s))
+    active = ((A >= 0) & (r <= 1.0 + eps_high)) | ((A < 0) & (r >= 1.0 - eps_low))
+    dl = np.where(active, -loss_scale * A * r, 0.0)
+    return loss, np.repeat(dl[:, None], logp.shape[-1], axis=-1), r, active
+
+
+def entropy_rows(z):
+    """Shannon entropy H = -sum_v p_v log p_v of softmax(z) along the last axis, and log p."""
+    m = z.max(axis=-1, keepdims=True)
+    logp_all = z - (m + np.log(np.exp(z - m).sum(axis=-1, keepdims=True)))
+    return -(np.exp(logp_all) * logp_all).sum(axis=-1), logp_all
+
+
+def objective(z, tgt, logp_old, adv_c, eps_low, eps_high, loss_scale, entropy_coef=0.0, ratio_level="token"):
+    """Surrogate minus entropy bonus (App. E: entropy coefficient 1e-3, no KL term):
+        loss = surrogate loss - entropy_coef * mean over the scored positions of H(pi(. | s)).
+    Returns (loss, dloss/dz, logp, ratio, active, mean entropy)."""
+    logp, prob = log_softmax_at(z, tgt)
+    if ratio_level == "chunk":
+        loss, dlogp, r, active = surrogate_chunk(logp, logp_old, adv_c, eps_low, eps_high, loss_scale)
+    else:
+        loss, dlogp, r, active = surrogate(logp, logp_old, adv_c, eps_low, eps_high, loss_scale)
+    onehot = np.zeros_like(prob)
+    np.put_along_axis(onehot, np.asarray(tgt, dtype=np.int64)[..., None], 1.0, axis=-1)
+    dz = dlogp[..., None] * (onehot - prob)
+    Hrow, logp_all = entropy_rows(z)
+    if entropy_coef != 0.0:
+        n_rows = Hrow.size
+        loss = loss - entropy_coef * float(Hrow.sum()) / n_rows
+        # dH/dz_v = -p_v (log p_v + H)
+        dz = dz + (entropy_coef / n_rows) * prob * (logp_all + Hrow[..., None])
+    return loss, dz, logp, r, active, float(Hrow.mean())
+
+
 def logp_only(weights, X, tgt, H, P):
     z, _ = forward(weights, X, H, P, keep_cache=False)
     return log_softmax_at(z, tgt)[0]
 
 
-def loss_only(weights, X, tgt, logp_old, adv_c, H, P, eps_low, eps_high, loss_scale):
+def loss_only(weights, X, tgt, logp_old, adv_c, H, P, eps_low, eps_high, loss_scale, entropy_coef=0.0,
+              ratio_level="token"):
     z, _ = forward(weights, X, H, P, keep_cache=False)
-    logp, _ = log_softmax_at(z, tgt)
-    return surrogate(logp, logp_old, adv_c, eps_low, eps_high, loss_scale)[0]
+    return objective(z, tgt, logp_old, adv_c, eps_low, eps_high, loss_scale, entropy_coef, ratio_level)[0]
 
 
-def fwd_bwd(weights, X, tgt, logp_old, adv_c, H, P, eps_low=0.2, eps_high=0.2, loss_scale=None):
+def fwd_bwd(weights, X, tgt, logp_old, adv_c, H, P, eps_low=0.2, eps_high=0.2, loss_scale=None, entropy_coef=0.0,
+            ratio_level="token"):
     """Masked GRPO actor update on the packed batch of kept chunks (Eq. 11).
 
     Returns (loss, logp [n,56], grads dict with the shapes of `weights`, stats).  `loss_scale`
-    defaults to the token mean 1/(56 n).  No gradient flows to the observation prefix; the
-    embedding gradient collects the rows at the action-token positions."""
+    defaults to the mean over the surrogate's terms: 1/(56 n) with one ratio per token, 1/n with one
+    ratio per chunk.  No gradient flows to the observation prefix; the embedding gradient collects
+    the rows at the action-token positions."""
     n, S, d = np.asarray(X).shape
     if loss_scale is None:
-        loss_scale = 1.0 / (ACT_DIM * n)
+        loss_scale = 1.0 / (ACT_DIM * n) if ratio_level == "token" else 1.0 / n
     z, cache = forward(weights, X, H, P)
     Wt = cache["W"]
     L = Wt["w_qkv"].shape[0]
     dh = d // H
     cos, sin = cache["cos"], cache["sin"]
     tgt = np.asarray(tgt, dtype=np.int64)
-    logp, prob = log_softmax_at(z, tgt)
-    loss, dlogp, r, active = surrogate(logp, logp_old, adv_c, eps_low, eps_high, loss_scale)
-
+    loss, dz, logp, r, active, mean_H = objective(z, tgt, logp_old, adv_c, eps_low, eps_high, loss_scale,
+                                                  entropy_coef, ratio_level)              # dz [n,56,V]
     grads = {k: np.zeros_like(v) for k, v in Wt.items()}
-    onehot = np.zeros_like(prob)
-    np.put_along_axis(onehot, tgt[..., None], 1.0, axis=-1)
-    dz = dlogp[..., None] * (onehot - prob)                                   # [n,56,V]
     V = dz.shape[-1]
     grads["w_h"] = dz.reshape(n * ACT_DIM, V).T @ cache["hf"].reshape(n * ACT_DIM, d)
     dhf = dz @ Wt["w_h"]
@@ -222,5 +264,5 @@ def fwd_bwd(weights, X, tgt, logp_old, adv_c, H, P, eps_low=0.2, eps_high=0.2, l
         for t in range(ACT_DIM):
             dE[tgt[j, t]] += dx[j, P + t]
     grads["e_act"] = dE
-    stats = dict(clip_frac=float(1.0 - active.mean()), mean_ratio=float(r.mean()))
+    stats = dict(clip_frac=float(1.0 - active.mean()), mean_ratio=float(r.mean()), entropy=mean_H)
     return loss, logp, grads, stats

@@ -244,3 +244,121 @@ def test_unclipped_on_policy_loss_is_eq11_and_zero_signal_cases():
     # a group with uniform rewards has zero advantages, hence exactly zero gradient
     _, _, g0, _ = ao.fwd_bwd(s["W"], X, tgt, logp, np.zeros(len(kept)), s["H"], s["P"], 0.2, 0.2, 1.0)
     assert all(np.all(v == 0.0) for v in g0.values())
+
+
+# ---- entropy bonus and chunk-level ratio (App. E; Eq. 2 / Eq. 11 written per chunk) -----------------
+@pytest.mark.parametrize("ratio_level,sigma", [("token", 0.01), ("token", 0.3), ("chunk", 0.001), ("chunk", 0.04)])
+def test_entropy_and_chunk_ratio_gradient_matches_finite_differences(ratio_level, sigma):
+    rng = np.random.default_rng(40)
+    d, H, P = 16, 2, 4
+    W = tiny_model(rng, d=d, H=H)
+    X, tgt, adv = tiny_batch(rng, W, P=P, d=d)
+    lpo = ao.logp_only(W, X, tgt, H, P) + sigma * rng.standard_normal((3, 56))
+    el, eh, coef = 0.2, 0.4, 0.05
+    loss, _, grads, stats = ao.fwd_bwd(W, X, tgt, lpo, adv, H, P, el, eh, loss_scale=1.0, entropy_coef=coef,
+                                        ratio_level=ratio_level)
+    if sigma in (0.3, 0.04):
+        assert 0.0 < stats["clip_frac"] < 1.0
+    else:
+        assert stats["clip_frac"] == 0.0
+
+    def f(Wp):
+        return ao.loss_only(Wp, rebuild_X(Wp, X, tgt, P), tgt, lpo, adv, H, P, el, eh, 1.0, coef, ratio_level)
+
+    assert f(W) == pytest.approx(loss, rel=1e-13)
+    for name in W:
+        for _ in range(3):
+            v = rng.standard_normal(W[name].shape)
+            h = 1e-6
+            Wp = dict(W); Wp[name] = W[name] + h * v
+            Wm = dict(W); Wm[name] = W[name] - h * v
+            fd = (f(Wp) - f(Wm)) / (2 * h)
+            assert float(np.sum(grads[name] * v)) == pytest.approx(fd, rel=3e-5, abs=1e-7), name
+
+
+def test_entropy_bonus_alone_matches_finite_differences_and_autograd():
+    """A = 0 leaves only the entropy term: gradient against autograd of -coef * mean H from library ops."""
+    rng = np.random.default_rng(41)
+    d, H, P = 32, 4, 5
+    W = tiny_model(rng, d=d, H=H, L=2)
+    X, tgt, _ = tiny_batch(rng, W, P=P, d=d)
+    lpo = ao.logp_only(W, X, tgt, H, P)
+    coef = 0.7
+    loss, _, grads, stats = ao.fwd_bwd(W, X, tgt, lpo, np.zeros(3), H, P, 0.2, 0.4, entropy_coef=coef)
+    Wt = {k: torch.tensor(v, dtype=torch.float64, requires_grad=True) for k, v in W.items()}
+    Xt = torch.tensor(X, dtype=torch.float64)
+    Xt = torch.cat([Xt[:, :P], Wt["e_act"][torch.tensor(tgt.astype(np.int64))]], dim=1)
+    z = _torch_forward_tracked(Wt, Xt, H, P)
+    ent = torch.distributions.Categorical(logits=z).entropy()
+    lt = -coef * ent.mean()
+    lt.backward()
+    assert float(lt.detach()) == pytest.approx(loss, rel=1e-12)
+    assert stats["entropy"] == pytest.approx(float(ent.mean().detach()), rel=1e-12)
+    for k in W:
+        assert np.allclose(grads[k], Wt[k].grad.numpy(), rtol=1e-8, atol=1e-13), k
+
+
+def test_full_paper_loss_matches_autograd_of_library_model():
+    """Asymmetric clip (0.2, 0.4) + entropy coefficient 1e-3, token-level and chunk-level ratios."""
+    rng = np.random.default_rng(42)
+    d, H, P = 32, 4, 5
+    W = tiny_model(rng, d=d, H=H, L=2)
+    X, tgt, adv = tiny_batch(rng, W, P=P, d=d)
+    base = ao.logp_only(W, X, tgt, H, P)
+    for level, sigma in (("token", 0.25), ("chunk", 0.04)):
+        lpo = base + sigma * rng.standard_normal((3, 56))
+        loss, _, grads, stats = ao.fwd_bwd(W, X, tgt, lpo, adv, H, P, 0.2, 0.4, entropy_coef=1e-3, ratio_level=level)
+        Wt = {k: torch.tensor(v, dtype=torch.float64, requires_grad=True) for k, v in W.items()}
+        Xt = torch.tensor(X, dtype=torch.float64)
+        Xt = torch.cat([Xt[:, :P], Wt["e_act"][torch.tensor(tgt.astype(np.int64))]], dim=1)
+        z = _torch_forward_tracked(Wt, Xt, H, P)
+        lsm = torch.log_softmax(z, -1)
+        lp = lsm.gather(-1, torch.tensor(tgt.astype(np.int64))[..., None])[..., 0]
+        if level == "token":
+            r = torch.exp(lp - torch.tensor(lpo)); A = torch.tensor(adv)[:, None]; denom = 56 * 3
+        else:
+            r = torch.exp(lp.sum(-1) - torch.tensor(lpo).sum(-1)); A = torch.tensor(adv); denom = 3
+        pg = -(torch.minimum(r * A, torch.clamp(r, 0.8, 1.4) * A)).sum() / denom
+        lt = pg - 1e-3 * (-(lsm.exp() * lsm).sum(-1)).mean()
+        lt.backward()
+        assert float(lt.detach()) == pytest.approx(loss, rel=1e-12)
+        for k in W:
+            assert np.allclose(grads[k], Wt[k].grad.numpy(), rtol=1e-8, atol=1e-12), (level, k)
+
+
+def test_zero_head_gives_uniform_policy_entropy_log256_and_no_entropy_gradient():
+    rng = np.random.default_rng(43)
+    W = tiny_model(rng)
+    W["w_h"] = np.zeros_like(W["w_h"])
+    X, tgt, adv = tiny_batch(rng, W)
+    lpo = np.full((3, 56), -np.log(256.0))
+    loss, logp, grads, stats = ao.fwd_bwd(W, X, tgt, lpo, np.zeros(3), 2, 4, entropy_coef=0.5)
+    assert stats["entropy"] == pytest.approx(np.log(256.0), rel=1e-14)
+    assert loss == pytest.approx(-0.5 * np.log(256.0), rel=1e-14)
+    assert np.allclose(logp, -np.log(256.0))
+    assert all(np.abs(g).max() < 1e-15 for g in grads.values())          # the uniform policy maximises H
+
+
+def test_chunk_level_ratio_on_policy_identity_and_joint_clipping():
+    rng = np.random.default_rng(44)
+    W = tiny_model(rng)
+    X, tgt, adv = tiny_batch(rng, W)
+    base = ao.logp_only(W, X, tgt, 2, 4)
+    # on-policy: every ratio is 1, both forms give -scale * A * grad(sum of log-probs)
+    _, _, g_tok, _ = ao.fwd_bwd(W, X, tgt, base, adv, 2, 4, loss_scale=0.01)
+    _, _, g_chk, st = ao.fwd_bwd(W, X, tgt, base, adv, 2, 4, loss_scale=0.01, ratio_level="chunk")
+    assert st["mean_ratio"] == pytest.approx(1.0, abs=1e-12)
+    for k in W:
+        assert np.allclose(g_tok[k], g_chk[k], rtol=1e-9, atol=1e-14), k
+    # every token ratio e^0.01 is inside the clip range, the joint ratio e^0.56 is not
+    lpo = base - 0.01
+    _, _, _, st_tok = ao.fwd_bwd(W, X, tgt, lpo, adv, 2, 4, 0.2, 0.4)
+    loss, _, g, st_chk = ao.fwd_bwd(W, X, tgt, lpo, adv, 2, 4, 0.2, 0.4, ratio_level="chunk")
+    assert st_tok["clip_frac"] == 0.0
+    assert st_chk["mean_ratio"] == pytest.approx(np.exp(0.56), rel=1e-12)
+    assert st_chk["clip_frac"] == pytest.approx(2 / 3)                     # the two chunks with A > 0
+    assert loss == pytest.approx(-(1.4 * 1.2 + np.exp(0.56) * -0.8 + 1.4 * 0.4) / 3, rel=1e-12)
+    # only the A < 0 chunk (index 1) still carries gradient: compare with that chunk alone
+    _, _, g1, _ = ao.fwd_bwd(W, X[1:2], tgt[1:2], lpo[1:2], adv[1:2], 2, 4, 0.2, 0.4, loss_scale=1 / 3, ratio_level="chunk")
+    for k in W:
+        assert np.allclose(g[k], g1[k], rtol=1e-9, atol=1e-14), k
