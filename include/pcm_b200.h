@@ -238,21 +238,25 @@ int grpo_pack_chunks(pcm_ctx* ctx, const pcm_batch* batch, const grpo_model_cfg*
 /* ---- Eq. 11 ------------------------------------------------------------------------------------ */
 #define GRPO_FWD_ONLY 1u       /* forward only: writes logp (and loss), touches no gradient       */
 #define GRPO_ACCUMULATE 2u     /* add into grads instead of overwriting them                      */
+#define GRPO_CHUNK_RATIO 4u    /* one importance ratio per chunk (joint of its 56 tokens) instead of per token */
 
 typedef struct {
   float eps_low;               /* clip range [1 - eps_low, 1 + eps_high]                          */
   float eps_high;
-  float loss_scale;            /* <= 0: token mean 1 / (56 * n_kept)                              */
+  float loss_scale;            /* <= 0: mean over the surrogate's terms, 1 / (56 * n_kept) per token,
+                                  1 / n_kept with GRPO_CHUNK_RATIO                                */
   int32_t mb_chunks;           /* chunks per micro-batch, >= 1                                    */
   uint32_t flags;
-  int32_t reserved;
+  float entropy_coef;          /* App. E: 1e-3; the loss subtracts entropy_coef * mean entropy    */
 } grpo_loss_cfg;
 
 typedef struct {
   float loss;
-  float clip_frac;             /* fraction of action tokens whose surrogate gradient is clipped   */
+  float clip_frac;             /* fraction of ratios (tokens, or chunks with GRPO_CHUNK_RATIO) whose gradient is clipped */
   float mean_ratio;
+  float entropy;               /* mean over the scored positions of H(pi(. | s)), in nats          */
   int32_t n_launches;          /* kernels launched by this call                                   */
+  int32_t reserved;
   uint64_t workspace_high_water;
 } grpo_stats;
 
@@ -264,7 +268,9 @@ size_t grpo_workspace_bytes(const grpo_model_cfg* cfg, int32_t mb_chunks, uint32
  *     loss = -loss_scale * sum_{kept chunks} sum_{j<56} min(r_j A, clip(r_j, 1-eps_low, 1+eps_high) A),
  *     r_j = exp(logp_j - lpo_j), logp_j = log softmax(z_j)[tgt_j], z_j = head(position P-1+j).
  * A term's gradient is r_j A when (A >= 0 and r_j <= 1+eps_high) or (A < 0 and r_j >= 1-eps_low),
- * else 0.  The batch is processed in micro-batches of mb_chunks chunks; gradients accumulate in
+ * else 0.  With GRPO_CHUNK_RATIO the inner sum is one term per chunk with r = exp(sum_j (logp_j - lpo_j)).
+ * The entropy bonus of App. E subtracts entropy_coef * (1 / (56 n_kept)) * sum over the scored positions of
+ * H(softmax(z_j)) from the loss (entropy_coef = 0: none).  The batch is processed in micro-batches of mb_chunks chunks; gradients accumulate in
  * fp32, so the micro-batch size only changes the rounding order.  No gradient reaches the
  * observation prefix.
  * Outputs: device loss[1] f32; device logp[n_kept][56] f32 (may be NULL); grads (ignored with

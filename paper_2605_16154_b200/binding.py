@@ -22,7 +22,7 @@ _lib = C.CDLL(LIB_PATH)
 ACT_DIM = 56
 N_BINS = 256
 GRPO_F32, GRPO_BF16 = 0, 1
-GRPO_FWD_ONLY, GRPO_ACCUMULATE = 1, 2
+GRPO_FWD_ONLY, GRPO_ACCUMULATE, GRPO_CHUNK_RATIO = 1, 2, 4
 MASK_PCM, MASK_RANDOM, MASK_FULL = 0, 1, 2
 
 STATUS_NAMES = {0: "PCM_OK", -1: "PCM_ERR_ARG", -2: "PCM_ERR_SHAPE", -3: "PCM_ERR_WORKSPACE", -4: "PCM_ERR_CUDA",
@@ -70,12 +70,12 @@ class grpo_packed(C.Structure):
 
 class grpo_loss_cfg(C.Structure):
     _fields_ = [("eps_low", C.c_float), ("eps_high", C.c_float), ("loss_scale", C.c_float), ("mb_chunks", C.c_int32),
-                ("flags", C.c_uint32), ("reserved", C.c_int32)]
+                ("flags", C.c_uint32), ("entropy_coef", C.c_float)]
 
 
 class grpo_stats(C.Structure):
-    _fields_ = [("loss", C.c_float), ("clip_frac", C.c_float), ("mean_ratio", C.c_float), ("n_launches", C.c_int32),
-                ("workspace_high_water", C.c_uint64)]
+    _fields_ = [("loss", C.c_float), ("clip_frac", C.c_float), ("mean_ratio", C.c_float), ("entropy", C.c_float),
+                ("n_launches", C.c_int32), ("reserved", C.c_int32), ("workspace_high_water", C.c_uint64)]
 
 
 class grpo_adamw_cfg(C.Structure):
@@ -313,7 +313,8 @@ def grpo_workspace_bytes(model: Model, mb_chunks: int, flags: int = 0) -> int:
 def grpo_actor_fwd_bwd(model: Model, packed: Packed, eps_low: float = 0.2, eps_high: float = 0.2,
                        loss_scale: float = 0.0, mb_chunks: int = 64, flags: int = 0,
                        workspace: Optional[torch.Tensor] = None, want_stats: bool = True,
-                       logp: Optional[torch.Tensor] = None, loss: Optional[torch.Tensor] = None):
+                       logp: Optional[torch.Tensor] = None, loss: Optional[torch.Tensor] = None,
+                       entropy_coef: float = 0.0):
     """Returns (loss tensor[1] on the device, logp [n_kept, 56], grads dict or None, stats or None)."""
     dev = torch.device("cuda")
     mb = max(1, min(mb_chunks, max(packed.n_kept, 1)))
@@ -329,7 +330,7 @@ def grpo_actor_fwd_bwd(model: Model, packed: Packed, eps_low: float = 0.2, eps_h
         loss = torch.zeros(1, dtype=torch.float32, device=dev)
     if logp is None:
         logp = torch.empty((packed.n_kept, ACT_DIM), dtype=torch.float32, device=dev)
-    lc = grpo_loss_cfg(eps_low, eps_high, loss_scale, mb, flags, 0)
+    lc = grpo_loss_cfg(eps_low, eps_high, loss_scale, mb, flags, entropy_coef)
     fwd_only = bool(flags & GRPO_FWD_ONLY)
     grads = None
     if not fwd_only:

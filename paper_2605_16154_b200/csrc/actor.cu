@@ -288,87 +288,131 @@ __global__ void swiglu_bwd_kernel(const T* __restrict__ gu, const T* __restrict_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Loss over the 256-bin head: one warp per scored row.  z fp32 [rows][256] logits in, dz T out.
-// Per-CTA partial sums {surrogate, clipped count, ratio} go to part[blockIdx][3].
+// Loss over the 256-bin head: one CTA per chunk, warp w scores rows 7w .. 7w+6 of the chunk's 56.
+// z fp32 [rows][256] logits in, dz T out.  Token level: one clipped ratio per row.  Chunk level: the rows'
+// log-ratios are summed over the CTA in a fixed order and one clipped ratio serves all 56 rows.
+// The entropy bonus adds ent_scale * p_v (log p_v + H) to dz (ent_scale = coefficient / scored rows).
+// Per-CTA partial sums {surrogate, clipped count, ratio, entropy} go to part[blockIdx][4].
 // ------------------------------------------------------------------------------------------------
+constexpr int LOSS_ROWS_PER_WARP = ACT / 8;
+static_assert(ACT % 8 == 0, "a chunk's rows are split evenly over the CTA's eight warps");
+
 template <typename T>
 __global__ void __launch_bounds__(256)
-loss_rows_kernel(const float* __restrict__ z, const uint8_t* __restrict__ tgt, const float* __restrict__ lpo,
-                 const float* __restrict__ adv_c, float eps_low, float eps_high, float loss_scale,
-                 T* __restrict__ dz, float* __restrict__ logp_out, float* __restrict__ part, long long rows,
-                 int fwd_only) {
-  __shared__ float red[8][3];
+loss_chunk_kernel(const float* __restrict__ z, const uint8_t* __restrict__ tgt, const float* __restrict__ lpo,
+                  const float* __restrict__ adv_c, float eps_low, float eps_high, float loss_scale, float ent_scale,
+                  int chunk_ratio, T* __restrict__ dz, float* __restrict__ logp_out, float* __restrict__ part,
+                  int fwd_only) {
+  __shared__ float red[8][4];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long r = (long long)blockIdx.x * 8 + warp;
-  float my_s = 0.f, my_clip = 0.f, my_ratio = 0.f;
-  if (r < rows) {
-    float v[8];
+  const long long chunk = blockIdx.x;
+  const float A = adv_c[chunk];
+  const float lo = 1.f - eps_low, hi = 1.f + eps_high;
+  float v[LOSS_ROWS_PER_WARP][8];
+  float lse[LOSS_ROWS_PER_WARP], ent[LOSS_ROWS_PER_WARP], dlogp[LOSS_ROWS_PER_WARP];
+  int tg[LOSS_ROWS_PER_WARP];
+  float my_s = 0.f, my_clip = 0.f, my_ratio = 0.f, my_ent = 0.f, dsum = 0.f;
+#pragma unroll
+  for (int i = 0; i < LOSS_ROWS_PER_WARP; ++i) {
+    const long long r = chunk * ACT + warp * LOSS_ROWS_PER_WARP + i;
     const float4 a = *reinterpret_cast<const float4*>(z + r * NB + lane * 8);
     const float4 b = *reinterpret_cast<const float4*>(z + r * NB + lane * 8 + 4);
-    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-    float mx = v[0];
+    v[i][0] = a.x; v[i][1] = a.y; v[i][2] = a.z; v[i][3] = a.w;
+    v[i][4] = b.x; v[i][5] = b.y; v[i][6] = b.z; v[i][7] = b.w;
+    float mx = v[i][0];
 #pragma unroll
-    for (int e = 1; e < 8; ++e) mx = fmaxf(mx, v[e]);
+    for (int e = 1; e < 8; ++e) mx = fmaxf(mx, v[i][e]);
 #pragma unroll
     for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    float se = 0.f;
+    float se = 0.f, sz = 0.f;                             // sum e^(z - mx), sum e^(z - mx) (z - mx)
 #pragma unroll
-    for (int e = 0; e < 8; ++e) se += expf(v[e] - mx);
-    se = warp_sum(se);
-    const float lse = mx + logf(se);
-    const int t = tgt[r];
-    float mine = v[0];                                    // this lane's value at sub-index t & 7
-#pragma unroll
-    for (int e = 1; e < 8; ++e) mine = ((t & 7) == e) ? v[e] : mine;
-    const float zt = __shfl_sync(0xffffffffu, mine, t >> 3);
-    const float logp = zt - lse;
-    const float A = adv_c[r / ACT];
-    const float ratio = expf(logp - lpo[r]);
-    const float lo = 1.f - eps_low, hi = 1.f + eps_high;
-    const float clipped = fminf(fmaxf(ratio, lo), hi);
-    const float surr = fminf(ratio * A, clipped * A);
-    const bool active = (A >= 0.f && ratio <= hi) || (A < 0.f && ratio >= lo);
-    const float dlogp = active ? -loss_scale * A * ratio : 0.f;
-    if (lane == 0) {
-      if (logp_out) logp_out[r] = logp;
-      my_s = surr; my_clip = active ? 0.f : 1.f; my_ratio = ratio;
+    for (int e = 0; e < 8; ++e) {
+      const float ex = expf(v[i][e] - mx);
+      se += ex;
+      sz += ex * (v[i][e] - mx);
     }
-    if (!fwd_only) {
+    se = warp_sum(se);
+    sz = warp_sum(sz);
+    const float lg = logf(se);
+    lse[i] = mx + lg;
+    ent[i] = lg - sz / se;                                // H = lse - sum p z
+    const int t = tgt[r];
+    tg[i] = t;
+    float mine = v[i][0];                                 // this lane's value at sub-index t & 7
+#pragma unroll
+    for (int e = 1; e < 8; ++e) mine = ((t & 7) == e) ? v[i][e] : mine;
+    const float zt = __shfl_sync(0xffffffffu, mine, t >> 3);
+    const float logp = zt - lse[i];
+    if (lane == 0 && logp_out) logp_out[r] = logp;
+    my_ent += ent[i];
+    if (chunk_ratio) {
+      dsum += logp - lpo[r];
+      dlogp[i] = 0.f;
+    } else {
+      const float ratio = expf(logp - lpo[r]);
+      const float clipped = fminf(fmaxf(ratio, lo), hi);
+      const bool active = (A >= 0.f && ratio <= hi) || (A < 0.f && ratio >= lo);
+      dlogp[i] = active ? -loss_scale * A * ratio : 0.f;
+      my_s += fminf(ratio * A, clipped * A);
+      my_clip += active ? 0.f : 1.f;
+      my_ratio += ratio;
+    }
+  }
+  if (chunk_ratio) {                                      // one ratio for the chunk: ordered sum over the warps
+    if (lane == 0) red[warp][0] = dsum;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w][0];
+    __syncthreads();
+    const float ratio = expf(tot);
+    const float clipped = fminf(fmaxf(ratio, lo), hi);
+    const bool active = (A >= 0.f && ratio <= hi) || (A < 0.f && ratio >= lo);
+#pragma unroll
+    for (int i = 0; i < LOSS_ROWS_PER_WARP; ++i) dlogp[i] = active ? -loss_scale * A * ratio : 0.f;
+    if (warp == 0) { my_s = fminf(ratio * A, clipped * A); my_clip = active ? 0.f : 1.f; my_ratio = ratio; }
+  }
+  if (!fwd_only) {
+#pragma unroll
+    for (int i = 0; i < LOSS_ROWS_PER_WARP; ++i) {
+      const long long r = chunk * ACT + warp * LOSS_ROWS_PER_WARP + i;
+      T* out = dz + r * NB + lane * 8;
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int col = lane * 8 + e;
-        const float p = expf(v[e] - lse);
-        stf(dz + r * NB + col, dlogp * ((col == t ? 1.f : 0.f) - p));
+        const float lp = v[i][e] - lse[i];
+        const float p = expf(lp);
+        stf(out + e, dlogp[i] * ((col == tg[i] ? 1.f : 0.f) - p) + ent_scale * p * (lp + ent[i]));
       }
     }
   }
-  if (lane == 0) { red[warp][0] = my_s; red[warp][1] = my_clip; red[warp][2] = my_ratio; }
+  if (lane == 0) { red[warp][0] = my_s; red[warp][1] = my_clip; red[warp][2] = my_ratio; red[warp][3] = my_ent; }
   __syncthreads();
-  if (threadIdx.x < 3) {
+  if (threadIdx.x < 4) {
     float s = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) s += red[w][threadIdx.x];
-    part[(size_t)blockIdx.x * 3 + threadIdx.x] = s;
+    part[(size_t)blockIdx.x * 4 + threadIdx.x] = s;
   }
 }
 
-// acc[0..2] += ordered sums of part; loss[0] = -loss_scale * acc[0]   (single CTA, fixed order)
-__global__ void loss_reduce_kernel(const float* __restrict__ part, int nblk, float loss_scale,
+// acc[0..3] += ordered sums of part; loss[0] = -loss_scale * acc[0] - ent_scale * acc[3]   (single CTA, fixed order)
+__global__ void loss_reduce_kernel(const float* __restrict__ part, int nblk, float loss_scale, float ent_scale,
                                    float* __restrict__ acc, float* __restrict__ loss) {
-  __shared__ double sh[256][3];
-  double s[3] = {0, 0, 0};
+  __shared__ double sh[256][4];
+  double s[4] = {0, 0, 0, 0};
   for (int b = threadIdx.x; b < nblk; b += blockDim.x)
-    for (int e = 0; e < 3; ++e) s[e] += (double)part[(size_t)b * 3 + e];
-  for (int e = 0; e < 3; ++e) sh[threadIdx.x][e] = s[e];
+    for (int e = 0; e < 4; ++e) s[e] += (double)part[(size_t)b * 4 + e];
+  for (int e = 0; e < 4; ++e) sh[threadIdx.x][e] = s[e];
   __syncthreads();
   for (int off = 128; off; off >>= 1) {
     if (threadIdx.x < off)
-      for (int e = 0; e < 3; ++e) sh[threadIdx.x][e] += sh[threadIdx.x + off][e];
+      for (int e = 0; e < 4; ++e) sh[threadIdx.x][e] += sh[threadIdx.x + off][e];
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    for (int e = 0; e < 3; ++e) acc[e] += (float)sh[0][e];
-    loss[0] = -loss_scale * acc[0];
+    for (int e = 0; e < 4; ++e) acc[e] += (float)sh[0][e];
+    loss[0] = -loss_scale * acc[0] - ent_scale * acc[3];
   }
 }
 
@@ -461,7 +505,7 @@ static void carve(Workspace& w, unsigned char* base, const grpo_model_cfg& c, in
   }
   w.hs = a.take(R * d * es); w.rstdf = (float*)a.take(R * 4); w.z = (float*)a.take(R * NB * 4);
   w.dz = a.take(R * NB * es);
-  w.loss_part = (float*)a.take(((R + 7) / 8) * 3 * 4); w.loss_acc = (float*)a.take(256);
+  w.loss_part = (float*)a.take((size_t)mb * 4 * 4); w.loss_acc = (float*)a.take(256);
   if (!fwd_only) {
     w.dx = (float*)a.take(M * d * 4); w.dx_t = a.take(M * d * es); w.dact = a.take(M * 4 * d * es);
     w.dgu = a.take(M * 8 * d * es); w.dh = (float*)a.take(M * d * 4); w.dattn = a.take(M * d * es);
@@ -494,7 +538,10 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
   const bool fwd_only = lc->flags & GRPO_FWD_ONLY;
   const int n = pk->n_kept;
   const int mb_max = lc->mb_chunks < n ? lc->mb_chunks : (n > 0 ? n : 1);
-  const float loss_scale = lc->loss_scale > 0.f ? lc->loss_scale : 1.0f / ((float)ACT * (float)(n > 0 ? n : 1));
+  const bool chunk_ratio = lc->flags & GRPO_CHUNK_RATIO;
+  const float n_terms = (chunk_ratio ? 1.f : (float)ACT) * (float)(n > 0 ? n : 1);
+  const float loss_scale = lc->loss_scale > 0.f ? lc->loss_scale : 1.0f / n_terms;
+  const float ent_scale = lc->entropy_coef / ((float)ACT * (float)(n > 0 ? n : 1));   // coefficient x token mean
   const long long launches0 = g_launches.load();
 
   Workspace w;
@@ -606,14 +653,15 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     PCM_LAUNCH_CHECK();
     prof_end(s, 0.0, (double)R * d * (es + 4.0));
     TRY(G(Ri, NB, d, w.hs, d, true, w_h, d, true, dt, w.z, NB, DT_F32, nullptr, 0));
-    const int loss_blocks = ceil_div(R, 8);
+    const int loss_blocks = mb;                           // one CTA per chunk
     prof_begin(PC_LOSS, s);
-    loss_rows_kernel<T><<<loss_blocks, 256, 0, s>>>(w.z, tgt, lpo, advc, lc->eps_low, lc->eps_high, loss_scale,
-                                                  (T*)w.dz, logp ? logp + (long long)c0 * ACT : nullptr, w.loss_part,
-                                                  R, fwd_only ? 1 : 0);
+    loss_chunk_kernel<T><<<loss_blocks, 256, 0, s>>>(w.z, tgt, lpo, advc, lc->eps_low, lc->eps_high, loss_scale, ent_scale,
+                                                   chunk_ratio ? 1 : 0, (T*)w.dz,
+                                                   logp ? logp + (long long)c0 * ACT : nullptr, w.loss_part,
+                                                   fwd_only ? 1 : 0);
     PCM_LAUNCH_CHECK();
     prof_end(s, 0.0, (double)R * NB * (4.0 + (fwd_only ? 0.0 : es)));
-    loss_reduce_kernel<<<1, 256, 0, s>>>(w.loss_part, loss_blocks, loss_scale, w.loss_acc, loss);
+    loss_reduce_kernel<<<1, 256, 0, s>>>(w.loss_part, loss_blocks, loss_scale, ent_scale, w.loss_acc, loss);
     PCM_LAUNCH_CHECK();
     if (fwd_only) continue;
 
@@ -687,14 +735,16 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
 #undef TRY
 
   if (stats) {
-    float acc[3] = {0, 0, 0}, l = 0;
+    float acc[4] = {0, 0, 0, 0}, l = 0;
     PCM_CUDA_TRY(cudaMemcpyAsync(acc, w.loss_acc, sizeof(acc), cudaMemcpyDeviceToHost, s));
     PCM_CUDA_TRY(cudaMemcpyAsync(&l, loss, sizeof(float), cudaMemcpyDeviceToHost, s));
     PCM_CUDA_TRY(cudaStreamSynchronize(s));
-    const float tokens = (float)n * ACT;
+    const float tokens = (float)n * ACT, terms = chunk_ratio ? (float)n : tokens;
     stats->loss = l;
-    stats->clip_frac = tokens > 0 ? acc[1] / tokens : 0.f;
-    stats->mean_ratio = tokens > 0 ? acc[2] / tokens : 0.f;
+    stats->clip_frac = terms > 0 ? acc[1] / terms : 0.f;
+    stats->mean_ratio = terms > 0 ? acc[2] / terms : 0.f;
+    stats->entropy = tokens > 0 ? acc[3] / tokens : 0.f;
+    stats->reserved = 0;
     stats->n_launches = (int32_t)(g_launches.load() - launches0);
     stats->workspace_high_water = w.bytes;
     const int tcs = tcgen05_poll_status();

@@ -64,9 +64,10 @@ def device_packed(B, PL, model, hp):
     return pk
 
 
-def oracle_update(hp, eps_low=0.2, eps_high=0.2, loss_scale=None):
+def oracle_update(hp, eps_low=0.2, eps_high=0.2, loss_scale=None, entropy_coef=0.0, ratio_level="token"):
     w = hp["w"]
-    return ao.fwd_bwd(hp["weights"], hp["X"], hp["tgt"], hp["lpo"], hp["adv_c"], w.H, w.P, eps_low, eps_high, loss_scale)
+    return ao.fwd_bwd(hp["weights"], hp["X"], hp["tgt"], hp["lpo"], hp["adv_c"], w.H, w.P, eps_low, eps_high, loss_scale,
+                      entropy_coef, ratio_level)
 
 
 def grads_to_numpy(grads):

@@ -30,7 +30,7 @@ def test_binding_struct_sizes_match_the_header_layout():
     assert ctypes.sizeof(B.grpo_model) == 24 + 9 * 8
     assert ctypes.sizeof(B.grpo_packed) == 8 + 5 * 8
     assert ctypes.sizeof(B.grpo_loss_cfg) == 24
-    assert ctypes.sizeof(B.grpo_stats) == 24
+    assert ctypes.sizeof(B.grpo_stats) == 32
     assert set(B.EXPORTED) == set(_declared())
 
 

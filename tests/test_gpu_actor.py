@@ -72,12 +72,15 @@ def test_attention_fwd_bwd(dtype, dh, S, H, n_seq):
 
 
 # ------------------------------------------------------------------ end to end
-def _compare(B, PL, hp, tol_grad, tol_loss_rel=None, tol_loss_abs=None, mb=64, eps=(0.2, 0.2), loss_scale=None):
+def _compare(B, PL, hp, tol_grad, tol_loss_rel=None, tol_loss_abs=None, mb=64, eps=(0.2, 0.2), loss_scale=None,
+             entropy_coef=0.0, ratio_level="token", tol_ratio=None):
     w = hp["w"]
     model = PL.upload_model(w, hp["weights"])
     pk = device_packed(B, PL, model, hp)
-    loss_o, logp_o, grads_o, stats_o = oracle_update(hp, eps[0], eps[1], loss_scale)
-    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, pk, eps[0], eps[1], loss_scale or 0.0, mb_chunks=mb)
+    loss_o, logp_o, grads_o, stats_o = oracle_update(hp, eps[0], eps[1], loss_scale, entropy_coef, ratio_level)
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, pk, eps[0], eps[1], loss_scale or 0.0, mb_chunks=mb,
+                                                    flags=B.GRPO_CHUNK_RATIO if ratio_level == "chunk" else 0,
+                                                    entropy_coef=entropy_coef)
     loss = float(loss.item())
     if tol_loss_rel is not None:
         assert abs(loss - loss_o) <= tol_loss_rel * abs(loss_o) + 1e-9
@@ -88,6 +91,8 @@ def _compare(B, PL, hp, tol_grad, tol_loss_rel=None, tol_loss_abs=None, mb=64, e
     assert max(errs.values()) < tol_grad, errs
     assert abs(stats.clip_frac - stats_o["clip_frac"]) < 0.02
     assert stats.n_launches > 0
+    assert stats.entropy == pytest.approx(stats_o["entropy"], rel=1e-5 if w.dtype == "f32" else 5e-3)
+    assert stats.mean_ratio == pytest.approx(stats_o["mean_ratio"], rel=tol_ratio or (1e-4 if w.dtype == "f32" else 2e-2))
     return model, pk, (loss, logp, g, stats), (loss_o, logp_o, grads_o, stats_o), errs
 
 
@@ -120,6 +125,37 @@ def test_c0_fp32_paper_clip_and_heavy_clipping():
     hp = host_problem(w, seed=4, sigma=0.3, lpo_mode="uniform")
     _, _, got, ref, _ = _compare(B, PL, hp, F32_TOL, tol_loss_rel=F32_TOL, eps=(0.2, 0.4), loss_scale=1.0 / w.n_traj)
     assert ref[3]["clip_frac"] > 0.1
+
+
+@pytest.mark.parametrize("coef", [1e-3, 0.05])
+def test_c0_fp32_paper_loss_asymmetric_clip_and_entropy_bonus(coef):
+    """App. E's loss: clip (0.2, 0.4), entropy coefficient 1e-3 (and a larger one so its gradient dominates)."""
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"].with_(gamma_std=0.1)
+    hp = host_problem(w, seed=5, sigma=0.25)
+    _, pk, got, ref, _ = _compare(B, PL, hp, F32_TOL, tol_loss_rel=F32_TOL, eps=(0.2, 0.4), entropy_coef=coef, mb=5)
+    assert 0.02 < ref[3]["clip_frac"] < 0.9 and 0.5 < ref[3]["entropy"] < np.log(256.0)
+    # the entropy term alone (zero advantages): loss = -coef * mean entropy
+    hp0 = dict(hp); hp0["adv_c"] = np.zeros_like(hp["adv_c"])
+    _, _, got0, ref0, _ = _compare(B, PL, hp0, F32_TOL, tol_loss_rel=F32_TOL, eps=(0.2, 0.4), entropy_coef=coef)
+    assert got0[0] == pytest.approx(-coef * got0[3].entropy, rel=1e-5)
+
+
+@pytest.mark.parametrize("sigma,mb", [(0.0, 64), (0.03, 64), (0.03, 5), (0.2, 7)])
+def test_c0_fp32_chunk_level_ratio(sigma, mb):
+    """One importance ratio per chunk; sigma 0 is on-policy, 0.03 mixes clipped and unclipped chunks,
+    0.2 clips nearly every chunk with A > 0."""
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"].with_(gamma_std=0.1)
+    hp = host_problem(w, seed=6, sigma=sigma)
+    _, pk, got, ref, _ = _compare(B, PL, hp, 5e-5 if sigma == 0.2 else F32_TOL, tol_loss_rel=5e-5, eps=(0.2, 0.4),
+                                  entropy_coef=1e-3, ratio_level="chunk", mb=mb)
+    n = len(hp["kept"])
+    assert round(got[3].clip_frac * n) == round(ref[3]["clip_frac"] * n)          # the same chunks clipped
+    if sigma == 0.0:
+        assert ref[3]["clip_frac"] == 0.0
+    if sigma == 0.03:
+        assert 0.0 < ref[3]["clip_frac"] < 1.0
 
 
 def test_c0_full_pipeline_through_the_c_abi():
@@ -175,6 +211,22 @@ def test_bf16_end_to_end(case, backend, monkeypatch):
     _, _, got, ref, errs = _compare(B, PL, hp, BF16_GRAD_TOL, tol_loss_abs=BF16_LOSS_TOL, mb=2)
     assert np.max(np.abs(got[1].cpu().numpy() - ref[1])) < 0.04          # well inside the clip margin
     assert got[3].clip_frac == pytest.approx(ref[3]["clip_frac"], abs=1e-6)   # same clip decisions
+
+
+def test_bf16_entropy_bonus_and_chunk_ratio():
+    B, PL = _mods()
+    kw = dict(BF16_CASES["small"])
+    max_kept = kw.pop("max_kept")
+    w = synth.WORKLOADS["C1"].with_(gamma_std=0.1, force_mixed=True, p_succ=0.5, **kw)
+    hp = host_problem(w, seed=2, max_kept=max_kept, clip_margin=0.05, eps=(0.2, 0.4))
+    _compare(B, PL, hp, BF16_GRAD_TOL, tol_loss_abs=BF16_LOSS_TOL, mb=2, eps=(0.2, 0.4), entropy_coef=0.05)
+    # on-policy chunk ratios (r = 1 in the oracle): no chunk near a clip boundary.  The chunk's log-ratio adds
+    # the bf16 rounding of 56 log-probs (each a few 1e-3), so the ratio, which scales the whole chunk's
+    # gradient, carries a relative error of several per cent: the bound here is 0.15 instead of 2e-2.
+    hp1 = host_problem(w, seed=2, max_kept=max_kept, sigma=0.0)
+    _, _, got, ref, _ = _compare(B, PL, hp1, 0.15, tol_loss_abs=0.15, mb=2, eps=(0.2, 0.4), entropy_coef=1e-3,
+                                 ratio_level="chunk", tol_ratio=0.15)
+    assert got[3].clip_frac == 0.0 and ref[3]["clip_frac"] == 0.0
 
 
 def test_argument_errors():
