@@ -114,6 +114,71 @@ def score_phases(traj_off, tok, phase, reward, G: int, n_phases: int):
     return C, valid, n_valid, C_group, valid_group
 
 
+ACT_FIX_BITS = 32            # continuous actions are summed as integers in units of 2^-32
+ACT_ABS_MAX = 4096.0         # |a| bound that keeps every sum below 2^63 for up to 2^18 chunks per group
+
+
+def score_phases_float(traj_off, act, phase, reward, G: int, n_phases: int):
+    """Eq. 5 on continuous chunk actions: act is float32 [n_chunks, 56] (the 7-DoF x 8-step action of each
+    chunk as the policy emitted it, before or instead of tokenisation).
+
+    Same groups, skip rules and reductions as score_phases.  So that the result does not depend on
+    the order of a floating-point sum, every action value is first read as the integer
+    round-half-even(a * 2^32) (exact for |a| >= 2^-9 in float32, off by at most 2^-33 below), the sums over
+    chunks are exact integers, and the means, differences, squares, the ascending-dimension sum and the
+    square root are individually rounded fp64 operations; the unit 2^-32 is applied once at the end.
+    A value that is not finite or exceeds ACT_ABS_MAX in magnitude is counted as 0 and reported in `bad`.
+
+    Returns (C, valid, n_valid_groups, C_group, valid_group, bad) with the shapes of score_phases.
+    """
+    traj_off = np.asarray(traj_off)
+    act = np.asarray(act, dtype=np.float32)
+    n_groups = (traj_off.size - 1) // G
+    C_group = np.zeros((n_groups, n_phases), dtype=np.float64)
+    valid_group = np.zeros((n_groups, n_phases), dtype=np.uint8)
+    unit = 2.0 ** (-ACT_FIX_BITS)
+    bad = 0
+    for g in range(n_groups):
+        S = [[[0] * ACT_DIM for _ in range(2)] for _ in range(n_phases)]      # Python ints: exact
+        n = [[0, 0] for _ in range(n_phases)]
+        for i in range(g * G, (g + 1) * G):
+            o = 1 if reward[i] else 0
+            for ch in range(int(traj_off[i]), int(traj_off[i + 1])):
+                c = int(phase[ch])
+                row = act[ch]
+                for dim in range(ACT_DIM):
+                    a = float(row[dim])
+                    if not (abs(a) <= ACT_ABS_MAX):                           # also catches NaN
+                        bad += 1
+                        continue
+                    S[c][o][dim] += int(round(a * 4294967296.0))              # a * 2^32 is exact in fp64
+                n[c][o] += 1
+        for c in range(n_phases):
+            if n[c][1] == 0 or n[c][0] == 0:
+                continue
+            acc = 0.0
+            for dim in range(ACT_DIM):
+                diff = float(S[c][1][dim]) / float(n[c][1]) - float(S[c][0][dim]) / float(n[c][0])
+                acc = acc + diff * diff
+            C_group[g, c] = math.sqrt(acc) * unit
+            valid_group[g, c] = 1
+    C = np.zeros(n_phases, dtype=np.float64)
+    valid = np.zeros(n_phases, dtype=np.uint8)
+    n_valid = np.zeros(n_phases, dtype=np.int32)
+    for c in range(n_phases):
+        s = 0.0
+        cnt = 0
+        for g in range(n_groups):
+            if valid_group[g, c]:
+                s = s + C_group[g, c]
+                cnt += 1
+        n_valid[c] = cnt
+        if cnt > 0:
+            C[c] = s / float(cnt)
+            valid[c] = 1
+    return C, valid, n_valid, C_group, valid_group, bad
+
+
 # ----------------------------------------------------------------------------------------------
 # Eq. 7-9, Algorithm 1 - online keep-probability update
 # ----------------------------------------------------------------------------------------------

@@ -335,3 +335,72 @@ def test_default_mode_unchanged_by_the_ablation_switch():
         pa, qa, _ = po.update_keep_probs(a, C, [1] * 5)
         pb, qb, _ = po.update_keep_probs(b, C, [1] * 5)
         assert np.array_equal(pa, pb) and np.array_equal(qa, qb) and np.all(qa >= round(0.1 * (1 << 24)))
+
+
+# ---- Eq. 5 on continuous actions ------------------------------------------------------------------
+def test_float_scoring_matches_the_plain_definition_in_extended_precision():
+    """Brute force of Eq. 5 with exact rational arithmetic on the float32 inputs."""
+    from fractions import Fraction
+    rng = np.random.default_rng(11)
+    G, Kc, n_traj = 4, 3, 8
+    lens = rng.integers(3, 9, size=n_traj)
+    traj_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    N = int(traj_off[-1])
+    act = (rng.standard_normal((N, 56)) * np.exp(rng.uniform(-3, 2, size=(N, 1)))).astype(np.float32)
+    phase = rng.integers(0, Kc, size=N).astype(np.uint8)
+    reward = np.array([1, 0, 0, 1, 1, 1, 0, 1], dtype=np.uint8)
+    C, valid, nv, Cg, vg, bad = po.score_phases_float(traj_off, act, phase, reward, G, Kc)
+    assert bad == 0
+    for g in range(2):
+        for c in range(Kc):
+            rows = {0: [], 1: []}
+            for i in range(g * G, (g + 1) * G):
+                for ch in range(traj_off[i], traj_off[i + 1]):
+                    if phase[ch] == c:
+                        rows[int(reward[i])].append(ch)
+            if not rows[0] or not rows[1]:
+                assert vg[g, c] == 0
+                continue
+            tot = Fraction(0)
+            for dim in range(56):
+                m1 = sum(Fraction(float(act[ch, dim])) for ch in rows[1]) / len(rows[1])
+                m0 = sum(Fraction(float(act[ch, dim])) for ch in rows[0]) / len(rows[0])
+                tot += (m1 - m0) ** 2
+            assert Cg[g, c] == pytest.approx(math.sqrt(float(tot)), rel=1e-12, abs=1e-9)
+    for c in range(Kc):
+        if valid[c]:
+            assert C[c] == pytest.approx(np.mean([Cg[g, c] for g in range(2) if vg[g, c]]), rel=1e-15)
+
+
+def test_float_scoring_on_bin_centres_equals_token_scoring():
+    """De-tokenised actions a = -1 + (tok + 1/2) / 128 are exact in float32: both entry points agree."""
+    w = synth.WORKLOADS["C0"]
+    rb = synth.make_rollouts(w)
+    act = (-1.0 + (rb["tok"].astype(np.float64) + 0.5) / 128.0).astype(np.float32)
+    C_t, v_t, n_t, Cg_t, vg_t = po.score_phases(rb["traj_off"], rb["tok"], rb["phase"], rb["reward"], w.G, w.n_phases)
+    C_f, v_f, n_f, Cg_f, vg_f, bad = po.score_phases_float(rb["traj_off"], act, rb["phase"], rb["reward"], w.G, w.n_phases)
+    assert bad == 0 and np.array_equal(v_t, v_f) and np.array_equal(n_t, n_f) and np.array_equal(vg_t, vg_f)
+    assert np.allclose(Cg_f, Cg_t, rtol=1e-14, atol=0) and np.allclose(C_f, C_t, rtol=1e-14, atol=0)
+
+
+def test_float_scoring_is_invariant_to_chunk_order_and_flags_bad_values():
+    rng = np.random.default_rng(12)
+    G, Kc = 4, 2
+    traj_off = np.array([0, 5, 9, 15, 20], dtype=np.int32)
+    act = (rng.standard_normal((20, 56)) * 10.0 ** rng.integers(-6, 3, size=(20, 1))).astype(np.float32)
+    phase = rng.integers(0, Kc, size=20).astype(np.uint8)
+    reward = np.array([1, 0, 1, 0], dtype=np.uint8)
+    ref = po.score_phases_float(traj_off, act, phase, reward, G, Kc)
+    # reverse the chunks inside every trajectory: the sets per (phase, outcome) are unchanged
+    perm = np.concatenate([np.arange(traj_off[i], traj_off[i + 1])[::-1] for i in range(4)])
+    got = po.score_phases_float(traj_off, act[perm], phase[perm], reward, G, Kc)
+    assert np.array_equal(ref[0].view(np.uint64), got[0].view(np.uint64))          # bit-identical
+    # translation by a constant vector cancels in the difference of means (values on the 2^-32 grid stay exact)
+    shift = np.float32(0.5)
+    sh = po.score_phases_float(traj_off, (act.astype(np.float64) + 0.5).astype(np.float32), phase, reward, G, Kc)
+    assert np.allclose(sh[0], ref[0], rtol=1e-5)
+    bad = act.copy(); bad[3, 7] = np.nan; bad[11, 0] = np.inf; bad[12, 55] = 5000.0
+    out = po.score_phases_float(traj_off, bad, phase, reward, G, Kc)
+    assert out[5] == 3
+    zeroed = act.copy(); zeroed[3, 7] = 0; zeroed[11, 0] = 0; zeroed[12, 55] = 0
+    assert np.array_equal(out[0], po.score_phases_float(traj_off, zeroed, phase, reward, G, Kc)[0])
