@@ -117,6 +117,18 @@ int pcm_state_import(pcm_ctx* ctx, const void* host_buf, size_t bytes);
 int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* batch, double* C, uint8_t* valid,
                      int32_t* n_valid_groups, float* adv, pcm_stream stream);
 
+/* ---- Eq. 5 on continuous actions -----------------------------------------------------------------
+ * pcm_score_phases for policies whose chunk action is a float vector: act is device float32
+ * [n_chunks][56] (16-byte aligned), batch->tok is not read.  Groups, skip rules, reductions and outputs
+ * are those of pcm_score_phases with a = act.  To make the sums over chunks independent of their order
+ * every value is read as the integer round-half-even(a * 2^32) (exact for |a| >= 2^-9, off by at most
+ * 2^-33 below) and summed in 64-bit integers; the rest is the same chain of individually rounded fp64
+ * operations, with the unit 2^-32 applied once at the end.  Limits: |a| <= 4096 and finite (another value
+ * counts as 0 and raises the context's status word: PCM_ERR_DEVICE_DATA from pcm_poll_status);
+ * group_size * max_len <= 262144 chunks (PCM_ERR_SHAPE), so that no sum can overflow. */
+int pcm_score_phases_f32(pcm_ctx* ctx, const pcm_batch* batch, const float* act, double* C, uint8_t* valid,
+                         int32_t* n_valid_groups, float* adv, pcm_stream stream);
+
 /* ---- allocation-free variant of pcm_score_phases (the paper has no counterpart) -----------------
  * Same computation and outputs as pcm_score_phases, for callers that are not allowed to allocate
  * device memory: code that runs inside a region where the allocator is off limits (a serving or

@@ -111,6 +111,8 @@ _lib.grpo_gemm.argtypes = [C.c_int32, C.c_int32, C.c_int32, _P, C.c_int64, C.c_i
 _lib.grpo_attention.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P]
 _lib.pcm_score_phases_static.argtypes = [C.c_int32, C.c_int32, C.c_double, C.POINTER(pcm_batch), _P, _P, _P, _P, _P, _P]
 _lib.pcm_score_phases_static.restype = C.c_int
+_lib.pcm_score_phases_f32.argtypes = [_P, C.POINTER(pcm_batch), _P, _P, _P, _P, _P, _P]
+_lib.pcm_score_phases_f32.restype = C.c_int
 _lib.pcm_label_phases.argtypes = [_P, C.c_int32, _P, _P, _P, C.c_int32, _P, _P]
 _lib.pcm_label_phases.restype = C.c_int
 _lib.grpo_adamw_scratch_bytes.restype = C.c_size_t
@@ -130,7 +132,7 @@ EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", 
             "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
             "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static",
-            "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases")
+            "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases", "pcm_score_phases_f32")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -210,6 +212,20 @@ def pcm_score_phases(ctx: Context, batch: pcm_batch, want_adv: bool = True):
     adv = torch.empty(batch.n_traj, dtype=torch.float32, device=dev) if want_adv else None
     _check("pcm_score_phases", _lib.pcm_score_phases(ctx.handle, C.byref(batch), _ptr(Cc), _ptr(valid), _ptr(n_valid),
                                                      _ptr(adv), _stream()))
+    return Cc, valid, n_valid, adv
+
+
+def pcm_score_phases_f32(ctx: Context, batch: pcm_batch, act: torch.Tensor, want_adv: bool = True):
+    """Eq. 5 on continuous chunk actions: act float32 [n_chunks, 56]."""
+    assert act.dtype == torch.float32 and act.shape[-1] == ACT_DIM
+    dev = torch.device("cuda")
+    K = ctx.cfg.n_phases
+    Cc = torch.empty(K, dtype=torch.float64, device=dev)
+    valid = torch.empty(K, dtype=torch.uint8, device=dev)
+    n_valid = torch.empty(K, dtype=torch.int32, device=dev)
+    adv = torch.empty(batch.n_traj, dtype=torch.float32, device=dev) if want_adv else None
+    _check("pcm_score_phases_f32", _lib.pcm_score_phases_f32(ctx.handle, C.byref(batch), _ptr(act), _ptr(Cc), _ptr(valid),
+                                                             _ptr(n_valid), _ptr(adv), _stream()))
     return Cc, valid, n_valid, adv
 
 

@@ -16,6 +16,7 @@ constexpr unsigned STATUS_TIMEOUT = 1u;       // a bounded wait expired
 constexpr unsigned STATUS_BAD_PHASE = 2u;     // phase label >= n_phases
 constexpr unsigned STATUS_TOO_LONG = 4u;      // trajectory longer than max_len
 constexpr unsigned STATUS_BAD_OFFSETS = 8u;   // traj_off / kept_idx inconsistent with host sizes
+constexpr unsigned STATUS_BAD_ACTION = 16u;   // continuous action not finite or beyond the fixed-point range
 
 #define PCM_CUDA_TRY(expr)                         \
   do {                                             \

@@ -200,6 +200,123 @@ score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restr
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Eq. 5 on continuous actions (float32 [n_chunks][56]).  Every value is read as the integer
+// round-half-even(a * 2^32); sums over chunks are then exact 64-bit integers, independent of their order.
+// One CTA per group, a warp per trajectory; a chunk is 14 float4, so lanes 0..13 and 14..27 each walk one
+// contiguous half of the trajectory and keep four running sums per lane while the phase does not change.
+// ------------------------------------------------------------------------------------------------
+constexpr float ACT_ABS_MAX = 4096.f;                     // |a| * 2^32 <= 2^44; 2^18 chunks per group stay below 2^63
+constexpr int ACT_MAX_GROUP_CHUNKS = 1 << 18;
+
+__global__ void __launch_bounds__(256)
+score_groups_f32_kernel(const int32_t* __restrict__ traj_off, const float* __restrict__ act,
+                        const uint8_t* __restrict__ phase, const uint8_t* __restrict__ reward, int G, int n_phases,
+                        int max_len, double* __restrict__ c_group, uint8_t* __restrict__ valid_group,
+                        unsigned* __restrict__ status) {
+  extern __shared__ unsigned long long smf[];
+  unsigned long long* sums = smf;                                           // [n_phases][2][56], two's complement
+  unsigned* cnt = reinterpret_cast<unsigned*>(smf + n_phases * 2 * ACT);    // [n_phases][2]
+  const int g = blockIdx.x;
+  for (int i = threadIdx.x; i < n_phases * 2 * ACT; i += blockDim.x) sums[i] = 0ull;
+  for (int i = threadIdx.x; i < n_phases * 2; i += blockDim.x) cnt[i] = 0u;
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int slot = lane / 14, vec = lane - slot * 14;     // slots 0, 1 active; lanes 28..31 idle
+  for (int i = g * G + warp; i < (g + 1) * G; i += nwarps) {
+    const int o = reward[i] ? 1 : 0;
+    const int a = traj_off[i], b = traj_off[i + 1];
+    if (b - a > max_len || b < a) {
+      if (lane == 0) atomicOr(status, STATUS_TOO_LONG);
+      continue;
+    }
+    if (slot >= 2) continue;
+    const int per = (b - a + 1) >> 1;
+    const int c_lo = a + slot * per, c_hi = min(b, c_lo + per);
+    long long acc[4] = {0, 0, 0, 0};
+    unsigned run = 0;
+    int cur = -1;
+    auto flush = [&]() {
+      if (run) {
+        unsigned long long* sp = sums + (cur * 2 + o) * ACT + 4 * vec;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) atomicAdd(sp + e, (unsigned long long)acc[e]);
+        if (vec == 0) atomicAdd(cnt + cur * 2 + o, run);
+      }
+      acc[0] = acc[1] = acc[2] = acc[3] = 0;
+      run = 0;
+    };
+    constexpr int UNROLL = 4;
+    for (int c0 = c_lo; c0 < c_hi; c0 += UNROLL) {
+      float4 v[UNROLL];
+      int ph[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const int ch = c0 + u;
+        if (ch < c_hi) {
+          v[u] = __ldg(reinterpret_cast<const float4*>(act + (size_t)ch * ACT) + vec);
+          ph[u] = __ldg(phase + ch);
+        } else {
+          v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          ph[u] = -1;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        if (ph[u] < 0) continue;
+        if (ph[u] >= n_phases) {
+          atomicOr(status, STATUS_BAD_PHASE);
+          continue;
+        }
+        if (ph[u] != cur) {
+          flush();
+          cur = ph[u];
+        }
+        const float x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (fabsf(x[e]) <= ACT_ABS_MAX)                  // false for NaN as well
+            acc[e] += __double2ll_rn(__dmul_rn((double)x[e], 4294967296.0));
+          else
+            atomicOr(status, STATUS_BAD_ACTION);           // counted as 0
+        }
+        ++run;
+      }
+    }
+    flush();
+  }
+  __syncthreads();
+
+  __shared__ double sq[8][ACT];
+  for (int c = warp; c < n_phases; c += nwarps) {
+    const unsigned n_succ = cnt[c * 2 + 1], n_fail = cnt[c * 2 + 0];
+    const bool both = n_succ && n_fail;
+    if (both) {
+      const unsigned long long* s1 = sums + (c * 2 + 1) * ACT;
+      const unsigned long long* s0 = sums + (c * 2 + 0) * ACT;
+      for (int dim = lane; dim < ACT; dim += 32) {
+        const double m1 = __ddiv_rn(__ll2double_rn((long long)s1[dim]), (double)n_succ);
+        const double m0 = __ddiv_rn(__ll2double_rn((long long)s0[dim]), (double)n_fail);
+        const double diff = __dsub_rn(m1, m0);
+        sq[warp][dim] = __dmul_rn(diff, diff);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) {
+      double val = 0.0;
+      if (both) {
+        double acc = 0.0;
+        for (int dim = 0; dim < ACT; ++dim) acc = __dadd_rn(acc, sq[warp][dim]);
+        val = __dmul_rn(__dsqrt_rn(acc), 1.0 / 4294967296.0);
+      }
+      c_group[(size_t)g * n_phases + c] = val;
+      valid_group[(size_t)g * n_phases + c] = both ? 1 : 0;
+    }
+    __syncwarp();
+  }
+}
+
 // Blocks 0 .. n_phases-1: mean of C_{c,g} over valid groups.  One warp per phase loads 32 groups at a
 // time in parallel and adds them in ascending g (every lane runs the same chain, so the order of the
 // fp64 additions is exactly the sequential one).
@@ -545,6 +662,28 @@ int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* b, double* C, uint8_t* valid
                                              ctx->valid_group, ctx->status);
   PCM_LAUNCH_CHECK();
   prof_end(s, 0.0, (double)b->n_chunks * (ACT + 1));
+  const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
+  score_finalize_kernel<<<Kc + adv_blocks, 128, 0, s>>>(ctx->c_group, ctx->valid_group, ng, Kc, C, valid,
+                                                       n_valid_groups, b->reward, G, ctx->cfg.adv_eps, adv);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
+}
+
+int pcm_score_phases_f32(pcm_ctx* ctx, const pcm_batch* b, const float* act, double* C, uint8_t* valid,
+                         int32_t* n_valid_groups, float* adv, pcm_stream stream) {
+  int rc = check_batch(ctx, b);
+  if (rc) return rc;
+  if (!act || !b->reward || !C || !valid) return PCM_ERR_ARG;
+  if (((uintptr_t)act) & 15) return PCM_ERR_ARG;
+  const int G = ctx->cfg.group_size, Kc = ctx->cfg.n_phases, ng = b->n_traj / G;
+  if ((long long)G * b->max_len > ACT_MAX_GROUP_CHUNKS) return PCM_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t smem = (size_t)Kc * 2 * ACT * sizeof(unsigned long long) + (size_t)Kc * 2 * sizeof(unsigned);
+  prof_begin(PC_SCORE, s);
+  score_groups_f32_kernel<<<ng, 256, smem, s>>>(b->traj_off, act, b->phase, b->reward, G, Kc, b->max_len, ctx->c_group,
+                                                 ctx->valid_group, ctx->status);
+  PCM_LAUNCH_CHECK();
+  prof_end(s, 0.0, (double)b->n_chunks * (ACT * 4 + 1));
   const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
   score_finalize_kernel<<<Kc + adv_blocks, 128, 0, s>>>(ctx->c_group, ctx->valid_group, ng, Kc, C, valid,
                                                        n_valid_groups, b->reward, G, ctx->cfg.adv_eps, adv);

@@ -225,3 +225,73 @@ def test_bad_mask_mode_is_rejected():
     B, _ = _mods()
     with pytest.raises(RuntimeError):
         B.Context(4, 4, 4, mode=3)
+
+
+def _float_actions(rb, seed, scale_spread=True):
+    """Continuous stand-in for the chunk actions: bin centres plus seeded jitter, magnitudes over several decades."""
+    rng = np.random.default_rng(seed)
+    base = -1.0 + (rb["tok"].astype(np.float64) + 0.5) / 128.0
+    act = base + 0.01 * rng.standard_normal(base.shape)
+    if scale_spread:
+        act = act * np.exp(rng.uniform(-8, 3, size=(act.shape[0], 1)))
+    return act.astype(np.float32)
+
+
+@pytest.mark.parametrize("name", ["C0", "C4"])
+def test_float_action_scoring_bit_exact(name):
+    B, PL = _mods()
+    w = synth.WORKLOADS[name]
+    rb = synth.make_rollouts(w)
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=0, max_traj=w.n_traj)
+    batch = PL.upload_rollouts(w, rb)
+    for spread in (False, True):
+        act = _float_actions(rb, 3, spread)
+        Cc, valid, n_valid, adv = B.pcm_score_phases_f32(ctx, batch, PL.dev(act))
+        C_o, valid_o, nv_o, _, _, bad = po.score_phases_float(rb["traj_off"], act, rb["phase"], rb["reward"], w.G, w.n_phases)
+        assert bad == 0 and B.pcm_poll_status(ctx) == 0
+        assert np.array_equal(_np(Cc).view(np.uint64), C_o.view(np.uint64))
+        assert np.array_equal(_np(valid), valid_o) and np.array_equal(_np(n_valid), nv_o)
+        adv_o = po.advantages(rb["reward"], w.G, 1e-6).astype(np.float32)
+        assert np.array_equal(_np(adv).view(np.uint32), adv_o.view(np.uint32))
+    # exact bin centres: the float entry point reproduces the token entry point to rounding
+    centres = (-1.0 + (rb["tok"].astype(np.float64) + 0.5) / 128.0).astype(np.float32)
+    C_f = _np(B.pcm_score_phases_f32(ctx, batch, PL.dev(centres))[0])
+    C_t = _np(B.pcm_score_phases(ctx, batch)[0])
+    assert np.allclose(C_f, C_t, rtol=1e-14, atol=0)
+    ctx.close()
+
+
+def test_float_action_scoring_edge_cases():
+    B, PL = _mods()
+    rng = np.random.default_rng(2)
+    lengths = np.array([700, 3, 1, 0, 10, 10, 11, 10], dtype=np.int64)       # long, odd, single and empty trajectories
+    traj_off = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    total = int(traj_off[-1])
+    phase = rng.integers(0, 3, total).astype(np.uint8)
+    phase[:650] = 1                                                          # one long run in a single phase
+    reward = np.array([1, 0, 0, 1, 1, 1, 1, 1], dtype=np.uint8)              # second group uniform
+    act = (rng.standard_normal((total, 56)) * 10.0 ** rng.integers(-7, 4, size=(total, 1))).astype(np.float32)
+    act = np.clip(act, -4096, 4096)
+    act[5, 3] = 4096.0; act[6, 3] = -4096.0; act[7, 0] = 1e-30; act[8, 0] = -0.0
+    w = synth.WORKLOADS["C0"].with_(n_phases=3, G=4)
+    rb = {"traj_off": traj_off, "tok": np.zeros((total, 56), dtype=np.uint8), "phase": phase, "reward": reward}
+    ctx = B.Context(3, 2, 4, 5, 0.1, 1e-6, seed=0, max_traj=8)
+    batch = PL.upload_rollouts(w, rb)
+    Cc, valid, n_valid, _ = B.pcm_score_phases_f32(ctx, batch, PL.dev(act))
+    C_o, valid_o, nv_o, _, _, bad = po.score_phases_float(traj_off, act, phase, reward, 4, 3)
+    assert bad == 0 and B.pcm_poll_status(ctx) == 0
+    assert np.array_equal(_np(Cc).view(np.uint64), C_o.view(np.uint64))
+    assert np.array_equal(_np(valid), valid_o) and np.array_equal(_np(n_valid), nv_o) and nv_o.max() == 1
+    # values outside the range count as zero and are reported, on both sides
+    act_bad = act.copy(); act_bad[2, 9] = np.nan; act_bad[701, 0] = np.inf; act_bad[10, 55] = -5000.0
+    Cc, _, _, _ = B.pcm_score_phases_f32(ctx, batch, PL.dev(act_bad))
+    C_b, _, _, _, _, bad = po.score_phases_float(traj_off, act_bad, phase, reward, 4, 3)
+    assert bad == 3 and np.array_equal(_np(Cc).view(np.uint64), C_b.view(np.uint64))
+    assert B.pcm_poll_status(ctx) == -7 and B.pcm_poll_status(ctx) == 0
+    # host checks: misaligned action pointer, group too large for the 64-bit sums
+    with pytest.raises(RuntimeError):
+        B.pcm_score_phases_f32(ctx, batch, PL.dev(np.zeros(total * 56 + 1, dtype=np.float32))[1:].view(total, 56))
+    big = B.make_batch(PL.dev(traj_off), None, PL.dev(phase), PL.dev(reward), 70000)
+    with pytest.raises(RuntimeError):
+        B.pcm_score_phases_f32(ctx, big, PL.dev(act))
+    ctx.close()
