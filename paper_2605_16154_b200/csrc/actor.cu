@@ -838,5 +838,5 @@ extern "C" int grpo_attention(int32_t dtype, const void* qkv, void* out, float* 
     if (rc != PCM_OK) return rc;
   }
   PCM_CUDA_TRY(cudaStreamSynchronize(s));
-  return PCM_OK;
+  return tcgen05_poll_status();
 }

@@ -1,5 +1,7 @@
 // Dispatch of the attention entry points on the activation dtype: fp32 runs the SIMT kernels
 // (attention_f32.cu), bf16 the tensor-core kernels (attention_mma.cu).
+#include <cstdlib>
+
 #include "internal.h"
 
 namespace pcm {
@@ -10,11 +12,26 @@ int attention_bwd_f32(const void*, const void*, const void*, const float*, float
 int attention_bwd_bf16(const void*, const void*, const void*, const float*, float*, void*, int, int, int, int, const float2*,
                        cudaStream_t);
 
+bool attention_tc_supported(const void* qkv, const void* out, int S, int H, int dh);
+int attention_fwd_bf16_tc(const void*, void*, float*, int, int, int, int, cudaStream_t);
+
+// PCM_ATTN_TC=0 keeps bf16 attention on the warp-level (mma.sync) kernels, for comparison runs.
+static bool attn_tc_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("PCM_ATTN_TC");
+    v = (e && e[0] == '0') ? 0 : 1;
+  }
+  return v == 1;
+}
+
 int attention_fwd(int dtype, const void* qkv, void* out, float* lse, int n_seq, int S, int H, int dh,
                   cudaStream_t s) {
   if (S > 384 || n_seq > 65535) return PCM_ERR_SHAPE;
-  return dtype == DT_F32 ? attention_fwd_f32(qkv, out, lse, n_seq, S, H, dh, s)
-                         : attention_fwd_bf16(qkv, out, lse, n_seq, S, H, dh, s);
+  if (dtype == DT_F32) return attention_fwd_f32(qkv, out, lse, n_seq, S, H, dh, s);
+  if (attn_tc_enabled() && attention_tc_supported(qkv, out, S, H, dh))
+    return attention_fwd_bf16_tc(qkv, out, lse, n_seq, S, H, dh, s);
+  return attention_fwd_bf16(qkv, out, lse, n_seq, S, H, dh, s);
 }
 
 int attention_bwd(int dtype, const void* qkv, const void* out, const void* dout, const float* lse, float* dsum,

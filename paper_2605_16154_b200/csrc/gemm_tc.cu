@@ -978,7 +978,11 @@ int gemm_tcgen05(const GemmArgs& g, cudaStream_t s) {
   return launch_tc<128, EPI_NONE>(g, s);
 }
 
+int attention_tc_poll_status();
+
 int tcgen05_poll_status() {
+  const int arc = attention_tc_poll_status();
+  if (arc != PCM_OK) return arc;
   unsigned h = 0;
   if (cudaMemcpyFromSymbol(&h, g_tc_status, sizeof(h)) != cudaSuccess) return PCM_ERR_CUDA;
   if (h) {

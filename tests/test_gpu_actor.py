@@ -47,7 +47,9 @@ def test_gemm_simt_all_layouts(dtype, a_k, b_k):
 
 # ------------------------------------------------------------------ attention
 @pytest.mark.parametrize("dtype,dh,S,H,n_seq", [("f32", 32, 88, 4, 3), ("f32", 64, 45, 2, 2), ("bf16", 64, 312, 3, 2),
-                                                ("bf16", 128, 100, 2, 2), ("bf16", 32, 33, 2, 1)])
+                                                ("bf16", 128, 100, 2, 2), ("bf16", 32, 33, 2, 1),
+                                                ("bf16", 64, 384, 2, 3), ("bf16", 128, 312, 2, 2), ("bf16", 64, 17, 1, 1),
+                                                ("bf16", 64, 200, 16, 24), ("bf16", 128, 129, 16, 10)])
 def test_attention_fwd_bwd(dtype, dh, S, H, n_seq):
     B, PL = _mods()
     rng = np.random.default_rng(5)
