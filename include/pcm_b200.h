@@ -329,6 +329,12 @@ int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32
 int grpo_attention(int32_t dtype, const void* qkv, void* out, float* lse, const void* dout, void* dqkv,
                    float* scratch, int32_t n_seq, int32_t S, int32_t n_heads, int32_t head_dim, pcm_stream stream);
 
+/* Which bounded wait of the tensor-core attention kernels expired last (0 = none since the library was
+ * loaded): bit 0 set, bit 8 + k names the barrier (k = 0 K/V buffer free, 1 query buffer free, 2 K/V landed,
+ * 3 queries landed, 4 probabilities ready, 5 accumulator slot free, 6 output ready, 7 scores ready).
+ * Updated when a call returns PCM_ERR_DEVICE_TIMEOUT.  Host value, no GPU work. */
+uint32_t grpo_attention_wait_status(void);
+
 /* Per-kernel-class timing.  While enabled, every launch of the classes below is bracketed by a
  * pair of CUDA events on its stream; pcm_profile_read() synchronises the device, adds up elapsed
  * milliseconds, the algorithmic flops / bytes of the launches and their count since the last read,

@@ -132,7 +132,8 @@ EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", 
             "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
             "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static",
-            "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases", "pcm_score_phases_f32")
+            "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases", "pcm_score_phases_f32",
+            "grpo_attention_wait_status")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -386,6 +387,11 @@ def grpo_attention(qkv: torch.Tensor, n_seq: int, S: int, H: int, dh: int, dout:
     _check("grpo_attention", _lib.grpo_attention(dt, _ptr(qkv), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dqkv),
                                                  _ptr(scratch), n_seq, S, H, dh, _stream()))
     return out, lse, dqkv
+
+
+def grpo_attention_wait_status() -> int:
+    _lib.grpo_attention_wait_status.restype = C.c_uint32
+    return int(_lib.grpo_attention_wait_status())
 
 
 def pcm_launch_count() -> int:

@@ -823,6 +823,9 @@ extern "C" int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t
   return tcgen05_poll_status();
 }
 
+namespace pcm { unsigned attention_tc_last_status(); }
+extern "C" uint32_t grpo_attention_wait_status(void) { return pcm::attention_tc_last_status(); }
+
 extern "C" int grpo_attention(int32_t dtype, const void* qkv, void* out, float* lse, const void* dout, void* dqkv,
                               float* scratch, int32_t n_seq, int32_t S, int32_t n_heads, int32_t head_dim,
                               pcm_stream stream) {

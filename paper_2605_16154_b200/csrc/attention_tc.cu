@@ -2,17 +2,21 @@
 //
 // One persistent CTA per SM walks (sequence, head) items.  The whole K and V of an item (S <= 384 rows)
 // sit in shared memory (TMA, 128-byte swizzle); query tiles of 128 rows stream through a small ring.
-// For a query tile the full score row block S = Q K^T (128 x n, n <= 384 columns, causal: only the
-// columns at or left of the tile's last row) is produced by tcgen05.mma into tensor memory, so the
-// softmax is a plain two-pass softmax over tensor memory (no running rescale): pass 1 takes the row
-// maximum, pass 2 writes P = exp(.) as packed bf16 back into tensor memory over the scores it has
-// consumed, and O = P V runs with P as the tensor-memory A operand and V as an MN-major shared-memory
-// B operand.  Probabilities never touch shared or global memory.
+// A query tile is processed as independent blocks of 128 keys (causal: the blocks at or left of the
+// diagonal).  For block j, tcgen05.mma puts S_j = Q K_j^T (128 x 128, fp32) into one of the score
+// buffers in tensor memory; the softmax warps take the block's own row maximum m_j, write
+// P_j = exp(S_j - m_j) as packed bf16 over the scores they have consumed and keep the row sums l_j;
+// O_j = P_j V_j then runs with P_j as the tensor-memory A operand and V_j as an MN-major shared-memory
+// B operand into its own accumulator slot.  Blocks never wait for one another (no running rescale);
+// the output warps combine the slots at the end of the tile:
+//   m = max_j m_j,  w_j = exp(m_j - m),  O = sum_j w_j O_j / sum_j w_j l_j,  lse = m + log(sum_j w_j l_j).
+// With two score buffers the tensor core works on one block while the softmax warps work on the other.
+// Probabilities never touch shared or global memory.
 //
-// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = tensor-memory allocation + MMA issue,
-// warps 2..9 = softmax and output (two per tensor-memory lane quadrant; the two split a tile's columns).
-// Every mbarrier wait is bounded; when one runs out the CTA latches a status bit, all roles leave at the
-// next tile boundary, tensor memory is released and the kernel returns.
+// Warp roles: warp 0 = TMA producer, warp 1 = tensor-memory allocation + MMA issue, warps 2..5 = output
+// (one per tensor-memory lane quadrant), then 8 softmax warps per score buffer (two per lane quadrant,
+// splitting the block's columns).  Every mbarrier wait is bounded; when one runs out the CTA latches a
+// status bit, all roles leave at their next block boundary, tensor memory is released and the kernel returns.
 #include <cuda.h>
 
 #include "async_ptx.cuh"
@@ -20,30 +24,54 @@
 
 namespace pcm {
 
-__device__ unsigned g_fa_status = 0;          // bit 0: a bounded wait expired
+__device__ unsigned g_fa_status = 0;          // bit 0: a bounded wait expired; bit 8 + site: which wait it was
+__device__ __forceinline__ void fa_timeout(int site) { atomicOr(&g_fa_status, 1u | (1u << (8 + site))); }
+enum { SITE_KV_EMPTY = 0, SITE_Q_EMPTY = 1, SITE_KV_FULL = 2, SITE_Q_FULL = 3, SITE_P_FULL = 4, SITE_O_EMPTY = 5, SITE_O_FULL = 6, SITE_S_FULL = 7 };
 
 namespace fatc {
 
 constexpr int BM = 128;                        // query rows per tile = tensor-memory lanes
-constexpr int THREADS = 320;
-constexpr int SM_WARPS = 8;                    // softmax warps
+constexpr int BN = 128;                        // keys per block
+constexpr int MAX_SLOTS = 3;                   // blocks per tile at most: S <= 384
+constexpr int S_MAX = BN * MAX_SLOTS;
+constexpr int SM_WARPS_PER_BUF = 8;
 constexpr unsigned long long WAIT_NS = 2000000000ull;
 constexpr int TMEM_COLS = 512;
-constexpr int S_COLS = 384;                    // score columns (fp32); P (packed bf16) overwrites consumed scores
-constexpr int O_COL = 384;                     // output accumulator: columns [384, 384 + DH)
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
+constexpr int OUT_BAR = 9;                     // named barrier of the four output warps (1..8: softmax warp pairs)
+constexpr int STAT_RING = 4;                   // tiles whose row statistics may be live at once
+
+template <int DH> struct Cfg {
+  static constexpr int NBUF = DH == 64 ? 2 : 1;                       // score buffers that fit beside the output slots
+  static constexpr int O_COL = NBUF * BN;                             // accumulator slot s: columns [O_COL + s DH, +DH)
+  static constexpr int NSLOT = (TMEM_COLS - O_COL) / DH;              // slots form a ring over all blocks of the CTA
+  static constexpr int THREADS = (2 + 4 + NBUF * SM_WARPS_PER_BUF) * 32;
+  static_assert(NSLOT >= MAX_SLOTS, "tensor memory plan does not fit");
+};
 
 struct Params {
   int n_seq, S, H, d;
   int n_items;                                 // n_seq * H
   int nq;                                      // query tiles per item
   int kv_rows;                                 // rows of K / V staged per item (multiple of 64)
-  int n_total;                                 // S rounded up to 16: columns of the widest score block
+  int n_total;                                 // S rounded up to 16: keys that take part in the MMAs
   int kv_stages, q_stages;
   float scale_log2;                            // log2(e) / sqrt(dh)
   __nv_bfloat16* out;
   float* lse;
+};
+
+// Walks the blocks of this CTA's items in issue order: item k, query tile t, key block j <= t.
+struct BlockIter {
+  int nq, k, t, j, tile;                       // tile = running count of query tiles (all items)
+  __device__ void init(int nq_) { nq = nq_; k = t = j = tile = 0; }
+  __device__ void next() {
+    if (j < t) { ++j; return; }
+    j = 0; ++tile;
+    if (t + 1 < nq) { ++t; } else { t = 0; ++k; }
+  }
+  __device__ void advance(int n) { for (int i = 0; i < n; ++i) next(); }
 };
 
 __device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* tmap, int x, int y, int z, uint64_t* bar) {
@@ -71,6 +99,13 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r
       "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const void* tmap, const void* smem_src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(tmap),
+               "r"(smem_u32(smem_src)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+// makes this thread's shared-memory writes visible to the asynchronous proxy (TMA)
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -105,9 +140,11 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n, int b_mn_major) {
 //   K ring   kv_stages x DH/64 slabs x kv_rows x 128 B     slab = 64 head-dim columns of every staged row
 //   V ring   the same
 //   Q ring   q_stages x DH/64 slabs x 128 rows x 128 B
-//   barriers, row statistics exchanged between the two warps of a lane quadrant
+//   output staging for the TMA store
+//   barriers; row statistics (m_j, l_j per tile of the ring, block and row); the maxima the two warps of a
+//   lane quadrant exchange
 struct Plan {
-  uint32_t k_off, v_off, q_off, bar_off, red_off, total;
+  uint32_t k_off, v_off, q_off, ostage_off, bar_off, stat_m_off, stat_l_off, red_off, total;
 };
 __host__ __device__ inline Plan make_plan(int dh, int kv_rows, int kv_stages, int q_stages) {
   Plan p;
@@ -116,50 +153,63 @@ __host__ __device__ inline Plan make_plan(int dh, int kv_rows, int kv_stages, in
   p.k_off = 0;
   p.v_off = p.k_off + kv_stages * kv_bytes;
   p.q_off = p.v_off + kv_stages * kv_bytes;
-  p.bar_off = p.q_off + q_stages * q_bytes;
-  p.red_off = p.bar_off + 256;
-  p.total = p.red_off + 2 * 2 * BM * 4 + 1024 /* alignment slack */;
+  p.ostage_off = p.q_off + q_stages * q_bytes;                       // 128 rows x 64 bf16 columns, swizzled
+  p.bar_off = p.ostage_off + BM * 128;
+  p.stat_m_off = p.bar_off + 256;
+  p.stat_l_off = p.stat_m_off + STAT_RING * MAX_SLOTS * BM * 4;
+  p.red_off = p.stat_l_off + STAT_RING * MAX_SLOTS * BM * 4;
+  p.total = p.red_off + 2 * 2 * 2 * BM * 4 + 1024 /* alignment slack */;
   return p;
 }
 
-
 template <int DH>
-__global__ void __launch_bounds__(THREADS, 1)
-fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const Params p) {
+__global__ void __launch_bounds__(Cfg<DH>::THREADS, 1)
+fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV,
+                 const __grid_constant__ CUtensorMap tmO, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int NSLAB = DH / 64;
+  constexpr int NBUF = Cfg<DH>::NBUF;
+  constexpr int O_COL = Cfg<DH>::O_COL;
+  constexpr int NSLOT = Cfg<DH>::NSLOT;
   constexpr uint32_t Q_SLAB = BM * 128u, Q_BYTES = NSLAB * Q_SLAB;
   const uint32_t raw_addr = smem_u32(smem_raw);
   uint8_t* base = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
   const Plan pl = make_plan(DH, p.kv_rows, p.kv_stages, p.q_stages);
   const uint32_t kv_slab = (uint32_t)p.kv_rows * 128u, kv_bytes = NSLAB * kv_slab;
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + pl.bar_off);
-  uint64_t* kv_full = bars;                    // [2] producer -> MMA, K and V of one item
+  uint64_t* kv_full = bars;                    // [2] producer -> MMA: K and V of one item
   uint64_t* kv_empty = bars + 2;               // [2] MMA -> producer
   uint64_t* q_full = bars + 4;                 // [2]
   uint64_t* q_empty = bars + 6;                // [2]
-  uint64_t* s_full = bars + 8;                 // MMA -> softmax: scores of a tile are in tensor memory
-  uint64_t* p_full = bars + 9;                 // softmax -> MMA: probabilities are in tensor memory (8 warp arrivals)
-  uint64_t* o_full = bars + 10;                // MMA -> softmax: the tile's output is in tensor memory
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11);
+  uint64_t* s_full = bars + 8;                 // [2] MMA -> softmax: a block's scores are in the buffer
+  uint64_t* p_full = bars + 10;                // [2] softmax -> MMA: the block's probabilities are in the buffer (8 warp arrivals)
+  uint64_t* o_full = bars + 12;                // [2] MMA -> output warps: every slot of the tile is complete
+  uint64_t* o_empty = bars + 14;               // [2] output warps -> MMA: the tile's slots may be overwritten (4 warp
+                                               //     arrivals); tiles alternate between the two barriers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile uint32_t* abort_flag = tmem_slot + 1;
-  float* red_max = reinterpret_cast<float*>(base + pl.red_off);   // [2][128]
-  float* red_sum = red_max + 2 * BM;                              // [2][128]
+  float* stat_m = reinterpret_cast<float*>(base + pl.stat_m_off);   // [STAT_RING][MAX_SLOTS][128]
+  float* stat_l = reinterpret_cast<float*>(base + pl.stat_l_off);   // [STAT_RING][MAX_SLOTS][128]
+  float* red_max = reinterpret_cast<float*>(base + pl.red_off);     // [2][2][128]
+  float* red_sum = red_max + 2 * 2 * BM;                            // [2][2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_local = ((int)blockIdx.x < p.n_items) ? (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const int n_tiles = n_local * p.nq;
+  const int n_blocks = n_local * (p.nq * (p.nq + 1) / 2);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
       mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1);
       mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 1);
+      mbar_init(&s_full[s], 1); mbar_init(&p_full[s], SM_WARPS_PER_BUF);
     }
-    mbar_init(s_full, 1); mbar_init(p_full, SM_WARPS); mbar_init(o_full, 1);
+    mbar_init(&o_full[0], 1); mbar_init(&o_full[1], 1); mbar_init(&o_empty[0], 4); mbar_init(&o_empty[1], 4);
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmKV);
+    prefetch_tmap(&tmO);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, TMEM_COLS);
@@ -176,9 +226,9 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       bool ok = true;
       for (int k = 0; k < n_local && ok && !*abort_flag; ++k) {
         const int item = blockIdx.x + k * gridDim.x, seq = item / p.H, h = item - seq * p.H;
-        const int st = k % p.kv_stages;
-        const unsigned ph = (unsigned)(k / p.kv_stages) & 1u;
-        if (!mbar_wait_bounded(&kv_empty[st], ph ^ 1u, WAIT_NS)) { ok = false; break; }
+        const int st = k & (p.kv_stages - 1);                          // stages are 1 or 2
+        const unsigned ph = (unsigned)(k >> (p.kv_stages - 1)) & 1u;
+        if (!mbar_wait_bounded(&kv_empty[st], ph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; break; }
         mbar_expect_tx(&kv_full[st], 2 * kv_bytes);
         uint8_t* ks = base + pl.k_off + st * kv_bytes;
         uint8_t* vs = base + pl.v_off + st * kv_bytes;
@@ -188,133 +238,292 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             tma_load_3d(vs + sl * kv_slab + rb * 8192, &tmKV, 2 * p.d + h * DH + sl * 64, rb * 64, seq, &kv_full[st]);
           }
         for (int t = 0; t < p.nq; ++t) {
-          const int g = k * p.nq + t, qs = g % p.q_stages;
-          const unsigned qph = (unsigned)(g / p.q_stages) & 1u;
-          if (*abort_flag || !mbar_wait_bounded(&q_empty[qs], qph ^ 1u, WAIT_NS)) { ok = false; break; }
+          const int g = k * p.nq + t, qs = g & (p.q_stages - 1);
+          const unsigned qph = (unsigned)(g >> (p.q_stages - 1)) & 1u;
+          if (*abort_flag) { ok = false; break; }
+          if (!mbar_wait_bounded(&q_empty[qs], qph ^ 1u, WAIT_NS)) { fa_timeout(SITE_Q_EMPTY); ok = false; break; }
           mbar_expect_tx(&q_full[qs], Q_BYTES);
           uint8_t* qd = base + pl.q_off + qs * Q_BYTES;
           for (int sl = 0; sl < NSLAB; ++sl)
             tma_load_3d(qd + sl * Q_SLAB, &tmQ, h * DH + sl * 64, t * BM, seq, &q_full[qs]);
         }
       }
-      if (!ok) { *abort_flag = 1; atomicOr(&g_fa_status, 1u); }
+      if (!ok) *abort_flag = 1;
     }
   } else if (warp == 1) {
     if (lane == 0) {
       // ------------------------------ MMA issuer ------------------------------
+      // One thread issues every MMA, so its instruction count per MMA matters (the MMAs are short: 32-64
+      // tensor-core cycles): descriptors are built once and advanced by adding constants to their low word,
+      // the block loops are unrolled, and ring positions are kept as counters instead of being divided out.
       bool ok = true;
-      const uint32_t k_base = smem_u32(base + pl.k_off), v_base = smem_u32(base + pl.v_off);
-      const uint32_t q_base = smem_u32(base + pl.q_off);
-      // S(g) = Q K^T for local tile g: columns 0 .. n-1 of the score block
-      auto issue_scores = [&](int g) {
-        const int k = g / p.nq, t = g - k * p.nq, st = k % p.kv_stages, qs = g % p.q_stages;
-        if (t == 0 && !mbar_wait_bounded(&kv_full[st], (unsigned)(k / p.kv_stages) & 1u, WAIT_NS)) { ok = false; return; }
-        if (!mbar_wait_bounded(&q_full[qs], (unsigned)(g / p.q_stages) & 1u, WAIT_NS)) { ok = false; return; }
+      const uint32_t kslab16 = kv_slab >> 4;                           // descriptor units (16 bytes)
+      const uint64_t dq0 = smem_desc(smem_u32(base + pl.q_off), 16u, 1024u);
+      const uint64_t dk0 = smem_desc(smem_u32(base + pl.k_off), 16u, 1024u);
+      const uint64_t dv0 = smem_desc(smem_u32(base + pl.v_off), kv_slab, 1024u);
+      const uint32_t dq_hi = (uint32_t)(dq0 >> 32), dk_hi = (uint32_t)(dk0 >> 32), dv_hi = (uint32_t)(dv0 >> 32);
+      const uint32_t dq_lo = (uint32_t)dq0, dk_lo = (uint32_t)dk0, dv_lo = (uint32_t)dv0;
+      const int kv_mask = p.kv_stages - 1, kv_shift = p.kv_stages - 1;  // stages are 1 or 2
+      const int q_mask = p.q_stages - 1, q_shift = p.q_stages - 1;
+      const int nb_tail = p.n_total - (p.nq - 1) * BN;                  // keys in an item's last block (multiple of 16)
+      const uint32_t idesc_s_full = idesc_bf16(BN, 0), idesc_s_tail = idesc_bf16(nb_tail, 0);
+      const uint32_t idesc_pv = idesc_bf16(DH, 1);
+      auto desc = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; };
+      // S_j = Q K_j^T for the block `it` points at, into score buffer `buf`
+      auto issue_scores = [&](const BlockIter& it, int buf) {
+        const int st = it.k & kv_mask, qs = it.tile & q_mask;
+        if (it.t == 0 && it.j == 0 && !mbar_wait_bounded(&kv_full[st], (unsigned)(it.k >> kv_shift) & 1u, WAIT_NS)) {
+          fa_timeout(SITE_KV_FULL); ok = false; return;
+        }
+        if (it.j == 0 && !mbar_wait_bounded(&q_full[qs], (unsigned)(it.tile >> q_shift) & 1u, WAIT_NS)) {
+          fa_timeout(SITE_Q_FULL); ok = false; return;
+        }
         tc_fence_after();
-        const int n = min(p.n_total, (t + 1) * BM);
-        const uint32_t qa = q_base + qs * Q_BYTES, ka = k_base + st * kv_bytes;
-        for (int c0 = 0; c0 < n; c0 += 128) {
-          const int nn = min(128, n - c0);
-          const uint32_t idesc = idesc_bf16(nn, 0);
+        const uint32_t qa = dq_lo + (uint32_t)qs * (Q_BYTES >> 4);
+        const uint32_t ka = dk_lo + (uint32_t)st * (kv_bytes >> 4) + (uint32_t)it.j * (BN * 128 >> 4);
+        const uint32_t idesc = (it.j == p.nq - 1) ? idesc_s_tail : idesc_s_full;
+        const uint32_t d_col = tmem_base + (uint32_t)(buf * BN);
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks) {
-            const uint64_t da = smem_desc(qa + (ks >> 2) * Q_SLAB + (ks & 3) * 32, 16u, 1024u);
-            const uint64_t db = smem_desc(ka + (ks >> 2) * kv_slab + c0 * 128 + (ks & 3) * 32, 16u, 1024u);
-            umma_bf16(tmem_base + (uint32_t)c0, da, db, idesc, ks > 0 ? 1u : 0u);
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const uint32_t qo = (uint32_t)((ks >> 2) * (Q_SLAB >> 4) + (ks & 3) * 2);
+          const uint32_t ko = (uint32_t)(ks >> 2) * kslab16 + (uint32_t)((ks & 3) * 2);
+          if (ks == 0) umma_bf16(d_col, desc(qa + qo, dq_hi), desc(ka + ko, dk_hi), idesc, 0u);
+          else umma_bf16(d_col, desc(qa + qo, dq_hi), desc(ka + ko, dk_hi), idesc, 1u);
+        }
+        umma_commit(&s_full[buf]);
+        if (it.j == it.t) umma_commit(&q_empty[qs]);    // the tile's last block: its queries may be replaced
+      };
+      BlockIter ahead, cur;
+      ahead.init(p.nq); cur.init(p.nq);
+      int b_ahead = 0, released = 0;             // released = tiles whose slots the output warps have handed back
+      int hist[NSLOT];                           // tile of the last NSLOT blocks, oldest first: hist[0] used this block's slot
+#pragma unroll
+      for (int i = 0; i < NSLOT; ++i) hist[i] = -1;
+      for (; b_ahead < NBUF && b_ahead < n_blocks && ok; ++b_ahead) { issue_scores(ahead, b_ahead); ahead.next(); }
+      int buf = 0, slot = 0, buf_phase = 0;
+      for (int b = 0; b < n_blocks && ok; ++b) {
+        const int st = cur.k & kv_mask;
+        if (*abort_flag) { ok = false; break; }
+        if (!mbar_wait_bounded(&p_full[buf], (unsigned)buf_phase, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
+        // the accumulator slot must have been read by the output warps of the tile that used it last.  Releases are
+        // consumed in tile order and at least up to tile - 2: with the tiles alternating between two barriers, the
+        // phase waited for is then never a whole lap behind its barrier
+        const int need = max(hist[0], cur.tile - 2);
+        while (released <= need && ok) {
+          if (!mbar_wait_bounded(&o_empty[released & 1], (unsigned)(released >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_O_EMPTY); ok = false; }
+          ++released;
+        }
+        if (!ok) break;
+#pragma unroll
+        for (int i = 0; i + 1 < NSLOT; ++i) hist[i] = hist[i + 1];
+        hist[NSLOT - 1] = cur.tile;
+        tc_fence_after();
+        // O_j = P_j V_j: P from the score buffer in two segments (one per softmax warp of a quadrant)
+        const uint32_t va = dv_lo + (uint32_t)st * (kv_bytes >> 4) + (uint32_t)cur.j * (BN * 128 >> 4);
+        const uint32_t d_col = tmem_base + (uint32_t)(O_COL + slot * DH);
+        const uint32_t a_base = tmem_base + (uint32_t)(buf * BN);
+        if (cur.j < p.nq - 1 || nb_tail == BN) {
+          // full block: keys 0..63 packed in columns 0..31, keys 64..127 in columns 64..95
+#pragma unroll
+          for (int i = 0; i < BN / 16; ++i) {
+            const uint32_t a_col = a_base + (uint32_t)(i < 4 ? i * 8 : 64 + (i - 4) * 8);
+            if (i == 0) umma_bf16_ts(d_col, a_col, desc(va + (uint32_t)(i * 128), dv_hi), idesc_pv, 0u);
+            else umma_bf16_ts(d_col, a_col, desc(va + (uint32_t)(i * 128), dv_hi), idesc_pv, 1u);
+          }
+        } else {
+          const int nsl = (nb_tail + 31) >> 5, seg_a = ((nsl + 1) >> 1) * 32;
+          for (int kv0 = 0; kv0 < nb_tail; kv0 += 16) {
+            const uint32_t a_col = a_base + (kv0 < seg_a ? (uint32_t)(kv0 >> 1) : (uint32_t)(seg_a + ((kv0 - seg_a) >> 1)));
+            umma_bf16_ts(d_col, a_col, desc(va + (uint32_t)(kv0 * 8), dv_hi), idesc_pv, kv0 > 0 ? 1u : 0u);
           }
         }
-        umma_commit(s_full);
-        umma_commit(&q_empty[qs]);             // the query tile may be replaced once these MMAs have read it
-      };
-      if (n_tiles > 0) issue_scores(0);
-      for (int g = 0; g < n_tiles && ok; ++g) {
-        const int k = g / p.nq, t = g - k * p.nq, st = k % p.kv_stages;
-        if (*abort_flag || !mbar_wait_bounded(p_full, (unsigned)g & 1u, WAIT_NS)) { ok = false; break; }
-        tc_fence_after();
-        // O = P V: P from tensor memory in two segments (one per softmax warp of a quadrant), V MN-major from shared memory
-        const int n = min(p.n_total, (t + 1) * BM);
-        const int nsl = (n + 31) >> 5, seg_a = ((nsl + 1) >> 1) * 32;
-        const uint32_t idesc = idesc_bf16(DH, 1);
-        const uint32_t va = v_base + st * kv_bytes;
-        for (int kv0 = 0; kv0 < n; kv0 += 16) {
-          const uint32_t a_col = kv0 < seg_a ? (uint32_t)(kv0 >> 1) : (uint32_t)(seg_a + ((kv0 - seg_a) >> 1));
-          const uint64_t db = smem_desc(va + kv0 * 128, kv_slab, 1024u);
-          umma_bf16_ts(tmem_base + O_COL, tmem_base + a_col, db, idesc, kv0 > 0 ? 1u : 0u);
+        if (cur.j == cur.t) {
+          umma_commit(&o_full[cur.tile & 1]);
+          if (cur.t == p.nq - 1) umma_commit(&kv_empty[st]);          // last use of this item's K and V
         }
-        umma_commit(o_full);
-        if (t == p.nq - 1) umma_commit(&kv_empty[st]);   // last use of this item's K and V
-        if (g + 1 < n_tiles) issue_scores(g + 1);
+        cur.next();
+        // the buffer's next scores: issued after the MMAs above, which read P from it
+        if (b_ahead < n_blocks) { issue_scores(ahead, buf); ahead.next(); ++b_ahead; }
+        if (++buf == NBUF) { buf = 0; buf_phase ^= 1; }
+        if (++slot == NSLOT) slot = 0;
       }
-      if (!ok) { *abort_flag = 1; atomicOr(&g_fa_status, 1u); }
+      if (!ok) *abort_flag = 1;
     }
-  } else {
-    // ------------------------------ softmax + output: warps 2..9 ------------------------------
-    const int quad = warp & 3, half = (warp - 2) >> 2;
-    const int row = quad * 32 + lane;
+  } else if (warp < 6) {
+    // ------------------------------ output: warps 2..5 ------------------------------
+    // Combines the tile's accumulator slots, stages the bf16 result in shared memory in the 128-byte-swizzled
+    // layout of the output tensor map (64 columns at a time) and lets one TMA store write it: rows past the end
+    // of the sequence are clipped by the tensor map.
+    const int quad = warp & 3, row = quad * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const float c2 = p.scale_log2;
+    uint8_t* stage_row = base + pl.ostage_off + row * 128;
+    const bool storer = warp == 2 && lane == 0;
     bool dead = false;
+    int b0 = 0;                                // index of the tile's first block among this CTA's blocks
     for (int g = 0; g < n_tiles; ++g) {
-      named_bar_sync(1, SM_WARPS * 32);
-      if (*abort_flag) break;                  // read after the barrier: the same answer in all softmax warps
+      named_bar_sync(OUT_BAR, 128);
+      if (*abort_flag) break;                  // read after the barrier: the same answer in all four warps
       const int k = g / p.nq, t = g - k * p.nq;
       const int item = blockIdx.x + k * gridDim.x, seq = item / p.H, h = item - seq * p.H;
-      const int n = min(p.n_total, (t + 1) * BM);
-      const int nsl = (n + 31) >> 5, sl_a = (nsl + 1) >> 1;
-      const int sl_lo = half ? sl_a : 0, sl_hi = half ? nsl : sl_a;
-      const int qi = t * BM + row, qc = min(qi, p.S - 1);             // rows past the sequence are computed but not stored
-      const int q_warp_min = min(t * BM + quad * 32, p.S - 1);
-      auto wait_all = [&](uint64_t* bar, unsigned parity) {
+      {
         int ok = 1;
         if (lane == 0) {
-          ok = (!dead && !*abort_flag && mbar_wait_bounded(bar, parity, WAIT_NS * 2ull)) ? 1 : 0;
-          if (!ok) { *abort_flag = 1; atomicOr(&g_fa_status, 1u); }
+          ok = *abort_flag ? 0 : 1;
+          if (ok && !mbar_wait_bounded(&o_full[g & 1], (unsigned)(g >> 1) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_O_FULL); ok = 0; }
+          if (!ok) *abort_flag = 1;
         }
         if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
-      };
-      wait_all(s_full, (unsigned)g & 1u);
+      }
+      tc_fence_after();
+      const int nj = t + 1, ring = g & (STAT_RING - 1);
+      const int qi = t * BM + row;
+      float mj[MAX_SLOTS], w[MAX_SLOTS];
+      float m = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < MAX_SLOTS; ++j) {
+        mj[j] = j < nj ? stat_m[(ring * MAX_SLOTS + j) * BM + row] : -INFINITY;
+        m = fmaxf(m, mj[j]);
+      }
+      float L = 0.f;
+#pragma unroll
+      for (int j = 0; j < MAX_SLOTS; ++j) {
+        w[j] = j < nj ? ex2_approx((mj[j] - m) * c2) : 0.f;
+        if (j < nj) L = fmaf(w[j], stat_l[(ring * MAX_SLOTS + j) * BM + row], L);
+      }
+      const float inv = 1.f / L;
+#pragma unroll
+      for (int j = 0; j < MAX_SLOTS; ++j) w[j] *= inv;
+#pragma unroll 1
+      for (int cb = 0; cb < DH; cb += 64) {
+        if (storer) bulk_wait_read_all();      // the previous store has finished reading the staging buffer
+        named_bar_sync(OUT_BAR, 128);
+#pragma unroll 1
+        for (int cc = 0; cc < 64; cc += 32) {
+          float acc[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+          if (!dead) {
+#pragma unroll
+            for (int j = 0; j < MAX_SLOTS; ++j) {
+              if (j < nj) {
+                int sl = b0 + j;
+                sl -= (sl / NSLOT) * NSLOT;
+                uint32_t r[32];
+                tmem_ld_32x32(lane_addr + (uint32_t)(O_COL + sl * DH + cb + cc), r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) acc[e] = fmaf(w[j], __uint_as_float(r[e]), acc[e]);
+              }
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            uint4 o;
+            o.x = pack_bf16x2(acc[e], acc[e + 1]); o.y = pack_bf16x2(acc[e + 2], acc[e + 3]);
+            o.z = pack_bf16x2(acc[e + 4], acc[e + 5]); o.w = pack_bf16x2(acc[e + 6], acc[e + 7]);
+            const int chunk = (cc + e) >> 3;                            // 16-byte chunk of the 128-byte row
+            *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) = o;
+          }
+        }
+        fence_proxy_async_smem();
+        named_bar_sync(OUT_BAR, 128);
+        if (storer && !dead) {
+          tma_store_3d(&tmO, base + pl.ostage_off, h * DH + cb, t * BM, seq);
+          bulk_commit();
+        }
+      }
+      if (!dead && qi < p.S) p.lse[((long long)seq * p.H + h) * p.S + qi] = (m * c2 + log2f(L)) * LN2;
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0 && !dead) mbar_arrive(&o_empty[g & 1]);
+      b0 += nj;
+    }
+    if (storer) bulk_wait_read_all();
+  } else {
+    // ------------------------------ softmax: 8 warps per score buffer ------------------------------
+    const int sw = warp - 6, buf = sw / SM_WARPS_PER_BUF, wq = sw % SM_WARPS_PER_BUF;
+    const int quad = warp & 3, half = wq >> 2;                        // warps 6..9 -> quadrants 2,3,0,1
+    const int row = quad * 32 + lane;
+    const int pair_bar = 1 + buf * 4 + quad;                          // named barrier of the two warps sharing these rows
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN);
+    float* my_red = red_max + (buf * 2 + half) * BM + row;
+    const float* other_red = red_max + (buf * 2 + (half ^ 1)) * BM + row;
+    const float c2 = p.scale_log2;
+    bool dead = false;
+    BlockIter it;
+    it.init(p.nq);
+    it.advance(buf);
+    for (int b = buf; b < n_blocks; b += NBUF, it.advance(NBUF)) {
+      named_bar_sync(pair_bar, 64);
+      if (*abort_flag) break;                  // read after the barrier: the same answer in both warps of the pair
+      const int nb = min(BN, p.n_total - it.j * BN);
+      const int nsl = (nb + 31) >> 5, sl_a = (nsl + 1) >> 1;
+      const int sl_lo = half ? sl_a : 0, sl_hi = half ? nsl : sl_a;
+      const bool diag = it.j == it.t;
+      // last valid column of this row inside a diagonal block (rows past the sequence are computed, never stored)
+      const int lim = min(it.t * BM + row, p.S - 1) - it.j * BN;
+      const int lim_warp = min(it.t * BM + quad * 32, p.S - 1) - it.j * BN;
+      {
+        int ok = 1;
+        if (lane == 0) {
+          ok = *abort_flag ? 0 : 1;
+          if (ok && !mbar_wait_bounded(&s_full[buf], (unsigned)(b / NBUF) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
+          if (!ok) *abort_flag = 1;
+        }
+        if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
+      }
       tc_fence_after();
       // pass 1: row maximum over this warp's slices of 32 columns
-      float m = -INFINITY;
+      float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
       if (!dead) {
         for (int sl = sl_lo; sl < sl_hi; ++sl) {
           uint32_t r[32];
           tmem_ld_32x32(lane_addr + (uint32_t)(sl * 32), r);
           tmem_ld_wait();
-          if (sl * 32 + 31 <= q_warp_min) {
+          if (!diag || sl * 32 + 31 <= lim_warp) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) m = fmaxf(m, __uint_as_float(r[e]));
+            for (int e = 0; e < 32; e += 4) {
+              m0 = fmaxf(m0, __uint_as_float(r[e])); m1 = fmaxf(m1, __uint_as_float(r[e + 1]));
+              m2 = fmaxf(m2, __uint_as_float(r[e + 2])); m3 = fmaxf(m3, __uint_as_float(r[e + 3]));
+            }
           } else {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) m = (sl * 32 + e <= qc) ? fmaxf(m, __uint_as_float(r[e])) : m;
+            for (int e = 0; e < 32; e += 4) {
+              m0 = (sl * 32 + e <= lim) ? fmaxf(m0, __uint_as_float(r[e])) : m0;
+              m1 = (sl * 32 + e + 1 <= lim) ? fmaxf(m1, __uint_as_float(r[e + 1])) : m1;
+              m2 = (sl * 32 + e + 2 <= lim) ? fmaxf(m2, __uint_as_float(r[e + 2])) : m2;
+              m3 = (sl * 32 + e + 3 <= lim) ? fmaxf(m3, __uint_as_float(r[e + 3])) : m3;
+            }
           }
         }
       }
-      red_max[half * BM + row] = m;
-      named_bar_sync(2, SM_WARPS * 32);
-      m = fmaxf(m, red_max[(half ^ 1) * BM + row]);                    // column 0 is never masked: finite
+      float m = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      *my_red = m;
+      named_bar_sync(pair_bar, 64);
+      m = fmaxf(m, *other_red);                                        // column 0 of a block is never masked: finite
       const float mc = m * c2;
-      // pass 2: P = exp2(s c - m c), packed bf16 written over scores this warp has already consumed
-      float sum = 0.f;
+      // pass 2: P = exp2(s c - m c) as packed bf16 over scores this warp has already consumed
+      float sum0 = 0.f, sum1 = 0.f;
       if (!dead) {
         for (int sl = sl_lo; sl < sl_hi; ++sl) {
           uint32_t r[32], pk[16];
           tmem_ld_32x32(lane_addr + (uint32_t)(sl * 32), r);
           tmem_ld_wait();
-          if (sl * 32 + 31 <= q_warp_min) {
+          if (!diag || sl * 32 + 31 <= lim_warp) {
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
               const float p0 = ex2_approx(fmaf(__uint_as_float(r[e]), c2, -mc));
               const float p1 = ex2_approx(fmaf(__uint_as_float(r[e + 1]), c2, -mc));
-              sum += p0 + p1;
+              sum0 += p0; sum1 += p1;
               pk[e >> 1] = pack_bf16x2(p0, p1);
             }
           } else {
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
-              const float p0 = (sl * 32 + e <= qc) ? ex2_approx(fmaf(__uint_as_float(r[e]), c2, -mc)) : 0.f;
-              const float p1 = (sl * 32 + e + 1 <= qc) ? ex2_approx(fmaf(__uint_as_float(r[e + 1]), c2, -mc)) : 0.f;
-              sum += p0 + p1;
+              const float p0 = (sl * 32 + e <= lim) ? ex2_approx(fmaf(__uint_as_float(r[e]), c2, -mc)) : 0.f;
+              const float p1 = (sl * 32 + e + 1 <= lim) ? ex2_approx(fmaf(__uint_as_float(r[e + 1]), c2, -mc)) : 0.f;
+              sum0 += p0; sum1 += p1;
               pk[e >> 1] = pack_bf16x2(p0, p1);
             }
           }
@@ -323,37 +532,18 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         tmem_st_wait();
       }
-      red_sum[half * BM + row] = sum;
+      // the quadrant's other warp adds its row sums; one of the two publishes the block's statistics
+      red_sum[(buf * 2 + half) * BM + row] = sum0 + sum1;
+      named_bar_sync(pair_bar, 64);
+      if (half == 0) {
+        const int ring = it.tile & (STAT_RING - 1);
+        stat_l[(ring * MAX_SLOTS + it.j) * BM + row] = sum0 + sum1 + red_sum[(buf * 2 + 1) * BM + row];
+        stat_m[(ring * MAX_SLOTS + it.j) * BM + row] = m;
+      }
+      __threadfence_block();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0 && !dead) mbar_arrive(p_full);
-      named_bar_sync(2, SM_WARPS * 32);
-      const float tot = sum + red_sum[(half ^ 1) * BM + row];
-      wait_all(o_full, (unsigned)g & 1u);
-      tc_fence_after();
-      if (!dead) {
-        const float inv = 1.f / tot;
-        __nv_bfloat16* op = p.out + ((long long)seq * p.S + qi) * p.d + h * DH + half * (DH / 2);
-#pragma unroll
-        for (int cc = 0; cc < DH / 2; cc += 32) {
-          uint32_t r[32];
-          tmem_ld_32x32(lane_addr + (uint32_t)(O_COL + half * (DH / 2) + cc), r);
-          tmem_ld_wait();
-          if (qi < p.S) {
-#pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              uint4 o;
-              o.x = pack_bf16x2(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv);
-              o.y = pack_bf16x2(__uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
-              o.z = pack_bf16x2(__uint_as_float(r[e + 4]) * inv, __uint_as_float(r[e + 5]) * inv);
-              o.w = pack_bf16x2(__uint_as_float(r[e + 6]) * inv, __uint_as_float(r[e + 7]) * inv);
-              *reinterpret_cast<uint4*>(op + cc + e) = o;
-            }
-          }
-        }
-        if (half == 0 && qi < p.S) p.lse[((long long)seq * p.H + h) * p.S + qi] = (mc + log2f(tot)) * LN2;
-      }
-      tc_fence_before();                       // the next tile's P V overwrites the accumulator only after these reads
+      if (lane == 0 && !dead) mbar_arrive(&p_full[buf]);
     }
   }
 
@@ -439,13 +629,15 @@ static int fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int S, 
   CUtensorMap tmQ, tmKV;
   if (!make_seq_tmap(&tmQ, qkv, n_seq, S, 3LL * d, 3LL * d, BM) || !make_seq_tmap(&tmKV, qkv, n_seq, S, 3LL * d, 3LL * d, 64))
     return PCM_ERR_CUDA;
+  CUtensorMap tmO;
+  if (!make_seq_tmap(&tmO, out, n_seq, S, d, d, BM)) return PCM_ERR_CUDA;
   static bool attr_done = false;
   if (!attr_done) {
     PCM_CUDA_TRY(cudaFuncSetAttribute(fa_tc_fwd_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT));
     attr_done = true;
   }
   const int grid = p.n_items < attn_sm_count() ? p.n_items : attn_sm_count();
-  fa_tc_fwd_kernel<DH><<<grid, THREADS, smem, s>>>(tmQ, tmKV, p);
+  fa_tc_fwd_kernel<DH><<<grid, Cfg<DH>::THREADS, smem, s>>>(tmQ, tmKV, tmO, p);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
 }
@@ -454,7 +646,7 @@ static int fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int S, 
 
 bool attention_tc_supported(const void* qkv, const void* out, int S, int H, int dh) {
   if (dh != 64 && dh != 128) return false;
-  if (S < 1 || S > fatc::S_COLS) return false;
+  if (S < 1 || S > fatc::S_MAX) return false;
   if ((((uintptr_t)qkv) | ((uintptr_t)out)) & 15) return false;
   (void)H;
   return fatc::attn_encode_fn() != nullptr;
@@ -466,6 +658,10 @@ int attention_fwd_bf16_tc(const void* qkv, void* out, float* lse, int n_seq, int
   return dh == 64 ? fatc::fwd_launch<64>(qkv, out, lse, n_seq, S, H, s) : fatc::fwd_launch<128>(qkv, out, lse, n_seq, S, H, s);
 }
 
+static unsigned g_fa_last_status = 0;
+// The raw status word of the last expired wait (bit 8 + site says which barrier): for diagnostics.
+unsigned attention_tc_last_status() { return g_fa_last_status; }
+
 // Reads and clears this file's device status word (synchronous copy).
 int attention_tc_poll_status() {
   unsigned h = 0;
@@ -473,6 +669,7 @@ int attention_tc_poll_status() {
   if (h) {
     unsigned z = 0;
     cudaMemcpyToSymbol(g_fa_status, &z, sizeof(z));
+    g_fa_last_status = h;
     return PCM_ERR_DEVICE_TIMEOUT;
   }
   return PCM_OK;
