@@ -40,7 +40,7 @@ constexpr int TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float LN2 = 0.6931471805599453f;
 constexpr int OUT_BAR = 9;                     // named barrier of the four output warps (1..8: softmax warp pairs)
-constexpr int STAT_RING = 4;                   // tiles whose row statistics may be live at once
+constexpr int STAT_RING = 3;                   // tiles whose row statistics may be live at once
 
 template <int DH> struct Cfg {
   static constexpr int NBUF = DH == 64 ? 2 : 1;                       // score buffers that fit beside the output slots
@@ -157,8 +157,8 @@ __host__ __device__ inline Plan make_plan(int dh, int kv_rows, int kv_stages, in
   p.bar_off = p.ostage_off + BM * 128;
   p.stat_m_off = p.bar_off + 256;
   p.stat_l_off = p.stat_m_off + STAT_RING * MAX_SLOTS * BM * 4;
-  p.red_off = p.stat_l_off + STAT_RING * MAX_SLOTS * BM * 4;
-  p.total = p.red_off + 2 * 2 * 2 * BM * 4 + 1024 /* alignment slack */;
+  p.red_off = p.stat_l_off + STAT_RING * MAX_SLOTS * 2 * BM * 4;
+  p.total = p.red_off + 2 * 2 * BM * 4 + 1024 /* alignment slack */;
   return p;
 }
 
@@ -189,9 +189,8 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   float* stat_m = reinterpret_cast<float*>(base + pl.stat_m_off);   // [STAT_RING][MAX_SLOTS][128]
-  float* stat_l = reinterpret_cast<float*>(base + pl.stat_l_off);   // [STAT_RING][MAX_SLOTS][128]
+  float* stat_l = reinterpret_cast<float*>(base + pl.stat_l_off);   // [STAT_RING][MAX_SLOTS][2][128]: one partial sum per softmax warp of a quadrant
   float* red_max = reinterpret_cast<float*>(base + pl.red_off);     // [2][2][128]
-  float* red_sum = red_max + 2 * 2 * BM;                            // [2][2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_local = ((int)blockIdx.x < p.n_items) ? (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
@@ -269,6 +268,7 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint32_t idesc_s_full = idesc_bf16(BN, 0), idesc_s_tail = idesc_bf16(nb_tail, 0);
       const uint32_t idesc_pv = idesc_bf16(DH, 1);
       auto desc = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; };
+      int released = 0;                          // tiles whose slots and statistics the output warps have handed back
       // S_j = Q K_j^T for the block `it` points at, into score buffer `buf`
       auto issue_scores = [&](const BlockIter& it, int buf) {
         const int st = it.k & kv_mask, qs = it.tile & q_mask;
@@ -278,6 +278,12 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (it.j == 0 && !mbar_wait_bounded(&q_full[qs], (unsigned)(it.tile >> q_shift) & 1u, WAIT_NS)) {
           fa_timeout(SITE_Q_FULL); ok = false; return;
         }
+        // the statistics ring holds STAT_RING tiles: this tile's softmax overwrites those of tile - STAT_RING
+        while (it.j == 0 && released <= it.tile - STAT_RING && ok) {
+          if (!mbar_wait_bounded(&o_empty[released & 1], (unsigned)(released >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_O_EMPTY); ok = false; }
+          ++released;
+        }
+        if (!ok) return;
         tc_fence_after();
         const uint32_t qa = dq_lo + (uint32_t)qs * (Q_BYTES >> 4);
         const uint32_t ka = dk_lo + (uint32_t)st * (kv_bytes >> 4) + (uint32_t)it.j * (BN * 128 >> 4);
@@ -295,7 +301,7 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       };
       BlockIter ahead, cur;
       ahead.init(p.nq); cur.init(p.nq);
-      int b_ahead = 0, released = 0;             // released = tiles whose slots the output warps have handed back
+      int b_ahead = 0;
       int hist[NSLOT];                           // tile of the last NSLOT blocks, oldest first: hist[0] used this block's slot
 #pragma unroll
       for (int i = 0; i < NSLOT; ++i) hist[i] = -1;
@@ -376,7 +382,7 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
       }
       tc_fence_after();
-      const int nj = t + 1, ring = g & (STAT_RING - 1);
+      const int nj = t + 1, ring = g % STAT_RING;
       const int qi = t * BM + row;
       float mj[MAX_SLOTS], w[MAX_SLOTS];
       float m = -INFINITY;
@@ -389,7 +395,10 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
       for (int j = 0; j < MAX_SLOTS; ++j) {
         w[j] = j < nj ? ex2_approx((mj[j] - m) * c2) : 0.f;
-        if (j < nj) L = fmaf(w[j], stat_l[(ring * MAX_SLOTS + j) * BM + row], L);
+        if (j < nj) {
+          const float* lp = stat_l + ((ring * MAX_SLOTS + j) * 2) * BM + row;
+          L = fmaf(w[j], lp[0] + lp[BM], L);
+        }
       }
       const float inv = 1.f / L;
 #pragma unroll
@@ -532,13 +541,10 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         tmem_st_wait();
       }
-      // the quadrant's other warp adds its row sums; one of the two publishes the block's statistics
-      red_sum[(buf * 2 + half) * BM + row] = sum0 + sum1;
-      named_bar_sync(pair_bar, 64);
-      if (half == 0) {
-        const int ring = it.tile & (STAT_RING - 1);
-        stat_l[(ring * MAX_SLOTS + it.j) * BM + row] = sum0 + sum1 + red_sum[(buf * 2 + 1) * BM + row];
-        stat_m[(ring * MAX_SLOTS + it.j) * BM + row] = m;
+      {
+        const int ring = it.tile % STAT_RING;
+        stat_l[((ring * MAX_SLOTS + it.j) * 2 + half) * BM + row] = sum0 + sum1;
+        if (half == 0) stat_m[(ring * MAX_SLOTS + it.j) * BM + row] = m;
       }
       __threadfence_block();
       tc_fence_before();
