@@ -565,6 +565,538 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// backward
+// ------------------------------------------------------------------------------------------------
+// Two launches of one kernel template, both built like the forward pass (TMA producer, one MMA thread,
+// compute warps on tensor memory, output warps with a TMA store), both recomputing the probabilities
+// from the saved log-sum-exp:
+//   BW_DQ   item = (sequence, head, query tile i): the tile's Q_i and dO_i stay in shared memory, the key
+//           blocks j <= i stream by.  Per block: S = Q_i K_j^T and dP = dO_i V_j^T into tensor memory;
+//           the compute warps form dS = P o (dP - rowsum(dO o O)) with P = exp(S / sqrt(dh) - lse) and write
+//           it as packed bf16 over the scores; dQ_i += dS K_j with dS as the tensor-memory A operand.
+//           This launch also writes rowsum(dO o O) for the second one.
+//   BW_DKV  item = (sequence, head, key block j): K_j and V_j stay, the query tiles i >= j stream by.
+//           Per block: S^T = K_j Q_i^T and dP^T = V_j dO_i^T (rows = keys); P^T is written over S^T and
+//           dS^T over dP^T; dV_j += P^T dO_i and dK_j += dS^T Q_i.
+// The streamed tile is the B operand twice: K-major for the first two products, MN-major (same bytes,
+// another descriptor) for the accumulating ones.  Scores are double-buffered for head dim 64, so the
+// tensor core forms the next block's scores while the compute warps work.  The output warps scale by
+// 1 / sqrt(dh), rotate dQ and dK back through the rotary embedding when a table is given, and store.
+enum { BW_DQ = 0, BW_DKV = 1 };
+constexpr int BW_COMPUTE_WARPS = 16;            // four per tensor-memory lane quadrant: one 32-column slice each
+constexpr int BW_THREADS = (2 + 4 + BW_COMPUTE_WARPS) * 32;
+constexpr int BW_COMPUTE_BAR = 10;              // named barrier of the compute warps
+constexpr int BW_OUT_BAR = 11;                  // named barrier of the output warps
+
+template <int DH> struct BwCfg {
+  static constexpr int NSBUF = DH == 64 ? 2 : 1;                      // score buffers
+  static constexpr int DP_COL = NSBUF * BN;                           // dP buffer
+  static constexpr int ACC_COL = DP_COL + BN;                         // two accumulators of DH columns
+  static constexpr int FIX_STAGES = DH == 64 ? 2 : 1;                 // resident operand pairs (this item's and the next)
+  static constexpr int STR_STAGES = NSBUF + 1;                        // streamed operand pairs in flight
+  static constexpr uint32_t TILE_BYTES = (DH / 64) * BM * 128u;       // one 128-row operand tile: DH/64 slabs of 16 KB
+  static_assert(ACC_COL + 2 * DH <= TMEM_COLS, "tensor memory plan does not fit");
+};
+
+struct BwParams {
+  int n_seq, S, H, d;
+  int n_items;                                  // n_seq * H * nq
+  int nq;                                       // 128-row tiles per sequence
+  int n_total;                                  // S rounded up to 16
+  float scale, scale_log2;                      // 1 / sqrt(dh), log2(e) / sqrt(dh)
+  const float* lse;                             // [n_seq][H][S]
+  float* dsum;                                  // [n_seq][H][S]: written by BW_DQ, read by BW_DKV
+  const __nv_bfloat16* out;                     // [n_seq*S][d]
+  const __nv_bfloat16* dout;                    // [n_seq*S][d]
+  const float2* rope_tab;                       // [S][dh/2] (cos, sin) or nullptr
+};
+
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+
+// Walks this CTA's items and their blocks in issue order.  Item = ((sequence * H + head) * nq + tile); a BW_DQ
+// item streams the key blocks 0 .. tile, a BW_DKV item the query tiles tile .. nq - 1.
+struct BwIter {
+  int nq, mode, grid, n_items;
+  int k, item, tt, u, cnt, b;                   // k = local item count, b = local block count
+  __device__ void setup() {
+    if (item < n_items) {
+      tt = item % nq;
+      cnt = mode == BW_DQ ? tt + 1 : nq - tt;
+      u = 0;
+    }
+  }
+  __device__ void init(int nq_, int mode_, int n_items_) {
+    nq = nq_; mode = mode_; n_items = n_items_; grid = gridDim.x;
+    k = 0; b = 0; item = blockIdx.x;
+    setup();
+  }
+  __device__ bool valid() const { return item < n_items; }
+  __device__ bool first() const { return u == 0; }
+  __device__ bool last() const { return u == cnt - 1; }
+  __device__ int stile() const { return mode == BW_DQ ? u : tt + u; }   // index of the streamed tile in its sequence
+  __device__ bool diag() const { return stile() == tt; }
+  __device__ void next() {
+    ++b;
+    if (++u == cnt) { ++k; item += grid; setup(); }
+  }
+};
+
+// Shared-memory plan of the backward kernel (bytes, after 1024-byte alignment): resident pairs, streamed
+// pairs, output staging, barriers, per-column or per-row statistics.
+struct BwPlan {
+  uint32_t fix_off, str_off, ostage_off, bar_off, stat_off, total;
+};
+template <int DH>
+__host__ __device__ inline BwPlan bw_make_plan() {
+  BwPlan p;
+  p.fix_off = 0;
+  p.str_off = p.fix_off + BwCfg<DH>::FIX_STAGES * 2 * BwCfg<DH>::TILE_BYTES;
+  p.ostage_off = p.str_off + BwCfg<DH>::STR_STAGES * 2 * BwCfg<DH>::TILE_BYTES;
+  p.bar_off = p.ostage_off + BM * 128;
+  p.stat_off = p.bar_off + 256;
+  p.total = p.stat_off + 2 * 2 * BM * 4 + 1024 /* alignment slack */;
+  return p;
+}
+
+template <int DH, int MODE>
+__global__ void __launch_bounds__(BW_THREADS, 1)
+fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constant__ CUtensorMap tmDO,
+                 const __grid_constant__ CUtensorMap tmDQKV, const BwParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  using C = BwCfg<DH>;
+  constexpr int NSLAB = DH / 64;
+  constexpr int NSBUF = C::NSBUF;
+  constexpr uint32_t TILE = C::TILE_BYTES, PAIR = 2 * TILE;
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  uint8_t* base = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
+  const BwPlan pl = bw_make_plan<DH>();
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + pl.bar_off);
+  uint64_t* fix_full = bars;                   // [2] producer -> MMA: an item's resident pair has landed
+  uint64_t* fix_empty = bars + 2;              // [2] MMA -> producer
+  uint64_t* str_full = bars + 4;               // [3] producer -> MMA: a block's streamed pair has landed
+  uint64_t* str_empty = bars + 7;              // [3] MMA -> producer
+  uint64_t* sdp_full = bars + 10;              // MMA -> compute: S and dP of a block are in tensor memory
+  uint64_t* p_ready = bars + 11;               // compute -> MMA: P / dS of the block are in tensor memory (16 warp arrivals)
+  uint64_t* acc_full = bars + 12;              // [2] MMA -> output warps: the item's accumulators are complete
+  uint64_t* acc_empty = bars + 14;             // [2] output warps -> MMA (4 warp arrivals); items alternate between the two
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* stat = reinterpret_cast<float*>(base + pl.stat_off);        // BW_DKV: [2][2][128] column statistics; BW_DQ: [4][128] partial row sums
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nb_tail = p.n_total - (p.nq - 1) * BN;                  // rows of a sequence's last tile that take part (multiple of 16)
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&fix_full[s], 1); mbar_init(&fix_empty[s], 1);
+      mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4);
+    }
+    for (int s = 0; s < 3; ++s) { mbar_init(&str_full[s], 1); mbar_init(&str_empty[s], 1); }
+    mbar_init(sdp_full, 1); mbar_init(p_ready, BW_COMPUTE_WARPS);
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmQKV);
+    prefetch_tmap(&tmDO);
+    prefetch_tmap(&tmDQKV);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------ TMA producer ------------------------------
+      // BW_DQ: resident = (Q_i, dO_i), streamed = (K_j, V_j).  BW_DKV: resident = (K_j, V_j), streamed = (Q_i, dO_i).
+      bool ok = true;
+      BwIter it;
+      it.init(p.nq, MODE, p.n_items);
+      int fs = 0, fph = 0, ss = 0, sph = 0;
+      auto load_pair = [&](uint8_t* dst, bool qdo, int h, int tile, int seq, uint64_t* bar) {
+        for (int sl = 0; sl < NSLAB; ++sl) {
+          if (qdo) {
+            tma_load_3d(dst + sl * 16384, &tmQKV, h * DH + sl * 64, tile * BM, seq, bar);
+            tma_load_3d(dst + TILE + sl * 16384, &tmDO, h * DH + sl * 64, tile * BM, seq, bar);
+          } else {
+            tma_load_3d(dst + sl * 16384, &tmQKV, p.d + h * DH + sl * 64, tile * BM, seq, bar);
+            tma_load_3d(dst + TILE + sl * 16384, &tmQKV, 2 * p.d + h * DH + sl * 64, tile * BM, seq, bar);
+          }
+        }
+      };
+      while (it.valid() && ok && !*abort_flag) {
+        const int sh = it.item / p.nq, h = sh % p.H, seq = sh / p.H;
+        if (it.first()) {
+          if (!mbar_wait_bounded(&fix_empty[fs], (unsigned)fph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; break; }
+          mbar_expect_tx(&fix_full[fs], PAIR);
+          load_pair(base + pl.fix_off + fs * PAIR, MODE == BW_DQ, h, it.tt, seq, &fix_full[fs]);
+          if (++fs == C::FIX_STAGES) { fs = 0; fph ^= 1; }
+        }
+        if (!mbar_wait_bounded(&str_empty[ss], (unsigned)sph ^ 1u, WAIT_NS)) { fa_timeout(SITE_Q_EMPTY); ok = false; break; }
+        mbar_expect_tx(&str_full[ss], PAIR);
+        load_pair(base + pl.str_off + ss * PAIR, MODE == BW_DKV, h, it.stile(), seq, &str_full[ss]);
+        if (++ss == C::STR_STAGES) { ss = 0; sph ^= 1; }
+        it.next();
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------ MMA issuer ------------------------------
+      bool ok = true;
+      auto desc = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; };
+      const uint64_t dfk = smem_desc(smem_u32(base + pl.fix_off), 16u, 1024u);        // resident tiles: K-major A operands
+      const uint64_t dsk = smem_desc(smem_u32(base + pl.str_off), 16u, 1024u);        // streamed tiles, K-major B
+      const uint64_t dsm = smem_desc(smem_u32(base + pl.str_off), 16384u, 1024u);     // streamed tiles, MN-major B
+      const uint32_t dfk_lo = (uint32_t)dfk, dfk_hi = (uint32_t)(dfk >> 32);
+      const uint32_t dsk_lo = (uint32_t)dsk, dsk_hi = (uint32_t)(dsk >> 32);
+      const uint32_t dsm_lo = (uint32_t)dsm, dsm_hi = (uint32_t)(dsm >> 32);
+      const uint32_t idesc_full = idesc_bf16(BN, 0), idesc_tail = idesc_bf16(nb_tail, 0), idesc_acc = idesc_bf16(DH, 1);
+      // ring positions of the three issue streams: scores (furthest ahead), dP, accumulation
+      struct Pos { BwIter it; int fs, ss, sph, fph; };
+      auto pos_init = [&](Pos& q) { q.it.init(p.nq, MODE, p.n_items); q.fs = q.ss = q.sph = q.fph = 0; };
+      auto pos_next = [&](Pos& q) {
+        const bool item_end = q.it.last();
+        q.it.next();
+        if (++q.ss == C::STR_STAGES) { q.ss = 0; q.sph ^= 1; }
+        if (item_end && ++q.fs == C::FIX_STAGES) { q.fs = 0; q.fph ^= 1; }
+      };
+      Pos ps, pd, pc;                           // scores / dP / current (accumulating) block
+      pos_init(ps); pos_init(pd); pos_init(pc);
+      // first product of a block: scores into buffer sb.  Waits for the block's operands (first use of both).
+      auto issue_scores = [&](Pos& q, int sb) {
+        if (q.it.first() && !mbar_wait_bounded(&fix_full[q.fs], (unsigned)q.fph, WAIT_NS)) { fa_timeout(SITE_KV_FULL); ok = false; return; }
+        if (!mbar_wait_bounded(&str_full[q.ss], (unsigned)q.sph, WAIT_NS)) { fa_timeout(SITE_Q_FULL); ok = false; return; }
+        tc_fence_after();
+        const uint32_t a = dfk_lo + (uint32_t)q.fs * (PAIR >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4);
+        const uint32_t idesc = (q.it.stile() == p.nq - 1) ? idesc_tail : idesc_full;
+        const uint32_t d_col = tmem_base + (uint32_t)(sb * BN);
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const uint32_t o = (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
+          if (ks == 0) umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 0u);
+          else umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 1u);
+        }
+      };
+      // second product of a block: dP from the second tiles of both pairs; then both are announced
+      auto issue_dp = [&](Pos& q) {
+        const uint32_t a = dfk_lo + (uint32_t)q.fs * (PAIR >> 4) + (TILE >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4) + (TILE >> 4);
+        const uint32_t idesc = (q.it.stile() == p.nq - 1) ? idesc_tail : idesc_full;
+        const uint32_t d_col = tmem_base + (uint32_t)C::DP_COL;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const uint32_t o = (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
+          if (ks == 0) umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 0u);
+          else umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 1u);
+        }
+        umma_commit(sdp_full);
+      };
+      // accumulating product: D (+)= A[tensor memory, packed bf16 at a_col0] * streamed tile `which` read MN-major
+      auto issue_acc = [&](const Pos& q, uint32_t d_col, uint32_t a_col0, int which, bool fresh) {
+        const uint32_t bq = dsm_lo + (uint32_t)q.ss * (PAIR >> 4) + (uint32_t)which * (TILE >> 4);
+        const int nk = (q.it.stile() == p.nq - 1 ? nb_tail : BN) >> 4;          // 16-row steps of the streamed tile
+#pragma unroll
+        for (int kk = 0; kk < BN / 16; ++kk) {
+          if (kk < nk) {
+            const uint32_t a_col = a_col0 + (uint32_t)((kk >> 1) * 32 + (kk & 1) * 8);   // slice kk/2, half kk%2
+            umma_bf16_ts(d_col, a_col, desc(bq + (uint32_t)(kk * 128), dsm_hi), idesc_acc, (kk > 0 || !fresh) ? 1u : 0u);
+          }
+        }
+      };
+      // prologue: scores and dP of block 0, scores of block 1 when there is a second score buffer
+      if (ps.it.valid()) {
+        issue_scores(ps, 0);
+        if (ok) { issue_dp(pd); pos_next(ps); pos_next(pd); }
+        if (NSBUF == 2 && ok && ps.it.valid()) { issue_scores(ps, 1); if (ok) pos_next(ps); }
+      }
+      int sb = 0, rph = 0;                      // score buffer and p_ready parity of the current block
+      while (pc.it.valid() && ok) {
+        if (*abort_flag) { ok = false; break; }
+        if (!mbar_wait_bounded(p_ready, (unsigned)rph, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
+        const int k = pc.it.k;
+        if (pc.it.first()) {
+          // BW_DQ alternates between two accumulators: the one of item k was last read for item k - 2;
+          // BW_DKV uses both accumulators for every item: wait for item k - 1
+          const int prev = MODE == BW_DQ ? k - 2 : k - 1;
+          if (prev >= 0 && !mbar_wait_bounded(&acc_empty[prev & 1], (unsigned)(prev >> 1) & 1u, WAIT_NS)) {
+            fa_timeout(SITE_O_EMPTY); ok = false; break;
+          }
+        }
+        tc_fence_after();
+        const uint32_t s_col = tmem_base + (uint32_t)(sb * BN), dp_col = tmem_base + (uint32_t)C::DP_COL;
+        const uint32_t acc0 = tmem_base + (uint32_t)C::ACC_COL, acc1 = acc0 + DH;
+        const bool fresh = pc.it.first();
+        if (MODE == BW_DKV) {
+          issue_acc(pc, acc0, dp_col, 0, fresh);                       // dK += dS^T Q_i (dS^T sits in the dP buffer)
+          if (NSBUF == 2) {
+            if (pd.it.valid()) { issue_dp(pd); pos_next(pd); }         // the dP buffer is free again: next block's dP
+            issue_acc(pc, acc1, s_col, 1, fresh);                      // dV += P^T dO_i
+          } else {
+            issue_acc(pc, acc1, s_col, 1, fresh);
+          }
+        } else {
+          if (NSBUF == 2 && pd.it.valid()) { issue_dp(pd); pos_next(pd); }   // dS went over the scores: dP is free
+          issue_acc(pc, (k & 1) ? acc1 : acc0, s_col, 0, fresh);       // dQ += dS K_j
+        }
+        umma_commit(&str_empty[pc.ss]);                                // the streamed pair has been read for the last time
+        if (pc.it.last()) {
+          umma_commit(&acc_full[k & 1]);
+          umma_commit(&fix_empty[pc.fs]);
+        }
+        pos_next(pc);
+        // this block's score buffer is free once the accumulation above has read it: scores of the block after next
+        // (or, with one buffer, scores and dP of the next block)
+        if (ps.it.valid()) { issue_scores(ps, sb); if (ok) pos_next(ps); }
+        if (NSBUF == 1 && ok && pd.it.valid()) { issue_dp(pd); pos_next(pd); }
+        if (++sb == NSBUF) sb = 0;
+        rph ^= 1;
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp < 6) {
+    // ------------------------------ output: warps 2..5 ------------------------------
+    // Scale by 1 / sqrt(dh) (dQ, dK), rotate back through the rotary embedding, stage 64 columns at a time in
+    // the swizzled layout of the gradient tensor map, TMA store (rows past the sequence are clipped).
+    const int quad = warp & 3, row = quad * 32 + lane;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    uint8_t* stage_row = base + pl.ostage_off + row * 128;
+    const bool storer = warp == 2 && lane == 0;
+    constexpr int HALF = DH / 2;
+    bool dead = false;
+    BwIter it;
+    it.init(p.nq, MODE, p.n_items);
+    while (it.valid()) {
+      named_bar_sync(BW_OUT_BAR, 128);
+      if (*abort_flag) break;                  // read after the barrier: the same answer in all four warps
+      const int k = it.k, tile = it.tt;
+      const int sh = it.item / p.nq, h = sh % p.H, seq = sh / p.H;
+      {
+        int ok = 1;
+        if (lane == 0) {
+          ok = *abort_flag ? 0 : 1;
+          if (ok && !mbar_wait_bounded(&acc_full[k & 1], (unsigned)(k >> 1) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_O_FULL); ok = 0; }
+          if (!ok) *abort_flag = 1;
+        }
+        if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
+      }
+      tc_fence_after();
+      const int pos = min(tile * BM + row, p.S - 1);                  // position of this row in its sequence
+      constexpr int N_OUT = MODE == BW_DQ ? 1 : 2;                     // dQ | dK, dV
+#pragma unroll 1
+      for (int o = 0; o < N_OUT; ++o) {
+        const uint32_t acc = lane_addr + (uint32_t)(C::ACC_COL + (MODE == BW_DQ ? (k & 1) : o) * DH);
+        const bool rotate = p.rope_tab != nullptr && !(MODE == BW_DKV && o == 1);   // dV is not rotated
+        const float sc = (MODE == BW_DKV && o == 1) ? 1.f : p.scale;
+        const int x0 = (MODE == BW_DQ ? 0 : (o == 0 ? p.d : 2 * p.d)) + h * DH;
+#pragma unroll 1
+        for (int cb = 0; cb < DH; cb += 64) {
+          if (storer) bulk_wait_read_all();    // the previous store has finished reading the staging buffer
+          named_bar_sync(BW_OUT_BAR, 128);
+#pragma unroll 1
+          for (int cc = 0; cc < 64; cc += 32) {
+            const int c0 = cb + cc;                                     // first output column of this chunk
+            float v[32];
+            if (!dead) {
+              uint32_t r[32];
+              tmem_ld_32x32(acc + (uint32_t)c0, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]) * sc;
+              if (rotate) {
+                // pair (c, c + HALF): lo' = lo cos + hi sin, hi' = hi cos - lo sin
+                const bool is_lo = c0 < HALF;
+                uint32_t q[32];
+                tmem_ld_32x32(acc + (uint32_t)(is_lo ? c0 + HALF : c0 - HALF), q);
+                tmem_ld_wait();
+                const float2* tab = p.rope_tab + (long long)pos * HALF + (is_lo ? c0 : c0 - HALF);
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                  const float4 cs = *reinterpret_cast<const float4*>(tab + e);      // (cos, sin) of two pairs
+                  const float o0 = __uint_as_float(q[e]) * sc, o1 = __uint_as_float(q[e + 1]) * sc;
+                  v[e] = is_lo ? v[e] * cs.x + o0 * cs.y : v[e] * cs.x - o0 * cs.y;
+                  v[e + 1] = is_lo ? v[e + 1] * cs.z + o1 * cs.w : v[e + 1] * cs.z - o1 * cs.w;
+                }
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) v[e] = 0.f;
+            }
+#pragma unroll
+            for (int e = 0; e < 32; e += 8) {
+              uint4 ov;
+              ov.x = pack_bf16x2(v[e], v[e + 1]); ov.y = pack_bf16x2(v[e + 2], v[e + 3]);
+              ov.z = pack_bf16x2(v[e + 4], v[e + 5]); ov.w = pack_bf16x2(v[e + 6], v[e + 7]);
+              const int chunk = (cc + e) >> 3;
+              *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) = ov;
+            }
+          }
+          fence_proxy_async_smem();
+          named_bar_sync(BW_OUT_BAR, 128);
+          if (storer && !dead) {
+            tma_store_3d(&tmDQKV, base + pl.ostage_off, x0 + cb, tile * BM, seq);
+            bulk_commit();
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0 && !dead) mbar_arrive(&acc_empty[k & 1]);
+      // advance to the next item
+      const int cnt = it.cnt;
+      for (int i = 0; i < cnt; ++i) it.next();
+    }
+    if (storer) bulk_wait_read_all();
+  } else {
+    // ------------------------------ compute: 16 warps, one 32-column slice each ------------------------------
+    const int cw = warp - 6, quad = warp & 3, slice = cw >> 2;        // warps 6..9 -> quadrants 2,3,0,1
+    const int row = quad * 32 + lane;
+    const int ct = threadIdx.x - 6 * 32;                              // 0..511 within the compute warps
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const float c2 = p.scale_log2;
+    bool dead = false;
+    float lse2_row = INFINITY, dsum_row = 0.f;                         // BW_DQ: this row's statistics
+    BwIter it;
+    it.init(p.nq, MODE, p.n_items);
+    for (int b = 0; it.valid(); ++b, it.next()) {
+      const int sh = it.item / p.nq, h = sh % p.H, seq = sh / p.H;
+      const long long stat_base = ((long long)seq * p.H + h) * p.S;
+      float* cstat = stat + (b & 1) * 2 * BM;                          // BW_DKV: [lse * log2 e | rowsum(dO o O)] of the streamed queries
+      if (MODE == BW_DKV) {
+        if (ct < 2 * BM) {
+          const int c = ct & (BM - 1), qi = it.stile() * BM + c;
+          float v;
+          if (ct < BM) v = qi < p.S ? p.lse[stat_base + qi] * LOG2E : INFINITY;   // +inf: probability 0 past the sequence
+          else v = qi < p.S ? p.dsum[stat_base + qi] : 0.f;
+          cstat[ct] = v;
+        }
+      } else if (it.first()) {
+        // rowsum(dO o O) of this query row: each of the quadrant's four warps takes a quarter of the columns
+        const int qi = it.tt * BM + row;
+        float part = 0.f;
+        if (qi < p.S) {
+          const long long off = ((long long)seq * p.S + qi) * p.d + h * DH + slice * (DH / 4);
+#pragma unroll
+          for (int e = 0; e < DH / 4; e += 8) {
+            const uint4 a = *reinterpret_cast<const uint4*>(p.out + off + e);
+            const uint4 g = *reinterpret_cast<const uint4*>(p.dout + off + e);
+            const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+            const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 af = __bfloat1622float2(ah[i]), gf = __bfloat1622float2(gh[i]);
+              part = fmaf(af.x, gf.x, part);
+              part = fmaf(af.y, gf.y, part);
+            }
+          }
+          lse2_row = p.lse[stat_base + qi] * LOG2E;
+        } else {
+          lse2_row = INFINITY;
+        }
+        stat[slice * BM + row] = part;
+      }
+      named_bar_sync(BW_COMPUTE_BAR, BW_COMPUTE_WARPS * 32);           // statistics visible; also the block boundary for leaving
+      if (*abort_flag) break;
+      if (MODE == BW_DQ && it.first()) {
+        dsum_row = (stat[row] + stat[BM + row]) + (stat[2 * BM + row] + stat[3 * BM + row]);
+        const int qi = it.tt * BM + row;
+        if (slice == 0 && qi < p.S) p.dsum[stat_base + qi] = dsum_row;
+      }
+      {
+        int ok = 1;
+        if (lane == 0) {
+          ok = (dead || *abort_flag) ? 0 : 1;
+          if (ok && !mbar_wait_bounded(sdp_full, (unsigned)b & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
+          if (!ok) *abort_flag = 1;
+        }
+        if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
+      }
+      tc_fence_after();
+      const int nbc = it.stile() == p.nq - 1 ? nb_tail : BN;           // columns of this block
+      if (!dead && slice * 32 < nbc) {
+        const uint32_t s_addr = lane_addr + (uint32_t)((b % NSBUF) * BN + slice * 32);
+        const uint32_t dp_addr = lane_addr + (uint32_t)(C::DP_COL + slice * 32);
+        // causal mask on the diagonal block.  BW_DQ: column (key) <= row (query).  BW_DKV: column (query) >= row (key).
+        // 0 = every element of this warp's slice is kept, 1 = mixed, 2 = every element is masked
+        int mode_mask = 0;
+        if (it.diag()) mode_mask = slice == quad ? 1 : ((MODE == BW_DQ ? slice > quad : slice < quad) ? 2 : 0);
+#pragma unroll 1
+        for (int hc = 0; hc < 32; hc += 16) {
+          uint32_t pp[8], pd8[8];
+          if (mode_mask == 2) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { pp[e] = 0u; pd8[e] = 0u; }
+          } else {
+            uint32_t rs[16], rd[16];
+            tmem_ld_32x16(s_addr + (uint32_t)hc, rs);
+            tmem_ld_32x16(dp_addr + (uint32_t)hc, rd);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) {
+              float pr[2], ds[2];
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {
+                const int c = slice * 32 + hc + e + u;                  // column inside the block
+                const float l2 = MODE == BW_DQ ? lse2_row : cstat[c];
+                const float dsm = MODE == BW_DQ ? dsum_row : cstat[BM + c];
+                float pv = ex2_approx(fmaf(__uint_as_float(rs[e + u]), c2, -l2));
+                if (mode_mask == 1) {
+                  const bool keep = MODE == BW_DQ ? (c <= row) : (c >= row);
+                  pv = keep ? pv : 0.f;
+                }
+                pr[u] = pv;
+                ds[u] = pv * (__uint_as_float(rd[e + u]) - dsm);
+              }
+              pp[e >> 1] = pack_bf16x2(pr[0], pr[1]);
+              pd8[e >> 1] = pack_bf16x2(ds[0], ds[1]);
+            }
+          }
+          // packed results go over the first 16 columns of this warp's own slice (already consumed for hc = 0;
+          // for hc = 16 the columns written, 8..15, were read in the first half)
+          if (MODE == BW_DQ) {
+            tmem_st_32x8(s_addr + (uint32_t)(hc >> 1), pd8);           // dS over the scores
+          } else {
+            tmem_st_32x8(s_addr + (uint32_t)(hc >> 1), pp);            // P^T over S^T
+            tmem_st_32x8(dp_addr + (uint32_t)(hc >> 1), pd8);          // dS^T over dP^T
+          }
+        }
+        tmem_st_wait();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0 && !dead) mbar_arrive(p_ready);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);   // let copies still in flight land before shared memory goes away
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
@@ -648,6 +1180,47 @@ static int fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int S, 
   return PCM_OK;
 }
 
+
+template <int DH, int MODE>
+static int bwd_launch_one(const CUtensorMap& tmQKV, const CUtensorMap& tmDO, const CUtensorMap& tmDQKV, const BwParams& p,
+                          cudaStream_t s) {
+  const BwPlan pl = bw_make_plan<DH>();
+  if (pl.total > SMEM_LIMIT) return PCM_ERR_SHAPE;
+  const uint32_t smem = pl.total < SMEM_FLOOR ? SMEM_FLOOR : pl.total;
+  static bool attr_done = false;
+  if (!attr_done) {
+    PCM_CUDA_TRY(cudaFuncSetAttribute(fa_tc_bwd_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT));
+    attr_done = true;
+  }
+  const int grid = p.n_items < attn_sm_count() ? p.n_items : attn_sm_count();
+  fa_tc_bwd_kernel<DH, MODE><<<grid, BW_THREADS, smem, s>>>(tmQKV, tmDO, tmDQKV, p);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
+}
+
+template <int DH>
+static int bwd_launch(const void* qkv, const void* out, const void* dout, const float* lse, float* dsum, void* dqkv,
+                      int n_seq, int S, int H, const float2* rope_tab, cudaStream_t s) {
+  const int d = H * DH;
+  BwParams p;
+  p.n_seq = n_seq; p.S = S; p.H = H; p.d = d;
+  p.nq = (S + BM - 1) / BM;
+  p.n_items = n_seq * H * p.nq;
+  p.n_total = ((S + 15) / 16) * 16;
+  p.scale = 1.f / sqrtf((float)DH);
+  p.scale_log2 = LOG2E / sqrtf((float)DH);
+  p.lse = lse; p.dsum = dsum;
+  p.out = (const __nv_bfloat16*)out; p.dout = (const __nv_bfloat16*)dout;
+  p.rope_tab = rope_tab;
+  CUtensorMap tmQKV, tmDO, tmDQKV;
+  if (!make_seq_tmap(&tmQKV, qkv, n_seq, S, 3LL * d, 3LL * d, BM) || !make_seq_tmap(&tmDO, dout, n_seq, S, d, d, BM) ||
+      !make_seq_tmap(&tmDQKV, dqkv, n_seq, S, 3LL * d, 3LL * d, BM))
+    return PCM_ERR_CUDA;
+  const int rc = bwd_launch_one<DH, BW_DQ>(tmQKV, tmDO, tmDQKV, p, s);     // also writes rowsum(dO o O) for the second launch
+  if (rc != PCM_OK) return rc;
+  return bwd_launch_one<DH, BW_DKV>(tmQKV, tmDO, tmDQKV, p, s);
+}
+
 }  // namespace fatc
 
 bool attention_tc_supported(const void* qkv, const void* out, int S, int H, int dh) {
@@ -656,6 +1229,14 @@ bool attention_tc_supported(const void* qkv, const void* out, int S, int H, int 
   if ((((uintptr_t)qkv) | ((uintptr_t)out)) & 15) return false;
   (void)H;
   return fatc::attn_encode_fn() != nullptr;
+}
+
+int attention_bwd_bf16_tc(const void* qkv, const void* out, const void* dout, const float* lse, float* dsum, void* dqkv,
+                          int n_seq, int S, int H, int dh, const float2* rope_tab, cudaStream_t s) {
+  if (!attention_tc_supported(qkv, out, S, H, dh) || ((((uintptr_t)dout) | ((uintptr_t)dqkv)) & 15)) return PCM_ERR_SHAPE;
+  if (n_seq < 1) return PCM_OK;
+  return dh == 64 ? fatc::bwd_launch<64>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s)
+                  : fatc::bwd_launch<128>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s);
 }
 
 int attention_fwd_bf16_tc(const void* qkv, void* out, float* lse, int n_seq, int S, int H, int dh, cudaStream_t s) {
