@@ -597,6 +597,7 @@ template <int DH> struct BwCfg {
   static constexpr int FIX_STAGES = DH == 64 ? 2 : 1;                 // resident operand pairs (this item's and the next)
   static constexpr int STR_STAGES = NSBUF + 1;                        // streamed operand pairs in flight
   static constexpr uint32_t TILE_BYTES = (DH / 64) * BM * 128u;       // one 128-row operand tile: DH/64 slabs of 16 KB
+  static constexpr bool O_IN_SMEM = DH == 64;                         // BW_DQ also keeps O_i resident (rowsum(dO o O) from shared memory)
   static_assert(ACC_COL + 2 * DH <= TMEM_COLS, "tensor memory plan does not fit");
 };
 
@@ -630,29 +631,28 @@ __device__ __forceinline__ void tmem_st_32x8(uint32_t taddr, const uint32_t (&r)
 
 // Walks this CTA's items and their blocks in issue order.  Item = ((sequence * H + head) * nq + tile); a BW_DQ
 // item streams the key blocks 0 .. tile, a BW_DKV item the query tiles tile .. nq - 1.
+struct BwShape { int nq, mode, grid, n_items; };
 struct BwIter {
-  int nq, mode, grid, n_items;
   int k, item, tt, u, cnt, b;                   // k = local item count, b = local block count
-  __device__ void setup() {
-    if (item < n_items) {
-      tt = item % nq;
-      cnt = mode == BW_DQ ? tt + 1 : nq - tt;
+  __device__ void setup(const BwShape& sh) {
+    if (item < sh.n_items) {
+      tt = item % sh.nq;
+      cnt = sh.mode == BW_DQ ? tt + 1 : sh.nq - tt;
       u = 0;
     }
   }
-  __device__ void init(int nq_, int mode_, int n_items_) {
-    nq = nq_; mode = mode_; n_items = n_items_; grid = gridDim.x;
+  __device__ void init(const BwShape& sh) {
     k = 0; b = 0; item = blockIdx.x;
-    setup();
+    setup(sh);
   }
-  __device__ bool valid() const { return item < n_items; }
+  __device__ bool valid(const BwShape& sh) const { return item < sh.n_items; }
   __device__ bool first() const { return u == 0; }
   __device__ bool last() const { return u == cnt - 1; }
-  __device__ int stile() const { return mode == BW_DQ ? u : tt + u; }   // index of the streamed tile in its sequence
-  __device__ bool diag() const { return stile() == tt; }
-  __device__ void next() {
+  __device__ int stile(const BwShape& sh) const { return sh.mode == BW_DQ ? u : tt + u; }   // index of the streamed tile in its sequence
+  __device__ bool diag(const BwShape& sh) const { return stile(sh) == tt; }
+  __device__ void next(const BwShape& sh) {
     ++b;
-    if (++u == cnt) { ++k; item += grid; setup(); }
+    if (++u == cnt) { ++k; item += sh.grid; setup(sh); }
   }
 };
 
@@ -661,11 +661,12 @@ struct BwIter {
 struct BwPlan {
   uint32_t fix_off, str_off, ostage_off, bar_off, stat_off, total;
 };
-template <int DH>
+template <int DH, int MODE>
 __host__ __device__ inline BwPlan bw_make_plan() {
   BwPlan p;
+  constexpr int n_fix = (MODE == BW_DQ && BwCfg<DH>::O_IN_SMEM) ? 3 : 2;     // tiles per resident group
   p.fix_off = 0;
-  p.str_off = p.fix_off + BwCfg<DH>::FIX_STAGES * 2 * BwCfg<DH>::TILE_BYTES;
+  p.str_off = p.fix_off + BwCfg<DH>::FIX_STAGES * n_fix * BwCfg<DH>::TILE_BYTES;
   p.ostage_off = p.str_off + BwCfg<DH>::STR_STAGES * 2 * BwCfg<DH>::TILE_BYTES;
   p.bar_off = p.ostage_off + BM * 128;
   p.stat_off = p.bar_off + 256;
@@ -676,7 +677,7 @@ __host__ __device__ inline BwPlan bw_make_plan() {
 template <int DH, int MODE>
 __global__ void __launch_bounds__(BW_THREADS, 1)
 fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constant__ CUtensorMap tmDO,
-                 const __grid_constant__ CUtensorMap tmDQKV, const BwParams p) {
+                 const __grid_constant__ CUtensorMap tmOUT, const __grid_constant__ CUtensorMap tmDQKV, const BwParams p) {
   extern __shared__ uint8_t smem_raw[];
   using C = BwCfg<DH>;
   constexpr int NSLAB = DH / 64;
@@ -684,7 +685,9 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   constexpr uint32_t TILE = C::TILE_BYTES, PAIR = 2 * TILE;
   const uint32_t raw_addr = smem_u32(smem_raw);
   uint8_t* base = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
-  const BwPlan pl = bw_make_plan<DH>();
+  const BwPlan pl = bw_make_plan<DH, MODE>();
+  constexpr bool O_SMEM = MODE == BW_DQ && C::O_IN_SMEM;
+  constexpr uint32_t FIXB = (O_SMEM ? 3u : 2u) * TILE;              // bytes of a resident group
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + pl.bar_off);
   uint64_t* fix_full = bars;                   // [2] producer -> MMA: an item's resident pair has landed
   uint64_t* fix_empty = bars + 2;              // [2] MMA -> producer
@@ -693,18 +696,20 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   uint64_t* sdp_full = bars + 10;              // MMA -> compute: S and dP of a block are in tensor memory
   uint64_t* p_ready = bars + 11;               // compute -> MMA: P / dS of the block are in tensor memory (16 warp arrivals)
   uint64_t* acc_full = bars + 12;              // [2] MMA -> output warps: the item's accumulators are complete
-  uint64_t* acc_empty = bars + 14;             // [2] output warps -> MMA (4 warp arrivals); items alternate between the two
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* acc_empty = bars + 14;             // [2] output warps -> MMA (4 warp arrivals): dQ / dK accumulator read; items alternate
+  uint64_t* accv_empty = bars + 16;            // [2] the same for the dV accumulator
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   float* stat = reinterpret_cast<float*>(base + pl.stat_off);        // BW_DKV: [2][2][128] column statistics; BW_DQ: [4][128] partial row sums
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nb_tail = p.n_total - (p.nq - 1) * BN;                  // rows of a sequence's last tile that take part (multiple of 16)
+  const BwShape shp = {p.nq, MODE, (int)gridDim.x, p.n_items};
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
       mbar_init(&fix_full[s], 1); mbar_init(&fix_empty[s], 1);
-      mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4);
+      mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); mbar_init(&accv_empty[s], 4);
     }
     for (int s = 0; s < 3; ++s) { mbar_init(&str_full[s], 1); mbar_init(&str_empty[s], 1); }
     mbar_init(sdp_full, 1); mbar_init(p_ready, BW_COMPUTE_WARPS);
@@ -712,6 +717,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
     fence_mbar_init();
     prefetch_tmap(&tmQKV);
     prefetch_tmap(&tmDO);
+    prefetch_tmap(&tmOUT);
     prefetch_tmap(&tmDQKV);
   }
   if (warp == 1) {
@@ -729,7 +735,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       // BW_DQ: resident = (Q_i, dO_i), streamed = (K_j, V_j).  BW_DKV: resident = (K_j, V_j), streamed = (Q_i, dO_i).
       bool ok = true;
       BwIter it;
-      it.init(p.nq, MODE, p.n_items);
+      it.init(shp);
       int fs = 0, fph = 0, ss = 0, sph = 0;
       auto load_pair = [&](uint8_t* dst, bool qdo, int h, int tile, int seq, uint64_t* bar) {
         for (int sl = 0; sl < NSLAB; ++sl) {
@@ -742,19 +748,35 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
           }
         }
       };
-      while (it.valid() && ok && !*abort_flag) {
+      int fix_issued = 0;                         // items whose resident group has been requested
+      auto load_resident = [&](int item) {
+        const int sh = item / p.nq, h = sh % p.H, seq = sh / p.H, tile = item - sh * p.nq;
+        if (!mbar_wait_bounded(&fix_empty[fs], (unsigned)fph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; return; }
+        mbar_expect_tx(&fix_full[fs], FIXB);
+        uint8_t* dst = base + pl.fix_off + fs * FIXB;
+        load_pair(dst, MODE == BW_DQ, h, tile, seq, &fix_full[fs]);
+        if (O_SMEM)
+          for (int sl = 0; sl < NSLAB; ++sl) tma_load_3d(dst + 2 * TILE + sl * 16384, &tmOUT, h * DH + sl * 64, tile * BM, seq, &fix_full[fs]);
+        if (++fs == C::FIX_STAGES) { fs = 0; fph ^= 1; }
+        ++fix_issued;
+      };
+      while (it.valid(shp) && ok && !*abort_flag) {
         const int sh = it.item / p.nq, h = sh % p.H, seq = sh / p.H;
-        if (it.first()) {
-          if (!mbar_wait_bounded(&fix_empty[fs], (unsigned)fph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; break; }
-          mbar_expect_tx(&fix_full[fs], PAIR);
-          load_pair(base + pl.fix_off + fs * PAIR, MODE == BW_DQ, h, it.tt, seq, &fix_full[fs]);
-          if (++fs == C::FIX_STAGES) { fs = 0; fph ^= 1; }
-        }
+        const bool first = it.first();
+        if (first && fix_issued <= it.k) load_resident(it.item);
+        if (!ok) break;
         if (!mbar_wait_bounded(&str_empty[ss], (unsigned)sph ^ 1u, WAIT_NS)) { fa_timeout(SITE_Q_EMPTY); ok = false; break; }
         mbar_expect_tx(&str_full[ss], PAIR);
-        load_pair(base + pl.str_off + ss * PAIR, MODE == BW_DKV, h, it.stile(), seq, &str_full[ss]);
+        load_pair(base + pl.str_off + ss * PAIR, MODE == BW_DKV, h, it.stile(shp), seq, &str_full[ss]);
         if (++ss == C::STR_STAGES) { ss = 0; sph ^= 1; }
-        it.next();
+        // With a second resident stage the next item's group is requested now, so that its load overlaps this item's
+        // blocks.  It comes after this item's first streamed pair: the stage it waits for is released at the end of the
+        // previous item, and the MMA thread gets there only once that pair has been issued.
+        if (first && C::FIX_STAGES == 2 && fix_issued == it.k + 1 && it.item + (long long)gridDim.x < p.n_items) {
+          load_resident(it.item + gridDim.x);
+          if (!ok) break;
+        }
+        it.next(shp);
       }
       if (!ok) *abort_flag = 1;
     }
@@ -772,10 +794,10 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       const uint32_t idesc_full = idesc_bf16(BN, 0), idesc_tail = idesc_bf16(nb_tail, 0), idesc_acc = idesc_bf16(DH, 1);
       // ring positions of the three issue streams: scores (furthest ahead), dP, accumulation
       struct Pos { BwIter it; int fs, ss, sph, fph; };
-      auto pos_init = [&](Pos& q) { q.it.init(p.nq, MODE, p.n_items); q.fs = q.ss = q.sph = q.fph = 0; };
+      auto pos_init = [&](Pos& q) { q.it.init(shp); q.fs = q.ss = q.sph = q.fph = 0; };
       auto pos_next = [&](Pos& q) {
         const bool item_end = q.it.last();
-        q.it.next();
+        q.it.next(shp);
         if (++q.ss == C::STR_STAGES) { q.ss = 0; q.sph ^= 1; }
         if (item_end && ++q.fs == C::FIX_STAGES) { q.fs = 0; q.fph ^= 1; }
       };
@@ -786,8 +808,8 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         if (q.it.first() && !mbar_wait_bounded(&fix_full[q.fs], (unsigned)q.fph, WAIT_NS)) { fa_timeout(SITE_KV_FULL); ok = false; return; }
         if (!mbar_wait_bounded(&str_full[q.ss], (unsigned)q.sph, WAIT_NS)) { fa_timeout(SITE_Q_FULL); ok = false; return; }
         tc_fence_after();
-        const uint32_t a = dfk_lo + (uint32_t)q.fs * (PAIR >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4);
-        const uint32_t idesc = (q.it.stile() == p.nq - 1) ? idesc_tail : idesc_full;
+        const uint32_t a = dfk_lo + (uint32_t)q.fs * (FIXB >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4);
+        const uint32_t idesc = (q.it.stile(shp) == p.nq - 1) ? idesc_tail : idesc_full;
         const uint32_t d_col = tmem_base + (uint32_t)(sb * BN);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks) {
@@ -798,8 +820,8 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       };
       // second product of a block: dP from the second tiles of both pairs; then both are announced
       auto issue_dp = [&](Pos& q) {
-        const uint32_t a = dfk_lo + (uint32_t)q.fs * (PAIR >> 4) + (TILE >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4) + (TILE >> 4);
-        const uint32_t idesc = (q.it.stile() == p.nq - 1) ? idesc_tail : idesc_full;
+        const uint32_t a = dfk_lo + (uint32_t)q.fs * (FIXB >> 4) + (TILE >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4) + (TILE >> 4);
+        const uint32_t idesc = (q.it.stile(shp) == p.nq - 1) ? idesc_tail : idesc_full;
         const uint32_t d_col = tmem_base + (uint32_t)C::DP_COL;
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks) {
@@ -812,7 +834,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       // accumulating product: D (+)= A[tensor memory, packed bf16 at a_col0] * streamed tile `which` read MN-major
       auto issue_acc = [&](const Pos& q, uint32_t d_col, uint32_t a_col0, int which, bool fresh) {
         const uint32_t bq = dsm_lo + (uint32_t)q.ss * (PAIR >> 4) + (uint32_t)which * (TILE >> 4);
-        const int nk = (q.it.stile() == p.nq - 1 ? nb_tail : BN) >> 4;          // 16-row steps of the streamed tile
+        const int nk = (q.it.stile(shp) == p.nq - 1 ? nb_tail : BN) >> 4;          // 16-row steps of the streamed tile
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk) {
           if (kk < nk) {
@@ -822,13 +844,13 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         }
       };
       // prologue: scores and dP of block 0, scores of block 1 when there is a second score buffer
-      if (ps.it.valid()) {
+      if (ps.it.valid(shp)) {
         issue_scores(ps, 0);
         if (ok) { issue_dp(pd); pos_next(ps); pos_next(pd); }
-        if (NSBUF == 2 && ok && ps.it.valid()) { issue_scores(ps, 1); if (ok) pos_next(ps); }
+        if (NSBUF == 2 && ok && ps.it.valid(shp)) { issue_scores(ps, 1); if (ok) pos_next(ps); }
       }
       int sb = 0, rph = 0;                      // score buffer and p_ready parity of the current block
-      while (pc.it.valid() && ok) {
+      while (pc.it.valid(shp) && ok) {
         if (*abort_flag) { ok = false; break; }
         if (!mbar_wait_bounded(p_ready, (unsigned)rph, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
         const int k = pc.it.k;
@@ -846,14 +868,13 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         const bool fresh = pc.it.first();
         if (MODE == BW_DKV) {
           issue_acc(pc, acc0, dp_col, 0, fresh);                       // dK += dS^T Q_i (dS^T sits in the dP buffer)
-          if (NSBUF == 2) {
-            if (pd.it.valid()) { issue_dp(pd); pos_next(pd); }         // the dP buffer is free again: next block's dP
-            issue_acc(pc, acc1, s_col, 1, fresh);                      // dV += P^T dO_i
-          } else {
-            issue_acc(pc, acc1, s_col, 1, fresh);
+          if (NSBUF == 2 && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }   // the dP buffer is free again: next block's dP
+          if (fresh && k >= 1 && !mbar_wait_bounded(&accv_empty[(k - 1) & 1], (unsigned)((k - 1) >> 1) & 1u, WAIT_NS)) {
+            fa_timeout(SITE_O_EMPTY); ok = false; break;
           }
+          issue_acc(pc, acc1, s_col, 1, fresh);                        // dV += P^T dO_i
         } else {
-          if (NSBUF == 2 && pd.it.valid()) { issue_dp(pd); pos_next(pd); }   // dS went over the scores: dP is free
+          if (NSBUF == 2 && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }   // dS went over the scores: dP is free
           issue_acc(pc, (k & 1) ? acc1 : acc0, s_col, 0, fresh);       // dQ += dS K_j
         }
         umma_commit(&str_empty[pc.ss]);                                // the streamed pair has been read for the last time
@@ -864,8 +885,8 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         pos_next(pc);
         // this block's score buffer is free once the accumulation above has read it: scores of the block after next
         // (or, with one buffer, scores and dP of the next block)
-        if (ps.it.valid()) { issue_scores(ps, sb); if (ok) pos_next(ps); }
-        if (NSBUF == 1 && ok && pd.it.valid()) { issue_dp(pd); pos_next(pd); }
+        if (ps.it.valid(shp)) { issue_scores(ps, sb); if (ok) pos_next(ps); }
+        if (NSBUF == 1 && ok && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }
         if (++sb == NSBUF) sb = 0;
         rph ^= 1;
       }
@@ -874,7 +895,8 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   } else if (warp < 6) {
     // ------------------------------ output: warps 2..5 ------------------------------
     // Scale by 1 / sqrt(dh) (dQ, dK), rotate back through the rotary embedding, stage 64 columns at a time in
-    // the swizzled layout of the gradient tensor map, TMA store (rows past the sequence are clipped).
+    // the swizzled layout of the gradient tensor map, TMA store (rows past the sequence are clipped).  An
+    // accumulator is handed back to the MMA thread as soon as it has been read into registers.
     const int quad = warp & 3, row = quad * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint8_t* stage_row = base + pl.ostage_off + row * 128;
@@ -882,8 +904,26 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
     constexpr int HALF = DH / 2;
     bool dead = false;
     BwIter it;
-    it.init(p.nq, MODE, p.n_items);
-    while (it.valid()) {
+    it.init(shp);
+    // one staged box: 64 bf16 columns of this row from v[0..63], then the TMA store
+    auto stage_box = [&](const float (&v)[64], int x, int tile, int seq) {
+      if (storer) bulk_wait_read_all();        // the previous store has finished reading the staging buffer
+      named_bar_sync(BW_OUT_BAR, 128);
+#pragma unroll
+      for (int e = 0; e < 64; e += 8) {
+        uint4 ov;
+        ov.x = pack_bf16x2(v[e], v[e + 1]); ov.y = pack_bf16x2(v[e + 2], v[e + 3]);
+        ov.z = pack_bf16x2(v[e + 4], v[e + 5]); ov.w = pack_bf16x2(v[e + 6], v[e + 7]);
+        *reinterpret_cast<uint4*>(stage_row + (((e >> 3) ^ (row & 7)) << 4)) = ov;
+      }
+      fence_proxy_async_smem();
+      named_bar_sync(BW_OUT_BAR, 128);
+      if (storer && !dead) {
+        tma_store_3d(&tmDQKV, base + pl.ostage_off, x, tile * BM, seq);
+        bulk_commit();
+      }
+    };
+    while (it.valid(shp)) {
       named_bar_sync(BW_OUT_BAR, 128);
       if (*abort_flag) break;                  // read after the barrier: the same answer in all four warps
       const int k = it.k, tile = it.tt;
@@ -906,62 +946,78 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         const bool rotate = p.rope_tab != nullptr && !(MODE == BW_DKV && o == 1);   // dV is not rotated
         const float sc = (MODE == BW_DKV && o == 1) ? 1.f : p.scale;
         const int x0 = (MODE == BW_DQ ? 0 : (o == 0 ? p.d : 2 * p.d)) + h * DH;
-#pragma unroll 1
-        for (int cb = 0; cb < DH; cb += 64) {
-          if (storer) bulk_wait_read_all();    // the previous store has finished reading the staging buffer
-          named_bar_sync(BW_OUT_BAR, 128);
-#pragma unroll 1
-          for (int cc = 0; cc < 64; cc += 32) {
-            const int c0 = cb + cc;                                     // first output column of this chunk
-            float v[32];
-            if (!dead) {
-              uint32_t r[32];
-              tmem_ld_32x32(acc + (uint32_t)c0, r);
-              tmem_ld_wait();
+        uint64_t* release = (MODE == BW_DKV && o == 1) ? &accv_empty[k & 1] : &acc_empty[k & 1];
+        if constexpr (DH == 64) {
+          float v[64];
+          if (!dead) {
+            uint32_t r0[32], r1[32];
+            tmem_ld_32x32(acc, r0);
+            tmem_ld_32x32(acc + 32u, r1);
+            tmem_ld_wait();
 #pragma unroll
-              for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]) * sc;
-              if (rotate) {
-                // pair (c, c + HALF): lo' = lo cos + hi sin, hi' = hi cos - lo sin
-                const bool is_lo = c0 < HALF;
-                uint32_t q[32];
-                tmem_ld_32x32(acc + (uint32_t)(is_lo ? c0 + HALF : c0 - HALF), q);
-                tmem_ld_wait();
-                const float2* tab = p.rope_tab + (long long)pos * HALF + (is_lo ? c0 : c0 - HALF);
+            for (int e = 0; e < 32; ++e) { v[e] = __uint_as_float(r0[e]) * sc; v[32 + e] = __uint_as_float(r1[e]) * sc; }
+          } else {
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                  const float4 cs = *reinterpret_cast<const float4*>(tab + e);      // (cos, sin) of two pairs
-                  const float o0 = __uint_as_float(q[e]) * sc, o1 = __uint_as_float(q[e + 1]) * sc;
-                  v[e] = is_lo ? v[e] * cs.x + o0 * cs.y : v[e] * cs.x - o0 * cs.y;
-                  v[e + 1] = is_lo ? v[e + 1] * cs.z + o1 * cs.w : v[e + 1] * cs.z - o1 * cs.w;
-                }
-              }
-            } else {
+            for (int e = 0; e < 64; ++e) v[e] = 0.f;
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0 && !dead) mbar_arrive(release);                // the accumulator is in registers
+          if (rotate) {
+            // pair (c, c + 32): lo' = lo cos + hi sin, hi' = hi cos - lo sin
+            const float2* tab = p.rope_tab + (long long)pos * HALF;
 #pragma unroll
-              for (int e = 0; e < 32; ++e) v[e] = 0.f;
-            }
-#pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              uint4 ov;
-              ov.x = pack_bf16x2(v[e], v[e + 1]); ov.y = pack_bf16x2(v[e + 2], v[e + 3]);
-              ov.z = pack_bf16x2(v[e + 4], v[e + 5]); ov.w = pack_bf16x2(v[e + 6], v[e + 7]);
-              const int chunk = (cc + e) >> 3;
-              *reinterpret_cast<uint4*>(stage_row + ((chunk ^ (row & 7)) << 4)) = ov;
+            for (int e = 0; e < 32; e += 2) {
+              const float4 cs = *reinterpret_cast<const float4*>(tab + e);      // (cos, sin) of two pairs
+              const float l0 = v[e], h0 = v[32 + e], l1 = v[e + 1], h1 = v[33 + e];
+              v[e] = l0 * cs.x + h0 * cs.y; v[32 + e] = h0 * cs.x - l0 * cs.y;
+              v[e + 1] = l1 * cs.z + h1 * cs.w; v[33 + e] = h1 * cs.z - l1 * cs.w;
             }
           }
-          fence_proxy_async_smem();
-          named_bar_sync(BW_OUT_BAR, 128);
-          if (storer && !dead) {
-            tma_store_3d(&tmDQKV, base + pl.ostage_off, x0 + cb, tile * BM, seq);
-            bulk_commit();
+          stage_box(v, x0, tile, seq);
+        } else {
+#pragma unroll 1
+          for (int cb = 0; cb < DH; cb += 64) {
+            float v[64];
+#pragma unroll
+            for (int cc = 0; cc < 64; cc += 32) {
+              const int c0 = cb + cc;                                   // first output column of this chunk
+              if (!dead) {
+                uint32_t r[32];
+                tmem_ld_32x32(acc + (uint32_t)c0, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[cc + e] = __uint_as_float(r[e]) * sc;
+                if (rotate) {
+                  const bool is_lo = c0 < HALF;
+                  tmem_ld_32x32(acc + (uint32_t)(is_lo ? c0 + HALF : c0 - HALF), r);
+                  tmem_ld_wait();
+                  const float2* tab = p.rope_tab + (long long)pos * HALF + (is_lo ? c0 : c0 - HALF);
+#pragma unroll
+                  for (int e = 0; e < 32; e += 2) {
+                    const float4 cs = *reinterpret_cast<const float4*>(tab + e);
+                    const float o0 = __uint_as_float(r[e]) * sc, o1 = __uint_as_float(r[e + 1]) * sc;
+                    v[cc + e] = is_lo ? v[cc + e] * cs.x + o0 * cs.y : v[cc + e] * cs.x - o0 * cs.y;
+                    v[cc + e + 1] = is_lo ? v[cc + e + 1] * cs.z + o1 * cs.w : v[cc + e + 1] * cs.z - o1 * cs.w;
+                  }
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[cc + e] = 0.f;
+              }
+            }
+            if (cb + 64 == DH) {                                        // last read of this accumulator
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0 && !dead) mbar_arrive(release);
+            }
+            stage_box(v, x0 + cb, tile, seq);
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0 && !dead) mbar_arrive(&acc_empty[k & 1]);
       // advance to the next item
       const int cnt = it.cnt;
-      for (int i = 0; i < cnt; ++i) it.next();
+      for (int i = 0; i < cnt; ++i) it.next(shp);
     }
     if (storer) bulk_wait_read_all();
   } else {
@@ -973,25 +1029,66 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
     const float c2 = p.scale_log2;
     bool dead = false;
     float lse2_row = INFINITY, dsum_row = 0.f;                         // BW_DQ: this row's statistics
+    int cfs = 0;                                                       // BW_DQ: resident stage of the current item
     BwIter it;
-    it.init(p.nq, MODE, p.n_items);
-    for (int b = 0; it.valid(); ++b, it.next()) {
+    it.init(shp);
+    // BW_DKV: lse * log2(e) (threads 0..127) and rowsum(dO o O) (threads 128..255) of one streamed query tile
+    auto load_col_stat = [&](const BwIter& q) -> float {
+      const int sh = q.item / p.nq, h = sh % p.H, seq = sh / p.H;
+      const long long sb0 = ((long long)seq * p.H + h) * p.S;
+      const int qi = q.stile(shp) * BM + (ct & (BM - 1));
+      if (ct < BM) return qi < p.S ? p.lse[sb0 + qi] * LOG2E : INFINITY;   // +inf: probability 0 past the sequence
+      return qi < p.S ? p.dsum[sb0 + qi] : 0.f;
+    };
+    if (MODE == BW_DKV && it.valid(shp) && ct < 2 * BM) stat[ct] = load_col_stat(it);
+    for (int b = 0; it.valid(shp); ++b, it.next(shp)) {
       const int sh = it.item / p.nq, h = sh % p.H, seq = sh / p.H;
       const long long stat_base = ((long long)seq * p.H + h) * p.S;
-      float* cstat = stat + (b & 1) * 2 * BM;                          // BW_DKV: [lse * log2 e | rowsum(dO o O)] of the streamed queries
-      if (MODE == BW_DKV) {
-        if (ct < 2 * BM) {
-          const int c = ct & (BM - 1), qi = it.stile() * BM + c;
-          float v;
-          if (ct < BM) v = qi < p.S ? p.lse[stat_base + qi] * LOG2E : INFINITY;   // +inf: probability 0 past the sequence
-          else v = qi < p.S ? p.dsum[stat_base + qi] : 0.f;
-          cstat[ct] = v;
+      float* cstat = stat + (b & 1) * 2 * BM;                          // BW_DKV: statistics of this block's queries
+      named_bar_sync(BW_COMPUTE_BAR, BW_COMPUTE_WARPS * 32);           // statistics visible; also the block boundary for leaving
+      if (*abort_flag) break;
+      // BW_DKV: the next block's statistics are fetched now and stored at the end of this block
+      float next_stat = 0.f;
+      BwIter nx = it;
+      nx.next(shp);
+      const bool have_next = MODE == BW_DKV && nx.valid(shp) && ct < 2 * BM;
+      if (have_next) next_stat = load_col_stat(nx);
+      if (MODE == BW_DQ && it.first()) {
+        const int qi = it.tt * BM + row;
+        lse2_row = qi < p.S ? p.lse[stat_base + qi] * LOG2E : INFINITY;
+      }
+      {
+        int ok = 1;
+        if (lane == 0) {
+          ok = (dead || *abort_flag) ? 0 : 1;
+          if (ok && !mbar_wait_bounded(sdp_full, (unsigned)b & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
+          if (!ok) *abort_flag = 1;
         }
-      } else if (it.first()) {
-        // rowsum(dO o O) of this query row: each of the quadrant's four warps takes a quarter of the columns
+        if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
+      }
+      if (MODE == BW_DQ && it.first()) {
+        // rowsum(dO o O) of this query row: each of the quadrant's four warps takes a quarter of the columns.  The
+        // item's tiles have landed (the scores above were formed from them).
         const int qi = it.tt * BM + row;
         float part = 0.f;
-        if (qi < p.S) {
+        if (O_SMEM) {
+          const uint8_t* g_row = base + pl.fix_off + cfs * FIXB + TILE + row * 128;      // dO_i, 128-byte-swizzled rows
+          const uint8_t* o_row = g_row + TILE;                                            // O_i
+#pragma unroll
+          for (int cix = 0; cix < 2; ++cix) {
+            const int chunk = ((slice * 2 + cix) ^ (row & 7)) << 4;
+            const uint4 a = *reinterpret_cast<const uint4*>(o_row + chunk);
+            const uint4 g = *reinterpret_cast<const uint4*>(g_row + chunk);
+            const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+            const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 af = __bfloat1622float2(ah[i]), gf = __bfloat1622float2(gh[i]);
+              part = fmaf(af.x, gf.x, part);
+              part = fmaf(af.y, gf.y, part);
+            }
+          }
+        } else if (qi < p.S) {
           const long long off = ((long long)seq * p.S + qi) * p.d + h * DH + slice * (DH / 4);
 #pragma unroll
           for (int e = 0; e < DH / 4; e += 8) {
@@ -1006,37 +1103,22 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
               part = fmaf(af.y, gf.y, part);
             }
           }
-          lse2_row = p.lse[stat_base + qi] * LOG2E;
-        } else {
-          lse2_row = INFINITY;
         }
         stat[slice * BM + row] = part;
-      }
-      named_bar_sync(BW_COMPUTE_BAR, BW_COMPUTE_WARPS * 32);           // statistics visible; also the block boundary for leaving
-      if (*abort_flag) break;
-      if (MODE == BW_DQ && it.first()) {
+        named_bar_sync(BW_COMPUTE_BAR, BW_COMPUTE_WARPS * 32);
         dsum_row = (stat[row] + stat[BM + row]) + (stat[2 * BM + row] + stat[3 * BM + row]);
-        const int qi = it.tt * BM + row;
         if (slice == 0 && qi < p.S) p.dsum[stat_base + qi] = dsum_row;
-      }
-      {
-        int ok = 1;
-        if (lane == 0) {
-          ok = (dead || *abort_flag) ? 0 : 1;
-          if (ok && !mbar_wait_bounded(sdp_full, (unsigned)b & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
-          if (!ok) *abort_flag = 1;
-        }
-        if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
+        if (++cfs == C::FIX_STAGES) cfs = 0;
       }
       tc_fence_after();
-      const int nbc = it.stile() == p.nq - 1 ? nb_tail : BN;           // columns of this block
+      const int nbc = it.stile(shp) == p.nq - 1 ? nb_tail : BN;           // columns of this block
       if (!dead && slice * 32 < nbc) {
         const uint32_t s_addr = lane_addr + (uint32_t)((b % NSBUF) * BN + slice * 32);
         const uint32_t dp_addr = lane_addr + (uint32_t)(C::DP_COL + slice * 32);
         // causal mask on the diagonal block.  BW_DQ: column (key) <= row (query).  BW_DKV: column (query) >= row (key).
         // 0 = every element of this warp's slice is kept, 1 = mixed, 2 = every element is masked
         int mode_mask = 0;
-        if (it.diag()) mode_mask = slice == quad ? 1 : ((MODE == BW_DQ ? slice > quad : slice < quad) ? 2 : 0);
+        if (it.diag(shp)) mode_mask = slice == quad ? 1 : ((MODE == BW_DQ ? slice > quad : slice < quad) ? 2 : 0);
 #pragma unroll 1
         for (int hc = 0; hc < 32; hc += 16) {
           uint32_t pp[8], pd8[8];
@@ -1082,6 +1164,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       tc_fence_before();
       __syncwarp();
       if (lane == 0 && !dead) mbar_arrive(p_ready);
+      if (have_next) stat[((b + 1) & 1) * 2 * BM + ct] = next_stat;
     }
   }
 
@@ -1182,9 +1265,9 @@ static int fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int S, 
 
 
 template <int DH, int MODE>
-static int bwd_launch_one(const CUtensorMap& tmQKV, const CUtensorMap& tmDO, const CUtensorMap& tmDQKV, const BwParams& p,
+static int bwd_launch_one(const CUtensorMap& tmQKV, const CUtensorMap& tmDO, const CUtensorMap& tmOUT, const CUtensorMap& tmDQKV, const BwParams& p,
                           cudaStream_t s) {
-  const BwPlan pl = bw_make_plan<DH>();
+  const BwPlan pl = bw_make_plan<DH, MODE>();
   if (pl.total > SMEM_LIMIT) return PCM_ERR_SHAPE;
   const uint32_t smem = pl.total < SMEM_FLOOR ? SMEM_FLOOR : pl.total;
   static bool attr_done = false;
@@ -1193,7 +1276,7 @@ static int bwd_launch_one(const CUtensorMap& tmQKV, const CUtensorMap& tmDO, con
     attr_done = true;
   }
   const int grid = p.n_items < attn_sm_count() ? p.n_items : attn_sm_count();
-  fa_tc_bwd_kernel<DH, MODE><<<grid, BW_THREADS, smem, s>>>(tmQKV, tmDO, tmDQKV, p);
+  fa_tc_bwd_kernel<DH, MODE><<<grid, BW_THREADS, smem, s>>>(tmQKV, tmDO, tmOUT, tmDQKV, p);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
 }
@@ -1212,13 +1295,14 @@ static int bwd_launch(const void* qkv, const void* out, const void* dout, const 
   p.lse = lse; p.dsum = dsum;
   p.out = (const __nv_bfloat16*)out; p.dout = (const __nv_bfloat16*)dout;
   p.rope_tab = rope_tab;
-  CUtensorMap tmQKV, tmDO, tmDQKV;
+  CUtensorMap tmQKV, tmDO, tmOUT, tmDQKV;
   if (!make_seq_tmap(&tmQKV, qkv, n_seq, S, 3LL * d, 3LL * d, BM) || !make_seq_tmap(&tmDO, dout, n_seq, S, d, d, BM) ||
+      !make_seq_tmap(&tmOUT, out, n_seq, S, d, d, BM) ||
       !make_seq_tmap(&tmDQKV, dqkv, n_seq, S, 3LL * d, 3LL * d, BM))
     return PCM_ERR_CUDA;
-  const int rc = bwd_launch_one<DH, BW_DQ>(tmQKV, tmDO, tmDQKV, p, s);     // also writes rowsum(dO o O) for the second launch
+  const int rc = bwd_launch_one<DH, BW_DQ>(tmQKV, tmDO, tmOUT, tmDQKV, p, s);     // also writes rowsum(dO o O) for the second launch
   if (rc != PCM_OK) return rc;
-  return bwd_launch_one<DH, BW_DKV>(tmQKV, tmDO, tmDQKV, p, s);
+  return bwd_launch_one<DH, BW_DKV>(tmQKV, tmDO, tmOUT, tmDQKV, p, s);
 }
 
 }  // namespace fatc
