@@ -595,9 +595,11 @@ template <int DH> struct BwCfg {
   static constexpr int DP_COL = NSBUF * BN;                           // dP buffer
   static constexpr int ACC_COL = DP_COL + BN;                         // two accumulators of DH columns
   static constexpr int FIX_STAGES = DH == 64 ? 2 : 1;                 // resident operand pairs (this item's and the next)
-  static constexpr int STR_STAGES = NSBUF + 1;                        // streamed operand pairs in flight
+  // streamed operand pairs in flight: a pair is held from its load until the block's last product has read it
+  // (two blocks after its scores were issued), and its successor's load takes about a block and a half to land
+  static constexpr int STR_STAGES = DH == 64 ? 4 : 2;
   static constexpr uint32_t TILE_BYTES = (DH / 64) * BM * 128u;       // one 128-row operand tile: DH/64 slabs of 16 KB
-  static constexpr bool O_IN_SMEM = DH == 64;                         // BW_DQ also keeps O_i resident (rowsum(dO o O) from shared memory)
+  static constexpr bool O_IN_SMEM = false;                            // BW_DQ could keep O_i resident too; the shared memory goes to the streamed ring instead
   static_assert(ACC_COL + 2 * DH <= TMEM_COLS, "tensor memory plan does not fit");
 };
 
@@ -691,10 +693,10 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + pl.bar_off);
   uint64_t* fix_full = bars;                   // [2] producer -> MMA: an item's resident pair has landed
   uint64_t* fix_empty = bars + 2;              // [2] MMA -> producer
-  uint64_t* str_full = bars + 4;               // [3] producer -> MMA: a block's streamed pair has landed
-  uint64_t* str_empty = bars + 7;              // [3] MMA -> producer
-  uint64_t* sdp_full = bars + 10;              // MMA -> compute: S and dP of a block are in tensor memory
-  uint64_t* p_ready = bars + 11;               // compute -> MMA: P / dS of the block are in tensor memory (16 warp arrivals)
+  uint64_t* str_full = bars + 4;               // [4] producer -> MMA: a block's streamed pair has landed
+  uint64_t* str_empty = bars + 8;              // [4] MMA -> producer
+  uint64_t* sdp_full = bars + 20;              // MMA -> compute: S and dP of a block are in tensor memory
+  uint64_t* p_ready = bars + 21;               // compute -> MMA: P / dS of the block are in tensor memory (16 warp arrivals)
   uint64_t* acc_full = bars + 12;              // [2] MMA -> output warps: the item's accumulators are complete
   uint64_t* acc_empty = bars + 14;             // [2] output warps -> MMA (4 warp arrivals): dQ / dK accumulator read; items alternate
   uint64_t* accv_empty = bars + 16;            // [2] the same for the dV accumulator
@@ -711,7 +713,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       mbar_init(&fix_full[s], 1); mbar_init(&fix_empty[s], 1);
       mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); mbar_init(&accv_empty[s], 4);
     }
-    for (int s = 0; s < 3; ++s) { mbar_init(&str_full[s], 1); mbar_init(&str_empty[s], 1); }
+    for (int s = 0; s < 4; ++s) { mbar_init(&str_full[s], 1); mbar_init(&str_empty[s], 1); }
     mbar_init(sdp_full, 1); mbar_init(p_ready, BW_COMPUTE_WARPS);
     *abort_flag = 0;
     fence_mbar_init();
@@ -905,17 +907,21 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
     bool dead = false;
     BwIter it;
     it.init(shp);
-    // one staged box: 64 bf16 columns of this row from v[0..63], then the TMA store
-    auto stage_box = [&](const float (&v)[64], int x, int tile, int seq) {
+    // a staged box = 64 bf16 columns of every row: begin, two chunks of 32 columns, end (which issues the TMA store)
+    auto stage_begin = [&]() {
       if (storer) bulk_wait_read_all();        // the previous store has finished reading the staging buffer
       named_bar_sync(BW_OUT_BAR, 128);
+    };
+    auto stage_chunk = [&](const float* v, int cc) {
 #pragma unroll
-      for (int e = 0; e < 64; e += 8) {
+      for (int e = 0; e < 32; e += 8) {
         uint4 ov;
         ov.x = pack_bf16x2(v[e], v[e + 1]); ov.y = pack_bf16x2(v[e + 2], v[e + 3]);
         ov.z = pack_bf16x2(v[e + 4], v[e + 5]); ov.w = pack_bf16x2(v[e + 6], v[e + 7]);
-        *reinterpret_cast<uint4*>(stage_row + (((e >> 3) ^ (row & 7)) << 4)) = ov;
+        *reinterpret_cast<uint4*>(stage_row + ((((cc + e) >> 3) ^ (row & 7)) << 4)) = ov;
       }
+    };
+    auto stage_end = [&](int x, int tile, int seq) {
       fence_proxy_async_smem();
       named_bar_sync(BW_OUT_BAR, 128);
       if (storer && !dead) {
@@ -974,20 +980,24 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
               v[e + 1] = l1 * cs.z + h1 * cs.w; v[33 + e] = h1 * cs.z - l1 * cs.w;
             }
           }
-          stage_box(v, x0, tile, seq);
+          stage_begin();
+          stage_chunk(v, 0);
+          stage_chunk(v + 32, 32);
+          stage_end(x0, tile, seq);
         } else {
 #pragma unroll 1
           for (int cb = 0; cb < DH; cb += 64) {
-            float v[64];
-#pragma unroll
+            stage_begin();
+#pragma unroll 1
             for (int cc = 0; cc < 64; cc += 32) {
               const int c0 = cb + cc;                                   // first output column of this chunk
+              float v[32];
               if (!dead) {
                 uint32_t r[32];
                 tmem_ld_32x32(acc + (uint32_t)c0, r);
                 tmem_ld_wait();
 #pragma unroll
-                for (int e = 0; e < 32; ++e) v[cc + e] = __uint_as_float(r[e]) * sc;
+                for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]) * sc;
                 if (rotate) {
                   const bool is_lo = c0 < HALF;
                   tmem_ld_32x32(acc + (uint32_t)(is_lo ? c0 + HALF : c0 - HALF), r);
@@ -997,21 +1007,22 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
                   for (int e = 0; e < 32; e += 2) {
                     const float4 cs = *reinterpret_cast<const float4*>(tab + e);
                     const float o0 = __uint_as_float(r[e]) * sc, o1 = __uint_as_float(r[e + 1]) * sc;
-                    v[cc + e] = is_lo ? v[cc + e] * cs.x + o0 * cs.y : v[cc + e] * cs.x - o0 * cs.y;
-                    v[cc + e + 1] = is_lo ? v[cc + e + 1] * cs.z + o1 * cs.w : v[cc + e + 1] * cs.z - o1 * cs.w;
+                    v[e] = is_lo ? v[e] * cs.x + o0 * cs.y : v[e] * cs.x - o0 * cs.y;
+                    v[e + 1] = is_lo ? v[e + 1] * cs.z + o1 * cs.w : v[e + 1] * cs.z - o1 * cs.w;
                   }
                 }
               } else {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) v[cc + e] = 0.f;
+                for (int e = 0; e < 32; ++e) v[e] = 0.f;
               }
+              if (c0 + 32 == DH) {                                      // last read of this accumulator
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0 && !dead) mbar_arrive(release);
+              }
+              stage_chunk(v, cc);
             }
-            if (cb + 64 == DH) {                                        // last read of this accumulator
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0 && !dead) mbar_arrive(release);
-            }
-            stage_box(v, x0 + cb, tile, seq);
+            stage_end(x0 + cb, tile, seq);
           }
         }
       }
@@ -1041,6 +1052,16 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       return qi < p.S ? p.dsum[sb0 + qi] : 0.f;
     };
     if (MODE == BW_DKV && it.valid(shp) && ct < 2 * BM) stat[ct] = load_col_stat(it);
+    // BW_DQ: this row's quarter (DH/4 columns) of the item's forward output, zero past the sequence
+    uint4 o_pref[DH / 32];
+    auto load_o_quarter = [&](int item) {
+      const int sh = item / p.nq, h = sh % p.H, seq = sh / p.H, qi = (item - sh * p.nq) * BM + row;
+      const __nv_bfloat16* src = p.out + ((long long)seq * p.S + qi) * p.d + h * DH + slice * (DH / 4);
+#pragma unroll
+      for (int cix = 0; cix < DH / 32; ++cix)
+        o_pref[cix] = qi < p.S ? *reinterpret_cast<const uint4*>(src + cix * 8) : make_uint4(0u, 0u, 0u, 0u);
+    };
+    if (MODE == BW_DQ && it.valid(shp)) load_o_quarter(it.item);
     for (int b = 0; it.valid(shp); ++b, it.next(shp)) {
       const int sh = it.item / p.nq, h = sh % p.H, seq = sh / p.H;
       const long long stat_base = ((long long)seq * p.H + h) * p.S;
@@ -1071,13 +1092,15 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         // item's tiles have landed (the scores above were formed from them).
         const int qi = it.tt * BM + row;
         float part = 0.f;
-        if (O_SMEM) {
-          const uint8_t* g_row = base + pl.fix_off + cfs * FIXB + TILE + row * 128;      // dO_i, 128-byte-swizzled rows
-          const uint8_t* o_row = g_row + TILE;                                            // O_i
+        {
+          // dO_i sits in the resident group (128-byte-swizzled rows, DH/64 slabs); this row's quarter of O_i was
+          // fetched from global memory one item ahead
+          const int c0 = slice * (DH / 4);                              // first column of this warp's quarter
+          const uint8_t* g_row = base + pl.fix_off + cfs * FIXB + TILE + (c0 >> 6) * 16384 + row * 128;
 #pragma unroll
-          for (int cix = 0; cix < 2; ++cix) {
-            const int chunk = ((slice * 2 + cix) ^ (row & 7)) << 4;
-            const uint4 a = *reinterpret_cast<const uint4*>(o_row + chunk);
+          for (int cix = 0; cix < DH / 32; ++cix) {
+            const int chunk = ((((c0 & 63) >> 3) + cix) ^ (row & 7)) << 4;
+            const uint4 a = o_pref[cix];
             const uint4 g = *reinterpret_cast<const uint4*>(g_row + chunk);
             const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
             const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g);
@@ -1088,21 +1111,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
               part = fmaf(af.y, gf.y, part);
             }
           }
-        } else if (qi < p.S) {
-          const long long off = ((long long)seq * p.S + qi) * p.d + h * DH + slice * (DH / 4);
-#pragma unroll
-          for (int e = 0; e < DH / 4; e += 8) {
-            const uint4 a = *reinterpret_cast<const uint4*>(p.out + off + e);
-            const uint4 g = *reinterpret_cast<const uint4*>(p.dout + off + e);
-            const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
-            const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float2 af = __bfloat1622float2(ah[i]), gf = __bfloat1622float2(gh[i]);
-              part = fmaf(af.x, gf.x, part);
-              part = fmaf(af.y, gf.y, part);
-            }
-          }
+          if (it.item + (long long)gridDim.x < p.n_items) load_o_quarter(it.item + gridDim.x);   // the next item's
         }
         stat[slice * BM + row] = part;
         named_bar_sync(BW_COMPUTE_BAR, BW_COMPUTE_WARPS * 32);
