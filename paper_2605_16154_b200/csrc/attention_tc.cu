@@ -594,10 +594,12 @@ template <int DH> struct BwCfg {
   static constexpr int NSBUF = DH == 64 ? 2 : 1;                      // score buffers
   static constexpr int DP_COL = NSBUF * BN;                           // dP buffer
   static constexpr int ACC_COL = DP_COL + BN;                         // two accumulators of DH columns
-  static constexpr int FIX_STAGES = DH == 64 ? 2 : 1;                 // resident operand pairs (this item's and the next)
+  // resident operand pairs: an item's pair can only be requested once the item FIX_STAGES back has ended, and items
+  // are as short as one block, so three stages are needed to request it a whole item ahead of its use
+  static constexpr int FIX_STAGES = DH == 64 ? 3 : 1;
   // streamed operand pairs in flight: a pair is held from its load until the block's last product has read it
   // (two blocks after its scores were issued), and its successor's load takes about a block and a half to land
-  static constexpr int STR_STAGES = DH == 64 ? 4 : 2;
+  static constexpr int STR_STAGES = DH == 64 ? 3 : 2;
   static constexpr uint32_t TILE_BYTES = (DH / 64) * BM * 128u;       // one 128-row operand tile: DH/64 slabs of 16 KB
   static constexpr bool O_IN_SMEM = false;                            // BW_DQ could keep O_i resident too; the shared memory goes to the streamed ring instead
   static_assert(ACC_COL + 2 * DH <= TMEM_COLS, "tensor memory plan does not fit");
@@ -691,16 +693,16 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   constexpr bool O_SMEM = MODE == BW_DQ && C::O_IN_SMEM;
   constexpr uint32_t FIXB = (O_SMEM ? 3u : 2u) * TILE;              // bytes of a resident group
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + pl.bar_off);
-  uint64_t* fix_full = bars;                   // [2] producer -> MMA: an item's resident pair has landed
-  uint64_t* fix_empty = bars + 2;              // [2] MMA -> producer
-  uint64_t* str_full = bars + 4;               // [4] producer -> MMA: a block's streamed pair has landed
-  uint64_t* str_empty = bars + 8;              // [4] MMA -> producer
+  uint64_t* fix_full = bars;                   // [3] producer -> MMA: an item's resident pair has landed
+  uint64_t* fix_empty = bars + 3;              // [3] MMA -> producer
+  uint64_t* str_full = bars + 6;               // [4] producer -> MMA: a block's streamed pair has landed
+  uint64_t* str_empty = bars + 10;             // [4] MMA -> producer
   uint64_t* sdp_full = bars + 20;              // MMA -> compute: S and dP of a block are in tensor memory
   uint64_t* p_ready = bars + 21;               // compute -> MMA: P / dS of the block are in tensor memory (16 warp arrivals)
-  uint64_t* acc_full = bars + 12;              // [2] MMA -> output warps: the item's accumulators are complete
-  uint64_t* acc_empty = bars + 14;             // [2] output warps -> MMA (4 warp arrivals): dQ / dK accumulator read; items alternate
-  uint64_t* accv_empty = bars + 16;            // [2] the same for the dV accumulator
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
+  uint64_t* acc_full = bars + 14;              // [2] MMA -> output warps: the item's accumulators are complete
+  uint64_t* acc_empty = bars + 16;             // [2] output warps -> MMA (4 warp arrivals): dQ / dK accumulator read; items alternate
+  uint64_t* accv_empty = bars + 18;            // [2] the same for the dV accumulator
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   float* stat = reinterpret_cast<float*>(base + pl.stat_off);        // BW_DKV: [2][2][128] column statistics; BW_DQ: [4][128] partial row sums
 
@@ -709,10 +711,8 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   const BwShape shp = {p.nq, MODE, (int)gridDim.x, p.n_items};
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&fix_full[s], 1); mbar_init(&fix_empty[s], 1);
-      mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); mbar_init(&accv_empty[s], 4);
-    }
+    for (int s = 0; s < 3; ++s) { mbar_init(&fix_full[s], 1); mbar_init(&fix_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); mbar_init(&accv_empty[s], 4); }
     for (int s = 0; s < 4; ++s) { mbar_init(&str_full[s], 1); mbar_init(&str_empty[s], 1); }
     mbar_init(sdp_full, 1); mbar_init(p_ready, BW_COMPUTE_WARPS);
     *abort_flag = 0;
@@ -771,13 +771,13 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         mbar_expect_tx(&str_full[ss], PAIR);
         load_pair(base + pl.str_off + ss * PAIR, MODE == BW_DKV, h, it.stile(shp), seq, &str_full[ss]);
         if (++ss == C::STR_STAGES) { ss = 0; sph ^= 1; }
-        // With a second resident stage the next item's group is requested now, so that its load overlaps this item's
-        // blocks.  It comes after this item's first streamed pair: the stage it waits for is released at the end of the
-        // previous item, and the MMA thread gets there only once that pair has been issued.
-        if (first && C::FIX_STAGES == 2 && fix_issued == it.k + 1 && it.item + (long long)gridDim.x < p.n_items) {
-          load_resident(it.item + gridDim.x);
-          if (!ok) break;
-        }
+        // Resident groups of the following items are requested as far ahead as there are free stages, so that their
+        // loads overlap this item's blocks.  Only a stage that is free right now is taken (one poll per block): this
+        // thread also feeds the streamed ring and must not sit in a wait for an item to end.
+        while (ok && fix_issued < it.k + C::FIX_STAGES && blockIdx.x + (long long)fix_issued * gridDim.x < p.n_items &&
+               mbar_try_wait(&fix_empty[fs], (unsigned)fph ^ 1u))
+          load_resident(blockIdx.x + fix_issued * gridDim.x);
+        if (!ok) break;
         it.next(shp);
       }
       if (!ok) *abort_flag = 1;
