@@ -635,18 +635,16 @@ __device__ __forceinline__ void tmem_st_32x8(uint32_t taddr, const uint32_t (&r)
 
 // Walks this CTA's items and their blocks in issue order.  Item = ((sequence * H + head) * nq + tile); a BW_DQ
 // item streams the key blocks 0 .. tile, a BW_DKV item the query tiles tile .. nq - 1.
-struct BwShape { int nq, mode, grid, n_items; };
+struct BwShape { int nq, mode, grid, n_items, gmod; };   // gmod = grid % nq: how the tile index moves from item to item
 struct BwIter {
   int k, item, tt, u, cnt, b;                   // k = local item count, b = local block count
   __device__ void setup(const BwShape& sh) {
-    if (item < sh.n_items) {
-      tt = item % sh.nq;
-      cnt = sh.mode == BW_DQ ? tt + 1 : sh.nq - tt;
-      u = 0;
-    }
+    cnt = sh.mode == BW_DQ ? tt + 1 : sh.nq - tt;
+    u = 0;
   }
   __device__ void init(const BwShape& sh) {
     k = 0; b = 0; item = blockIdx.x;
+    tt = item % sh.nq;
     setup(sh);
   }
   __device__ bool valid(const BwShape& sh) const { return item < sh.n_items; }
@@ -656,7 +654,12 @@ struct BwIter {
   __device__ bool diag(const BwShape& sh) const { return stile(sh) == tt; }
   __device__ void next(const BwShape& sh) {
     ++b;
-    if (++u == cnt) { ++k; item += sh.grid; setup(sh); }
+    if (++u == cnt) {
+      ++k; item += sh.grid;
+      tt += sh.gmod;
+      if (tt >= sh.nq) tt -= sh.nq;
+      setup(sh);
+    }
   }
 };
 
@@ -708,7 +711,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nb_tail = p.n_total - (p.nq - 1) * BN;                  // rows of a sequence's last tile that take part (multiple of 16)
-  const BwShape shp = {p.nq, MODE, (int)gridDim.x, p.n_items};
+  const BwShape shp = {p.nq, MODE, (int)gridDim.x, p.n_items, (int)(gridDim.x % p.nq)};
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 3; ++s) { mbar_init(&fix_full[s], 1); mbar_init(&fix_empty[s], 1); }
@@ -1048,14 +1051,17 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       const int sh = q.item / p.nq, h = sh % p.H, seq = sh / p.H;
       const long long sb0 = ((long long)seq * p.H + h) * p.S;
       const int qi = q.stile(shp) * BM + (ct & (BM - 1));
-      if (ct < BM) return qi < p.S ? p.lse[sb0 + qi] * LOG2E : INFINITY;   // +inf: probability 0 past the sequence
+      // raw values: the scaling by log2(e) happens where the value is stored, so that the load has a block to land
+      if (ct < BM) return qi < p.S ? p.lse[sb0 + qi] : INFINITY;          // +inf: probability 0 past the sequence
       return qi < p.S ? p.dsum[sb0 + qi] : 0.f;
     };
-    if (MODE == BW_DKV && it.valid(shp) && ct < 2 * BM) stat[ct] = load_col_stat(it);
+    if (MODE == BW_DKV && it.valid(shp) && ct < 2 * BM) stat[ct] = load_col_stat(it) * (ct < BM ? LOG2E : 1.f);
     // BW_DQ: this row's quarter (DH/4 columns) of the item's forward output, zero past the sequence
     uint4 o_pref[DH / 32];
+    float lse_pref = INFINITY;                                         // BW_DQ: this row's log-sum-exp (+inf past the sequence)
     auto load_o_quarter = [&](int item) {
       const int sh = item / p.nq, h = sh % p.H, seq = sh / p.H, qi = (item - sh * p.nq) * BM + row;
+      lse_pref = qi < p.S ? p.lse[((long long)seq * p.H + h) * p.S + qi] : INFINITY;
       const __nv_bfloat16* src = p.out + ((long long)seq * p.S + qi) * p.d + h * DH + slice * (DH / 4);
 #pragma unroll
       for (int cix = 0; cix < DH / 32; ++cix)
@@ -1074,10 +1080,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       nx.next(shp);
       const bool have_next = MODE == BW_DKV && nx.valid(shp) && ct < 2 * BM;
       if (have_next) next_stat = load_col_stat(nx);
-      if (MODE == BW_DQ && it.first()) {
-        const int qi = it.tt * BM + row;
-        lse2_row = qi < p.S ? p.lse[stat_base + qi] * LOG2E : INFINITY;
-      }
+      if (MODE == BW_DQ && it.first()) lse2_row = lse_pref * LOG2E;     // fetched one item ahead
       {
         int ok = 1;
         if (lane == 0) {
@@ -1173,7 +1176,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       tc_fence_before();
       __syncwarp();
       if (lane == 0 && !dead) mbar_arrive(p_ready);
-      if (have_next) stat[((b + 1) & 1) * 2 * BM + ct] = next_stat;
+      if (have_next) stat[((b + 1) & 1) * 2 * BM + ct] = next_stat * (ct < BM ? LOG2E : 1.f);
     }
   }
 
