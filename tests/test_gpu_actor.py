@@ -49,7 +49,10 @@ def test_gemm_simt_all_layouts(dtype, a_k, b_k):
 @pytest.mark.parametrize("dtype,dh,S,H,n_seq", [("f32", 32, 88, 4, 3), ("f32", 64, 45, 2, 2), ("bf16", 64, 312, 3, 2),
                                                 ("bf16", 128, 100, 2, 2), ("bf16", 32, 33, 2, 1),
                                                 ("bf16", 64, 384, 2, 3), ("bf16", 128, 312, 2, 2), ("bf16", 64, 17, 1, 1),
-                                                ("bf16", 64, 200, 16, 24), ("bf16", 128, 129, 16, 10)])
+                                                ("bf16", 64, 200, 16, 24), ("bf16", 128, 129, 16, 10),
+                                                ("bf16", 64, 128, 2, 2), ("bf16", 64, 129, 2, 2), ("bf16", 64, 256, 1, 3),
+                                                ("bf16", 64, 257, 3, 1), ("bf16", 128, 384, 1, 2), ("bf16", 64, 1, 2, 2),
+                                                ("bf16", 128, 16, 1, 3), ("bf16", 64, 312, 16, 20)])
 def test_attention_fwd_bwd(dtype, dh, S, H, n_seq):
     B, PL = _mods()
     rng = np.random.default_rng(5)
