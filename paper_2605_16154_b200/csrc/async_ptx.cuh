@@ -35,13 +35,26 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 // Waits for the phase with the given parity for at most `limit_ns` nanoseconds of wall time;
 // false when the wait ran out (the caller records the failure and unwinds).
+// A poll with a suspend-time hint: the thread may sleep inside the instruction until the phase completes or the
+// hint (nanoseconds) runs out, instead of spinning through issue slots.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, unsigned parity, unsigned hint_ns) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, unsigned parity, unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
   for (;;) {
 #pragma unroll 1
-    for (int it = 0; it < 256; ++it)
-      if (mbar_try_wait(bar, parity)) return true;
+    for (int it = 0; it < 64; ++it)
+      if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
     if (global_timer_ns() - t0 > limit_ns) return false;
   }
 }

@@ -74,30 +74,6 @@ struct BlockIter {
   __device__ void advance(int n) { for (int i = 0; i < n; ++i) next(); }
 };
 
-// Bounded wait whose polls carry a suspend-time hint: the thread may sleep inside the instruction until the phase
-// completes (or the hint runs out) instead of spinning through issue slots that the compute warps need.
-__device__ __forceinline__ bool fa_try_wait_hint(uint64_t* bar, unsigned parity, unsigned hint_ns) {
-  unsigned ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool fa_wait_bounded(uint64_t* bar, unsigned parity, unsigned long long limit_ns) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_timer_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int it = 0; it < 64; ++it)
-      if (fa_try_wait_hint(bar, parity, 4000u)) return true;
-    if (global_timer_ns() - t0 > limit_ns) return false;
-  }
-}
-
 __device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* tmap, int x, int y, int z, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
@@ -251,7 +227,7 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const int item = blockIdx.x + k * gridDim.x, seq = item / p.H, h = item - seq * p.H;
         const int st = k & (p.kv_stages - 1);                          // stages are 1 or 2
         const unsigned ph = (unsigned)(k >> (p.kv_stages - 1)) & 1u;
-        if (!fa_wait_bounded(&kv_empty[st], ph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; break; }
+        if (!mbar_wait_bounded(&kv_empty[st], ph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; break; }
         mbar_expect_tx(&kv_full[st], 2 * kv_bytes);
         uint8_t* ks = base + pl.k_off + st * kv_bytes;
         uint8_t* vs = base + pl.v_off + st * kv_bytes;
@@ -264,7 +240,7 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           const int g = k * p.nq + t, qs = g & (p.q_stages - 1);
           const unsigned qph = (unsigned)(g >> (p.q_stages - 1)) & 1u;
           if (*abort_flag) { ok = false; break; }
-          if (!fa_wait_bounded(&q_empty[qs], qph ^ 1u, WAIT_NS)) { fa_timeout(SITE_Q_EMPTY); ok = false; break; }
+          if (!mbar_wait_bounded(&q_empty[qs], qph ^ 1u, WAIT_NS)) { fa_timeout(SITE_Q_EMPTY); ok = false; break; }
           mbar_expect_tx(&q_full[qs], Q_BYTES);
           uint8_t* qd = base + pl.q_off + qs * Q_BYTES;
           for (int sl = 0; sl < NSLAB; ++sl)
@@ -296,15 +272,15 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // S_j = Q K_j^T for the block `it` points at, into score buffer `buf`
       auto issue_scores = [&](const BlockIter& it, int buf) {
         const int st = it.k & kv_mask, qs = it.tile & q_mask;
-        if (it.t == 0 && it.j == 0 && !fa_wait_bounded(&kv_full[st], (unsigned)(it.k >> kv_shift) & 1u, WAIT_NS)) {
+        if (it.t == 0 && it.j == 0 && !mbar_wait_bounded(&kv_full[st], (unsigned)(it.k >> kv_shift) & 1u, WAIT_NS)) {
           fa_timeout(SITE_KV_FULL); ok = false; return;
         }
-        if (it.j == 0 && !fa_wait_bounded(&q_full[qs], (unsigned)(it.tile >> q_shift) & 1u, WAIT_NS)) {
+        if (it.j == 0 && !mbar_wait_bounded(&q_full[qs], (unsigned)(it.tile >> q_shift) & 1u, WAIT_NS)) {
           fa_timeout(SITE_Q_FULL); ok = false; return;
         }
         // the statistics ring holds STAT_RING tiles: this tile's softmax overwrites those of tile - STAT_RING
         while (it.j == 0 && released <= it.tile - STAT_RING && ok) {
-          if (!fa_wait_bounded(&o_empty[released & 1], (unsigned)(released >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_O_EMPTY); ok = false; }
+          if (!mbar_wait_bounded(&o_empty[released & 1], (unsigned)(released >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_O_EMPTY); ok = false; }
           ++released;
         }
         if (!ok) return;
@@ -334,13 +310,13 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       for (int b = 0; b < n_blocks && ok; ++b) {
         const int st = cur.k & kv_mask;
         if (*abort_flag) { ok = false; break; }
-        if (!fa_wait_bounded(&p_full[buf], (unsigned)buf_phase, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
+        if (!mbar_wait_bounded(&p_full[buf], (unsigned)buf_phase, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
         // the accumulator slot must have been read by the output warps of the tile that used it last.  Releases are
         // consumed in tile order and at least up to tile - 2: with the tiles alternating between two barriers, the
         // phase waited for is then never a whole lap behind its barrier
         const int need = max(hist[0], cur.tile - 2);
         while (released <= need && ok) {
-          if (!fa_wait_bounded(&o_empty[released & 1], (unsigned)(released >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_O_EMPTY); ok = false; }
+          if (!mbar_wait_bounded(&o_empty[released & 1], (unsigned)(released >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_O_EMPTY); ok = false; }
           ++released;
         }
         if (!ok) break;
@@ -400,7 +376,7 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         int ok = 1;
         if (lane == 0) {
           ok = *abort_flag ? 0 : 1;
-          if (ok && !fa_wait_bounded(&o_full[g & 1], (unsigned)(g >> 1) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_O_FULL); ok = 0; }
+          if (ok && !mbar_wait_bounded(&o_full[g & 1], (unsigned)(g >> 1) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_O_FULL); ok = 0; }
           if (!ok) *abort_flag = 1;
         }
         if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
@@ -501,7 +477,7 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         int ok = 1;
         if (lane == 0) {
           ok = *abort_flag ? 0 : 1;
-          if (ok && !fa_wait_bounded(&s_full[buf], (unsigned)(b / NBUF) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
+          if (ok && !mbar_wait_bounded(&s_full[buf], (unsigned)(b / NBUF) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
           if (!ok) *abort_flag = 1;
         }
         if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
@@ -780,7 +756,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       int fix_issued = 0;                         // items whose resident group has been requested
       auto load_resident = [&](int item) {
         const int sh = item / p.nq, h = sh % p.H, seq = sh / p.H, tile = item - sh * p.nq;
-        if (!fa_wait_bounded(&fix_empty[fs], (unsigned)fph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; return; }
+        if (!mbar_wait_bounded(&fix_empty[fs], (unsigned)fph ^ 1u, WAIT_NS)) { fa_timeout(SITE_KV_EMPTY); ok = false; return; }
         mbar_expect_tx(&fix_full[fs], FIXB);
         uint8_t* dst = base + pl.fix_off + fs * FIXB;
         load_pair(dst, MODE == BW_DQ, h, tile, seq, &fix_full[fs]);
@@ -794,7 +770,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         const bool first = it.first();
         if (first && fix_issued <= it.k) load_resident(it.item);
         if (!ok) break;
-        if (!fa_wait_bounded(&str_empty[ss], (unsigned)sph ^ 1u, WAIT_NS)) { fa_timeout(SITE_Q_EMPTY); ok = false; break; }
+        if (!mbar_wait_bounded(&str_empty[ss], (unsigned)sph ^ 1u, WAIT_NS)) { fa_timeout(SITE_Q_EMPTY); ok = false; break; }
         mbar_expect_tx(&str_full[ss], PAIR);
         load_pair(base + pl.str_off + ss * PAIR, MODE == BW_DKV, h, it.stile(shp), seq, &str_full[ss]);
         if (++ss == C::STR_STAGES) { ss = 0; sph ^= 1; }
@@ -834,8 +810,8 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       pos_init(ps); pos_init(pd); pos_init(pc);
       // first product of a block: scores into buffer sb.  Waits for the block's operands (first use of both).
       auto issue_scores = [&](Pos& q, int sb) {
-        if (q.it.first() && !fa_wait_bounded(&fix_full[q.fs], (unsigned)q.fph, WAIT_NS)) { fa_timeout(SITE_KV_FULL); ok = false; return; }
-        if (!fa_wait_bounded(&str_full[q.ss], (unsigned)q.sph, WAIT_NS)) { fa_timeout(SITE_Q_FULL); ok = false; return; }
+        if (q.it.first() && !mbar_wait_bounded(&fix_full[q.fs], (unsigned)q.fph, WAIT_NS)) { fa_timeout(SITE_KV_FULL); ok = false; return; }
+        if (!mbar_wait_bounded(&str_full[q.ss], (unsigned)q.sph, WAIT_NS)) { fa_timeout(SITE_Q_FULL); ok = false; return; }
         tc_fence_after();
         const uint32_t a = dfk_lo + (uint32_t)q.fs * (FIXB >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4);
         const uint32_t idesc = (q.it.stile(shp) == p.nq - 1) ? idesc_tail : idesc_full;
@@ -881,13 +857,13 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       int sb = 0, rph = 0;                      // score buffer and p_ready parity of the current block
       while (pc.it.valid(shp) && ok) {
         if (*abort_flag) { ok = false; break; }
-        if (!fa_wait_bounded(p_ready, (unsigned)rph, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
+        if (!mbar_wait_bounded(p_ready, (unsigned)rph, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
         const int k = pc.it.k;
         if (pc.it.first()) {
           // BW_DQ alternates between two accumulators: the one of item k was last read for item k - 2;
           // BW_DKV uses both accumulators for every item: wait for item k - 1
           const int prev = MODE == BW_DQ ? k - 2 : k - 1;
-          if (prev >= 0 && !fa_wait_bounded(&acc_empty[prev & 1], (unsigned)(prev >> 1) & 1u, WAIT_NS)) {
+          if (prev >= 0 && !mbar_wait_bounded(&acc_empty[prev & 1], (unsigned)(prev >> 1) & 1u, WAIT_NS)) {
             fa_timeout(SITE_O_EMPTY); ok = false; break;
           }
         }
@@ -898,7 +874,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         if (MODE == BW_DKV) {
           issue_acc(pc, acc0, dp_col, 0, fresh);                       // dK += dS^T Q_i (dS^T sits in the dP buffer)
           if (NSBUF == 2 && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }   // the dP buffer is free again: next block's dP
-          if (fresh && k >= 1 && !fa_wait_bounded(&accv_empty[(k - 1) & 1], (unsigned)((k - 1) >> 1) & 1u, WAIT_NS)) {
+          if (fresh && k >= 1 && !mbar_wait_bounded(&accv_empty[(k - 1) & 1], (unsigned)((k - 1) >> 1) & 1u, WAIT_NS)) {
             fa_timeout(SITE_O_EMPTY); ok = false; break;
           }
           issue_acc(pc, acc1, s_col, 1, fresh);                        // dV += P^T dO_i
@@ -965,7 +941,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         int ok = 1;
         if (lane == 0) {
           ok = *abort_flag ? 0 : 1;
-          if (ok && !fa_wait_bounded(&acc_full[k & 1], (unsigned)(k >> 1) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_O_FULL); ok = 0; }
+          if (ok && !mbar_wait_bounded(&acc_full[k & 1], (unsigned)(k >> 1) & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_O_FULL); ok = 0; }
           if (!ok) *abort_flag = 1;
         }
         if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
@@ -1109,7 +1085,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         int ok = 1;
         if (lane == 0) {
           ok = (dead || *abort_flag) ? 0 : 1;
-          if (ok && !fa_wait_bounded(sdp_full, (unsigned)b & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
+          if (ok && !mbar_wait_bounded(sdp_full, (unsigned)b & 1u, WAIT_NS * 2ull)) { fa_timeout(SITE_S_FULL); ok = 0; }
           if (!ok) *abort_flag = 1;
         }
         if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
