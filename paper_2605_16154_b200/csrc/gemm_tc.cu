@@ -610,6 +610,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 //   acc_full[b]  (each)    <- multicast commit from the leader's MMA thread
 //   acc_empty[b] (leader)  <- the epilogue warps of both CTAs
 // ------------------------------------------------------------------------------------------------
+// Position of a CTA pair's current tile in the (split, m, n) grid, n fastest, advanced by a fixed stride without
+// divisions: the stride is decomposed once.
+struct TileWalk {
+  int split, m, n, d_split, d_m, d_n;
+  __device__ void init(int first, int stride, int tiles_m, int tiles_n) {
+    const int tiles_mn = tiles_m * tiles_n;
+    split = first / tiles_mn;
+    int r = first - split * tiles_mn;
+    m = r / tiles_n; n = r - m * tiles_n;
+    d_split = stride / tiles_mn;
+    r = stride - d_split * tiles_mn;
+    d_m = r / tiles_n; d_n = r - d_m * tiles_n;
+  }
+  __device__ void next(int tiles_m, int tiles_n) {
+    n += d_n;
+    if (n >= tiles_n) { n -= tiles_n; ++m; }
+    m += d_m;
+    if (m >= tiles_m) { m -= tiles_m; ++split; }
+    split += d_split;
+  }
+};
+
 constexpr int T2_BN = 256;
 constexpr int T2_STAGES = 5;
 constexpr int T2_A_BYTES = TC_BM * TC_BK * 2;          // 16 KB: this CTA's 128 rows of A
@@ -662,20 +684,24 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   if (warp == 0) {
     if (lane == 0) {
       // ------------------------------ TMA producer (both CTAs) ------------------------------
-      unsigned it = 0;
-      for (int tile = pair; tile < total_tiles && !*abort_flag; tile += n_pairs) {
-        const int split = tile / tiles_mn, mn = tile - split * tiles_mn;
-        const int m0 = (mn / p.tiles_n) * (2 * TC_BM) + (int)rank * TC_BM;      // this CTA's rows
-        const int n0 = (mn % p.tiles_n) * BN;
+      // One thread: ring positions and the tile walk are kept as counters (no division or modulo per k-block), so
+      // that a k-block costs it less than the 512 tensor-core cycles the block's four MMAs take.
+      const uint32_t bar0 = mapa_shared(smem_u32(&full[0]), 0);               // the leader's barriers count both CTAs' bytes
+      TileWalk tw;
+      tw.init(pair, n_pairs, p.tiles_m, p.tiles_n);
+      int st = 0;
+      unsigned ph = 0;
+      bool ok = true;
+      for (int tile = pair; tile < total_tiles && ok && !*abort_flag; tile += n_pairs, tw.next(p.tiles_m, p.tiles_n)) {
+        const int m0 = tw.m * (2 * TC_BM) + (int)rank * TC_BM;                  // this CTA's rows
+        const int n0 = tw.n * BN;
         const int nb0 = n0 + (int)rank * (BN / 2);                              // this CTA's columns of B
-        const int kb_lo = split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
-        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
-          const int st = it % T2_STAGES;
-          const unsigned ph = (it / T2_STAGES) & 1u;
-          if (!mbar_wait_bounded(&empty[st], ph ^ 1u, TC_WAIT_LIMIT_NS)) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); break; }
+        const int kb_lo = tw.split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
+          if (!mbar_wait_bounded(&empty[st], ph ^ 1u, TC_WAIT_LIMIT_NS)) { ok = false; break; }
           uint8_t* sa = tiles + st * T2_STAGE_BYTES;
           uint8_t* sb = sa + T2_A_BYTES;
-          const uint32_t bar = mapa_shared(smem_u32(&full[st]), 0);             // the leader's barrier counts both CTAs' bytes
+          const uint32_t bar = bar0 + (uint32_t)st * 8u;
           if (leader) mbar_expect_tx(&full[st], 2 * T2_STAGE_BYTES);
           const int k0 = kb * TC_BK;
           if (p.a_kmajor) {
@@ -693,40 +719,50 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
             for (int b = 0; b < 2; ++b) tma_load_2d_pair(sb + b * 8192, &tmB, nb0 + b * 64, k0, bar);
           }
+          if (++st == T2_STAGES) { st = 0; ph ^= 1u; }
         }
       }
+      if (!ok) { *abort_flag = 1; atomicOr(&g_tc_status, 1u); }
     }
   } else if (warp == 1) {
     if (lane == 0 && leader) {
       // ------------------------------ MMA issuer (leader CTA only) ------------------------------
+      // The four MMAs of a k-block take 512 tensor-core cycles; this thread must spend less than that per k-block
+      // (a poll of an already completed barrier alone costs about 125 cycles).  Descriptors are therefore built once
+      // and advanced by adding constants to their low word, and the ring position is a counter.
       constexpr uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                                       ((uint32_t)((2 * TC_BM) >> 4) << 24);
       const uint32_t idesc = idesc_base | ((p.a_kmajor ? 0u : 1u) << 15) | ((p.b_kmajor ? 0u : 1u) << 16);
       const uint32_t a_lbo = p.a_kmajor ? 16u : 8192u, b_lbo = p.b_kmajor ? 16u : 8192u;
-      const uint32_t a_step = p.a_kmajor ? 32u : 2048u, b_step = p.b_kmajor ? 32u : 2048u;
-      unsigned it = 0, tcount = 0;
+      const uint32_t a_step16 = (p.a_kmajor ? 32u : 2048u) >> 4, b_step16 = (p.b_kmajor ? 32u : 2048u) >> 4;
+      const uint64_t da0 = make_smem_desc(smem_u32(tiles), a_lbo, 1024u);
+      const uint64_t db0 = make_smem_desc(smem_u32(tiles) + T2_A_BYTES, b_lbo, 1024u);
+      const uint32_t da_hi = (uint32_t)(da0 >> 32), db_hi = (uint32_t)(db0 >> 32);
+      const uint32_t da_lo = (uint32_t)da0, db_lo = (uint32_t)db0;
+      auto desc = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; };
+      TileWalk tw;
+      tw.init(pair, n_pairs, p.tiles_m, p.tiles_n);
+      unsigned tcount = 0, ph = 0;
+      int st = 0;
+      uint32_t st_off = 0;                       // st * stage bytes, in descriptor units of 16 bytes
       bool ok = true;
-      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++tcount) {
-        const int split = tile / tiles_mn;
-        const int kb_lo = split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++tcount, tw.next(p.tiles_m, p.tiles_n)) {
+        const int kb_lo = tw.split * p.kb_per_split, kb_hi = min(kb_lo + p.kb_per_split, num_kb_total);
         const unsigned ab = tcount & 1u, aph = (tcount >> 1) & 1u;
         if (*abort_flag || !mbar_wait_bounded(&acc_empty[ab], aph ^ 1u, TC_WAIT_LIMIT_NS)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_acc = tmem_base + ab * BN;
-        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
-          const int st = it % T2_STAGES;
-          const unsigned ph = (it / T2_STAGES) & 1u;
-          if (*abort_flag || !mbar_wait_bounded(&full[st], ph, TC_WAIT_LIMIT_NS)) { ok = false; break; }
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
+          if (!mbar_wait_bounded(&full[st], ph, TC_WAIT_LIMIT_NS)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_u32(tiles + st * T2_STAGE_BYTES);
-          const uint32_t sb = sa + T2_A_BYTES;
+          const uint32_t alo = da_lo + st_off, blo = db_lo + st_off;
+          umma_bf16_pair(tmem_acc, desc(alo, da_hi), desc(blo, db_hi), idesc, kb > kb_lo ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < TC_BK / 16; ++k) {
-            const uint64_t da = make_smem_desc(sa + k * a_step, a_lbo, 1024u);
-            const uint64_t db = make_smem_desc(sb + k * b_step, b_lbo, 1024u);
-            umma_bf16_pair(tmem_acc, da, db, idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
-          }
+          for (int k = 1; k < TC_BK / 16; ++k)
+            umma_bf16_pair(tmem_acc, desc(alo + k * a_step16, da_hi), desc(blo + k * b_step16, db_hi), idesc, 1u);
           umma_commit_pair(&empty[st], 3);     // both CTAs may refill the stage
+          st_off += T2_STAGE_BYTES >> 4;
+          if (++st == T2_STAGES) { st = 0; st_off = 0; ph ^= 1u; }
         }
         if (ok) umma_commit_pair(&acc_full[ab], 3);
       }
