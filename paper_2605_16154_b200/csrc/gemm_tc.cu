@@ -637,10 +637,12 @@ constexpr int T2_STAGES = 5;
 constexpr int T2_A_BYTES = TC_BM * TC_BK * 2;          // 16 KB: this CTA's 128 rows of A
 constexpr int T2_B_BYTES = (T2_BN / 2) * TC_BK * 2;    // 16 KB: this CTA's 128 columns of B
 constexpr int T2_STAGE_BYTES = T2_A_BYTES + T2_B_BYTES;
+constexpr int T2_PRODUCER_B_WARP = 10;               // after the eight epilogue warps 2..9
+constexpr int T2_THREADS = TC_THREADS + 32;
 constexpr int T2_SMEM_TOTAL = T2_STAGES * T2_STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES;   // ring + slack + barriers + epilogue staging
 
 template <int EPI>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(T2_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int BN = T2_BN;
@@ -681,11 +683,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == T2_PRODUCER_B_WARP) {
     if (lane == 0) {
-      // ------------------------------ TMA producer (both CTAs) ------------------------------
-      // One thread: ring positions and the tile walk are kept as counters (no division or modulo per k-block), so
-      // that a k-block costs it less than the 512 tensor-core cycles the block's four MMAs take.
+      // ------------------------------ TMA producers (both CTAs) ------------------------------
+      // Two threads per CTA, one per operand (warp 0: A, warp 10: B): a TMA issue costs its thread about a hundred
+      // cycles, and a k-block must cost each producer well under the 512 tensor-core cycles it feeds.  Ring positions
+      // and the tile walk are counters (no division or modulo per k-block).
+      const bool load_a = warp == 0;
       const uint32_t bar0 = mapa_shared(smem_u32(&full[0]), 0);               // the leader's barriers count both CTAs' bytes
       TileWalk tw;
       tw.init(pair, n_pairs, p.tiles_m, p.tiles_n);
@@ -702,15 +706,16 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           uint8_t* sa = tiles + st * T2_STAGE_BYTES;
           uint8_t* sb = sa + T2_A_BYTES;
           const uint32_t bar = bar0 + (uint32_t)st * 8u;
-          if (leader) mbar_expect_tx(&full[st], 2 * T2_STAGE_BYTES);
           const int k0 = kb * TC_BK;
-          if (p.a_kmajor) {
-            tma_load_2d_pair(sa, &tmA, k0, m0, bar);                            // box {64 k, 128 m}
-          } else {
+          if (load_a) {
+            if (leader) mbar_expect_tx(&full[st], 2 * T2_STAGE_BYTES);
+            if (p.a_kmajor) {
+              tma_load_2d_pair(sa, &tmA, k0, m0, bar);                          // box {64 k, 128 m}
+            } else {
 #pragma unroll
-            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sa + b * 8192, &tmA, m0 + b * 64, k0, bar);   // box {64 m, 64 k}
-          }
-          if (EPI == EPI_SWIGLU_FWD) {
+              for (int b = 0; b < 2; ++b) tma_load_2d_pair(sa + b * 8192, &tmA, m0 + b * 64, k0, bar);   // box {64 m, 64 k}
+            }
+          } else if (EPI == EPI_SWIGLU_FWD) {
             // accumulator columns [0,128) = gate (leader's half of B), [128,256) = up (the peer's half)
             tma_load_2d_pair(sb, &tmB, k0, (leader ? 0 : p.up_row0) + n0 / 2, bar);                 // box {64 k, 128 n}
           } else if (p.b_kmajor) {
@@ -963,7 +968,7 @@ static int launch_tc2(const GemmArgs& g, cudaStream_t s) {
   const int pairs = (int)(total < n_pairs_max ? total : n_pairs_max);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
-  cfg.blockDim = dim3(TC_THREADS);
+  cfg.blockDim = dim3(T2_THREADS);
   cfg.dynamicSmemBytes = T2_SMEM_TOTAL;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
