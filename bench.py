@@ -24,9 +24,9 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 # DRAM traffic of the dominant kernel from one ncu capture (profiles/gemm_tc2_kernel_M19968_N3072_K1024_ncu.md):
-# dram__bytes_read.sum + dram__bytes_write.sum = 120.1 MB for the QKV-shaped launch at M = 19968 rows against
+# dram__bytes_read.sum + dram__bytes_write.sum = 119.6 MB for the QKV-shaped launch at M = 19968 rows against
 # 169.9 MB of algorithmic bytes; traffic grows in proportion to the rows for a fixed weight matrix.
-GEMM_TRAFFIC_CAPTURE = {"rows": 19968, "n": 3072, "k": 1024, "dram_bytes": 120.1e6, "algorithmic_bytes": 169.9e6}
+GEMM_TRAFFIC_CAPTURE = {"rows": 19968, "n": 3072, "k": 1024, "dram_bytes": 119.6e6, "algorithmic_bytes": 169.9e6}
 
 METRIC = "kept_chunks_per_s_actor_fwd_bwd"
 UNIT = "chunks/s"
