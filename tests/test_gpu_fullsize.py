@@ -113,3 +113,33 @@ def test_eight_chunk_update_of_the_full_model_against_the_oracle(c1):
     assert max(errs.values()) < 2e-2, (errs, float(loss.item()), loss_o)
     assert abs(float(loss.item()) - loss_o) < 1e-3
     assert stats.clip_frac == pytest.approx(stats_o["clip_frac"], abs=1e-6)
+
+
+def test_attention_at_the_full_batch_shape_on_sampled_sequences_and_heads():
+    """grpo_attention on the shape one C1 layer runs (384 sequences of 312 tokens, 16 heads of 64: every CTA of the
+    persistent kernels walks about 40 items); forward and backward checked against the oracle on sampled
+    (sequence, head) pairs, which are independent problems."""
+    from paper_2605_16154_b200 import binding as B, pipeline as PL
+    n_seq, S, H, dh = 384, 312, 16, 64
+    d = H * dh
+    g = torch.Generator(device="cuda").manual_seed(3)
+    qkv = torch.randn((n_seq * S, 3 * d), generator=g, device="cuda").to(torch.bfloat16)
+    do = torch.randn((n_seq * S, d), generator=g, device="cuda").to(torch.bfloat16)
+    out, lse, dqkv = B.grpo_attention(qkv, n_seq, S, H, dh, dout=do)
+    rng = np.random.default_rng(0)
+    picks = [(0, 0), (n_seq - 1, H - 1), (147, 5), (148, 6)] + [(int(rng.integers(n_seq)), int(rng.integers(H))) for _ in range(8)]
+    for s_i, h_i in picks:
+        rows = slice(s_i * S, (s_i + 1) * S)
+        cols = lambda part: slice(part * d + h_i * dh, part * d + (h_i + 1) * dh)
+        blk = qkv[rows].float().cpu().numpy().astype(np.float64)
+        q, k, v = (blk[:, cols(i)][None, None] for i in range(3))
+        o, p = ao.causal_attention(q, k, v)
+        go = do[rows, h_i * dh:(h_i + 1) * dh].float().cpu().numpy().astype(np.float64)[None, None]
+        dq, dk, dv = ao.causal_attention_bwd(go, q, k, v, p)
+        got = dqkv[rows].float().cpu().numpy()
+        assert rel_fro(out[rows, h_i * dh:(h_i + 1) * dh].float().cpu().numpy(), o[0, 0]) < 1e-2, (s_i, h_i)
+        assert rel_fro(got[:, cols(0)], dq[0, 0]) < 2e-2, (s_i, h_i)
+        assert rel_fro(got[:, cols(1)], dk[0, 0]) < 2e-2, (s_i, h_i)
+        assert rel_fro(got[:, cols(2)], dv[0, 0]) < 2e-2, (s_i, h_i)
+        lse_o = np.log(np.exp(q[0, 0] @ k[0, 0].T / np.sqrt(dh) + np.triu(np.full((S, S), -np.inf), 1)).sum(-1))
+        assert np.max(np.abs(lse[s_i, h_i].cpu().numpy() - lse_o)) < 2e-2, (s_i, h_i)
