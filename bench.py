@@ -340,7 +340,7 @@ def run_cuda(args):
             "config": {"workload": w.name, "kept_chunks_per_step": n_kept, "chunks_per_step": total,
                        "tokens_per_step": n_kept * w.S, "mb_chunks": mb, "l2": "inputs_larger_than_l2",
                        "multi_gpu": "independent replicas, no collective"},
-            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "tensor", "kernel": "gemm_tc2_kernel", "achieved": achieved, "peak": peak,
                          "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
                          "traffic": GEMM_TRAFFIC_CAPTURE["dram_bytes"] * (n_kept * w.S) / GEMM_TRAFFIC_CAPTURE["rows"]
                          if (w.d == 1024 and mb >= n_kept) else None,
