@@ -1,6 +1,7 @@
-// bf16 causal attention inside each chunk's sequence on the 5th-generation tensor cores (forward).
+// bf16 causal attention inside each chunk's sequence on the 5th-generation tensor cores: the forward pass
+// (described here) and, further down, the backward pass (one kernel template launched for dQ and for dK / dV).
 //
-// One persistent CTA per SM walks (sequence, head) items.  The whole K and V of an item (S <= 384 rows)
+// Forward.  One persistent CTA per SM walks (sequence, head) items.  The whole K and V of an item (S <= 384 rows)
 // sit in shared memory (TMA, 128-byte swizzle); query tiles of 128 rows stream through a small ring.
 // A query tile is processed as independent blocks of 128 keys (causal: the blocks at or left of the
 // diagonal).  For block j, tcgen05.mma puts S_j = Q K_j^T (128 x 128, fp32) into one of the score
