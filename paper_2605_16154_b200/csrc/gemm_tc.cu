@@ -950,11 +950,21 @@ static int launch_tc2(const GemmArgs& g, cudaStream_t s) {
   const int n_pairs_max = sm_count() / 2;
   int splits = 1;
   if (p.reduce) {
+    // Split the contraction so that the work items fill whole waves of CTA pairs: with tiles x splits items on
+    // n_pairs_max pairs, ceil(items / pairs) waves run and the last one is as long as the others.  Among the
+    // candidates (at least 8 k-blocks per split) take the fullest waves, charging each extra split a little for its
+    // fp32 reduction traffic.
     const long long tiles = (long long)tiles_m * tiles_n;
-    long long want = (2 * n_pairs_max + tiles - 1) / tiles;
-    long long cap = num_kb / 8 > 0 ? num_kb / 8 : 1;
-    splits = (int)(want < cap ? want : cap);
-    if (splits < 1) splits = 1;
+    const int cap = num_kb / 8 > 0 ? (num_kb / 8 < 32 ? num_kb / 8 : 32) : 1;
+    double best = -1.0;
+    for (int cand = 1; cand <= cap; ++cand) {
+      const int per = (num_kb + cand - 1) / cand;
+      const int actual = (num_kb + per - 1) / per;                 // no empty split
+      const long long items = tiles * actual;
+      const long long waves = (items + n_pairs_max - 1) / n_pairs_max;
+      const double score = (double)items / (double)(waves * n_pairs_max) - 0.004 * actual;
+      if (score > best) { best = score; splits = actual; }
+    }
   }
   p.kb_per_split = (num_kb + splits - 1) / splits;
   splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;
