@@ -107,7 +107,7 @@ rmsnorm_fwd_kernel(const float* __restrict__ x, const T* __restrict__ gamma, T* 
 // ------------------------------------------------------------------------------------------------
 // RMSNorm backward.  dy fp32 [rows][d]; x fp32 (rows optionally gathered); dx_out = dx_in + dx is
 // written through the same row map, in fp32 and in T.  Per-CTA partial sums of
-// dgamma = sum_rows dy * x * rstd go to part[blockIdx][d]; a second kernel adds them up in order.
+// dgamma = sum_rows dy * x * rstd go to part[blockIdx][d]; a second kernel adds them up in a fixed order.
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -163,13 +163,25 @@ rmsnorm_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ x, co
   }
 }
 
-// out[c] += sum_b part[b][c] in ascending b
-__global__ void colsum_accumulate_kernel(const float* __restrict__ part, int nblk, int d, float* __restrict__ out) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= d) return;
+// out[c] += sum_b part[b][c].  A CTA takes 32 columns; its eight warps each add every eighth row in ascending order
+// (coalesced 128-byte reads), and the eight partial sums are then added in warp order: a fixed association, so the
+// result does not depend on timing.
+__global__ void __launch_bounds__(256)
+colsum_accumulate_kernel(const float* __restrict__ part, int nblk, int d, float* __restrict__ out) {
+  __shared__ float red[8][32];
+  const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
   float s = 0.f;
-  for (int b = 0; b < nblk; ++b) s += part[(size_t)b * d + c];
-  out[c] += s;
+  if (c < d)
+    for (int b = slice; b < nblk; b += 8) s += part[(size_t)b * d + c];
+  red[slice][lane] = s;
+  __syncthreads();
+  if (slice == 0 && c < d) {
+    float t = red[0][lane];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) t += red[w][lane];
+    out[c] += t;
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -682,7 +694,7 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
                                                        d, mS, mP);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)rows * d * ((dx_in ? 16.0 : 12.0) + es));
-      colsum_accumulate_kernel<<<ceil_div(d, 256), 256, 0, s>>>(w.norm_part, blocks, d, dgamma);
+      colsum_accumulate_kernel<<<ceil_div(d, 32), 256, 0, s>>>(w.norm_part, blocks, d, dgamma);
       PCM_LAUNCH_CHECK();
       return PCM_OK;
     };
