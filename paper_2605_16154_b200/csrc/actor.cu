@@ -105,13 +105,13 @@ rmsnorm_fwd_kernel(const float* __restrict__ x, const T* __restrict__ gamma, T* 
 }
 
 // ------------------------------------------------------------------------------------------------
-// RMSNorm backward.  dy fp32 [rows][d]; x fp32 (rows optionally gathered); dx_out = dx_in + dx is
+// RMSNorm backward.  dy [rows][d] in fp32 or in the activation type T; x fp32 (rows optionally gathered); dx_out = dx_in + dx is
 // written through the same row map, in fp32 and in T.  Per-CTA partial sums of
 // dgamma = sum_rows dy * x * rstd go to part[blockIdx][d]; a second kernel adds them up in a fixed order.
 // ------------------------------------------------------------------------------------------------
-template <typename T>
+template <typename T, typename DY>
 __global__ void __launch_bounds__(256)
-rmsnorm_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ rstd,
+rmsnorm_bwd_kernel(const DY* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ rstd,
                    const T* __restrict__ gamma, const float* dx_in, float* dx_out, T* __restrict__ dx_out_t,
                    float* __restrict__ part, long long rows, int d, int map_S, int map_P) {
   extern __shared__ float red[];                         // [8 warps][d]
@@ -122,23 +122,23 @@ rmsnorm_bwd_kernel(const float* __restrict__ dy, const float* __restrict__ x, co
   for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
     const long long xr_i = map_row(r, map_S, map_P);
     const float* xr = x + xr_i * d;
-    const float* dyr = dy + r * d;
+    const DY* dyr = dy + r * d;
     const float rs = rstd[r];
     float dot = 0.f;
     for (int c = lane * 4; c < d; c += 128) {
       const float4 xv = *reinterpret_cast<const float4*>(xr + c);
-      const float4 gv = *reinterpret_cast<const float4*>(dyr + c);
-      float gm[4];
+      float gm[4], gy[4];
+      load4<DY>(dyr + c, gy);
       load4<T>(gamma + c, gm);
-      dot += gv.x * gm[0] * xv.x + gv.y * gm[1] * xv.y + gv.z * gm[2] * xv.z + gv.w * gm[3] * xv.w;
+      dot += gy[0] * gm[0] * xv.x + gy[1] * gm[1] * xv.y + gy[2] * gm[2] * xv.z + gy[3] * gm[3] * xv.w;
     }
     dot = warp_sum(dot);
     const float coef = dot * rs * rs * rs / (float)d;    // mean(dn * n) * rstd, with n = x * rstd
     for (int c = lane * 4; c < d; c += 128) {
       const float4 xv = *reinterpret_cast<const float4*>(xr + c);
-      const float4 gv = *reinterpret_cast<const float4*>(dyr + c);
       const float xa[4] = {xv.x, xv.y, xv.z, xv.w};
-      const float ga[4] = {gv.x, gv.y, gv.z, gv.w};
+      float ga[4];
+      load4<DY>(dyr + c, ga);
       float o[4], gm[4];
       load4<T>(gamma + c, gm);
 #pragma unroll
@@ -685,20 +685,28 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     PCM_CUDA_TRY(cudaMemsetAsync(w.dx_t, 0, (size_t)M * d * sizeof(T), s));
     const size_t nb_smem = (size_t)8 * d * sizeof(float);
     if (nb_smem > 48 * 1024)
-      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
-    auto norm_bwd = [&](const float* dy, const float* x, const float* rstd, const T* gamma, const float* dx_in,
+    {
+      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
+      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
+    }
+    // dy_is_t: the incoming gradient is stored in the activation type (the per-layer dh), else in fp32
+    auto norm_bwd = [&](const void* dy, bool dy_is_t, const float* x, const float* rstd, const T* gamma, const float* dx_in,
                         long long rows, int mS, int mP, float* dgamma) -> int {
       const int blocks = (int)(rows / 8 + 1 < NORM_BWD_BLOCKS ? rows / 8 + 1 : NORM_BWD_BLOCKS);
       prof_begin(PC_NORM, s);
-      rmsnorm_bwd_kernel<T><<<blocks, 256, nb_smem, s>>>(dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t, w.norm_part, rows,
-                                                       d, mS, mP);
+      if (dy_is_t)
+        rmsnorm_bwd_kernel<T, T><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t, w.norm_part,
+                                                               rows, d, mS, mP);
+      else
+        rmsnorm_bwd_kernel<T, float><<<blocks, 256, nb_smem, s>>>((const float*)dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t,
+                                                                   w.norm_part, rows, d, mS, mP);
       PCM_LAUNCH_CHECK();
-      prof_end(s, 0.0, (double)rows * d * ((dx_in ? 16.0 : 12.0) + es));
+      prof_end(s, 0.0, (double)rows * d * ((dx_in ? 12.0 : 8.0) + (dy_is_t ? es : 4.0) + es));
       colsum_accumulate_kernel<<<ceil_div(d, 32), 256, 0, s>>>(w.norm_part, blocks, d, dgamma);
       PCM_LAUNCH_CHECK();
       return PCM_OK;
     };
-    TRY(norm_bwd(w.dhs, w.x[L], w.rstdf, gf, nullptr, R, S, P, gr->gf));
+    TRY(norm_bwd(w.dhs, false, w.x[L], w.rstdf, gf, nullptr, R, S, P, gr->gf));
 
     for (int l = L - 1; l >= 0; --l) {
       LayerActs& la = w.la[l];
@@ -719,8 +727,8 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       }
       TRY(G(8 * d, d, Mi, w.dgu, 8 * d, false, la.h2, d, false, dt, gr->w_gu + l * 8 * dd, d, DT_F32,
             gr->w_gu + l * 8 * dd, d));
-      TRY(G(Mi, d, 8 * d, w.dgu, 8 * d, true, w_gu + l * 8 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
-      TRY(norm_bwd(w.dh, la.x_mid, la.rstd2, g2 + (size_t)l * d, w.dx, M, 0, 0, gr->g2 + (size_t)l * d));
+      TRY(G(Mi, d, 8 * d, w.dgu, 8 * d, true, w_gu + l * 8 * dd, d, false, dt, w.dh, d, dt, nullptr, 0));
+      TRY(norm_bwd(w.dh, true, la.x_mid, la.rstd2, g2 + (size_t)l * d, w.dx, M, 0, 0, gr->g2 + (size_t)l * d));
       // attention block: x_mid = x_in + attn W_o^T
       TRY(G(d, d, Mi, w.dx_t, d, false, la.attn, d, false, dt, gr->w_o + l * dd, d, DT_F32, gr->w_o + l * dd, d));
       TRY(G(Mi, d, d, w.dx_t, d, true, w_o + l * dd, d, false, dt, w.dattn, d, dt, nullptr, 0));
@@ -736,8 +744,8 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       }
       TRY(G(3 * d, d, Mi, w.dqkv, 3 * d, false, la.h1, d, false, dt, gr->w_qkv + l * 3 * dd, d, DT_F32,
             gr->w_qkv + l * 3 * dd, d));
-      TRY(G(Mi, d, 3 * d, w.dqkv, 3 * d, true, w_qkv + l * 3 * dd, d, false, dt, w.dh, d, DT_F32, nullptr, 0));
-      TRY(norm_bwd(w.dh, w.x[l], la.rstd1, g1 + (size_t)l * d, w.dx, M, 0, 0, gr->g1 + (size_t)l * d));
+      TRY(G(Mi, d, 3 * d, w.dqkv, 3 * d, true, w_qkv + l * 3 * dd, d, false, dt, w.dh, d, dt, nullptr, 0));
+      TRY(norm_bwd(w.dh, true, w.x[l], la.rstd1, g1 + (size_t)l * d, w.dx, M, 0, 0, gr->g1 + (size_t)l * d));
     }
     prof_begin(PC_EMBED, s);
     embed_grad_kernel<<<dim3(NB, ceil_div(d, 256)), 256, 0, s>>>(w.dx, tgt, mb, S, P, d, gr->e_act);
