@@ -1228,6 +1228,15 @@ static bool make_seq_tmap(CUtensorMap* tm, const void* base, int n_seq, int S, l
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// cudaFuncSetAttribute applies to the current device: remember per function which devices already have it
+static bool attr_needed(unsigned long long* seen_mask) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+  if (*seen_mask & (1ull << dev)) return false;
+  *seen_mask |= 1ull << dev;
+  return true;
+}
+
 static int attn_sm_count() {
   static int n = 0;
   if (!n) {
@@ -1265,11 +1274,9 @@ static int fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int S, 
     return PCM_ERR_CUDA;
   CUtensorMap tmO;
   if (!make_seq_tmap(&tmO, out, n_seq, S, d, d, BM)) return PCM_ERR_CUDA;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_devices = 0;
+  if (attr_needed(&attr_devices))
     PCM_CUDA_TRY(cudaFuncSetAttribute(fa_tc_fwd_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT));
-    attr_done = true;
-  }
   const int grid = p.n_items < attn_sm_count() ? p.n_items : attn_sm_count();
   fa_tc_fwd_kernel<DH><<<grid, Cfg<DH>::THREADS, smem, s>>>(tmQ, tmKV, tmO, p);
   PCM_LAUNCH_CHECK();
@@ -1283,11 +1290,9 @@ static int bwd_launch_one(const CUtensorMap& tmQKV, const CUtensorMap& tmDO, con
   const BwPlan pl = bw_make_plan<DH, MODE>();
   if (pl.total > SMEM_LIMIT) return PCM_ERR_SHAPE;
   const uint32_t smem = pl.total < SMEM_FLOOR ? SMEM_FLOOR : pl.total;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_devices = 0;
+  if (attr_needed(&attr_devices))
     PCM_CUDA_TRY(cudaFuncSetAttribute(fa_tc_bwd_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT));
-    attr_done = true;
-  }
   const int grid = p.n_items < attn_sm_count() ? p.n_items : attn_sm_count();
   fa_tc_bwd_kernel<DH, MODE><<<grid, BW_THREADS, smem, s>>>(tmQKV, tmDO, tmOUT, tmDQKV, p);
   PCM_LAUNCH_CHECK();
