@@ -877,6 +877,15 @@ static void fill_params(TcParams& p, const GemmArgs& g) {
   p.kb_per_split = 1; p.tiles_m = p.tiles_n = p.splits = 1;
 }
 
+// cudaFuncSetAttribute applies to the current device: remember per function which devices already have it
+static bool attr_needed(unsigned long long* seen_mask) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+  if (*seen_mask & (1ull << dev)) return false;
+  *seen_mask |= 1ull << dev;
+  return true;
+}
+
 static int sm_count() {
   static int n = 0;
   if (!n) {
@@ -912,11 +921,9 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   }
   p.kb_per_split = (num_kb + splits - 1) / splits;
   splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;          // no empty split
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_devices = 0;
+  if (attr_needed(&attr_devices))
     PCM_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<BN>::TOTAL));
-    attr_done = true;
-  }
   p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits;
   const long long total = (long long)tiles_m * tiles_n * splits;
   const int grid = (int)(total < sm_count() ? total : sm_count());      // persistent: one CTA per SM walks the tile list
@@ -969,11 +976,9 @@ static int launch_tc2(const GemmArgs& g, cudaStream_t s) {
   p.kb_per_split = (num_kb + splits - 1) / splits;
   splits = (num_kb + p.kb_per_split - 1) / p.kb_per_split;
   p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static unsigned long long attr_devices = 0;
+  if (attr_needed(&attr_devices))
     PCM_CUDA_TRY(cudaFuncSetAttribute(gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, T2_SMEM_TOTAL));
-    attr_done = true;
-  }
   const long long total = (long long)tiles_m * tiles_n * splits;
   const int pairs = (int)(total < n_pairs_max ? total : n_pairs_max);
   cudaLaunchConfig_t cfg = {};
