@@ -163,6 +163,76 @@ rmsnorm_bwd_kernel(const DY* __restrict__ dy, const float* __restrict__ x, const
   }
 }
 
+// The same for d = 128 NV with the whole row in registers: every load of a row (x, dy, the incoming residual
+// gradient) is issued before the first use, nothing is read twice, gamma and the dgamma partial sums of this lane's
+// columns stay in registers for the life of the CTA.  Fewer, fatter warps: the kernel is HBM-bound and needs bytes
+// in flight, not occupancy.
+template <typename T, typename DY, int NV>
+__global__ void __launch_bounds__(256)
+rmsnorm_bwd_rows_kernel(const DY* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ rstd,
+                        const T* __restrict__ gamma, const float* dx_in, float* dx_out, T* __restrict__ dx_out_t,
+                        float* __restrict__ part, long long rows, int map_S, int map_P) {
+  constexpr int d = NV * 128;
+  extern __shared__ float red[];                         // [8 warps][d]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float gm[NV][4], acc[NV][4];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    load4<T>(gamma + k * 128 + lane * 4, gm[k]);
+    acc[k][0] = acc[k][1] = acc[k][2] = acc[k][3] = 0.f;
+  }
+  for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
+    const long long xr_i = map_row(r, map_S, map_P);
+    const float* xr = x + xr_i * d + lane * 4;
+    const DY* dyr = dy + r * d + lane * 4;
+    float4 xv[NV], pv[NV];
+    float gy[NV][4];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      xv[k] = *reinterpret_cast<const float4*>(xr + k * 128);
+      load4<DY>(dyr + k * 128, gy[k]);
+    }
+    if (dx_in) {
+#pragma unroll
+      for (int k = 0; k < NV; ++k) pv[k] = *reinterpret_cast<const float4*>(dx_in + xr_i * d + lane * 4 + k * 128);
+    } else {
+#pragma unroll
+      for (int k = 0; k < NV; ++k) pv[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const float rs = rstd[r];
+    float dot = 0.f;
+#pragma unroll
+    for (int k = 0; k < NV; ++k)
+      dot += gy[k][0] * gm[k][0] * xv[k].x + gy[k][1] * gm[k][1] * xv[k].y + gy[k][2] * gm[k][2] * xv[k].z +
+             gy[k][3] * gm[k][3] * xv[k].w;
+    dot = warp_sum(dot);
+    const float coef = dot * rs * rs * rs / (float)d;    // mean(dn * n) * rstd, with n = x * rstd
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      const float xa[4] = {xv[k].x, xv[k].y, xv[k].z, xv[k].w};
+      const float pa[4] = {pv[k].x, pv[k].y, pv[k].z, pv[k].w};
+      float o[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        o[e] = rs * gy[k][e] * gm[k][e] - coef * xa[e] + pa[e];
+        acc[k][e] += gy[k][e] * xa[e] * rs;
+      }
+      *reinterpret_cast<float4*>(dx_out + xr_i * d + lane * 4 + k * 128) = make_float4(o[0], o[1], o[2], o[3]);
+      store4<T>(dx_out_t + xr_i * d + lane * 4 + k * 128, o[0], o[1], o[2], o[3]);
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < NV; ++k)
+    *reinterpret_cast<float4*>(red + (size_t)warp * d + k * 128 + lane * 4) = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+  __syncthreads();
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += red[(size_t)w * d + c];
+    part[(size_t)blockIdx.x * d + c] = s;
+  }
+}
+
 // out[c] += sum_b part[b][c].  A CTA takes 32 columns; its eight warps each add every eighth row in ascending order
 // (coalesced 128-byte reads), and the eight partial sums are then added in warp order: a fixed association, so the
 // result does not depend on timing.
@@ -688,13 +758,17 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     {
       PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
       PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
+      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_rows_kernel<T, T, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
     }
     // dy_is_t: the incoming gradient is stored in the activation type (the per-layer dh), else in fp32
     auto norm_bwd = [&](const void* dy, bool dy_is_t, const float* x, const float* rstd, const T* gamma, const float* dx_in,
                         long long rows, int mS, int mP, float* dgamma) -> int {
       const int blocks = (int)(rows / 8 + 1 < NORM_BWD_BLOCKS ? rows / 8 + 1 : NORM_BWD_BLOCKS);
       prof_begin(PC_NORM, s);
-      if (dy_is_t)
+      if (dy_is_t && d == 1024)
+        rmsnorm_bwd_rows_kernel<T, T, 8><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t,
+                                                                       w.norm_part, rows, mS, mP);
+      else if (dy_is_t)
         rmsnorm_bwd_kernel<T, T><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t, w.norm_part,
                                                                rows, d, mS, mP);
       else
