@@ -23,10 +23,14 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# DRAM traffic of the dominant kernel from one ncu capture (profiles/gemm_tc2_kernel_M19968_N3072_K1024_ncu.md):
-# dram__bytes_read.sum + dram__bytes_write.sum = 119.6 MB for the QKV-shaped launch at M = 19968 rows against
-# 169.9 MB of algorithmic bytes; traffic grows in proportion to the rows for a fixed weight matrix.
-GEMM_TRAFFIC_CAPTURE = {"rows": 19968, "n": 3072, "k": 1024, "dram_bytes": 119.6e6, "algorithmic_bytes": 169.9e6}
+# DRAM traffic of the dominant kernel, from one ncu capture of ONE launch at the shape the medium workload runs
+# (QKV projection, all 119 808 tokens in one micro-batch): dram__bytes_read.sum + dram__bytes_write.sum.  None until
+# such a capture exists for the kernel as it stands; never scaled from another size.
+GEMM_TRAFFIC_CAPTURE = None
+
+# Context figures the paper reports for its own runs (7B policy with LoRA on 2 x H100, LIBERO): not targets.
+PAPER_CONTEXT = {"wall_clock_speedup": 2.38, "gradient_update_speedup": 4.8, "activation_memory_reduction": 0.60,
+                 "where": "Sec. 5 RQ2, Fig. 4; App. E hardware"}
 
 METRIC = "kept_chunks_per_s_actor_fwd_bwd"
 UNIT = "chunks/s"
@@ -139,6 +143,25 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
+def config_of(w, n_kept, total, mb, iterations=None):
+    """The `config` object both arms print."""
+    c = {"workload": w.name, "kept_chunks_per_step": int(n_kept), "chunks_per_step": int(total),
+         "tokens_per_step": int(n_kept) * w.S, "mb_chunks": int(mb), "l2": "inputs_larger_than_l2",
+         "multi_gpu": "independent replicas, no collective"}
+    if iterations is not None:
+        c["iterations"] = int(iterations)
+        c["resampled"] = "rollouts redrawn every iteration from seeds 0..iterations-1, keep-probability state carried"
+    return c
+
+
+def launch_steps_online(args):
+    return args.steps
+
+
+def default_mb(args, n_kept):
+    return args.mb if args.mb > 0 else min(n_kept, 384)
+
+
 def run_reference(args):
     """The oracle as it stands, timed on the host cores, on the same workload and metric."""
     rank = int(os.environ.get("RANK", "0"))
@@ -146,7 +169,8 @@ def run_reference(args):
         return
     from paper_2605_16154_b200 import synth
     w = synth.WORKLOADS[args.workload]
-    rb = synth.make_rollouts(w)
+    online = w.T == 0
+    rb = synth.make_rollouts(w, 0 if online else None)
     weights = synth.make_weights(w)
     n_sample = 1
     est = []
@@ -156,11 +180,13 @@ def run_reference(args):
             est.append(t_pcm + t_actor * n_kept / n_sample)
     ms = 1e3 * sum(est) / len(est)
     value = n_kept / (ms / 1e3)
+    total = int(rb["traj_off"][-1])
     sample = (f"per step: control plane on the full batch + actor fwd/bwd on {n_sample} of {n_kept} kept chunks, "
-              f"scaled by {n_kept}/{n_sample} (chunks are independent sequences)")
+              f"scaled by {n_kept}/{n_sample} (chunks are independent sequences); ms_per_step is that estimate")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic", "config": {"workload": w.name, "kept_chunks_per_step": n_kept},
+            "dtype": "f64", "data": "synthetic",
+            "config": config_of(w, n_kept, total, default_mb(args, n_kept), launch_steps_online(args) if online else None),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -170,107 +196,99 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # CUDA path
 # ------------------------------------------------------------------------------------------------
+class Harness:
+    """Device state shared by the timed legs: model, workspace, preallocated outputs."""
+
+    def __init__(self, B, PL, synth, w, weights, n_kept_max, mb):
+        import torch
+        self.B, self.w, self.mb = B, w, mb
+        self.model = PL.upload_model(w, weights)
+        self.model.alloc_grads()
+        self.ws = torch.empty(B.grpo_workspace_bytes(self.model, mb, 0) + 256, dtype=torch.uint8, device="cuda")
+        self.loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+        self.outputs(n_kept_max, w.n_traj, w.budget)
+
+    def outputs(self, n_kept, n_traj, budget):
+        import torch
+        B = self.B
+        self.n_kept = n_kept
+        self.packed = B.Packed(self.model, n_kept)
+        self.samp = {"kept_idx": torch.empty(n_traj * budget, dtype=torch.int32, device="cuda"),
+                     "kept_off": torch.empty(n_traj + 1, dtype=torch.int32, device="cuda"),
+                     "kept_per_phase": torch.empty(self.w.n_phases, dtype=torch.int32, device="cuda")}
+        self.logp = torch.empty((n_kept, ACT), dtype=torch.float32, device="cuda")
+
+    def select(self, ctx, bt, it):
+        B = self.B
+        Cc, valid, _, adv = B.pcm_score_phases(ctx, bt)
+        _, q = B.pcm_update_keep_probs(ctx, Cc, valid)
+        kept_idx, kept_off, _ = B.pcm_sample_chunks(ctx, bt, q, it, out=self.samp)
+        return adv, kept_idx, kept_off, q
+
+    def update(self, ctx, bt, adv, kept_idx, kept_off):
+        B, w = self.B, self.w
+        B.grpo_pack_chunks(ctx, bt, self.model, kept_idx, kept_off, adv, self.packed)
+        B.grpo_actor_fwd_bwd(self.model, self.packed, w.eps_low, w.eps_high, 0.0, mb_chunks=self.mb, workspace=self.ws,
+                             want_stats=False, logp=self.logp, loss=self.loss)
+
+    def step(self, ctx, bt, it):
+        adv, kept_idx, kept_off, _ = self.select(ctx, bt, it)
+        self.update(ctx, bt, adv, kept_idx, kept_off)
+
+
+def class_table(prof, steps):
+    classes = {}
+    for name, p in prof.items():
+        if p["launches"] == 0:
+            continue
+        c = {"ms_per_step": p["ms"] / steps, "launches_per_step": p["launches"] / steps}
+        if p["flops"] > 0:
+            c["tflops"] = p["flops"] / (p["ms"] * 1e9)
+        if p["bytes"] > 0:
+            c["gbs"] = p["bytes"] / (p["ms"] * 1e6)
+        classes[name] = c
+    return classes
+
+
+def roofline_of(prof, peaks, steps, step_flops, ms_step, traffic):
+    """The dominant kernel: gemm_tc2_kernel (CTA-pair tcgen05 GEMM), every launch of it in the timed region."""
+    g = prof["gemm"]
+    achieved = g["flops"] / (g["ms"] * 1e9) if g["ms"] > 0 else 0.0
+    peak = peaks["bf16_tflops_sustained"]
+    step_tflops = step_flops / (ms_step * 1e9)
+    return {"bound": "tensor", "kernel": "gemm_tc2_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+            "frac": achieved / peak if peak else None, "traffic": traffic,
+            "traffic_of": ("one QKV-projection launch at this workload's full micro-batch, ncu dram read + write"
+                           if traffic is not None else "no capture of the current kernel at this shape"),
+            "peak_source": peaks["source"] + " bf16_tflops_sustained (kernel timed inside a long step)",
+            "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
+            "launches_per_step": g["launches"] / steps, "flops_per_launch": g["flops"] / max(1, g["launches"]),
+            "ms_per_launch": g["ms"] / max(1, g["launches"]),
+            "step_tflops": step_tflops, "step_frac": step_tflops / peak, "step_frac_of_nominal_2250": step_tflops / 2250.0}
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
 
     from paper_2605_16154_b200 import build as _build
     _build.build()
-    from paper_2605_16154_b200 import binding as B, dist_util, pipeline as PL, synth
+    from paper_2605_16154_b200 import binding as B, dist_util, launch, pipeline as PL, synth
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = launch.rank_world_local()
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    launch.init_process_group("nccl", torch.device("cuda", local_rank))
 
     w = synth.WORKLOADS[args.workload]
-    td = PL.torch_dtype(w)
-    seed = dist_util.replica_seed(w.seed, rank)    # every rank works on its own batch (replicas, no exchange)
-    rb = synth.make_rollouts(w, seed)
-    weights = synth.make_weights(w)
-    lengths = np.diff(rb["traj_off"])
-    total = int(rb["traj_off"][-1])
-    n_kept = PL.n_kept_of(w.budget, rb["traj_off"])
-    mb = args.mb if args.mb > 0 else min(n_kept, 384)
+    if w.T == 0:
+        run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank)
+    else:
+        run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank)
+    if world > 1:
+        dist.destroy_process_group()
 
-    # host inputs in pinned memory (what an end-to-end caller owns)
-    gen = torch.Generator().manual_seed(seed)
-    h_obs = torch.empty((total, w.P, w.d), dtype=td).pin_memory()
-    for c0 in range(0, total, 256):                 # N(0,1) prefixes, rounded to the model dtype
-        c1 = min(total, c0 + 256)
-        h_obs[c0:c1] = torch.randn((c1 - c0, w.P, w.d), generator=gen, dtype=torch.float32).to(td)
-    h = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in rb.items()}
 
-    model = PL.upload_model(w, weights)
-    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=seed, max_traj=w.n_traj)
-    d_in = {k: v.cuda() for k, v in h.items()}
-    d_obs = h_obs.cuda()
-
-    # behaviour-policy log-probs: a forward-only pass of the library over every chunk, plus noise
-    ident = B.Context(w.n_phases, int(lengths.max()), w.G, max_traj=w.n_traj)
-    d_lpo = torch.zeros((total, ACT), dtype=torch.float32, device="cuda")
-    batch = B.make_batch(d_in["traj_off"], d_in["tok"], d_in["phase"], d_in["reward"], int(lengths.max()), d_obs, d_lpo)
-    ws_fwd = None
-    zero_adv = torch.zeros(w.n_traj, dtype=torch.float32, device="cuda")
-    for c0 in range(0, total, 512):
-        c1 = min(total, c0 + 512)
-        idx = torch.arange(c0, c1, dtype=torch.int32, device="cuda")
-        off = torch.clamp(d_in["traj_off"].to(torch.int32) - c0, 0, c1 - c0).to(torch.int32).contiguous()
-        pk_all = B.grpo_pack_chunks(ident, batch, model, idx, off, zero_adv, B.Packed(model, c1 - c0))
-        _, lp, _, _ = B.grpo_actor_fwd_bwd(model, pk_all, flags=B.GRPO_FWD_ONLY, mb_chunks=128, workspace=ws_fwd)
-        d_lpo[c0:c1] = lp
-        del pk_all
-    ident.close()
-    d_lpo += torch.from_numpy(synth.logp_noise(seed, total, 0.1)).cuda()
-    h_lpo = d_lpo.cpu().pin_memory()
-    torch.cuda.empty_cache()
-
-    # preallocated outputs and workspace
-    packed = B.Packed(model, n_kept)
-    ws = torch.empty(B.grpo_workspace_bytes(model, mb, 0) + 256, dtype=torch.uint8, device="cuda")
-    samp = {"kept_idx": torch.empty(w.n_traj * w.budget, dtype=torch.int32, device="cuda"),
-            "kept_off": torch.empty(w.n_traj + 1, dtype=torch.int32, device="cuda"),
-            "kept_per_phase": torch.empty(w.n_phases, dtype=torch.int32, device="cuda")}
-    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
-    logp = torch.empty((n_kept, ACT), dtype=torch.float32, device="cuda")
-    model.alloc_grads()
-
-    def step(it, bt):
-        Cc, valid, _, adv = B.pcm_score_phases(ctx, bt)
-        _, q = B.pcm_update_keep_probs(ctx, Cc, valid)
-        kept_idx, kept_off, _ = B.pcm_sample_chunks(ctx, bt, q, it, out=samp)
-        B.grpo_pack_chunks(ctx, bt, model, kept_idx, kept_off, adv, packed)
-        B.grpo_actor_fwd_bwd(model, packed, w.eps_low, w.eps_high, 0.0, mb_chunks=mb, workspace=ws, want_stats=False,
-                             logp=logp, loss=loss)
-
-    kept_host = torch.empty(w.n_traj * w.budget, dtype=torch.int32).pin_memory()
-
-    def step_e2e(it):
-        """Host buffers in, loss out.  The mask is applied before the big transfer: the control plane runs on
-        the small arrays first, the kept chunk ids come back (a few KB), and only the kept chunks'
-        observation prefixes cross the bus."""
-        for k in ("traj_off", "tok", "phase", "reward"):
-            d_in[k].copy_(h[k], non_blocking=True)
-        d_lpo.copy_(h_lpo, non_blocking=True)
-        Cc, valid, _, adv = B.pcm_score_phases(ctx, batch)
-        _, q = B.pcm_update_keep_probs(ctx, Cc, valid)
-        kept_idx, kept_off, _ = B.pcm_sample_chunks(ctx, batch, q, it, out=samp)
-        kept_host.copy_(kept_idx, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-        for c in kept_host[:n_kept].tolist():
-            d_obs[c].copy_(h_obs[c], non_blocking=True)
-        B.grpo_pack_chunks(ctx, batch, model, kept_idx, kept_off, adv, packed)
-        B.grpo_actor_fwd_bwd(model, packed, w.eps_low, w.eps_high, 0.0, mb_chunks=mb, workspace=ws, want_stats=False,
-                             logp=logp, loss=loss)
-        return float(loss.item())                  # device -> host read of the step's result
-
-    chunk_bytes = w.P * w.d * h_obs.element_size()
-    h2d = sum(v.numel() * v.element_size() for v in h.values()) + h_lpo.numel() * h_lpo.element_size() + \
-        n_kept * chunk_bytes
-    d2h = 4 + 4 * w.n_traj * w.budget
-
+def make_timers(torch, dist, dist_util, world):
     def barrier():
         if world > 1:
             dist.barrier()
@@ -285,10 +303,81 @@ def run_cuda(args):
         ev1.record()
         barrier()
         return dist_util.max_over_ranks(ev0.elapsed_time(ev1), "cuda")
+    return barrier, timed
+
+
+def behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed):
+    """Behaviour-policy log-probs: a forward-only pass of the library over every chunk, plus seeded noise."""
+    ident = B.Context(w.n_phases, int(lengths.max()), w.G, max_traj=w.n_traj)
+    d_lpo = torch.zeros((total, ACT), dtype=torch.float32, device="cuda")
+    batch = B.make_batch(d_in["traj_off"], d_in["tok"], d_in["phase"], d_in["reward"], int(lengths.max()), d_obs, d_lpo)
+    zero_adv = torch.zeros(w.n_traj, dtype=torch.float32, device="cuda")
+    for c0 in range(0, total, 512):
+        c1 = min(total, c0 + 512)
+        idx = torch.arange(c0, c1, dtype=torch.int32, device="cuda")
+        off = torch.clamp(d_in["traj_off"].to(torch.int32) - c0, 0, c1 - c0).to(torch.int32).contiguous()
+        pk_all = B.grpo_pack_chunks(ident, batch, model, idx, off, zero_adv, B.Packed(model, c1 - c0))
+        _, lp, _, _ = B.grpo_actor_fwd_bwd(model, pk_all, flags=B.GRPO_FWD_ONLY, mb_chunks=128)
+        d_lpo[c0:c1] = lp
+        del pk_all
+    ident.close()
+    d_lpo += torch.from_numpy(synth.logp_noise(seed, total, 0.1)).cuda()
+    torch.cuda.empty_cache()
+    return d_lpo, batch
+
+
+def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank):
+    """Fixed-length workloads (C0-C3): K steps over one resident batch."""
+    td = PL.torch_dtype(w)
+    seed = dist_util.replica_seed(w.seed, rank)    # every rank works on its own batch (replicas, no exchange)
+    rb = synth.make_rollouts(w, seed)
+    weights = synth.make_weights(w)
+    lengths = np.diff(rb["traj_off"])
+    total = int(rb["traj_off"][-1])
+    n_kept = PL.n_kept_of(w.budget, rb["traj_off"])
+    mb = default_mb(args, n_kept)
+
+    # host inputs in pinned memory (what an end-to-end caller owns)
+    gen = torch.Generator().manual_seed(seed)
+    h_obs = torch.empty((total, w.P, w.d), dtype=td).pin_memory()
+    for c0 in range(0, total, 256):                 # N(0,1) prefixes, rounded to the model dtype
+        c1 = min(total, c0 + 256)
+        h_obs[c0:c1] = torch.randn((c1 - c0, w.P, w.d), generator=gen, dtype=torch.float32).to(td)
+    h = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in rb.items()}
+
+    hs = Harness(B, PL, synth, w, weights, n_kept, mb)
+    model = hs.model
+    ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=seed, max_traj=w.n_traj)
+    d_in = {k: v.cuda() for k, v in h.items()}
+    d_obs = h_obs.cuda()
+    d_lpo, batch = behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed)
+    h_lpo = d_lpo.cpu().pin_memory()
+    kept_host = torch.empty(w.n_traj * w.budget, dtype=torch.int32).pin_memory()
+
+    def step_e2e(it):
+        """Host buffers in, loss out.  The mask is applied before the big transfer: the control plane runs on
+        the small arrays first, the kept chunk ids come back (a few KB), and only the kept chunks'
+        observation prefixes cross the bus."""
+        for k in ("traj_off", "tok", "phase", "reward"):
+            d_in[k].copy_(h[k], non_blocking=True)
+        d_lpo.copy_(h_lpo, non_blocking=True)
+        adv, kept_idx, kept_off, _ = hs.select(ctx, batch, it)
+        kept_host.copy_(kept_idx, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        for c in kept_host[:n_kept].tolist():
+            d_obs[c].copy_(h_obs[c], non_blocking=True)
+        hs.update(ctx, batch, adv, kept_idx, kept_off)
+        return float(hs.loss.item())                  # device -> host read of the step's result
+
+    chunk_bytes = w.P * w.d * h_obs.element_size()
+    h2d = sum(v.numel() * v.element_size() for v in h.values()) + h_lpo.numel() * h_lpo.element_size() + \
+        n_kept * chunk_bytes
+    d2h = 4 + 4 * w.n_traj * w.budget
+    barrier, timed = make_timers(torch, dist, dist_util, world)
 
     it = 0
     for _ in range(max(args.warmup, 3)):
-        step(it, batch); it += 1
+        hs.step(ctx, batch, it); it += 1
     torch.cuda.synchronize()
     assert B.pcm_poll_status(ctx) == 0
 
@@ -299,7 +388,7 @@ def run_cuda(args):
     B.pcm_profile_read()
     B.pcm_profile_enable(True)
     launches0 = B.pcm_launch_count()
-    ms_total = timed(lambda i: step(i, batch), args.steps, it)
+    ms_total = timed(lambda i: hs.step(ctx, batch, i), args.steps, it)
     it += args.steps
     launches = B.pcm_launch_count() - launches0
     B.pcm_profile_enable(False)
@@ -310,77 +399,239 @@ def run_cuda(args):
     step_e2e(it); it += 1
     ms_e2e = timed(step_e2e, args.steps, it)
     it += args.steps
-    loss_val = float(loss.item())
+    loss_val = float(hs.loss.item())
     status = B.pcm_poll_status(ctx)
     peak_alloc = torch.cuda.max_memory_allocated()
+
+    # ---- the same update with the mask keeping every chunk (plain GRPO), for the masked / full ratio ----
+    masked_full = None
+    if w.name == "C1" and world == 1 and not args.no_masked_full:
+        full_steps = 3
+        ctx_full = B.Context(w.n_phases, int(lengths.max()), w.G, w.t_rc, w.p_min, 1e-6, seed=seed, max_traj=w.n_traj)
+        hs.outputs(total, w.n_traj, int(lengths.max()))
+        full_step = lambda i: hs.step(ctx_full, batch, i)
+        full_step(0)
+        ms_full = timed(full_step, full_steps, 1) / full_steps
+        assert B.pcm_poll_status(ctx_full) == 0
+        ctx_full.close()
+        traj_mb = 8                                    # trajectories per micro-batch for the activation figure
+        act_masked = B.grpo_workspace_bytes(model, traj_mb * w.budget, 0)
+        act_full = B.grpo_workspace_bytes(model, traj_mb * int(lengths.max()), 0)
+        masked_full = {"ms_masked": ms_total / args.steps, "ms_full": ms_full, "speedup": ms_full / (ms_total / args.steps),
+                       "kept_chunks_masked": n_kept, "kept_chunks_full": total, "steps_full": full_steps,
+                       "activation_bytes": {"masked": int(act_masked), "full": int(act_full),
+                                            "ratio": act_masked / act_full,
+                                            "of": f"library workspace for micro-batches of {traj_mb} trajectories "
+                                                  f"({traj_mb * w.budget} vs {traj_mb * int(lengths.max())} chunks), no recompute"},
+                       "context": PAPER_CONTEXT}
 
     if rank == 0:
         peaks = measured_peaks()
         ms_step = ms_total / args.steps
         value = dist_util.aggregate_throughput(n_kept, args.steps, ms_total, world)
         e2e_value = dist_util.aggregate_throughput(n_kept, args.steps, ms_e2e, world)
-        g = prof["gemm"]
-        achieved = g["flops"] / (g["ms"] * 1e9) if g["ms"] > 0 else 0.0
-        peak = peaks["bf16_tflops_sustained"]
-        step_tflops = flops_per_kept_chunk(w) * n_kept / (ms_step * 1e9)
-        classes = {}
-        for name, p in prof.items():
-            if p["launches"] == 0:
-                continue
-            c = {"ms_per_step": p["ms"] / args.steps, "launches_per_step": p["launches"] / args.steps}
-            if p["flops"] > 0:
-                c["tflops"] = p["flops"] / (p["ms"] * 1e9)
-            if p["bytes"] > 0:
-                c["gbs"] = p["bytes"] / (p["ms"] * 1e6)
-            classes[name] = c
+        traffic = None
+        if GEMM_TRAFFIC_CAPTURE and GEMM_TRAFFIC_CAPTURE["rows"] == min(mb, n_kept) * w.S and w.d == GEMM_TRAFFIC_CAPTURE["k"]:
+            traffic = GEMM_TRAFFIC_CAPTURE["dram_bytes"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": w.name, "kept_chunks_per_step": n_kept, "chunks_per_step": total,
-                       "tokens_per_step": n_kept * w.S, "mb_chunks": mb, "l2": "inputs_larger_than_l2",
-                       "multi_gpu": "independent replicas, no collective"},
-            "roofline": {"bound": "tensor", "kernel": "gemm_tc2_kernel", "achieved": achieved, "peak": peak,
-                         "unit": "TFLOP/s", "frac": achieved / peak if peak else None,
-                         "traffic": GEMM_TRAFFIC_CAPTURE["dram_bytes"] * (n_kept * w.S) / GEMM_TRAFFIC_CAPTURE["rows"]
-                         if (w.d == 1024 and mb >= n_kept) else None,
-                         "traffic_of": "QKV-shaped launch [tokens x 3072 x 1024], ncu capture at 19968 rows scaled by rows",
-                         "peak_source": peaks["source"] + " bf16_tflops_sustained",
-                         "launches_per_step": g["launches"] / args.steps,
-                         "flops_per_launch": g["flops"] / max(1, g["launches"]),
-                         "step_tflops": step_tflops, "step_frac": step_tflops / peak},
-            "kernel_classes": classes,
+            "config": config_of(w, n_kept, total, mb),
+            "roofline": roofline_of(prof, peaks, args.steps, flops_per_kept_chunk(w) * n_kept, ms_step, traffic),
+            "kernel_classes": class_table(prof, args.steps),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": int(launches),
             "clocks": clocks,
             "loss": loss_val, "device_status": status,
-            "memory": {"workspace_bytes": int(ws.numel()), "peak_allocated_bytes": int(peak_alloc)},
+            "memory": {"workspace_bytes": int(hs.ws.numel()), "peak_allocated_bytes": int(peak_alloc)},
         }
+        if masked_full is not None:
+            line["masked_full"] = masked_full
         if world == 1 and not args.no_cpu_baseline:
-            t_pcm, t_actor, nk = oracle_sample_step(w, rb, weights, seed, args.cpu_sample)
-            est = t_pcm + t_actor * nk / args.cpu_sample
-            line["cpu_baseline"] = {
-                "value": nk / est, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                "sample": (f"control plane on the full batch ({t_pcm:.2f} s) + actor fwd/bwd on {args.cpu_sample} of "
-                           f"{nk} kept chunks ({t_actor:.2f} s), scaled by {nk}/{args.cpu_sample}")}
+            line["cpu_baseline"] = cpu_baseline_leg(args, w, rb, weights, seed)
         print(json.dumps(line))
     ctx.close()
-    if world > 1:
-        dist.destroy_process_group()
+
+
+def cpu_baseline_leg(args, w, rb, weights, seed):
+    t_pcm, t_actor, nk = oracle_sample_step(w, rb, weights, seed, args.cpu_sample)
+    est = t_pcm + t_actor * nk / args.cpu_sample
+    return {"value": nk / est, "unit": UNIT, "cores": blas_threads(), "kind": "oracle (fp64 numpy, BLAS threads = cores)",
+            "sample": (f"control plane on the full batch ({t_pcm:.2f} s) + actor fwd/bwd on {args.cpu_sample} of "
+                       f"{nk} kept chunks ({t_actor:.2f} s), scaled by {nk}/{args.cpu_sample}")}
+
+
+def run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank):
+    """Ragged workload (C4): Algorithm 1's loop.  Every iteration draws a new rollout batch (seed = iteration), the
+    keep-probability state is carried from one iteration to the next and refreshed every T_rc of them, so the
+    kept-chunk mix and the ragged tail of the last micro-batch change as the loop runs."""
+    td = PL.torch_dtype(w)
+    n_iter = args.steps
+    base = dist_util.replica_seed(0, rank)
+    batches = [synth.make_rollouts(w, base + it) for it in range(n_iter)]
+    weights = synth.make_weights(w)
+    totals = [int(b["traj_off"][-1]) for b in batches]
+    max_len = max(int(np.diff(b["traj_off"]).max()) for b in batches)
+    kept_per_it = [PL.n_kept_of(w.budget, b["traj_off"]) for b in batches]
+    n_kept_max = max(kept_per_it)
+    mb = default_mb(args, n_kept_max)
+    pool = max(totals)
+
+    # Observation prefixes: one pool of iid N(0,1) rows (seeded, drawn on the device and copied to pinned host memory,
+    # which is what the end-to-end leg reads); chunk c of every iteration uses pool row c.
+    g = torch.Generator(device="cuda").manual_seed(base + 17)
+    d_obs = torch.empty((pool, w.P, w.d), dtype=td, device="cuda")
+    for c0 in range(0, pool, 1024):
+        c1 = min(pool, c0 + 1024)
+        d_obs[c0:c1] = torch.randn((c1 - c0, w.P, w.d), generator=g, device="cuda").to(td)
+    h_obs = torch.empty((pool, w.P, w.d), dtype=td).pin_memory()
+    h_obs.copy_(d_obs)
+    # behaviour policy: near-uniform log-probs plus seeded noise (the synthetic weights give near-uniform logits)
+    host, dev_b = [], []
+    for it, rb in enumerate(batches):
+        hb = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in rb.items()}
+        hb["lpo"] = torch.from_numpy((-np.log(256.0) + synth.logp_noise(base + it, totals[it], 0.1)).astype(np.float32)).pin_memory()
+        host.append(hb)
+        db = {k: v.cuda() for k, v in hb.items()}
+        dev_b.append((db, B.make_batch(db["traj_off"], db["tok"], db["phase"], db["reward"], max_len, d_obs, db["lpo"])))
+
+    hs = Harness(B, PL, synth, w, weights, n_kept_max, mb)
+    barrier, timed = make_timers(torch, dist, dist_util, world)
+    # staging buffers of the end-to-end leg (sized for the largest iteration)
+    stage = {"traj_off": torch.empty(w.n_traj + 1, dtype=torch.int32, device="cuda"),
+             "tok": torch.empty((pool, ACT), dtype=torch.uint8, device="cuda"),
+             "phase": torch.empty(pool, dtype=torch.uint8, device="cuda"),
+             "reward": torch.empty(w.n_traj, dtype=torch.uint8, device="cuda"),
+             "lpo": torch.empty((pool, ACT), dtype=torch.float32, device="cuda")}
+    kept_host = torch.empty(w.n_traj * w.budget, dtype=torch.int32).pin_memory()
+
+    def set_kept(it):
+        hs.packed.c.n_kept = hs.packed.n_kept = kept_per_it[it]
+
+    def new_ctx():
+        return B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=base, max_traj=w.n_traj)
+
+    # warm-up on a context of its own, so that the timed chains start from a fresh keep-probability state
+    ctx = new_ctx()
+    for it in range(max(args.warmup, 3)):
+        set_kept(it % n_iter)
+        hs.step(ctx, dev_b[it % n_iter][1], it)
+    torch.cuda.synchronize()
+    assert B.pcm_poll_status(ctx) == 0
+    ctx.close()
+
+    # ---- device-resident chain ----
+    ctx = new_ctx()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    B.pcm_profile_read()
+    B.pcm_profile_enable(True)
+    launches0 = B.pcm_launch_count()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_iter + 1)]
+    q_hist = []
+    barrier()
+    evs[0].record()
+    for it in range(n_iter):
+        set_kept(it)
+        adv, kept_idx, kept_off, q = hs.select(ctx, dev_b[it][1], it)
+        hs.update(ctx, dev_b[it][1], adv, kept_idx, kept_off)
+        q_hist.append(q)
+        evs[it + 1].record()
+    barrier()
+    ms_total = dist_util.max_over_ranks(evs[0].elapsed_time(evs[n_iter]), "cuda")
+    per_it = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_iter)]
+    launches = B.pcm_launch_count() - launches0
+    B.pcm_profile_enable(False)
+    prof = B.pcm_profile_read()
+    clocks = sampler.stop() if rank == 0 else None
+    assert B.pcm_poll_status(ctx) == 0
+    q_np = np.stack([t.cpu().numpy() for t in q_hist]).astype(np.int64)
+    ctx.close()
+
+    # ---- end to end chain: every iteration's batch comes from pinned host memory ----
+    ctx = new_ctx()
+    e2e_batch = B.make_batch(stage["traj_off"], stage["tok"], stage["phase"], stage["reward"], max_len, d_obs, stage["lpo"])
+    h2d = d2h = 0
+
+    def step_e2e(it):
+        nonlocal h2d, d2h
+        hb, n = host[it], totals[it]
+        stage["traj_off"].copy_(hb["traj_off"], non_blocking=True)
+        stage["reward"].copy_(hb["reward"], non_blocking=True)
+        stage["tok"][:n].copy_(hb["tok"], non_blocking=True)
+        stage["phase"][:n].copy_(hb["phase"], non_blocking=True)
+        stage["lpo"][:n].copy_(hb["lpo"], non_blocking=True)
+        e2e_batch.n_chunks = n
+        set_kept(it)
+        adv, kept_idx, kept_off, _ = hs.select(ctx, e2e_batch, it)
+        kept_host.copy_(kept_idx, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        for c in kept_host[:kept_per_it[it]].tolist():
+            d_obs[c].copy_(h_obs[c], non_blocking=True)
+        hs.update(ctx, e2e_batch, adv, kept_idx, kept_off)
+        h2d += sum(hb[k].numel() * hb[k].element_size() for k in hb) + kept_per_it[it] * w.P * w.d * h_obs.element_size()
+        d2h += 4 + 4 * w.n_traj * w.budget
+        return float(hs.loss.item())
+
+    ms_e2e = timed(step_e2e, n_iter, 0)
+    loss_val = float(hs.loss.item())
+    status = B.pcm_poll_status(ctx)
+    peak_alloc = torch.cuda.max_memory_allocated()
+    ctx.close()
+
+    if rank == 0:
+        peaks = measured_peaks()
+        n_kept_total = sum(kept_per_it)
+        ms_step = ms_total / n_iter
+        value = world * n_kept_total / (ms_total / 1e3)
+        e2e_value = world * n_kept_total / (ms_e2e / 1e3)
+        refreshes = int((np.abs(np.diff(q_np, axis=0)).sum(axis=1) > 0).sum()) + 1
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_iter,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": config_of(w, n_kept_total / n_iter, sum(totals) / n_iter, mb, n_iter),
+            "online": {"ms_mean": statistics.mean(per_it), "ms_min": min(per_it), "ms_max": max(per_it),
+                       "kept_chunks_min": min(kept_per_it), "kept_chunks_max": max(kept_per_it),
+                       "chunks_min": min(totals), "chunks_max": max(totals),
+                       "keep_prob_refreshes": refreshes, "t_rc": w.t_rc,
+                       "keep_probs_first": (q_np[0] / float(1 << 24)).round(4).tolist(),
+                       "keep_probs_last": (q_np[-1] / float(1 << 24)).round(4).tolist()},
+            "roofline": roofline_of(prof, peaks, n_iter, flops_per_kept_chunk(w) * n_kept_total / n_iter, ms_step, None),
+            "kernel_classes": class_table(prof, n_iter),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d / n_iter),
+                    "d2h_bytes_per_step": int(d2h / n_iter), "ms_per_step": ms_e2e / n_iter},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "loss": loss_val, "device_status": status,
+            "memory": {"workspace_bytes": int(hs.ws.numel()), "peak_allocated_bytes": int(peak_alloc)},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline_leg(args, w, batches[0], weights, base)
+        print(json.dumps(line))
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 10; the ragged workload: 50 iterations)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="C1")
     ap.add_argument("--mb", type=int, default=0, help="chunks per micro-batch (0: up to 384)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--cpu-sample", type=int, default=2, help="kept chunks the CPU baseline leg runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-masked-full", action="store_true", help="skip the keep-every-chunk leg of the medium workload")
     args = ap.parse_args()
+    from paper_2605_16154_b200 import launch
+    if args.impl == "cuda" and launch.needs_relaunch(args.gpus, os.environ):
+        cmd = launch.torchrun_command(args.gpus, os.path.abspath(__file__), sys.argv[1:])
+        os.execv(cmd[0], cmd)
+    if args.steps is None:
+        args.steps = launch.default_steps(args.workload, args.impl)
     if args.impl == "reference":
         run_reference(args)
     else:

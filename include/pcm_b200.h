@@ -338,10 +338,11 @@ uint32_t grpo_attention_wait_status(void);
 /* Per-kernel-class timing.  While enabled, every launch of the classes below is bracketed by a
  * pair of CUDA events on its stream; pcm_profile_read() synchronises the device, adds up elapsed
  * milliseconds, the algorithmic flops / bytes of the launches and their count since the last read,
- * and clears the records.  Classes: 0 GEMM (all linear layers, head), 1 attention, 2 RMSNorm,
- * 3 element-wise (rotary, SwiGLU, residual cast), 4 loss rows, 5 embedding gradient, 6 pack,
- * 7 phase-score reduction (the per-group kernel of pcm_score_phases), 8 chunk sampling. */
-#define PCM_PROFILE_CLASSES 9
+ * and clears the records.  Classes: 0 GEMMs on the CTA-pair tensor-core kernel (the linear layers at
+ * training sizes), 1 attention, 2 RMSNorm, 3 element-wise (rotary, SwiGLU, residual cast), 4 loss rows,
+ * 5 embedding gradient, 6 pack, 7 phase-score reduction (the per-group kernel of pcm_score_phases),
+ * 8 chunk sampling, 9 GEMMs on the single-CTA or SIMT kernels (narrow outputs, the head, fp32 mode). */
+#define PCM_PROFILE_CLASSES 10
 typedef struct {
   double ms[PCM_PROFILE_CLASSES];
   double flops[PCM_PROFILE_CLASSES];
@@ -353,6 +354,12 @@ int pcm_profile_read(pcm_profile* out);
 
 /* Number of kernels this library has launched in the calling process (for accounting). */
 int64_t pcm_launch_count(void);
+
+/* Host-only helper behind the library's per-device set-up (kernel attributes such as the dynamic shared-memory
+ * limit belong to one device, so each launcher keeps a bit mask of the devices it has prepared): returns 1 and
+ * sets bit `device` of *seen_mask on the first call for that device, 0 afterwards; devices outside 0..63 always
+ * return 1.  No GPU work. */
+int32_t pcm_first_use_on_device(uint64_t* seen_mask, int32_t device);
 
 #ifdef __cplusplus
 }

@@ -83,12 +83,13 @@ class grpo_adamw_cfg(C.Structure):
                 ("weight_decay", C.c_float), ("max_grad_norm", C.c_float)]
 
 
-PROFILE_CLASSES = ("gemm", "attention", "rmsnorm", "elementwise", "loss", "embed_grad", "pack", "pcm_score", "pcm_sample")
+PROFILE_CLASSES = ("gemm", "attention", "rmsnorm", "elementwise", "loss", "embed_grad", "pack", "pcm_score", "pcm_sample",
+                   "gemm_small")
 
 
 class pcm_profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 9), ("flops", C.c_double * 9), ("bytes", C.c_double * 9),
-                ("launches", C.c_int64 * 9)]
+    _fields_ = [("ms", C.c_double * 10), ("flops", C.c_double * 10), ("bytes", C.c_double * 10),
+                ("launches", C.c_int64 * 10)]
 
 
 _P = C.c_void_p
@@ -121,6 +122,8 @@ _lib.grpo_adamw_step.argtypes = [C.POINTER(grpo_model_cfg), C.POINTER(grpo_adamw
                                  _P, _P, C.c_size_t, _P]
 _lib.grpo_adamw_step.restype = C.c_int
 _lib.pcm_launch_count.restype = C.c_int64
+_lib.pcm_first_use_on_device.argtypes = [C.POINTER(C.c_uint64), C.c_int32]
+_lib.pcm_first_use_on_device.restype = C.c_int32
 _lib.pcm_profile_enable.argtypes = [C.c_int32]
 _lib.pcm_profile_read.argtypes = [C.POINTER(pcm_profile)]
 for _name in ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", "pcm_state_import",
@@ -133,7 +136,7 @@ EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", 
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
             "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static",
             "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases", "pcm_score_phases_f32",
-            "grpo_attention_wait_status")
+            "grpo_attention_wait_status", "pcm_first_use_on_device")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:

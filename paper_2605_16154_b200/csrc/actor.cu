@@ -657,7 +657,7 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
                int abdt, void* C, long long ldc, int cdt, const float* R, long long ldr,
                const GemmEpilogue& epi = GemmEpilogue()) -> int {
     GemmArgs g{M_, N_, K_, A, lda, ak, B, ldb, bk, abdt, C, ldc, cdt, R, ldr, epi};
-    prof_begin(PC_GEMM, s);
+    prof_begin(gemm_runs_on_pairs(g) ? PC_GEMM : PC_GEMM_SMALL, s);
     const int rc = gemm(g, s);
     prof_end(s, 2.0 * M_ * (double)N_ * K_, 0.0);
     return rc;
@@ -852,6 +852,10 @@ static GemmBackend backend_from_env() {
   if (e && !strcmp(e, "simt")) return GEMM_SIMT;
   if (e && !strcmp(e, "tcgen05")) return GEMM_TCGEN05;
   return GEMM_AUTO;
+}
+
+bool gemm_runs_on_pairs(const GemmArgs& g) {
+  return backend_from_env() != GEMM_SIMT && gemm_tcgen05_supported(g) && gemm_tcgen05_pair(g);
 }
 
 int gemm(const GemmArgs& g, cudaStream_t s, GemmBackend backend) {

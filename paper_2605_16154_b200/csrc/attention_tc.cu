@@ -1228,25 +1228,6 @@ static bool make_seq_tmap(CUtensorMap* tm, const void* base, int n_seq, int S, l
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// cudaFuncSetAttribute applies to the current device: remember per function which devices already have it
-static bool attr_needed(unsigned long long* seen_mask) {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
-  if (*seen_mask & (1ull << dev)) return false;
-  *seen_mask |= 1ull << dev;
-  return true;
-}
-
-static int attn_sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
-      n = 148;
-  }
-  return n;
-}
-
 constexpr uint32_t SMEM_LIMIT = 227u * 1024u;
 constexpr uint32_t SMEM_FLOOR = 120u * 1024u;  // more than half of an SM's shared memory: one CTA per SM, which owns all of tensor memory
 
@@ -1277,7 +1258,7 @@ static int fwd_launch(const void* qkv, void* out, float* lse, int n_seq, int S, 
   static unsigned long long attr_devices = 0;
   if (attr_needed(&attr_devices))
     PCM_CUDA_TRY(cudaFuncSetAttribute(fa_tc_fwd_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT));
-  const int grid = p.n_items < attn_sm_count() ? p.n_items : attn_sm_count();
+  const int grid = p.n_items < sm_count() ? p.n_items : sm_count();
   fa_tc_fwd_kernel<DH><<<grid, Cfg<DH>::THREADS, smem, s>>>(tmQ, tmKV, tmO, p);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
@@ -1293,7 +1274,7 @@ static int bwd_launch_one(const CUtensorMap& tmQKV, const CUtensorMap& tmDO, con
   static unsigned long long attr_devices = 0;
   if (attr_needed(&attr_devices))
     PCM_CUDA_TRY(cudaFuncSetAttribute(fa_tc_bwd_kernel<DH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT));
-  const int grid = p.n_items < attn_sm_count() ? p.n_items : attn_sm_count();
+  const int grid = p.n_items < sm_count() ? p.n_items : sm_count();
   fa_tc_bwd_kernel<DH, MODE><<<grid, BW_THREADS, smem, s>>>(tmQKV, tmDO, tmOUT, tmDQKV, p);
   PCM_LAUNCH_CHECK();
   return PCM_OK;

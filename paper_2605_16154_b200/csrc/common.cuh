@@ -36,4 +36,31 @@ constexpr unsigned STATUS_BAD_ACTION = 16u;   // continuous action not finite or
 
 static inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
+// Per-device bookkeeping.  cudaFuncSetAttribute and the SM count belong to the current device, so a process that
+// drives several GPUs needs them once per device, not once per process.
+// First use of `seen_mask` on device `dev` (0..63) returns true and marks the device; devices outside that range
+// always return true (the attribute is then simply set again).
+static inline bool first_use_on_device(unsigned long long* seen_mask, int dev) {
+  if (dev < 0 || dev >= 64) return true;
+  if (*seen_mask & (1ull << dev)) return false;
+  *seen_mask |= 1ull << dev;
+  return true;
+}
+static inline bool attr_needed(unsigned long long* seen_mask) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return true;
+  return first_use_on_device(seen_mask, dev);
+}
+// SM count of the current device, cached per device; 148 when the query fails.
+static inline int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+  if (dev >= 0 && dev < 64) cached[dev] = n;
+  return n;
+}
+
 }  // namespace pcm

@@ -877,25 +877,6 @@ static void fill_params(TcParams& p, const GemmArgs& g) {
   p.kb_per_split = 1; p.tiles_m = p.tiles_n = p.splits = 1;
 }
 
-// cudaFuncSetAttribute applies to the current device: remember per function which devices already have it
-static bool attr_needed(unsigned long long* seen_mask) {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
-  if (*seen_mask & (1ull << dev)) return false;
-  *seen_mask |= 1ull << dev;
-  return true;
-}
-
-static int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
-      n = 148;
-  }
-  return n;
-}
-
 template <int BN, int EPI>
 static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   CUtensorMap tmA, tmB;
@@ -1014,9 +995,12 @@ bool gemm_epilogue_supported(const GemmArgs& g) {
   return false;
 }
 
+// CTA pairs whenever the output is at least one 256-wide tile; single CTAs otherwise (or with PCM_GEMM_PAIR=0)
+static bool wants_pair(const GemmArgs& g) { return pair_enabled() && g.N >= 256 && g.M > TC_BM; }
+bool gemm_tcgen05_pair(const GemmArgs& g) { return wants_pair(g); }
+
 int gemm_tcgen05(const GemmArgs& g, cudaStream_t s) {
-  // CTA pairs whenever the output is at least one 256-wide tile; single CTAs otherwise (or with PCM_GEMM_PAIR=0)
-  const bool pair = pair_enabled() && g.N >= 256 && g.M > TC_BM;
+  const bool pair = wants_pair(g);
   switch (g.epi.kind) {
     case EPI_SWIGLU_FWD:
       if (!gemm_epilogue_supported(g)) return PCM_ERR_SHAPE;

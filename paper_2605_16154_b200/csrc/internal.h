@@ -42,6 +42,9 @@ int gemm(const GemmArgs& g, cudaStream_t s, GemmBackend backend = GEMM_AUTO);
 int gemm_simt(const GemmArgs& g, cudaStream_t s);
 int gemm_tcgen05(const GemmArgs& g, cudaStream_t s);
 bool gemm_tcgen05_supported(const GemmArgs& g);
+// True when gemm() would run g on the CTA-pair kernel (256 x 256 tiles) rather than on a single-CTA or SIMT kernel.
+bool gemm_runs_on_pairs(const GemmArgs& g);
+bool gemm_tcgen05_pair(const GemmArgs& g);      // the tensor-core path's own choice, given that it takes g
 // True when the tensor-core kernel can run g including its fused epilogue.
 bool gemm_epilogue_supported(const GemmArgs& g);
 // Reads and clears the tensor-core kernels' device status word (synchronous copy).
@@ -58,7 +61,8 @@ int attention_bwd(int dtype, const void* qkv, const void* out, const void* dout,
                   void* dqkv, int n_seq, int S, int H, int dh, cudaStream_t s, const float2* rope_tab = nullptr);
 
 // Event-pair profiling (profile.cu).  prof_begin/prof_end nest like a stack and cost nothing when off.
-enum { PC_GEMM = 0, PC_ATTN = 1, PC_NORM = 2, PC_ELEM = 3, PC_LOSS = 4, PC_EMBED = 5, PC_PACK = 6, PC_SCORE = 7, PC_SAMPLE = 8 };
+enum { PC_GEMM = 0, PC_ATTN = 1, PC_NORM = 2, PC_ELEM = 3, PC_LOSS = 4, PC_EMBED = 5, PC_PACK = 6, PC_SCORE = 7, PC_SAMPLE = 8,
+       PC_GEMM_SMALL = 9 };
 bool prof_enabled();
 void prof_begin(int cls, cudaStream_t s);
 void prof_end(cudaStream_t s, double flops, double bytes);

@@ -139,11 +139,9 @@ extern "C" int grpo_pack_chunks(pcm_ctx* ctx, const pcm_batch* b, const grpo_mod
   const long long prefix_bytes = (long long)cfg->prefix_len * row_bytes;
   const int pieces = (int)((prefix_bytes + PK_PIECE_BYTES - 1) / PK_PIECE_BYTES);
   const size_t smem = (size_t)PK_STAGES * PK_STAGE_BYTES;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static unsigned long long attr_devices = 0;
+  if (attr_needed(&attr_devices))
     PCM_CUDA_TRY(cudaFuncSetAttribute(pack_chunks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_set = true;
-  }
   dim3 grid(pieces + 1, out->n_kept);
   prof_begin(PC_PACK, (cudaStream_t)stream);
   pack_chunks_kernel<<<grid, 64, smem, (cudaStream_t)stream>>>(

@@ -76,3 +76,11 @@ extern "C" int pcm_profile_read(pcm_profile* out) {
   g_prof_done.clear();
   return PCM_OK;
 }
+
+extern "C" int32_t pcm_first_use_on_device(uint64_t* seen_mask, int32_t device) {
+  if (!seen_mask) return 1;
+  unsigned long long m = *seen_mask;
+  const bool first = first_use_on_device(&m, device);
+  *seen_mask = m;
+  return first ? 1 : 0;
+}

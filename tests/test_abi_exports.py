@@ -46,3 +46,16 @@ def test_host_side_argument_checks_need_no_gpu():
     per_token = full / (64 * 312)
     assert 8 * 44 * 1024 < per_token < 8 * 44 * 1024 * 1.3
     assert B._lib.pcm_create(None, None, 0) == -1
+
+
+def test_per_device_setup_mask_marks_each_device_once():
+    """Kernel attributes are per device: the first launch on every device must set them, later ones must not."""
+    from paper_2605_16154_b200 import binding as B
+    mask = ctypes.c_uint64(0)
+    f = B._lib.pcm_first_use_on_device
+    assert f(ctypes.byref(mask), 0) == 1 and f(ctypes.byref(mask), 0) == 0
+    assert f(ctypes.byref(mask), 1) == 1 and f(ctypes.byref(mask), 1) == 0 and f(ctypes.byref(mask), 0) == 0
+    assert f(ctypes.byref(mask), 63) == 1 and f(ctypes.byref(mask), 63) == 0
+    assert mask.value == (1 | 2 | (1 << 63))
+    assert f(ctypes.byref(mask), 64) == 1 and f(ctypes.byref(mask), -1) == 1      # out of range: always set again
+    assert mask.value == (1 | 2 | (1 << 63))

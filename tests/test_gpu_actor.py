@@ -94,6 +94,10 @@ def _compare(B, PL, hp, tol_grad, tol_loss_rel=None, tol_loss_abs=None, mb=64, e
     g = grads_to_numpy(grads)
     errs = {k: rel_fro(g[k], grads_o[k]) for k in grads_o}
     assert max(errs.values()) < tol_grad, errs
+    if w.dtype == "f32":
+        # entry by entry as well: a few wrong small entries (one embedding row, one gain) hide under a norm
+        worst = {k: float(np.max(np.abs(g[k] - grads_o[k])) / np.max(np.abs(grads_o[k]))) for k in grads_o}
+        assert max(worst.values()) <= tol_grad, worst
     assert abs(stats.clip_frac - stats_o["clip_frac"]) < 0.02
     assert stats.n_launches > 0
     assert stats.entropy == pytest.approx(stats_o["entropy"], rel=1e-5 if w.dtype == "f32" else 5e-3)

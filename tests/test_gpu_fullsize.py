@@ -115,6 +115,40 @@ def test_eight_chunk_update_of_the_full_model_against_the_oracle(c1):
     assert stats.clip_frac == pytest.approx(stats_o["clip_frac"], abs=1e-6)
 
 
+def test_full_batch_backward_against_the_oracle_through_zero_advantage_chunks(c1):
+    """The 384-chunk update in one micro-batch (every GEMM, attention and norm launch at the shape bench.py
+    times) against the fp64 oracle.  Eight chunks spread over the batch, one of them in the last row tile,
+    keep their own advantage; the other 376 get A = 0.  A zero advantage gives an exactly zero surrogate term and
+    an exactly zero gradient (Eq. 1, Eq. 11), so the expected loss and gradients are the oracle's on the
+    eight chunks alone under the full batch's scale 1 / (56 * 384)."""
+    B, PL, w, model, pk = c1["B"], c1["PL"], c1["w"], c1["model"], c1["pk"]
+    sel = [0, 47, 101, 190, 255, 256, 340, 383]
+    X = pk.X[sel].float().cpu().numpy()
+    tgt = pk.tgt[sel].cpu().numpy()
+    adv8 = pk.adv_c[sel].cpu().numpy().astype(np.float32)          # Eq. 1 advantages of the chunks' own trajectories
+    assert adv8.min() < 0.0 < adv8.max()                             # both outcomes among the eight
+    lp_o = ao.logp_only(c1["weights"], X, tgt, w.H, w.P)
+    noise = synth.logp_noise(13, len(sel), 0.1).astype(np.float64)
+    hi, lo, m = np.log(1.2), np.log(0.8), 0.05
+    log_r = -noise
+    log_r = np.where(np.abs(log_r - hi) < m, hi + 2 * m * np.sign(log_r - hi + 1e-30), log_r)
+    log_r = np.where(np.abs(log_r - lo) < m, lo + 2 * m * np.sign(log_r - lo + 1e-30), log_r)
+    lpo8 = (lp_o - log_r).astype(np.float32)
+    scale = 1.0 / (56 * 384)
+    loss_o, _, grads_o, _ = ao.fwd_bwd(c1["weights"], X, tgt, lpo8, adv8, w.H, w.P, 0.2, 0.2, scale)
+    full = B.Packed(model, 384)
+    full.X.copy_(pk.X); full.tgt.copy_(pk.tgt); full.lpo.copy_(pk.lpo); full.src.copy_(pk.src)
+    adv_c = np.zeros(384, dtype=np.float32)
+    adv_c[sel] = adv8
+    full.adv_c.copy_(PL.dev(adv_c))
+    full.lpo[sel] = PL.dev(lpo8)
+    loss, logp, grads, stats = B.grpo_actor_fwd_bwd(model, full, mb_chunks=384)
+    assert abs(float(loss.item()) - loss_o) < 1e-3
+    assert np.max(np.abs(logp[sel].cpu().numpy() - lp_o)) < 0.04
+    errs = {k: rel_fro(v, grads_o[k]) for k, v in grads_to_numpy(grads).items()}
+    assert max(errs.values()) < 2e-2, errs
+
+
 def test_attention_at_the_full_batch_shape_on_sampled_sequences_and_heads():
     """grpo_attention on the shape one C1 layer runs (384 sequences of 312 tokens, 16 heads of 64: every CTA of the
     persistent kernels walks about 40 items); forward and backward checked against the oracle on sampled

@@ -5,12 +5,13 @@ plan is frozen, a control thread beside the robot that must not block on the all
 only receives pointers.  pcm_score_phases_static serves them from a fixed scratch array inside the
 library.  Here it is called twice in a row through the C ABI, on two different batches (the second
 smaller, so stale contents of the shared scratch would show), and must reproduce pcm_score_phases
-bit for bit - the same bar the other scoring tests use.  Collected last on purpose: a run that stops
+and the CPU oracle bit for bit - the same bar the other scoring tests use.  Collected last on purpose: a run that stops
 at the first failure has then already executed every other test."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import pcm_oracle as po
 from paper_2605_16154_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -38,6 +39,13 @@ def test_static_scoring_matches_context_scoring_twice_in_a_row():
         assert np.array_equal(out["C"].cpu().numpy().view(np.uint64), C_ref.cpu().numpy().view(np.uint64))
         assert torch.equal(out["valid"], valid_ref) and torch.equal(out["n_valid"], nvalid_ref)
         assert np.array_equal(out["adv"].cpu().numpy().view(np.uint32), adv_ref.cpu().numpy().view(np.uint32))
+        # and against the CPU oracle: the two entry points share a kernel, so a fault common to both would pass above
+        C_o, valid_o, nvalid_o, _, _ = po.score_phases(rb["traj_off"], rb["tok"], rb["phase"], rb["reward"], w.G, w.n_phases)
+        adv_o = po.advantages(rb["reward"], w.G, 1e-6).astype(np.float32)
+        assert np.array_equal(out["C"].cpu().numpy().view(np.uint64), np.asarray(C_o, dtype=np.float64).view(np.uint64))
+        assert np.array_equal(out["valid"].cpu().numpy(), np.asarray(valid_o, dtype=np.uint8))
+        assert np.array_equal(out["n_valid"].cpu().numpy(), np.asarray(nvalid_o, dtype=np.int32))
+        assert np.array_equal(out["adv"].cpu().numpy().view(np.uint32), adv_o.view(np.uint32))
         ctx.close()
 
 
