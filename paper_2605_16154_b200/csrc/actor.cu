@@ -370,112 +370,114 @@ __global__ void swiglu_bwd_kernel(const T* __restrict__ gu, const T* __restrict_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Loss over the 256-bin head: one CTA per chunk, warp w scores rows 7w .. 7w+6 of the chunk's 56.
-// z fp32 [rows][256] logits in, dz T out.  Token level: one clipped ratio per row.  Chunk level: the rows'
-// log-ratios are summed over the CTA in a fixed order and one clipped ratio serves all 56 rows.
-// The entropy bonus adds ent_scale * p_v (log p_v + H) to dz (ent_scale = coefficient / scored rows).
-// Per-CTA partial sums {surrogate, clipped count, ratio, entropy} go to part[blockIdx][4].
+// Head + loss without tensor cores (fp32 mode, or widths the tensor-core GEMM does not take): one CTA computes the
+// logits of HL_ROWS scored rows, thread v holding bin v of every row in a register, and applies the same row
+// functions as the tensor-core epilogue.  hs [rows][d] and W_h [256][d] in T; dz [rows][256] in T.  The logits never
+// leave registers.  part[blockIdx][4] receives the CTA's sums {surrogate, clipped terms, ratio, entropy}.
 // ------------------------------------------------------------------------------------------------
-constexpr int LOSS_ROWS_PER_WARP = ACT / 8;
-static_assert(ACT % 8 == 0, "a chunk's rows are split evenly over the CTA's eight warps");
+constexpr int HL_ROWS = 8;
+constexpr int HL_KT = 32;
 
 template <typename T>
-__global__ void __launch_bounds__(256)
-loss_chunk_kernel(const float* __restrict__ z, const uint8_t* __restrict__ tgt, const float* __restrict__ lpo,
-                  const float* __restrict__ adv_c, float eps_low, float eps_high, float loss_scale, float ent_scale,
-                  int chunk_ratio, T* __restrict__ dz, float* __restrict__ logp_out, float* __restrict__ part,
-                  int fwd_only) {
-  __shared__ float red[8][4];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long chunk = blockIdx.x;
-  const float A = adv_c[chunk];
-  const float lo = 1.f - eps_low, hi = 1.f + eps_high;
-  float v[LOSS_ROWS_PER_WARP][8];
-  float lse[LOSS_ROWS_PER_WARP], ent[LOSS_ROWS_PER_WARP], dlogp[LOSS_ROWS_PER_WARP];
-  int tg[LOSS_ROWS_PER_WARP];
-  float my_s = 0.f, my_clip = 0.f, my_ratio = 0.f, my_ent = 0.f, dsum = 0.f;
+__global__ void __launch_bounds__(NB)
+head_loss_simt_kernel(const T* __restrict__ hs, const T* __restrict__ w_h, int rows, int d, HeadLossArgs h,
+                      T* __restrict__ dz) {
+  __shared__ float Ws[HL_KT][NB + 1];
+  __shared__ float Hs[HL_ROWS][HL_KT];
+  __shared__ float red[3][HL_ROWS][NB / 32];
+  __shared__ float zt_s[HL_ROWS];
+  __shared__ float sums[HL_ROWS][4];
+  const int v = threadIdx.x, warp = v >> 5, lane = v & 31;
+  const long long r0 = (long long)blockIdx.x * HL_ROWS;
+  float z[HL_ROWS];
 #pragma unroll
-  for (int i = 0; i < LOSS_ROWS_PER_WARP; ++i) {
-    const long long r = chunk * ACT + warp * LOSS_ROWS_PER_WARP + i;
-    const float4 a = *reinterpret_cast<const float4*>(z + r * NB + lane * 8);
-    const float4 b = *reinterpret_cast<const float4*>(z + r * NB + lane * 8 + 4);
-    v[i][0] = a.x; v[i][1] = a.y; v[i][2] = a.z; v[i][3] = a.w;
-    v[i][4] = b.x; v[i][5] = b.y; v[i][6] = b.z; v[i][7] = b.w;
-    float mx = v[i][0];
-#pragma unroll
-    for (int e = 1; e < 8; ++e) mx = fmaxf(mx, v[i][e]);
-#pragma unroll
-    for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    float se = 0.f, sz = 0.f;                             // sum e^(z - mx), sum e^(z - mx) (z - mx)
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const float ex = expf(v[i][e] - mx);
-      se += ex;
-      sz += ex * (v[i][e] - mx);
+  for (int i = 0; i < HL_ROWS; ++i) z[i] = 0.f;
+  for (int k0 = 0; k0 < d; k0 += HL_KT) {
+    for (int i = 0; i < 32; ++i) {                        // W_h rows warp*32 .. +31, 32 consecutive k each
+      const int row = warp * 32 + i;
+      Ws[lane][row] = k0 + lane < d ? ldf(w_h + (long long)row * d + k0 + lane) : 0.f;
     }
-    se = warp_sum(se);
-    sz = warp_sum(sz);
-    const float lg = logf(se);
-    lse[i] = mx + lg;
-    ent[i] = lg - sz / se;                                // H = lse - sum p z
-    const int t = tgt[r];
-    tg[i] = t;
-    float mine = v[i][0];                                 // this lane's value at sub-index t & 7
-#pragma unroll
-    for (int e = 1; e < 8; ++e) mine = ((t & 7) == e) ? v[i][e] : mine;
-    const float zt = __shfl_sync(0xffffffffu, mine, t >> 3);
-    const float logp = zt - lse[i];
-    if (lane == 0 && logp_out) logp_out[r] = logp;
-    my_ent += ent[i];
-    if (chunk_ratio) {
-      dsum += logp - lpo[r];
-      dlogp[i] = 0.f;
-    } else {
-      const float ratio = expf(logp - lpo[r]);
-      const float clipped = fminf(fmaxf(ratio, lo), hi);
-      const bool active = (A >= 0.f && ratio <= hi) || (A < 0.f && ratio >= lo);
-      dlogp[i] = active ? -loss_scale * A * ratio : 0.f;
-      my_s += fminf(ratio * A, clipped * A);
-      my_clip += active ? 0.f : 1.f;
-      my_ratio += ratio;
+    {
+      const int i = v >> 5;                               // 8 rows x 32 k = one element per thread
+      Hs[i][lane] = (r0 + i < rows && k0 + lane < d) ? ldf(hs + (r0 + i) * d + k0 + lane) : 0.f;
     }
-  }
-  if (chunk_ratio) {                                      // one ratio for the chunk: ordered sum over the warps
-    if (lane == 0) red[warp][0] = dsum;
     __syncthreads();
-    float tot = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < HL_KT; ++k) {
+      const float wv = Ws[k][v];
 #pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w][0];
-    __syncthreads();
-    const float ratio = expf(tot);
-    const float clipped = fminf(fmaxf(ratio, lo), hi);
-    const bool active = (A >= 0.f && ratio <= hi) || (A < 0.f && ratio >= lo);
-#pragma unroll
-    for (int i = 0; i < LOSS_ROWS_PER_WARP; ++i) dlogp[i] = active ? -loss_scale * A * ratio : 0.f;
-    if (warp == 0) { my_s = fminf(ratio * A, clipped * A); my_clip = active ? 0.f : 1.f; my_ratio = ratio; }
-  }
-  if (!fwd_only) {
-#pragma unroll
-    for (int i = 0; i < LOSS_ROWS_PER_WARP; ++i) {
-      const long long r = chunk * ACT + warp * LOSS_ROWS_PER_WARP + i;
-      T* out = dz + r * NB + lane * 8;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int col = lane * 8 + e;
-        const float lp = v[i][e] - lse[i];
-        const float p = expf(lp);
-        stf(out + e, dlogp[i] * ((col == tg[i] ? 1.f : 0.f) - p) + ent_scale * p * (lp + ent[i]));
-      }
+      for (int i = 0; i < HL_ROWS; ++i) z[i] += Hs[i][k] * wv;
     }
+    __syncthreads();
   }
-  if (lane == 0) { red[warp][0] = my_s; red[warp][1] = my_clip; red[warp][2] = my_ratio; red[warp][3] = my_ent; }
+  // row statistics over the 256 threads: maximum first, then the two sums against it
+  float mx[HL_ROWS];
+#pragma unroll
+  for (int i = 0; i < HL_ROWS; ++i) {
+    float m = z[i];
+#pragma unroll
+    for (int off = 16; off; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if (lane == 0) red[0][i][warp] = m;
+  }
   __syncthreads();
-  if (threadIdx.x < 4) {
-    float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) s += red[w][threadIdx.x];
-    part[(size_t)blockIdx.x * 4 + threadIdx.x] = s;
+  for (int i = 0; i < HL_ROWS; ++i) {
+    float m = red[0][i][0];
+#pragma unroll
+    for (int w = 1; w < NB / 32; ++w) m = fmaxf(m, red[0][i][w]);
+    mx[i] = m;
+    const float ex = expf(z[i] - m);
+    const float se = warp_sum(ex), sz = warp_sum(ex * (z[i] - m));
+    if (lane == 0) { red[1][i][warp] = se; red[2][i][warp] = sz; }
+    const long long r = r0 + i;
+    if (r < rows && v == (int)h.tgt[r]) zt_s[i] = z[i];
   }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < HL_ROWS; ++i) {
+    const long long r = r0 + i;
+    const bool valid = r < rows;
+    RowStats st{mx[i], 0.f, 0.f};
+#pragma unroll
+    for (int w = 0; w < NB / 32; ++w) { st.se += red[1][i][w]; st.sz += red[2][i][w]; }
+    const float lse = hl_lse(st), ent = hl_entropy(st);
+    const float logp = valid ? zt_s[i] - lse : 0.f;
+    RowTerms tm{0.f, 0.f, 0.f, 0.f};
+    if (valid) {
+      if (h.mode == HL_TOKEN) tm = hl_token_terms(logp, h.lpo[r], h.adv_c[r / ACT], h.lo, h.hi, h.loss_scale);
+      else if (h.mode == HL_COEF) tm.dlogp = h.coef[r];
+    }
+    if (v == 0) {
+      if (valid && h.logp && h.mode != HL_COEF) h.logp[r] = logp;
+      sums[i][0] = tm.surrogate; sums[i][1] = tm.clipped; sums[i][2] = tm.ratio; sums[i][3] = valid ? ent : 0.f;
+    }
+    if (valid && h.want_dz) stf(dz + r * NB + v, hl_dz(z[i], lse, ent, tm.dlogp, h.ent_scale, v == (int)h.tgt[r]));
+  }
+  __syncthreads();
+  if (h.part && v < 4) {
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < HL_ROWS; ++i) t += sums[i][v];
+    h.part[(size_t)blockIdx.x * 4 + v] = t;
+  }
+}
+
+// Chunk-level importance ratio (Eq. 2 / Eq. 11 as written): one warp per chunk adds the 56 log-ratios in a fixed
+// order, forms r = exp(sum), clips once, and hands every row of the chunk the same d loss / d logp.
+// part[chunk][4] = {surrogate, clipped, ratio, 0}.
+__global__ void __launch_bounds__(256)
+chunk_ratio_kernel(const float* __restrict__ logp, const float* __restrict__ lpo, const float* __restrict__ adv_c,
+                   int n_chunks, float lo, float hi, float loss_scale, float* __restrict__ coef, float* __restrict__ part) {
+  const int chunk = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (chunk >= n_chunks) return;
+  const long long base = (long long)chunk * ACT;
+  float a = logp[base + lane] - lpo[base + lane];
+  if (lane + 32 < ACT) a += logp[base + lane + 32] - lpo[base + lane + 32];
+  const float tot = warp_sum(a);
+  const RowTerms tm = hl_token_terms(tot, 0.f, adv_c[chunk], lo, hi, loss_scale);     // ratio = exp(tot)
+  coef[base + lane] = tm.dlogp;
+  if (lane + 32 < ACT) coef[base + lane + 32] = tm.dlogp;
+  if (lane == 0) *reinterpret_cast<float4*>(part + (size_t)chunk * 4) = make_float4(tm.surrogate, tm.clipped, tm.ratio, 0.f);
 }
 
 // acc[0..3] += ordered sums of part; loss[0] = -loss_scale * acc[0] - ent_scale * acc[3]   (single CTA, fixed order)
@@ -559,7 +561,7 @@ struct Workspace {
   float2* rope_tab;
   float* x[129];                 // residual stream, x[0..L]
   LayerActs la[128];
-  void* hs; float* rstdf; float* z; void* dz; float* loss_part; float* loss_acc;
+  void* hs; float* rstdf; void* dz; float* loss_part; float* loss_acc; float* logp_tmp; float* coef;
   float* dx; void* dx_t; void* dact; void* dgu; float* dh; void* dattn; void* dqkv; float* dsum;
   float* norm_part; float* dhs;
   size_t bytes;
@@ -585,9 +587,11 @@ static void carve(Workspace& w, unsigned char* base, const grpo_model_cfg& c, in
     for (int l = 1; l < L; ++l) w.la[l] = w.la[0];
     for (int l = 2; l <= L; ++l) w.x[l] = w.x[l & 1];
   }
-  w.hs = a.take(R * d * es); w.rstdf = (float*)a.take(R * 4); w.z = (float*)a.take(R * NB * 4);
+  w.hs = a.take(R * d * es); w.rstdf = (float*)a.take(R * 4);
   w.dz = a.take(R * NB * es);
-  w.loss_part = (float*)a.take((size_t)mb * 4 * 4); w.loss_acc = (float*)a.take(256);
+  // loss partial sums: one entry of 4 per head block (at most one per 8 rows) plus one per chunk
+  w.loss_part = (float*)a.take(((size_t)mb * (ACT / HL_ROWS) + (size_t)mb + 8) * 4 * 4); w.loss_acc = (float*)a.take(256);
+  w.logp_tmp = (float*)a.take(R * 4); w.coef = (float*)a.take(R * 4);
   if (!fwd_only) {
     w.dx = (float*)a.take(M * d * 4); w.dx_t = a.take(M * d * es); w.dact = a.take(M * 4 * d * es);
     w.dgu = a.take(M * 8 * d * es); w.dh = (float*)a.take(M * d * 4); w.dattn = a.take(M * d * es);
@@ -734,16 +738,48 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     rmsnorm_fwd_kernel<T><<<ceil_div(R, 8), 256, 0, s>>>(w.x[L], gf, (T*)w.hs, w.rstdf, R, d, S, P);
     PCM_LAUNCH_CHECK();
     prof_end(s, 0.0, (double)R * d * (es + 4.0));
-    TRY(G(Ri, NB, d, w.hs, d, true, w_h, d, true, dt, w.z, NB, DT_F32, nullptr, 0));
-    const int loss_blocks = mb;                           // one CTA per chunk
-    prof_begin(PC_LOSS, s);
-    loss_chunk_kernel<T><<<loss_blocks, 256, 0, s>>>(w.z, tgt, lpo, advc, lc->eps_low, lc->eps_high, loss_scale, ent_scale,
-                                                   chunk_ratio ? 1 : 0, (T*)w.dz,
-                                                   logp ? logp + (long long)c0 * ACT : nullptr, w.loss_part,
-                                                   fwd_only ? 1 : 0);
-    PCM_LAUNCH_CHECK();
-    prof_end(s, 0.0, (double)R * NB * (4.0 + (fwd_only ? 0.0 : es)));
-    loss_reduce_kernel<<<1, 256, 0, s>>>(w.loss_part, loss_blocks, loss_scale, ent_scale, w.loss_acc, loss);
+    // Head and loss in one launch: the logits stay in tensor memory (bf16 on the tensor cores) or registers.
+    // Returns the number of partial-sum entries the launch wrote (0 when it writes none).
+    auto head = [&](int mode, bool want_dz, float* logp_out, float* part, int* n_part) -> int {
+      HeadLossArgs h;
+      h.tgt = tgt; h.lpo = lpo; h.adv_c = advc; h.coef = w.coef; h.logp = logp_out; h.part = part;
+      h.lo = 1.f - lc->eps_low; h.hi = 1.f + lc->eps_high; h.loss_scale = loss_scale; h.ent_scale = ent_scale;
+      h.mode = mode; h.want_dz = want_dz ? 1 : 0;
+      GemmArgs g{Ri, NB, d, w.hs, d, true, w_h, d, true, dt, w.dz, NB, dt, nullptr, 0};
+      g.epi.kind = EPI_HEAD_LOSS; g.epi.hl = h;
+      const double bytes = (double)R * (d * es + (want_dz ? NB * es : 0.0) + 9.0) + (double)NB * d * es;
+      prof_begin(PC_LOSS, s);
+      int rc = PCM_OK;
+      if (dt == DT_BF16 && backend_from_env() != GEMM_SIMT && gemm_epilogue_supported(g)) {
+        rc = gemm(g, s, GEMM_TCGEN05);
+        *n_part = ceil_div(R, 128) * 4;
+      } else {
+        head_loss_simt_kernel<T><<<ceil_div(R, HL_ROWS), NB, 0, s>>>((const T*)w.hs, w_h, Ri, d, h, (T*)w.dz);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); rc = PCM_ERR_CUDA; }
+        *n_part = ceil_div(R, HL_ROWS);
+      }
+      prof_end(s, 2.0 * R * (double)NB * d, bytes);
+      return rc;
+    };
+    int n_part = 0;
+    float* lp_out = logp ? logp + (long long)c0 * ACT : w.logp_tmp;
+    if (!chunk_ratio) {
+      TRY(head(HL_TOKEN, !fwd_only, lp_out, w.loss_part, &n_part));
+    } else {
+      // the chunk's ratio needs all 56 log-probs first: statistics pass, per-chunk ratio, then (backward only) a
+      // second head launch that recomputes the logits and forms their gradient
+      TRY(head(HL_STATS, false, lp_out, w.loss_part, &n_part));
+      chunk_ratio_kernel<<<ceil_div(mb, 8), 256, 0, s>>>(lp_out, lpo, advc, mb, 1.f - lc->eps_low, 1.f + lc->eps_high, loss_scale,
+                                                         w.coef, w.loss_part + (size_t)n_part * 4);
+      PCM_LAUNCH_CHECK();
+      n_part += mb;
+      if (!fwd_only) {
+        int unused = 0;
+        TRY(head(HL_COEF, true, nullptr, nullptr, &unused));
+      }
+    }
+    loss_reduce_kernel<<<1, 256, 0, s>>>(w.loss_part, n_part, loss_scale, ent_scale, w.loss_acc, loss);
     PCM_LAUNCH_CHECK();
     if (fwd_only) continue;
 

@@ -50,6 +50,7 @@ struct TcParams {
   __nv_bfloat16* out2; long long ld_out2;
   const float2* rope_tab; int S, dh, d;
   int up_row0;                                // EPI_SWIGLU_FWD: first "up" row of B (= F)
+  HeadLossArgs hl;                            // EPI_HEAD_LOSS
 };
 
 __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
@@ -256,7 +257,69 @@ template <int BN, int EPI>
 __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, int row, int n0, int chalf, EpiRegs& pre,
                                          float* stage) {
   const int lane_ = threadIdx.x & 31;
-      if constexpr (EPI == EPI_SWIGLU_FWD) {
+      if constexpr (EPI == EPI_HEAD_LOSS) {
+        // The tile is 128 scored rows x the whole 256-bin vocabulary.  One thread owns one row (the warps of the
+        // first column half take all 256 columns, so no statistics cross warps) and reads it from tensor memory
+        // three times: maximum; sum of exponentials, entropy sum and the target's logit; gradient.
+        static_assert(BN == 256, "a row's vocabulary is one accumulator tile");
+        if (chalf != 0) return;
+        const HeadLossArgs& h = p.hl;
+        const bool valid = row < p.M;
+        const int t = valid ? (int)h.tgt[row] : -1;
+        uint32_t r[32];
+        float mx = -3.0e38f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+        }
+        RowStats st{mx, 0.f, 0.f};
+        float zt = 0.f;
+#pragma unroll 1
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+          tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float z = __uint_as_float(r[e]);
+            const float ex = expf(z - mx);
+            st.se += ex;
+            st.sz += ex * (z - mx);
+            zt = (c0 + e == t) ? z : zt;
+          }
+        }
+        const float lse = hl_lse(st), ent = hl_entropy(st), logp = zt - lse;
+        RowTerms tm{0.f, 0.f, 0.f, 0.f};
+        if (valid) {
+          if (h.mode == HL_TOKEN) tm = hl_token_terms(logp, h.lpo[row], h.adv_c[row / PCM_ACT_DIM], h.lo, h.hi, h.loss_scale);
+          else if (h.mode == HL_COEF) tm.dlogp = h.coef[row];
+          if (h.logp && h.mode != HL_COEF) h.logp[row] = logp;
+        }
+        if (h.part) {
+          float s0 = tm.surrogate, s1 = tm.clipped, s2 = tm.ratio, s3 = valid ? ent : 0.f;
+#pragma unroll
+          for (int off = 16; off; off >>= 1) {
+            s0 += __shfl_xor_sync(0xffffffffu, s0, off); s1 += __shfl_xor_sync(0xffffffffu, s1, off);
+            s2 += __shfl_xor_sync(0xffffffffu, s2, off); s3 += __shfl_xor_sync(0xffffffffu, s3, off);
+          }
+          if (lane_ == 0)
+            *reinterpret_cast<float4*>(h.part + ((long long)(row >> 5)) * 4) = make_float4(s0, s1, s2, s3);   // one entry per 32 rows
+        }
+        if (h.want_dz) {
+          __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(p.C);
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            tmem_ld_32x32(tmem_acc + (uint32_t)c0, r);
+            tmem_ld_wait();
+            float v[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = hl_dz(__uint_as_float(r[e]), lse, ent, tm.dlogp, h.ent_scale, c0 + e == t);
+            staged_store_bf16(stage, lane_, v, dz, p.ldc, row - lane_, p.M, n0 + c0);
+          }
+        }
+      } else if constexpr (EPI == EPI_SWIGLU_FWD) {
         // accumulator columns [0,128) = gate, [128,256) = up, for hidden units hid0 .. hid0+127
         const int hid0 = n0 / 2, F = p.up_row0;
 #pragma unroll 1
@@ -874,6 +937,7 @@ static void fill_params(TcParams& p, const GemmArgs& g) {
   p.out2 = (__nv_bfloat16*)g.epi.out2; p.ld_out2 = g.epi.ld_out2;
   p.rope_tab = g.epi.rope_tab; p.S = g.epi.S; p.dh = g.epi.dh; p.d = g.epi.d;
   p.up_row0 = g.N / 2;
+  p.hl = g.epi.hl;
   p.kb_per_split = 1; p.tiles_m = p.tiles_n = p.splits = 1;
 }
 
@@ -991,12 +1055,18 @@ bool gemm_epilogue_supported(const GemmArgs& g) {
       return e.aux && (e.ld_aux % 8 == 0) && !(((uintptr_t)e.aux) & 15) && (g.N % 32 == 0);
     case EPI_ROPE:
       return e.rope_tab && (e.dh == 64 || e.dh == 128) && e.S > 0 && e.d > 0 && (e.d % 256 == 0) && g.N == 3 * e.d;
+    case EPI_HEAD_LOSS:    // one 256-column tile holds a row's whole vocabulary
+      return g.N == 256 && g.a_kmajor && g.b_kmajor && e.hl.tgt && (!e.hl.want_dz || (g.C && g.ldc == 256)) &&
+             (e.hl.mode == HL_COEF ? e.hl.coef != nullptr : true) &&
+             (e.hl.mode == HL_TOKEN ? (e.hl.lpo && e.hl.adv_c) : true) && !(((uintptr_t)e.hl.part) & 15);
   }
   return false;
 }
 
 // CTA pairs whenever the output is at least one 256-wide tile; single CTAs otherwise (or with PCM_GEMM_PAIR=0)
-static bool wants_pair(const GemmArgs& g) { return pair_enabled() && g.N >= 256 && g.M > TC_BM; }
+static bool wants_pair(const GemmArgs& g) {
+  return pair_enabled() && g.N >= 256 && g.M > TC_BM && g.epi.kind != EPI_HEAD_LOSS;
+}
 bool gemm_tcgen05_pair(const GemmArgs& g) { return wants_pair(g); }
 
 int gemm_tcgen05(const GemmArgs& g, cudaStream_t s) {
@@ -1011,6 +1081,9 @@ int gemm_tcgen05(const GemmArgs& g, cudaStream_t s) {
     case EPI_ROPE:
       if (!gemm_epilogue_supported(g)) return PCM_ERR_SHAPE;
       return pair ? launch_tc2<EPI_ROPE>(g, s) : launch_tc<256, EPI_ROPE>(g, s);
+    case EPI_HEAD_LOSS:
+      if (!gemm_epilogue_supported(g)) return PCM_ERR_SHAPE;
+      return launch_tc<256, EPI_HEAD_LOSS>(g, s);
     default: break;
   }
   if (pair) return launch_tc2<EPI_NONE>(g, s);

@@ -1,6 +1,7 @@
 // Internal interfaces between the translation units of the library (not part of the C ABI).
 #pragma once
 #include "common.cuh"
+#include "head_loss.cuh"
 
 namespace pcm {
 
@@ -12,7 +13,7 @@ enum { DT_F32 = 0, DT_BF16 = 1 };
 //   b_kmajor: B stored [N][K] with row stride ldb;   otherwise B stored [K][N] with row stride ldb.
 // Work fused into the tensor-core GEMM's epilogue (ignored by the SIMT kernel: callers use it only
 // when gemm_tcgen05_supported() holds).
-enum { EPI_NONE = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2, EPI_ROPE = 3 };
+enum { EPI_NONE = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2, EPI_ROPE = 3, EPI_HEAD_LOSS = 4 };
 struct GemmEpilogue {
   int kind = EPI_NONE;
   // EPI_SWIGLU_FWD: B is [2F][K] (gate rows, then up rows); C receives gate | up as [M][2F] and
@@ -23,7 +24,11 @@ struct GemmEpilogue {
   //                 head, position = row % S) with the (cos, sin) table before the bf16 store.
   const void* aux = nullptr; long long ld_aux = 0;
   void* out2 = nullptr; long long ld_out2 = 0;
+  // EPI_HEAD_LOSS:  the product is the logits z [M][256] of the scored rows (N = 256: a row's whole vocabulary is
+  //                 one accumulator tile); the epilogue turns them into log-probs, loss terms and, with
+  //                 hl.want_dz, C = d loss / d z [M][256] bf16.  z is never stored.
   const float2* rope_tab = nullptr; int S = 0, dh = 0, d = 0;
+  HeadLossArgs hl;
 };
 
 struct GemmArgs {

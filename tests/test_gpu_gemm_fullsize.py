@@ -4,8 +4,8 @@ so the oracle computes only the sampled ones).
 
 These shapes reach code the small cases do not: a persistent CTA pair walking tens of tiles with the
 tile position wrapping in all three indices, the wave-filling split of a 119 808-long contraction with
-the fp32 reduction epilogue, and row tiles at the very end of a 119 808-row operand.  Tolerances are
-those of the small GEMM cases: 1e-5 relative for fp32 outputs, 4e-3 for bf16 outputs."""
+the fp32 reduction epilogue, and row tiles at the very end of a 119 808-row operand.  Tolerances: 4e-3 for bf16 outputs as in the small GEMM cases;
+1e-4 for the fp32 weight-gradient reduction over 119 808 terms (derived where it is used)."""
 import numpy as np
 import pytest
 import torch
@@ -83,8 +83,12 @@ def test_weight_gradient_shape_tn_accumulates_into_a_non_zero_start(M, N):
     Xd = _f64(X)
     expect = _f64(dY[:, rows]).T @ Xd + start[rows].cpu().numpy().astype(np.float64)
     got = acc[rows].cpu().numpy()
-    assert rel_fro(got, expect) < 1e-5
+    # A contraction of 119 808 terms is about 830 accumulating MMAs per split and the fp32 accumulator is not
+    # rounded to nearest (addends are aligned and truncated), so the error is a small bias of up to one unit in
+    # the last place per accumulation: bounded by (K / 16 / splits) * 2^-23 ~ 1e-4 relative, measured 4.4e-5.
+    # The 1e-5 of the short contractions does not carry over; 1e-4 does, for the norm, per column tile and per entry.
+    tol = 1e-4
+    assert rel_fro(got, expect) < tol
     for lo in range(0, N, 256):
-        assert rel_fro(got[:, lo:lo + 256], expect[:, lo:lo + 256]) < 1e-5, lo
-    # every entry, not only the norm: the product's entries are O(sqrt(K)) = 350 on a start of O(100)
-    assert np.max(np.abs(got - expect)) < 1e-5 * np.max(np.abs(expect)) * 10
+        assert rel_fro(got[:, lo:lo + 256], expect[:, lo:lo + 256]) < tol, lo
+    assert np.max(np.abs(got - expect)) < tol * np.max(np.abs(expect))
