@@ -12,6 +12,12 @@ and the zero-gradient cases are checked as invariants.  The entropy bonus and th
 pinned by finite differences, by autograd of a library model, by H = log 256 for a zero head, and by the
 on-policy identity (chunk-level and token-level gradients coincide at r = 1 for equal scales).
 
+LoRA (App. E "Training": rank r = 32, alpha = 32): with `lora` given, every linear layer of the decoder computes
+y = x W^T + (alpha / r) (x A^T) B^T with the base weight W frozen; the low-rank branch is evaluated as written
+(never merged into W) and gradients go to A and B, the norm gains, the head and the action embedding.  Pinned by
+finite differences over A and B, by B = 0 giving the dense model's logits, and by the merged-weight identity
+(logits equal those of W + (alpha / r) B A; dA, dB equal the chain rule through the dense model's dW).
+
 Model (every kept chunk is its own sequence of S = P + 56 tokens): pre-norm decoder, RMSNorm,
 rotary position embedding on q and k (base 10000, pairs (i, i + dh/2)), causal softmax attention
 scaled by 1/sqrt(dh), SwiGLU MLP with hidden width 4d, final RMSNorm, linear head over 256 bins.
@@ -94,7 +100,38 @@ def causal_attention_bwd(do, q, k, v, p):
     return ds @ k, ds.transpose(0, 1, 3, 2) @ q, dv
 
 
-def forward(weights: Dict[str, np.ndarray], X, H: int, P: int, keep_cache: bool = True):
+LORA_PROJ = ("qkv", "o", "gu", "d")
+
+
+def lora_linear(x, W, A=None, B=None, scale=1.0):
+    """y = x W^T, plus the adapter's low-rank branch scale * (x A^T) B^T when A [r, in], B [out, r] are given."""
+    y = x @ W.T
+    if A is not None:
+        y = y + scale * ((x @ A.T) @ B.T)
+    return y
+
+
+def lora_linear_bwd(dy, x, W, A=None, B=None, scale=1.0):
+    """Input gradient of lora_linear and, with an adapter, (dA, dB); the base weight is frozen there.
+    Without an adapter returns (dx, dW)."""
+    in_f, out_f = W.shape[1], W.shape[0]
+    dy2, x2 = dy.reshape(-1, out_f), x.reshape(-1, in_f)
+    if A is None:
+        return dy @ W, dy2.T @ x2
+    u = dy @ B                                              # [.., r]
+    dx = dy @ W + scale * (u @ A)
+    dA = scale * (u.reshape(-1, A.shape[0]).T @ x2)
+    dB = scale * (dy2.T @ (x2 @ A.T))
+    return dx, (dA, dB)
+
+
+def _adapter(lora, name, l):
+    if lora is None:
+        return None, None, 1.0
+    return _f64(lora["a_" + name][l]), _f64(lora["b_" + name][l]), float(lora["alpha"]) / float(lora["rank"])
+
+
+def forward(weights: Dict[str, np.ndarray], X, H: int, P: int, keep_cache: bool = True, lora=None):
     """X [n, S, d] -> (z [n, 56, V] logits at the scored positions, cache)."""
     Wt = {k: _f64(v) for k, v in weights.items()}
     x = _f64(X)
@@ -106,19 +143,19 @@ def forward(weights: Dict[str, np.ndarray], X, H: int, P: int, keep_cache: bool 
     for l in range(L):
         x_in = x
         h1, rstd1 = rmsnorm(x_in, Wt["g1"][l])
-        qkv = h1 @ Wt["w_qkv"][l].T
+        qkv = lora_linear(h1, Wt["w_qkv"][l], *_adapter(lora, "qkv", l))
         # heads as [n, H, S, dh]
         q = rope(qkv[..., :d].reshape(n, S, H, dh), cos, sin).transpose(0, 2, 1, 3)
         k = rope(qkv[..., d:2 * d].reshape(n, S, H, dh), cos, sin).transpose(0, 2, 1, 3)
         v = qkv[..., 2 * d:].reshape(n, S, H, dh).transpose(0, 2, 1, 3)
         o, p = causal_attention(q, k, v)
         o = o.transpose(0, 2, 1, 3).reshape(n, S, d)
-        x_mid = x_in + o @ Wt["w_o"][l].T
+        x_mid = x_in + lora_linear(o, Wt["w_o"][l], *_adapter(lora, "o", l))
         h2, rstd2 = rmsnorm(x_mid, Wt["g2"][l])
-        gu = h2 @ Wt["w_gu"][l].T
+        gu = lora_linear(h2, Wt["w_gu"][l], *_adapter(lora, "gu", l))
         g, u = gu[..., :4 * d], gu[..., 4 * d:]
         act = silu(g) * u
-        x = x_mid + act @ Wt["w_d"][l].T
+        x = x_mid + lora_linear(act, Wt["w_d"][l], *_adapter(lora, "d", l))
         if keep_cache:
             layers.append(dict(x_in=x_in, rstd1=rstd1, h1=h1, q=q, k=k, v=v, p=p, o=o, x_mid=x_mid,
                                rstd2=rstd2, h2=h2, g=g, u=u, act=act))
@@ -194,29 +231,30 @@ def objective(z, tgt, logp_old, adv_c, eps_low, eps_high, loss_scale, entropy_co
     return loss, dz, logp, r, active, float(Hrow.mean())
 
 
-def logp_only(weights, X, tgt, H, P):
-    z, _ = forward(weights, X, H, P, keep_cache=False)
+def logp_only(weights, X, tgt, H, P, lora=None):
+    z, _ = forward(weights, X, H, P, keep_cache=False, lora=lora)
     return log_softmax_at(z, tgt)[0]
 
 
 def loss_only(weights, X, tgt, logp_old, adv_c, H, P, eps_low, eps_high, loss_scale, entropy_coef=0.0,
-              ratio_level="token"):
-    z, _ = forward(weights, X, H, P, keep_cache=False)
+              ratio_level="token", lora=None):
+    z, _ = forward(weights, X, H, P, keep_cache=False, lora=lora)
     return objective(z, tgt, logp_old, adv_c, eps_low, eps_high, loss_scale, entropy_coef, ratio_level)[0]
 
 
 def fwd_bwd(weights, X, tgt, logp_old, adv_c, H, P, eps_low=0.2, eps_high=0.2, loss_scale=None, entropy_coef=0.0,
-            ratio_level="token"):
+            ratio_level="token", lora=None):
     """Masked GRPO actor update on the packed batch of kept chunks (Eq. 11).
 
     Returns (loss, logp [n,56], grads dict with the shapes of `weights`, stats).  `loss_scale`
     defaults to the mean over the surrogate's terms: 1/(56 n) with one ratio per token, 1/n with one
     ratio per chunk.  No gradient flows to the observation prefix; the embedding gradient collects
-    the rows at the action-token positions."""
+    the rows at the action-token positions.  With `lora` the four base matrices of every layer are frozen:
+    their entries in `grads` are None and `grads` gains a_qkv, b_qkv, a_o, b_o, a_gu, b_gu, a_d, b_d."""
     n, S, d = np.asarray(X).shape
     if loss_scale is None:
         loss_scale = 1.0 / (ACT_DIM * n) if ratio_level == "token" else 1.0 / n
-    z, cache = forward(weights, X, H, P)
+    z, cache = forward(weights, X, H, P, lora=lora)
     Wt = cache["W"]
     L = Wt["w_qkv"].shape[0]
     dh = d // H
@@ -225,6 +263,22 @@ def fwd_bwd(weights, X, tgt, logp_old, adv_c, H, P, eps_low=0.2, eps_high=0.2, l
     loss, dz, logp, r, active, mean_H = objective(z, tgt, logp_old, adv_c, eps_low, eps_high, loss_scale,
                                                   entropy_coef, ratio_level)              # dz [n,56,V]
     grads = {k: np.zeros_like(v) for k, v in Wt.items()}
+    if lora is not None:
+        for name in LORA_PROJ:
+            grads["w_" + name] = None
+            grads["a_" + name] = np.zeros(np.asarray(lora["a_" + name]).shape)
+            grads["b_" + name] = np.zeros(np.asarray(lora["b_" + name]).shape)
+
+    def linear_bwd(name, l, dy, x_in_):
+        """dx of projection `name` in layer l; stores dW, or (dA, dB) when the base weight is frozen."""
+        A, B, sc = _adapter(lora, name, l)
+        dx_, gw = lora_linear_bwd(dy, x_in_, Wt["w_" + name][l], A, B, sc)
+        if lora is None:
+            grads["w_" + name][l] = gw
+        else:
+            grads["a_" + name][l], grads["b_" + name][l] = gw
+        return dx_
+
     V = dz.shape[-1]
     grads["w_h"] = dz.reshape(n * ACT_DIM, V).T @ cache["hf"].reshape(n * ACT_DIM, d)
     dhf = dz @ Wt["w_h"]
@@ -235,26 +289,22 @@ def fwd_bwd(weights, X, tgt, logp_old, adv_c, H, P, eps_low=0.2, eps_high=0.2, l
     for l in reversed(range(L)):
         c = cache["layers"][l]
         # x = x_mid + act @ W_d^T
-        grads["w_d"][l] = dx.reshape(n * S, d).T @ c["act"].reshape(n * S, 4 * d)
-        dact = dx @ Wt["w_d"][l]
+        dact = linear_bwd("d", l, dx, c["act"])
         sg = 1.0 / (1.0 + np.exp(-c["g"]))
         dg = dact * c["u"] * (sg * (1.0 + c["g"] * (1.0 - sg)))
         du = dact * (c["g"] * sg)
         dgu = np.concatenate([dg, du], axis=-1)
-        grads["w_gu"][l] = dgu.reshape(n * S, 8 * d).T @ c["h2"].reshape(n * S, d)
-        dh2 = dgu @ Wt["w_gu"][l]
+        dh2 = linear_bwd("gu", l, dgu, c["h2"])
         dxm, grads["g2"][l] = rmsnorm_bwd(dh2, c["x_mid"], c["rstd2"], Wt["g2"][l])
         dx_mid = dx + dxm
         # x_mid = x_in + o @ W_o^T
-        grads["w_o"][l] = dx_mid.reshape(n * S, d).T @ c["o"].reshape(n * S, d)
-        do = (dx_mid @ Wt["w_o"][l]).reshape(n, S, H, dh).transpose(0, 2, 1, 3)   # [n, H, S, dh]
+        do = linear_bwd("o", l, dx_mid, c["o"]).reshape(n, S, H, dh).transpose(0, 2, 1, 3)   # [n, H, S, dh]
         dq, dk, dv = causal_attention_bwd(do, c["q"], c["k"], c["v"], c["p"])
         dq = rope_bwd(dq.transpose(0, 2, 1, 3), cos, sin)                           # [n, S, H, dh]
         dk = rope_bwd(dk.transpose(0, 2, 1, 3), cos, sin)
         dv = dv.transpose(0, 2, 1, 3)
         dqkv = np.concatenate([dq.reshape(n, S, d), dk.reshape(n, S, d), dv.reshape(n, S, d)], axis=-1)
-        grads["w_qkv"][l] = dqkv.reshape(n * S, 3 * d).T @ c["h1"].reshape(n * S, d)
-        dh1 = dqkv @ Wt["w_qkv"][l]
+        dh1 = linear_bwd("qkv", l, dqkv, c["h1"])
         dxi, grads["g1"][l] = rmsnorm_bwd(dh1, c["x_in"], c["rstd1"], Wt["g1"][l])
         dx = dx_mid + dxi
 

@@ -362,3 +362,94 @@ def test_chunk_level_ratio_on_policy_identity_and_joint_clipping():
     _, _, g1, _ = ao.fwd_bwd(W, X[1:2], tgt[1:2], lpo[1:2], adv[1:2], 2, 4, 0.2, 0.4, loss_scale=1 / 3, ratio_level="chunk")
     for k in W:
         assert np.allclose(g[k], g1[k], rtol=1e-9, atol=1e-14), k
+
+
+# ------------------------------------------------------------------ LoRA (App. E: r = 32, alpha = 32)
+def tiny_lora(rng, W, rank=4, alpha=6.0, b_scale=0.2):
+    L, d = W["g1"].shape
+    dims = {"qkv": (d, 3 * d), "o": (d, d), "gu": (d, 8 * d), "d": (4 * d, d)}
+    lo = {"rank": rank, "alpha": alpha}
+    for name, (fin, fout) in dims.items():
+        lo["a_" + name] = 0.3 * rng.standard_normal((L, rank, fin))
+        lo["b_" + name] = b_scale * rng.standard_normal((L, fout, rank))
+    return lo
+
+
+def merged_weights(W, lo):
+    s = lo["alpha"] / lo["rank"]
+    Wm = dict(W)
+    for name in ao.LORA_PROJ:
+        Wm["w_" + name] = W["w_" + name] + s * np.einsum("lor,lri->loi", lo["b_" + name], lo["a_" + name])
+    return Wm
+
+
+def test_lora_with_zero_b_is_the_dense_model():
+    rng = np.random.default_rng(41)
+    W = tiny_model(rng)
+    X, tgt, adv = tiny_batch(rng, W)
+    lo = tiny_lora(rng, W, b_scale=0.0)
+    z0, _ = ao.forward(W, X, 2, 4)
+    z1, _ = ao.forward(W, X, 2, 4, lora=lo)
+    assert np.array_equal(z0, z1)
+    # B = 0: no signal reaches A, and dB is what the dense weight gradient projects onto A
+    lpo = ao.logp_only(W, X, tgt, 2, 4) + 0.01 * rng.standard_normal((3, 56))
+    _, _, g_dense, _ = ao.fwd_bwd(W, X, tgt, lpo, adv, 2, 4, loss_scale=1.0)
+    _, _, g, _ = ao.fwd_bwd(W, X, tgt, lpo, adv, 2, 4, loss_scale=1.0, lora=lo)
+    s = lo["alpha"] / lo["rank"]
+    for name in ao.LORA_PROJ:
+        assert g["w_" + name] is None
+        assert np.all(g["a_" + name] == 0.0)
+        expect = s * np.einsum("loi,lri->lor", g_dense["w_" + name], lo["a_" + name])
+        assert np.allclose(g["b_" + name], expect, rtol=1e-11, atol=1e-13)
+
+
+def test_lora_equals_the_merged_dense_model_and_its_chain_rule():
+    rng = np.random.default_rng(42)
+    W = tiny_model(rng)
+    X, tgt, adv = tiny_batch(rng, W)
+    lo = tiny_lora(rng, W)
+    Wm = merged_weights(W, lo)
+    z_l, _ = ao.forward(W, X, 2, 4, lora=lo)
+    z_m, _ = ao.forward(Wm, X, 2, 4)
+    assert np.allclose(z_l, z_m, rtol=1e-11, atol=1e-12)
+    assert not np.allclose(z_l, ao.forward(W, X, 2, 4)[0], atol=1e-3)          # the adapters do change the policy
+    lpo = ao.logp_only(Wm, X, tgt, 2, 4) + 0.2 * rng.standard_normal((3, 56))
+    loss_m, _, g_m, st_m = ao.fwd_bwd(Wm, X, tgt, lpo, adv, 2, 4, 0.2, 0.4, loss_scale=1.0, entropy_coef=1e-3)
+    loss_l, _, g_l, st_l = ao.fwd_bwd(W, X, tgt, lpo, adv, 2, 4, 0.2, 0.4, loss_scale=1.0, entropy_coef=1e-3, lora=lo)
+    assert loss_l == pytest.approx(loss_m, rel=1e-12)
+    assert 0.0 < st_l["clip_frac"] == pytest.approx(st_m["clip_frac"])
+    s = lo["alpha"] / lo["rank"]
+    for name in ao.LORA_PROJ:
+        dW = g_m["w_" + name]                                                   # W_eff = W + s B A
+        assert np.allclose(g_l["a_" + name], s * np.einsum("lor,loi->lri", lo["b_" + name], dW), rtol=1e-10, atol=1e-12)
+        assert np.allclose(g_l["b_" + name], s * np.einsum("loi,lri->lor", dW, lo["a_" + name]), rtol=1e-10, atol=1e-12)
+    for name in ("g1", "g2", "gf", "w_h", "e_act"):                             # the rest sees the same function
+        assert np.allclose(g_l[name], g_m[name], rtol=1e-10, atol=1e-12), name
+
+
+def test_lora_gradient_matches_central_finite_differences():
+    rng = np.random.default_rng(43)
+    W = tiny_model(rng)
+    X, tgt, adv = tiny_batch(rng, W)
+    lo = tiny_lora(rng, W)
+    lpo = ao.logp_only(W, X, tgt, 2, 4, lora=lo) + 0.01 * rng.standard_normal((3, 56))
+    loss, _, g, _ = ao.fwd_bwd(W, X, tgt, lpo, adv, 2, 4, 0.2, 0.4, loss_scale=1.0, lora=lo)
+
+    def f(lp):
+        return ao.loss_only(W, X, tgt, lpo, adv, 2, 4, 0.2, 0.4, 1.0, lora=lp)
+
+    assert f(lo) == pytest.approx(loss, rel=1e-13)
+    for name in ao.LORA_PROJ:
+        for key in ("a_" + name, "b_" + name):
+            v = rng.standard_normal(lo[key].shape)
+            h = 1e-5
+            lp = dict(lo); lp[key] = lo[key] + h * v
+            lm = dict(lo); lm[key] = lo[key] - h * v
+            fd = (f(lp) - f(lm)) / (2 * h)
+            assert float(np.sum(g[key] * v)) == pytest.approx(fd, rel=2e-6, abs=1e-9), key
+            flat = lo[key].reshape(-1)
+            for idx in rng.choice(flat.size, size=6, replace=False):
+                lp = dict(lo); a = lo[key].copy(); a.reshape(-1)[idx] += h; lp[key] = a
+                lm = dict(lo); b = lo[key].copy(); b.reshape(-1)[idx] -= h; lm[key] = b
+                fd = (f(lp) - f(lm)) / (2 * h)
+                assert g[key].reshape(-1)[idx] == pytest.approx(fd, rel=1e-5, abs=1e-9), (key, idx)
