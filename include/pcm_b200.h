@@ -293,6 +293,43 @@ int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* batch, const 
                        grpo_grads* grads, float* loss, float* logp, grpo_stats* stats,
                        void* workspace, size_t workspace_bytes, pcm_stream stream);
 
+/* ---- LoRA fine-tuning (App. E "Training": LoRA rank r = 32, alpha = 32) -----------------------------------
+ * The regime the paper trains in: the four weight matrices of every decoder layer stay frozen and each gets a
+ * low-rank adapter, y = x W^T + (alpha / rank) (x A^T) B^T.  The adapter branch is evaluated as written (never
+ * merged into W, which would round a small update away in bf16): t = (alpha / rank) x A^T is formed first and enters
+ * the same tensor-core accumulator as x W^T through a continuation of the contraction, before the fused rotary /
+ * SwiGLU epilogues; backward likewise with u = (alpha / rank) dy B, dx = dy W + u A, dA += u^T x, dB += dy^T t.
+ * No gradient of W_qkv, W_o, W_gu, W_d is formed (a third of the dense update's linear flops).
+ * Adapter tensors are device, in cfg.dtype; rank a multiple of 8, 8..64 (32 or 64 run entirely on the tensor-core
+ * kernels; other ranks send the adapters' own small products through the SIMT kernel). */
+typedef struct {
+  int32_t rank;
+  float alpha;                 /* scale = alpha / rank, > 0                                         */
+  const void* a_qkv;           /* [L][rank][d]                                                      */
+  const void* b_qkv;           /* [L][3d][rank]                                                     */
+  const void* a_o;             /* [L][rank][d]                                                      */
+  const void* b_o;             /* [L][d][rank]                                                      */
+  const void* a_gu;            /* [L][rank][d]                                                      */
+  const void* b_gu;            /* [L][8d][rank]                                                     */
+  const void* a_d;             /* [L][rank][4d]                                                     */
+  const void* b_d;             /* [L][d][rank]                                                      */
+} grpo_lora;
+
+/* fp32 gradients with the shapes of the adapter tensors (device). */
+typedef struct {
+  float* a_qkv; float* b_qkv; float* a_o; float* b_o; float* a_gu; float* b_gu; float* a_d; float* b_d;
+} grpo_lora_grads;
+
+/* Workspace of grpo_actor_fwd_bwd_lora (0 when cfg or rank is not supported). */
+size_t grpo_lora_workspace_bytes(const grpo_model_cfg* cfg, int32_t rank, int32_t mb_chunks, uint32_t flags);
+
+/* grpo_actor_fwd_bwd with adapters.  Same batch, loss configuration, outputs and error behaviour.  grads receives
+ * g1, g2, gf, w_h, e_act (its w_qkv, w_o, w_gu, w_d are ignored and may be NULL); lora_grads receives the adapter
+ * gradients (both ignored with GRPO_FWD_ONLY; GRPO_ACCUMULATE adds into both). */
+int grpo_actor_fwd_bwd_lora(const grpo_model* model, const grpo_lora* lora, const grpo_packed* batch,
+                            const grpo_loss_cfg* loss_cfg, grpo_grads* grads, grpo_lora_grads* lora_grads, float* loss,
+                            float* logp, grpo_stats* stats, void* workspace, size_t workspace_bytes, pcm_stream stream);
+
 /* ---- optimizer step (App. E: AdamW, lr 1e-5, betas (0.9, 0.999), weight decay 0, clipping at 2.0) -----
  * The step that follows grpo_actor_fwd_bwd.  Global L2 norm of all gradients (fp64 partial sums in a fixed
  * order), clip coefficient min(1, max_grad_norm / (norm + 1e-6)) (max_grad_norm = 0: no clipping), then per

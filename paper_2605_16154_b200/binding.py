@@ -78,6 +78,17 @@ class grpo_stats(C.Structure):
                 ("n_launches", C.c_int32), ("reserved", C.c_int32), ("workspace_high_water", C.c_uint64)]
 
 
+_LORA = ("a_qkv", "b_qkv", "a_o", "b_o", "a_gu", "b_gu", "a_d", "b_d")
+
+
+class grpo_lora(C.Structure):
+    _fields_ = [("rank", C.c_int32), ("alpha", C.c_float)] + [(n, C.c_void_p) for n in _LORA]
+
+
+class grpo_lora_grads(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _LORA]
+
+
 class grpo_adamw_cfg(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("weight_decay", C.c_float), ("max_grad_norm", C.c_float)]
@@ -107,6 +118,12 @@ _lib.grpo_workspace_bytes.argtypes = [C.POINTER(grpo_model_cfg), C.c_int32, C.c_
 _lib.grpo_workspace_bytes.restype = C.c_size_t
 _lib.grpo_actor_fwd_bwd.argtypes = [C.POINTER(grpo_model), C.POINTER(grpo_packed), C.POINTER(grpo_loss_cfg),
                                     C.POINTER(grpo_grads), _P, _P, C.POINTER(grpo_stats), _P, C.c_size_t, _P]
+_lib.grpo_lora_workspace_bytes.argtypes = [C.POINTER(grpo_model_cfg), C.c_int32, C.c_int32, C.c_uint32]
+_lib.grpo_lora_workspace_bytes.restype = C.c_size_t
+_lib.grpo_actor_fwd_bwd_lora.argtypes = [C.POINTER(grpo_model), C.POINTER(grpo_lora), C.POINTER(grpo_packed),
+                                         C.POINTER(grpo_loss_cfg), C.POINTER(grpo_grads), C.POINTER(grpo_lora_grads), _P, _P,
+                                         C.POINTER(grpo_stats), _P, C.c_size_t, _P]
+_lib.grpo_actor_fwd_bwd_lora.restype = C.c_int
 _lib.grpo_gemm.argtypes = [C.c_int32, C.c_int32, C.c_int32, _P, C.c_int64, C.c_int32, _P, C.c_int64, C.c_int32,
                            C.c_int32, _P, C.c_int64, C.c_int32, _P, C.c_int64, C.c_int32, _P]
 _lib.grpo_attention.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _P]
@@ -136,7 +153,8 @@ EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", 
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
             "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static",
             "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases", "pcm_score_phases_f32",
-            "grpo_attention_wait_status", "pcm_first_use_on_device")
+            "grpo_attention_wait_status", "pcm_first_use_on_device", "grpo_lora_workspace_bytes",
+            "grpo_actor_fwd_bwd_lora")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -304,6 +322,25 @@ class Model:
         return self.grads
 
 
+class Lora:
+    """Device adapter tensors (App. E: rank 32, alpha 32) of a Model, with the matching C structures."""
+
+    def __init__(self, model: Model, rank: int, alpha: float, tensors: Dict[str, torch.Tensor]):
+        self.rank, self.alpha = rank, alpha
+        self.tensors = {k: tensors[k].contiguous() for k in _LORA}
+        for k, t in self.tensors.items():
+            assert t.is_cuda and t.dtype == _torch_dtype(model.cfg.dtype), k
+        self.c = grpo_lora(rank, alpha, *[_ptr(self.tensors[k]) for k in _LORA])
+        self.grads: Optional[Dict[str, torch.Tensor]] = None
+        self.c_grads: Optional[grpo_lora_grads] = None
+
+    def alloc_grads(self) -> Dict[str, torch.Tensor]:
+        if self.grads is None:
+            self.grads = {k: torch.zeros(v.shape, dtype=torch.float32, device=v.device) for k, v in self.tensors.items()}
+            self.c_grads = grpo_lora_grads(*[_ptr(self.grads[k]) for k in _LORA])
+        return self.grads
+
+
 class Packed:
     """Caller-allocated dense batch of kept chunks."""
 
@@ -326,7 +363,9 @@ def grpo_pack_chunks(ctx: Context, batch: pcm_batch, model, kept_idx, kept_off, 
     return out
 
 
-def grpo_workspace_bytes(model: Model, mb_chunks: int, flags: int = 0) -> int:
+def grpo_workspace_bytes(model: Model, mb_chunks: int, flags: int = 0, lora: Optional[Lora] = None) -> int:
+    if lora is not None:
+        return int(_lib.grpo_lora_workspace_bytes(C.byref(model.cfg), lora.rank, mb_chunks, flags))
     return int(_lib.grpo_workspace_bytes(C.byref(model.cfg), mb_chunks, flags))
 
 
@@ -334,11 +373,13 @@ def grpo_actor_fwd_bwd(model: Model, packed: Packed, eps_low: float = 0.2, eps_h
                        loss_scale: float = 0.0, mb_chunks: int = 64, flags: int = 0,
                        workspace: Optional[torch.Tensor] = None, want_stats: bool = True,
                        logp: Optional[torch.Tensor] = None, loss: Optional[torch.Tensor] = None,
-                       entropy_coef: float = 0.0):
-    """Returns (loss tensor[1] on the device, logp [n_kept, 56], grads dict or None, stats or None)."""
+                       entropy_coef: float = 0.0, lora: Optional[Lora] = None):
+    """Returns (loss tensor[1] on the device, logp [n_kept, 56], grads dict or None, stats or None).
+    With `lora` the base matrices are frozen (their entries of the grads dict are left untouched) and the
+    adapter gradients are in lora.grads."""
     dev = torch.device("cuda")
     mb = max(1, min(mb_chunks, max(packed.n_kept, 1)))
-    need = grpo_workspace_bytes(model, mb, flags)
+    need = grpo_workspace_bytes(model, mb, flags, lora)
     if need == 0:
         raise PcmError("grpo_workspace_bytes", -2)
     if workspace is None:
@@ -356,9 +397,17 @@ def grpo_actor_fwd_bwd(model: Model, packed: Packed, eps_low: float = 0.2, eps_h
     if not fwd_only:
         grads = model.alloc_grads()
     stats = grpo_stats() if want_stats else None
-    rc = _lib.grpo_actor_fwd_bwd(C.byref(model.c_model), C.byref(packed.c), C.byref(lc),
-                                 C.byref(model.c_grads) if not fwd_only else None, _ptr(loss), _ptr(logp),
-                                 C.byref(stats) if stats is not None else None, ws_ptr, ws_bytes, _stream())
+    if lora is None:
+        rc = _lib.grpo_actor_fwd_bwd(C.byref(model.c_model), C.byref(packed.c), C.byref(lc),
+                                     C.byref(model.c_grads) if not fwd_only else None, _ptr(loss), _ptr(logp),
+                                     C.byref(stats) if stats is not None else None, ws_ptr, ws_bytes, _stream())
+    else:
+        if not fwd_only:
+            lora.alloc_grads()
+        rc = _lib.grpo_actor_fwd_bwd_lora(C.byref(model.c_model), C.byref(lora.c), C.byref(packed.c), C.byref(lc),
+                                          C.byref(model.c_grads) if not fwd_only else None,
+                                          C.byref(lora.c_grads) if not fwd_only else None, _ptr(loss), _ptr(logp),
+                                          C.byref(stats) if stats is not None else None, ws_ptr, ws_bytes, _stream())
     _check("grpo_actor_fwd_bwd", rc)
     return loss, logp, grads, stats
 

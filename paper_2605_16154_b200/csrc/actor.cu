@@ -77,6 +77,41 @@ __global__ void to_residual_kernel(const T* __restrict__ x, float* __restrict__ 
 }
 
 // ------------------------------------------------------------------------------------------------
+// Scored rows of the last layer.  Only positions P-1 .. P+54 of a chunk feed the head, so after the last attention
+// the layer continues on those 56 rows per chunk.  gather: compact row r <- full row map_row(r); scatter: the
+// reverse (the caller zeroes the full tensors first).  One thread moves four columns of both tensors.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void gather_scored_rows_kernel(const T* __restrict__ a_full, const float* __restrict__ x_full, T* __restrict__ a_s,
+                                          float* __restrict__ x_s, long long rows, int S, int P, int d) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = d / 4;
+  if (idx >= rows * per_row) return;
+  const long long r = idx / per_row;
+  const int c = (int)(idx - r * per_row) * 4;
+  const long long src = map_row(r, S, P) * d + c, dst = r * d + c;
+  float v[4];
+  load4<T>(a_full + src, v);
+  store4<T>(a_s + dst, v[0], v[1], v[2], v[3]);
+  *reinterpret_cast<float4*>(x_s + dst) = *reinterpret_cast<const float4*>(x_full + src);
+}
+
+template <typename T>
+__global__ void scatter_scored_rows_kernel(const T* __restrict__ a_s, const float* __restrict__ x_s, T* __restrict__ a_full,
+                                           float* __restrict__ x_full, long long rows, int S, int P, int d) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int per_row = d / 4;
+  if (idx >= rows * per_row) return;
+  const long long r = idx / per_row;
+  const int c = (int)(idx - r * per_row) * 4;
+  const long long dst = map_row(r, S, P) * d + c, src = r * d + c;
+  float v[4];
+  load4<T>(a_s + src, v);
+  store4<T>(a_full + dst, v[0], v[1], v[2], v[3]);
+  *reinterpret_cast<float4*>(x_full + dst) = *reinterpret_cast<const float4*>(x_s + src);
+}
+
+// ------------------------------------------------------------------------------------------------
 // RMSNorm forward: one warp per row.  x fp32 [.][d] (rows optionally gathered), h T [rows][d].
 // ------------------------------------------------------------------------------------------------
 template <typename T>
@@ -553,35 +588,47 @@ struct Arena {
   }
 };
 
+// The four linear maps of a decoder layer, in the order the adapter tensors of grpo_lora use.
+enum { PJ_QKV = 0, PJ_O = 1, PJ_GU = 2, PJ_D = 3 };
+
 struct LayerActs {
   void* h1; void* qkv; void* attn; float* lse; float* rstd1; float* x_mid; float* rstd2; void* h2; void* gu; void* act;
+  void* lt[4];                   // adapters: alpha/r * (input of the projection) A^T, kept for dB
 };
 
 struct Workspace {
   float2* rope_tab;
-  float* x[129];                 // residual stream, x[0..L]
+  float* x[129];                 // residual stream, x[0..L]; x[L] holds the scored rows only
   LayerActs la[128];
   void* hs; float* rstdf; void* dz; float* loss_part; float* loss_acc; float* logp_tmp; float* coef;
   float* dx; void* dx_t; void* dact; void* dgu; float* dh; void* dattn; void* dqkv; float* dsum;
   float* norm_part; float* dhs;
+  // the last layer's post-attention part runs on the scored rows only (nothing reads the others)
+  void* attn_s; float* xin_s; float* dxs; void* dxs_t; void* dattn_s;
+  void* lu;                      // adapters: alpha/r * (output gradient of the projection) B
   size_t bytes;
 };
 
-static void carve(Workspace& w, unsigned char* base, const grpo_model_cfg& c, int mb, bool fwd_only) {
+// lora_r: adapter rank (0: none).  keep_dact: the SwiGLU backward is not fused into the GEMM epilogue.
+static void carve(Workspace& w, unsigned char* base, const grpo_model_cfg& c, int mb, bool fwd_only, int lora_r,
+                  bool keep_dact) {
   Arena a{base, 0};
   const size_t es = c.dtype == GRPO_BF16 ? 2 : 4;
   const int S = c.prefix_len + ACT, d = c.d, H = c.n_heads, L = c.n_layers;
-  const size_t M = (size_t)mb * S, R = (size_t)mb * ACT;
+  const size_t M = (size_t)mb * S, R = (size_t)mb * ACT, r = (size_t)lora_r;
   w.rope_tab = (float2*)a.take((size_t)S * (d / H / 2) * sizeof(float2));
   // with backward every layer keeps its activations; forward-only reuses one layer's worth
   const int kept_layers = fwd_only ? 1 : L;
-  for (int l = 0; l <= (fwd_only ? 1 : L); ++l) w.x[l] = (float*)a.take(M * d * 4);
+  for (int l = 0; l <= (fwd_only ? 1 : L); ++l) w.x[l] = (float*)a.take(((!fwd_only && l == L) ? R : M) * d * 4);
   for (int l = 0; l < kept_layers; ++l) {
     LayerActs& la = w.la[l];
+    const size_t Mp = (!fwd_only && l == L - 1) ? R : M;          // rows of the post-attention part
     la.h1 = a.take(M * d * es); la.qkv = a.take(M * 3 * d * es); la.attn = a.take(M * d * es);
     la.lse = (float*)a.take((size_t)mb * H * S * 4); la.rstd1 = (float*)a.take(M * 4);
-    la.x_mid = (float*)a.take(M * d * 4); la.rstd2 = (float*)a.take(M * 4); la.h2 = a.take(M * d * es);
-    la.gu = a.take(M * 8 * d * es); la.act = a.take(M * 4 * d * es);
+    la.x_mid = (float*)a.take(Mp * d * 4); la.rstd2 = (float*)a.take(Mp * 4); la.h2 = a.take(Mp * d * es);
+    la.gu = a.take(Mp * 8 * d * es); la.act = a.take(Mp * 4 * d * es);
+    la.lt[PJ_QKV] = a.take(M * r * es);
+    for (int pj = PJ_O; pj <= PJ_D; ++pj) la.lt[pj] = a.take(Mp * r * es);
   }
   if (fwd_only) {
     for (int l = 1; l < L; ++l) w.la[l] = w.la[0];
@@ -592,11 +639,15 @@ static void carve(Workspace& w, unsigned char* base, const grpo_model_cfg& c, in
   // loss partial sums: one entry of 4 per head block (at most one per 8 rows) plus one per chunk
   w.loss_part = (float*)a.take(((size_t)mb * (ACT / HL_ROWS) + (size_t)mb + 8) * 4 * 4); w.loss_acc = (float*)a.take(256);
   w.logp_tmp = (float*)a.take(R * 4); w.coef = (float*)a.take(R * 4);
+  w.attn_s = a.take(R * d * es); w.xin_s = (float*)a.take(R * d * 4);
   if (!fwd_only) {
-    w.dx = (float*)a.take(M * d * 4); w.dx_t = a.take(M * d * es); w.dact = a.take(M * 4 * d * es);
+    w.dx = (float*)a.take(M * d * 4); w.dx_t = a.take(M * d * es);
+    w.dact = keep_dact ? a.take(M * 4 * d * es) : nullptr;
     w.dgu = a.take(M * 8 * d * es); w.dh = (float*)a.take(M * d * 4); w.dattn = a.take(M * d * es);
     w.dqkv = a.take(M * 3 * d * es); w.dsum = (float*)a.take((size_t)mb * H * S * 4);
     w.norm_part = (float*)a.take((size_t)NORM_BWD_BLOCKS * d * 4); w.dhs = (float*)a.take(R * d * 4);
+    w.dxs = (float*)a.take(R * d * 4); w.dxs_t = a.take(R * d * es); w.dattn_s = a.take(R * d * es);
+    w.lu = a.take(M * r * es);
   }
   w.bytes = a.off;
 }
@@ -613,11 +664,36 @@ static int check_cfg(const grpo_model_cfg* c) {
   return PCM_OK;
 }
 
+static int check_lora(const grpo_lora* lo) {
+  if (!lo) return PCM_ERR_ARG;
+  if (lo->rank < 8 || lo->rank > 64 || (lo->rank % 8)) return PCM_ERR_SHAPE;
+  if (!(lo->alpha > 0.f)) return PCM_ERR_ARG;
+  if (!lo->a_qkv || !lo->b_qkv || !lo->a_o || !lo->b_o || !lo->a_gu || !lo->b_gu || !lo->a_d || !lo->b_d) return PCM_ERR_ARG;
+  return PCM_OK;
+}
+
 static GemmBackend backend_from_env();
 
+// bf16 on the tensor-core path: SwiGLU and the rotary embedding run inside GEMM / attention epilogues
+static void fused_epilogues(const grpo_model_cfg& c, bool* swiglu, bool* rope) {
+  *swiglu = *rope = false;
+  if (c.dtype != GRPO_BF16 || backend_from_env() == GEMM_SIMT) return;
+  const int d = c.d, dh = d / c.n_heads;
+  // operand addresses only have to be aligned like real ones for the probe
+  void* any = reinterpret_cast<void*>(uintptr_t(4096));
+  GemmArgs probe{128, 8 * d, d, any, d, true, any, d, true, DT_BF16, any, 8 * d, DT_BF16, nullptr, 0};
+  probe.epi.kind = EPI_SWIGLU_FWD; probe.epi.out2 = any; probe.epi.ld_out2 = 4 * d;
+  *swiglu = gemm_epilogue_supported(probe);
+  GemmArgs probe2{128, 3 * d, d, any, d, true, any, d, true, DT_BF16, any, 3 * d, DT_BF16, nullptr, 0};
+  probe2.epi.kind = EPI_ROPE; probe2.epi.rope_tab = reinterpret_cast<const float2*>(any);
+  probe2.epi.S = c.prefix_len + ACT; probe2.epi.dh = dh; probe2.epi.d = d;
+  *rope = gemm_epilogue_supported(probe2);
+}
+
 template <typename T>
-static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* lc, grpo_grads* gr, float* loss,
-               float* logp, grpo_stats* stats, void* workspace, size_t workspace_bytes, cudaStream_t s) {
+static int run(const grpo_model* m, const grpo_lora* lo, const grpo_packed* pk, const grpo_loss_cfg* lc, grpo_grads* gr,
+               grpo_lora_grads* lg, float* loss, float* logp, grpo_stats* stats, void* workspace, size_t workspace_bytes,
+               cudaStream_t s) {
   const grpo_model_cfg& c = m->cfg;
   const int d = c.d, L = c.n_layers, H = c.n_heads, dh = d / H, P = c.prefix_len, S = P + ACT;
   const int dt = c.dtype == GRPO_BF16 ? DT_BF16 : DT_F32;
@@ -629,23 +705,47 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
   const float loss_scale = lc->loss_scale > 0.f ? lc->loss_scale : 1.0f / n_terms;
   const float ent_scale = lc->entropy_coef / ((float)ACT * (float)(n > 0 ? n : 1));   // coefficient x token mean
   const long long launches0 = g_launches.load();
+  const int r = lo ? lo->rank : 0;
+  const float lora_scale = lo ? lo->alpha / (float)lo->rank : 1.f;
 
+  bool fuse_swiglu = false, fuse_rope = false;
+  fused_epilogues(c, &fuse_swiglu, &fuse_rope);
   Workspace w;
   memset(&w, 0, sizeof(w));
-  carve(w, (unsigned char*)workspace, c, mb_max, fwd_only);
+  carve(w, (unsigned char*)workspace, c, mb_max, fwd_only, r, !fuse_swiglu);
   if (w.bytes > workspace_bytes) return PCM_ERR_WORKSPACE;
 
-  const T* w_qkv = (const T*)m->w_qkv; const T* w_o = (const T*)m->w_o; const T* w_gu = (const T*)m->w_gu;
-  const T* w_d = (const T*)m->w_d; const T* g1 = (const T*)m->g1; const T* g2 = (const T*)m->g2;
+  const T* g1 = (const T*)m->g1; const T* g2 = (const T*)m->g2;
   const T* gf = (const T*)m->gf; const T* w_h = (const T*)m->w_h;
+  // per projection: base weight [L][out][in], adapters A [L][r][in] and B [L][out][r], and their gradients
+  const int p_in[4] = {d, d, d, 4 * d}, p_out[4] = {3 * d, d, 8 * d, d};
+  const T* p_w[4] = {(const T*)m->w_qkv, (const T*)m->w_o, (const T*)m->w_gu, (const T*)m->w_d};
+  float* p_dw[4] = {nullptr, nullptr, nullptr, nullptr};
+  const T* p_a[4] = {nullptr, nullptr, nullptr, nullptr};
+  const T* p_b[4] = {nullptr, nullptr, nullptr, nullptr};
+  float* p_da[4] = {nullptr, nullptr, nullptr, nullptr};
+  float* p_db[4] = {nullptr, nullptr, nullptr, nullptr};
+  if (lo) {
+    const void* as[4] = {lo->a_qkv, lo->a_o, lo->a_gu, lo->a_d};
+    const void* bs[4] = {lo->b_qkv, lo->b_o, lo->b_gu, lo->b_d};
+    for (int pj = 0; pj < 4; ++pj) { p_a[pj] = (const T*)as[pj]; p_b[pj] = (const T*)bs[pj]; }
+    if (!fwd_only) {
+      float* das[4] = {lg->a_qkv, lg->a_o, lg->a_gu, lg->a_d};
+      float* dbs[4] = {lg->b_qkv, lg->b_o, lg->b_gu, lg->b_d};
+      for (int pj = 0; pj < 4; ++pj) { p_da[pj] = das[pj]; p_db[pj] = dbs[pj]; }
+    }
+  } else if (!fwd_only) {
+    p_dw[PJ_QKV] = gr->w_qkv; p_dw[PJ_O] = gr->w_o; p_dw[PJ_GU] = gr->w_gu; p_dw[PJ_D] = gr->w_d;
+  }
 
   // gradients start from zero unless the caller accumulates
   if (!fwd_only && !(lc->flags & GRPO_ACCUMULATE)) {
-    const size_t dd = (size_t)d * d;
-    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_qkv, 0, (size_t)L * 3 * dd * 4, s));
-    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_o, 0, (size_t)L * dd * 4, s));
-    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_gu, 0, (size_t)L * 8 * dd * 4, s));
-    PCM_CUDA_TRY(cudaMemsetAsync(gr->w_d, 0, (size_t)L * 4 * dd * 4, s));
+    for (int pj = 0; pj < 4; ++pj) {
+      const size_t io = (size_t)p_in[pj] * p_out[pj];
+      if (p_dw[pj]) PCM_CUDA_TRY(cudaMemsetAsync(p_dw[pj], 0, (size_t)L * io * 4, s));
+      if (p_da[pj]) PCM_CUDA_TRY(cudaMemsetAsync(p_da[pj], 0, (size_t)L * r * p_in[pj] * 4, s));
+      if (p_db[pj]) PCM_CUDA_TRY(cudaMemsetAsync(p_db[pj], 0, (size_t)L * r * p_out[pj] * 4, s));
+    }
     PCM_CUDA_TRY(cudaMemsetAsync(gr->g1, 0, (size_t)L * d * 4, s));
     PCM_CUDA_TRY(cudaMemsetAsync(gr->g2, 0, (size_t)L * d * 4, s));
     PCM_CUDA_TRY(cudaMemsetAsync(gr->gf, 0, (size_t)d * 4, s));
@@ -657,27 +757,57 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
   rope_table_kernel<<<ceil_div((long long)S * dh / 2, 256), 256, 0, s>>>(w.rope_tab, S, dh);
   PCM_LAUNCH_CHECK();
 
+  auto GX = [&](const GemmArgs& g) -> int {
+    prof_begin(gemm_runs_on_pairs(g) ? PC_GEMM : PC_GEMM_SMALL, s);
+    const int rc = gemm(g, s);
+    prof_end(s, 2.0 * g.M * (double)g.N * (g.K + g.K2), 0.0);
+    return rc;
+  };
   auto G = [&](int M_, int N_, int K_, const void* A, long long lda, bool ak, const void* B, long long ldb, bool bk,
                int abdt, void* C, long long ldc, int cdt, const float* R, long long ldr,
                const GemmEpilogue& epi = GemmEpilogue()) -> int {
     GemmArgs g{M_, N_, K_, A, lda, ak, B, ldb, bk, abdt, C, ldc, cdt, R, ldr, epi};
-    prof_begin(gemm_runs_on_pairs(g) ? PC_GEMM : PC_GEMM_SMALL, s);
-    const int rc = gemm(g, s);
-    prof_end(s, 2.0 * M_ * (double)N_ * K_, 0.0);
-    return rc;
+    return GX(g);
   };
 #define TRY(expr) do { int rc__ = (expr); if (rc__ != PCM_OK) return rc__; } while (0)
   const double es = (double)sizeof(T);
-  // bf16 on the tensor-core path: SwiGLU and the rotary embedding run inside GEMM / attention epilogues
-  bool fuse_swiglu = false, fuse_rope = false;
-  if (dt == DT_BF16 && backend_from_env() != GEMM_SIMT) {
-    GemmArgs probe{128, 8 * d, d, w.la[0].h2, d, true, w_gu, d, true, dt, w.la[0].gu, 8 * d, dt, nullptr, 0};
-    probe.epi.kind = EPI_SWIGLU_FWD; probe.epi.out2 = w.la[0].act; probe.epi.ld_out2 = 4 * d;
-    fuse_swiglu = gemm_epilogue_supported(probe);
-    GemmArgs probe2{128, 3 * d, d, w.la[0].h1, d, true, w_qkv, d, true, dt, w.la[0].qkv, 3 * d, dt, nullptr, 0};
-    probe2.epi.kind = EPI_ROPE; probe2.epi.rope_tab = w.rope_tab; probe2.epi.S = S; probe2.epi.dh = dh; probe2.epi.d = d;
-    fuse_rope = gemm_epilogue_supported(probe2);
-  }
+
+  // y[rows][out] = x W^T (+ R), with the adapter branch alpha/r (x A^T) B^T entering the same accumulator as a
+  // continuation of the contraction: t = alpha/r x A^T is formed first (and kept in t_buf for the backward pass).
+  auto lin_fwd = [&](int pj, int l, int rows, const void* x, void* t_buf, void* C, int cdt, const float* R,
+                     const GemmEpilogue& epi) -> int {
+    const int in = p_in[pj], out = p_out[pj];
+    GemmArgs g{rows, out, in, x, in, true, p_w[pj] + (size_t)l * out * in, in, true, dt, C, out, cdt, R, out, epi};
+    if (lo) {
+      GemmArgs gt{rows, r, in, x, in, true, p_a[pj] + (size_t)l * r * in, in, true, dt, t_buf, r, dt, nullptr, 0};
+      gt.alpha = lora_scale;
+      TRY(GX(gt));
+      g.A2 = t_buf; g.lda2 = r; g.B2 = p_b[pj] + (size_t)l * out * r; g.ldb2 = r; g.K2 = r;
+    }
+    return GX(g);
+  };
+  // Backward of the same map: dW += dy^T x (dense), or with adapters u = alpha/r dy B, dA += u^T x, dB += dy^T t
+  // (the base weight is frozen); then dX[rows][ldc >= in] = dy W (+ u A), again one contraction.
+  auto lin_bwd = [&](int pj, int l, int rows, const void* x, const void* t_buf, const void* dy, void* dX, int ldc, int cdt,
+                     const GemmEpilogue& epi) -> int {
+    const int in = p_in[pj], out = p_out[pj];
+    const T* W = p_w[pj] + (size_t)l * out * in;
+    GemmArgs g{rows, in, out, dy, out, true, W, in, false, dt, dX, ldc, cdt, nullptr, 0, epi};
+    if (!lo) {
+      float* dW = p_dw[pj] + (size_t)l * out * in;
+      TRY(G(out, in, rows, dy, out, false, x, in, false, dt, dW, in, DT_F32, dW, in));
+    } else {
+      GemmArgs gu{rows, r, out, dy, out, true, p_b[pj] + (size_t)l * out * r, r, false, dt, w.lu, r, dt, nullptr, 0};
+      gu.alpha = lora_scale;
+      TRY(GX(gu));
+      float* dA = p_da[pj] + (size_t)l * r * in;
+      float* dB = p_db[pj] + (size_t)l * out * r;
+      TRY(G(r, in, rows, w.lu, r, false, x, in, false, dt, dA, in, DT_F32, dA, in));
+      TRY(G(out, r, rows, dy, out, false, t_buf, r, false, dt, dB, r, DT_F32, dB, r));
+      g.A2 = w.lu; g.lda2 = r; g.B2 = p_a[pj] + (size_t)l * r * in; g.ldb2 = in; g.K2 = r;
+    }
+    return GX(g);
+  };
 
   for (int c0 = 0; c0 < n; c0 += mb_max) {
     const int mb = (n - c0) < mb_max ? (n - c0) : mb_max;
@@ -695,18 +825,17 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     prof_end(s, 0.0, (double)M * d * (es + 4.0));
     for (int l = 0; l < L; ++l) {
       LayerActs& la = w.la[l];
+      const bool last = l == L - 1;
       const float* x_in = w.x[l];
       float* x_out = w.x[l + 1];
       prof_begin(PC_NORM, s);
       rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(x_in, g1 + (size_t)l * d, (T*)la.h1, la.rstd1, M, d, 0, 0);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)M * d * (es + 4.0));
-      if (fuse_rope) {
-        GemmEpilogue e;
-        e.kind = EPI_ROPE; e.rope_tab = w.rope_tab; e.S = S; e.dh = dh; e.d = d;
-        TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0, e));
-      } else {
-        TRY(G(Mi, 3 * d, d, la.h1, d, true, w_qkv + (size_t)l * 3 * d * d, d, true, dt, la.qkv, 3 * d, dt, nullptr, 0));
+      GemmEpilogue e_qkv;
+      if (fuse_rope) { e_qkv.kind = EPI_ROPE; e_qkv.rope_tab = w.rope_tab; e_qkv.S = S; e_qkv.dh = dh; e_qkv.d = d; }
+      TRY(lin_fwd(PJ_QKV, l, Mi, la.h1, la.lt[PJ_QKV], la.qkv, dt, nullptr, e_qkv));
+      if (!fuse_rope) {
         prof_begin(PC_ELEM, s);
         rope_kernel<T><<<ceil_div(M * H * dh / Vec16<T>::N, 256), 256, 0, s>>>((T*)la.qkv, w.rope_tab, M, S, H, dh, 1.f);
         PCM_LAUNCH_CHECK();
@@ -715,27 +844,39 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       prof_begin(PC_ATTN, s);
       TRY(attention_fwd(dt, la.qkv, la.attn, la.lse, mb, S, H, dh, s));
       prof_end(s, 2.0 * S * (double)S * d * mb, (double)M * 4 * d * es);
-      TRY(G(Mi, d, d, la.attn, d, true, w_o + (size_t)l * d * d, d, true, dt, la.x_mid, d, DT_F32, x_in, d));
-      prof_begin(PC_NORM, s);
-      rmsnorm_fwd_kernel<T><<<ceil_div(M, 8), 256, 0, s>>>(la.x_mid, g2 + (size_t)l * d, (T*)la.h2, la.rstd2, M, d, 0, 0);
-      PCM_LAUNCH_CHECK();
-      prof_end(s, 0.0, (double)M * d * (es + 4.0));
-      if (fuse_swiglu) {
-        GemmEpilogue e;
-        e.kind = EPI_SWIGLU_FWD; e.out2 = la.act; e.ld_out2 = 4 * d;
-        TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0, e));
-      } else {
-        TRY(G(Mi, 8 * d, d, la.h2, d, true, w_gu + (size_t)l * 8 * d * d, d, true, dt, la.gu, 8 * d, dt, nullptr, 0));
+      // From here on the last layer works on the scored rows only: the head reads nothing else, so the other rows'
+      // values would be unread and their gradients exactly zero.
+      const long long Mp = last ? R : M;
+      const int Mpi = (int)Mp;
+      const void* attn_in = la.attn;
+      const float* resid = x_in;
+      if (last) {
         prof_begin(PC_ELEM, s);
-        swiglu_fwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, M, 4 * d);
+        gather_scored_rows_kernel<T><<<ceil_div(R * (d / 4), 256), 256, 0, s>>>((const T*)la.attn, x_in, (T*)w.attn_s, w.xin_s,
+                                                                              R, S, P, d);
         PCM_LAUNCH_CHECK();
-        prof_end(s, 0.0, (double)M * 4 * d * es * 3.0);
+        prof_end(s, 0.0, (double)R * d * (es + 4.0) * 2.0);
+        attn_in = w.attn_s; resid = w.xin_s;
       }
-      TRY(G(Mi, d, 4 * d, la.act, 4 * d, true, w_d + (size_t)l * 4 * d * d, 4 * d, true, dt, x_out, d, DT_F32, la.x_mid, d));
+      TRY(lin_fwd(PJ_O, l, Mpi, attn_in, la.lt[PJ_O], la.x_mid, DT_F32, resid, GemmEpilogue()));
+      prof_begin(PC_NORM, s);
+      rmsnorm_fwd_kernel<T><<<ceil_div(Mp, 8), 256, 0, s>>>(la.x_mid, g2 + (size_t)l * d, (T*)la.h2, la.rstd2, Mp, d, 0, 0);
+      PCM_LAUNCH_CHECK();
+      prof_end(s, 0.0, (double)Mp * d * (es + 4.0));
+      GemmEpilogue e_gu;
+      if (fuse_swiglu) { e_gu.kind = EPI_SWIGLU_FWD; e_gu.out2 = la.act; e_gu.ld_out2 = 4 * d; }
+      TRY(lin_fwd(PJ_GU, l, Mpi, la.h2, la.lt[PJ_GU], la.gu, dt, nullptr, e_gu));
+      if (!fuse_swiglu) {
+        prof_begin(PC_ELEM, s);
+        swiglu_fwd_kernel<T><<<ceil_div(Mp * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (T*)la.act, Mp, 4 * d);
+        PCM_LAUNCH_CHECK();
+        prof_end(s, 0.0, (double)Mp * 4 * d * es * 3.0);
+      }
+      TRY(lin_fwd(PJ_D, l, Mpi, la.act, la.lt[PJ_D], x_out, DT_F32, la.x_mid, GemmEpilogue()));
     }
-    // head on the scored rows only
+    // head on the scored rows (x[L] holds exactly those)
     prof_begin(PC_NORM, s);
-    rmsnorm_fwd_kernel<T><<<ceil_div(R, 8), 256, 0, s>>>(w.x[L], gf, (T*)w.hs, w.rstdf, R, d, S, P);
+    rmsnorm_fwd_kernel<T><<<ceil_div(R, 8), 256, 0, s>>>(w.x[L], gf, (T*)w.hs, w.rstdf, R, d, 0, 0);
     PCM_LAUNCH_CHECK();
     prof_end(s, 0.0, (double)R * d * (es + 4.0));
     // Head and loss in one launch: the logits stay in tensor memory (bf16 on the tensor cores) or registers.
@@ -784,11 +925,9 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
     if (fwd_only) continue;
 
     // ---------------- backward ----------------
-    // head: dW_h += dz^T hs ; dhs = dz W_h ; final norm backward scatters into dx
+    // head: dW_h += dz^T hs ; dhs = dz W_h
     TRY(G(NB, d, Ri, w.dz, NB, false, w.hs, d, false, dt, gr->w_h, d, DT_F32, gr->w_h, d));
     TRY(G(Ri, d, NB, w.dz, NB, true, w_h, d, false, dt, w.dhs, d, DT_F32, nullptr, 0));
-    PCM_CUDA_TRY(cudaMemsetAsync(w.dx, 0, (size_t)M * d * 4, s));
-    PCM_CUDA_TRY(cudaMemsetAsync(w.dx_t, 0, (size_t)M * d * sizeof(T), s));
     const size_t nb_smem = (size_t)8 * d * sizeof(float);
     if (nb_smem > 48 * 1024)
     {
@@ -796,52 +935,61 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
       PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
       PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_rows_kernel<T, T, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
     }
-    // dy_is_t: the incoming gradient is stored in the activation type (the per-layer dh), else in fp32
+    // dy_is_t: the incoming gradient is stored in the activation type (the per-layer dh), else in fp32.
+    // dx_out = dx_in + (gradient through the norm), in fp32 and in T.
     auto norm_bwd = [&](const void* dy, bool dy_is_t, const float* x, const float* rstd, const T* gamma, const float* dx_in,
-                        long long rows, int mS, int mP, float* dgamma) -> int {
+                        long long rows, float* dgamma, float* dx_out, T* dx_out_t) -> int {
       const int blocks = (int)(rows / 8 + 1 < NORM_BWD_BLOCKS ? rows / 8 + 1 : NORM_BWD_BLOCKS);
       prof_begin(PC_NORM, s);
       if (dy_is_t && d == 1024)
-        rmsnorm_bwd_rows_kernel<T, T, 8><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t,
-                                                                       w.norm_part, rows, mS, mP);
+        rmsnorm_bwd_rows_kernel<T, T, 8><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, dx_out, dx_out_t,
+                                                                       w.norm_part, rows, 0, 0);
       else if (dy_is_t)
-        rmsnorm_bwd_kernel<T, T><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t, w.norm_part,
-                                                               rows, d, mS, mP);
+        rmsnorm_bwd_kernel<T, T><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, dx_out, dx_out_t, w.norm_part,
+                                                               rows, d, 0, 0);
       else
-        rmsnorm_bwd_kernel<T, float><<<blocks, 256, nb_smem, s>>>((const float*)dy, x, rstd, gamma, dx_in, w.dx, (T*)w.dx_t,
-                                                                   w.norm_part, rows, d, mS, mP);
+        rmsnorm_bwd_kernel<T, float><<<blocks, 256, nb_smem, s>>>((const float*)dy, x, rstd, gamma, dx_in, dx_out, dx_out_t,
+                                                                   w.norm_part, rows, d, 0, 0);
       PCM_LAUNCH_CHECK();
       prof_end(s, 0.0, (double)rows * d * ((dx_in ? 12.0 : 8.0) + (dy_is_t ? es : 4.0) + es));
       colsum_accumulate_kernel<<<ceil_div(d, 32), 256, 0, s>>>(w.norm_part, blocks, d, dgamma);
       PCM_LAUNCH_CHECK();
       return PCM_OK;
     };
-    TRY(norm_bwd(w.dhs, false, w.x[L], w.rstdf, gf, nullptr, R, S, P, gr->gf));
+    // final norm: the gradient of the scored rows, kept compact until the last layer's attention block
+    TRY(norm_bwd(w.dhs, false, w.x[L], w.rstdf, gf, nullptr, R, gr->gf, w.dxs, (T*)w.dxs_t));
 
     for (int l = L - 1; l >= 0; --l) {
       LayerActs& la = w.la[l];
-      const size_t dd = (size_t)d * d;
+      const bool last = l == L - 1;
+      const long long Mp = last ? R : M;
+      const int Mpi = (int)Mp;
+      float* dxp = last ? w.dxs : w.dx;                     // residual gradient of the post-attention rows
+      T* dxp_t = last ? (T*)w.dxs_t : (T*)w.dx_t;
       // MLP: x_out = x_mid + act W_d^T
-      TRY(G(d, 4 * d, Mi, w.dx_t, d, false, la.act, 4 * d, false, dt, gr->w_d + l * 4 * dd, 4 * d, DT_F32,
-            gr->w_d + l * 4 * dd, 4 * d));
-      if (fuse_swiglu) {
-        GemmEpilogue e;
-        e.kind = EPI_SWIGLU_BWD; e.aux = la.gu; e.ld_aux = 8 * d;
-        TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dgu, 8 * d, dt, nullptr, 0, e));
-      } else {
-        TRY(G(Mi, 4 * d, d, w.dx_t, d, true, w_d + l * 4 * dd, 4 * d, false, dt, w.dact, 4 * d, dt, nullptr, 0));
+      GemmEpilogue e_d;
+      if (fuse_swiglu) { e_d.kind = EPI_SWIGLU_BWD; e_d.aux = la.gu; e_d.ld_aux = 8 * d; }
+      TRY(lin_bwd(PJ_D, l, Mpi, la.act, la.lt[PJ_D], dxp_t, fuse_swiglu ? w.dgu : w.dact, fuse_swiglu ? 8 * d : 4 * d, dt, e_d));
+      if (!fuse_swiglu) {
         prof_begin(PC_ELEM, s);
-        swiglu_bwd_kernel<T><<<ceil_div(M * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, M, 4 * d);
+        swiglu_bwd_kernel<T><<<ceil_div(Mp * 4 * d / Vec16<T>::N, 256), 256, 0, s>>>((const T*)la.gu, (const T*)w.dact, (T*)w.dgu, Mp, 4 * d);
         PCM_LAUNCH_CHECK();
-        prof_end(s, 0.0, (double)M * 4 * d * es * 5.0);
+        prof_end(s, 0.0, (double)Mp * 4 * d * es * 5.0);
       }
-      TRY(G(8 * d, d, Mi, w.dgu, 8 * d, false, la.h2, d, false, dt, gr->w_gu + l * 8 * dd, d, DT_F32,
-            gr->w_gu + l * 8 * dd, d));
-      TRY(G(Mi, d, 8 * d, w.dgu, 8 * d, true, w_gu + l * 8 * dd, d, false, dt, w.dh, d, dt, nullptr, 0));
-      TRY(norm_bwd(w.dh, true, la.x_mid, la.rstd2, g2 + (size_t)l * d, w.dx, M, 0, 0, gr->g2 + (size_t)l * d));
+      TRY(lin_bwd(PJ_GU, l, Mpi, la.h2, la.lt[PJ_GU], w.dgu, w.dh, d, dt, GemmEpilogue()));
+      TRY(norm_bwd(w.dh, true, la.x_mid, la.rstd2, g2 + (size_t)l * d, dxp, Mp, gr->g2 + (size_t)l * d, dxp, dxp_t));
       // attention block: x_mid = x_in + attn W_o^T
-      TRY(G(d, d, Mi, w.dx_t, d, false, la.attn, d, false, dt, gr->w_o + l * dd, d, DT_F32, gr->w_o + l * dd, d));
-      TRY(G(Mi, d, d, w.dx_t, d, true, w_o + l * dd, d, false, dt, w.dattn, d, dt, nullptr, 0));
+      TRY(lin_bwd(PJ_O, l, Mpi, last ? w.attn_s : la.attn, la.lt[PJ_O], dxp_t, last ? w.dattn_s : w.dattn, d, dt, GemmEpilogue()));
+      if (last) {
+        // back to all rows: the other rows of d(attn) and of the residual gradient are exactly zero
+        PCM_CUDA_TRY(cudaMemsetAsync(w.dattn, 0, (size_t)M * d * sizeof(T), s));
+        PCM_CUDA_TRY(cudaMemsetAsync(w.dx, 0, (size_t)M * d * 4, s));
+        prof_begin(PC_ELEM, s);
+        scatter_scored_rows_kernel<T><<<ceil_div(R * (d / 4), 256), 256, 0, s>>>((const T*)w.dattn_s, w.dxs, (T*)w.dattn, w.dx,
+                                                                               R, S, P, d);
+        PCM_LAUNCH_CHECK();
+        prof_end(s, 0.0, (double)M * d * (es + 4.0) + (double)R * d * (es + 4.0) * 2.0);
+      }
       prof_begin(PC_ATTN, s);
       TRY(attention_bwd(dt, la.qkv, la.attn, w.dattn, la.lse, w.dsum, w.dqkv, mb, S, H, dh, s,
                         fuse_rope ? w.rope_tab : nullptr));
@@ -852,10 +1000,8 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
         PCM_LAUNCH_CHECK();
         prof_end(s, 0.0, (double)M * 2 * d * es * 2.0);
       }
-      TRY(G(3 * d, d, Mi, w.dqkv, 3 * d, false, la.h1, d, false, dt, gr->w_qkv + l * 3 * dd, d, DT_F32,
-            gr->w_qkv + l * 3 * dd, d));
-      TRY(G(Mi, d, 3 * d, w.dqkv, 3 * d, true, w_qkv + l * 3 * dd, d, false, dt, w.dh, d, dt, nullptr, 0));
-      TRY(norm_bwd(w.dh, true, w.x[l], la.rstd1, g1 + (size_t)l * d, w.dx, M, 0, 0, gr->g1 + (size_t)l * d));
+      TRY(lin_bwd(PJ_QKV, l, Mi, la.h1, la.lt[PJ_QKV], w.dqkv, w.dh, d, dt, GemmEpilogue()));
+      TRY(norm_bwd(w.dh, true, w.x[l], la.rstd1, g1 + (size_t)l * d, w.dx, M, gr->g1 + (size_t)l * d, w.dx, (T*)w.dx_t));
     }
     prof_begin(PC_EMBED, s);
     embed_grad_kernel<<<dim3(NB, ceil_div(d, 256)), 256, 0, s>>>(w.dx, tgt, mb, S, P, d, gr->e_act);
@@ -883,6 +1029,7 @@ static int run(const grpo_model* m, const grpo_packed* pk, const grpo_loss_cfg* 
   return PCM_OK;
 }
 
+
 static GemmBackend backend_from_env() {
   const char* e = getenv("PCM_GEMM_BACKEND");
   if (e && !strcmp(e, "simt")) return GEMM_SIMT;
@@ -909,17 +1056,28 @@ int gemm(const GemmArgs& g, cudaStream_t s, GemmBackend backend) {
 
 using namespace pcm;
 
-extern "C" size_t grpo_workspace_bytes(const grpo_model_cfg* cfg, int32_t mb_chunks, uint32_t flags) {
+static size_t workspace_bytes_for(const grpo_model_cfg* cfg, int rank, int32_t mb_chunks, uint32_t flags) {
   if (check_cfg(cfg) != PCM_OK || mb_chunks < 1) return 0;
+  bool fuse_swiglu = false, fuse_rope = false;
+  fused_epilogues(*cfg, &fuse_swiglu, &fuse_rope);
   Workspace w;
   memset(&w, 0, sizeof(w));
-  carve(w, nullptr, *cfg, mb_chunks, flags & GRPO_FWD_ONLY);
+  carve(w, nullptr, *cfg, mb_chunks, flags & GRPO_FWD_ONLY, rank, !fuse_swiglu);
   return w.bytes;
 }
 
-extern "C" int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* batch, const grpo_loss_cfg* lc,
-                                  grpo_grads* grads, float* loss, float* logp, grpo_stats* stats, void* workspace,
-                                  size_t workspace_bytes, pcm_stream stream) {
+extern "C" size_t grpo_workspace_bytes(const grpo_model_cfg* cfg, int32_t mb_chunks, uint32_t flags) {
+  return workspace_bytes_for(cfg, 0, mb_chunks, flags);
+}
+
+extern "C" size_t grpo_lora_workspace_bytes(const grpo_model_cfg* cfg, int32_t rank, int32_t mb_chunks, uint32_t flags) {
+  if (rank < 8 || rank > 64 || (rank % 8)) return 0;
+  return workspace_bytes_for(cfg, rank, mb_chunks, flags);
+}
+
+static int actor_entry(const grpo_model* model, const grpo_lora* lora, const grpo_packed* batch, const grpo_loss_cfg* lc,
+                       grpo_grads* grads, grpo_lora_grads* lgrads, float* loss, float* logp, grpo_stats* stats,
+                       void* workspace, size_t workspace_bytes, pcm_stream stream) {
   if (!model || !batch || !lc || !loss || !workspace) return PCM_ERR_ARG;
   int rc = check_cfg(&model->cfg);
   if (rc) return rc;
@@ -930,15 +1088,32 @@ extern "C" int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* ba
   if (batch->n_kept > 0 && (!batch->X || !batch->tgt || !batch->lpo || !batch->adv_c)) return PCM_ERR_ARG;
   const bool fwd_only = lc->flags & GRPO_FWD_ONLY;
   if (!fwd_only) {
-    if (!grads || !grads->w_qkv || !grads->w_o || !grads->w_gu || !grads->w_d || !grads->g1 || !grads->g2 ||
-        !grads->gf || !grads->w_h || !grads->e_act)
+    if (!grads || !grads->g1 || !grads->g2 || !grads->gf || !grads->w_h || !grads->e_act) return PCM_ERR_ARG;
+    if (!lora && (!grads->w_qkv || !grads->w_o || !grads->w_gu || !grads->w_d)) return PCM_ERR_ARG;
+    if (lora && (!lgrads || !lgrads->a_qkv || !lgrads->b_qkv || !lgrads->a_o || !lgrads->b_o || !lgrads->a_gu ||
+                 !lgrads->b_gu || !lgrads->a_d || !lgrads->b_d))
       return PCM_ERR_ARG;
   }
   if (((uintptr_t)workspace) & 255) return PCM_ERR_WORKSPACE;
   cudaStream_t s = (cudaStream_t)stream;
   if (model->cfg.dtype == GRPO_BF16)
-    return run<__nv_bfloat16>(model, batch, lc, grads, loss, logp, stats, workspace, workspace_bytes, s);
-  return run<float>(model, batch, lc, grads, loss, logp, stats, workspace, workspace_bytes, s);
+    return run<__nv_bfloat16>(model, lora, batch, lc, grads, lgrads, loss, logp, stats, workspace, workspace_bytes, s);
+  return run<float>(model, lora, batch, lc, grads, lgrads, loss, logp, stats, workspace, workspace_bytes, s);
+}
+
+extern "C" int grpo_actor_fwd_bwd(const grpo_model* model, const grpo_packed* batch, const grpo_loss_cfg* lc,
+                                  grpo_grads* grads, float* loss, float* logp, grpo_stats* stats, void* workspace,
+                                  size_t workspace_bytes, pcm_stream stream) {
+  return actor_entry(model, nullptr, batch, lc, grads, nullptr, loss, logp, stats, workspace, workspace_bytes, stream);
+}
+
+extern "C" int grpo_actor_fwd_bwd_lora(const grpo_model* model, const grpo_lora* lora, const grpo_packed* batch,
+                                       const grpo_loss_cfg* lc, grpo_grads* grads, grpo_lora_grads* lora_grads, float* loss,
+                                       float* logp, grpo_stats* stats, void* workspace, size_t workspace_bytes,
+                                       pcm_stream stream) {
+  const int rc = check_lora(lora);
+  if (rc) return rc;
+  return actor_entry(model, lora, batch, lc, grads, lora_grads, loss, logp, stats, workspace, workspace_bytes, stream);
 }
 
 extern "C" int grpo_gemm(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_kmajor, const void* B,

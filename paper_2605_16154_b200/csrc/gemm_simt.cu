@@ -16,7 +16,8 @@ template <typename TI, typename TC>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(int M, int N, int K, const TI* __restrict__ A, long long sam, long long sak,
                  const TI* __restrict__ B, long long sbn, long long sbk, TC* C, long long ldc,
-                 const float* R, long long ldr) {
+                 const float* R, long long ldr, int K2, const TI* __restrict__ A2, long long sam2, long long sak2,
+                 const TI* __restrict__ B2, long long sbn2, long long sbk2, float alpha) {
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float Bs[SG_BK][SG_BN + 4];
   const int tid = threadIdx.x;
@@ -24,6 +25,11 @@ gemm_simt_kernel(int M, int N, int K, const TI* __restrict__ A, long long sam, l
   const int tx = tid & 15, ty = tid >> 4;                 // 16 x 16 threads, 4 x 4 outputs each
   float acc[4][4] = {};
   const bool a_k_fast = (sak == 1), b_k_fast = (sbk == 1);
+  for (int seg = 0; seg < 2; ++seg) {                     // the contraction, then its optional continuation
+  if (seg == 1) {
+    if (K2 <= 0) break;
+    A = A2; B = B2; K = K2; sam = sam2; sak = sak2; sbn = sbn2; sbk = sbk2;
+  }
   for (int k0 = 0; k0 < K; k0 += SG_BK) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -54,6 +60,7 @@ gemm_simt_kernel(int M, int N, int K, const TI* __restrict__ A, long long sam, l
     }
     __syncthreads();
   }
+  }
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int m = m0 + ty * 4 + i;
@@ -62,7 +69,7 @@ gemm_simt_kernel(int M, int N, int K, const TI* __restrict__ A, long long sam, l
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
       if (n >= N) continue;
-      float v = acc[i][j];
+      float v = alpha * acc[i][j];
       if (R) v += R[(long long)m * ldr + n];
       if constexpr (sizeof(TC) == 4) C[(long long)m * ldc + n] = v;
       else C[(long long)m * ldc + n] = __float2bfloat16_rn(v);
@@ -77,7 +84,9 @@ static int launch_simt(const GemmArgs& g, cudaStream_t s) {
   dim3 grid(ceil_div(g.N, SG_BN), ceil_div(g.M, SG_BM));
   if (grid.y > 65535) return PCM_ERR_SHAPE;
   gemm_simt_kernel<TI, TC><<<grid, 256, 0, s>>>(g.M, g.N, g.K, (const TI*)g.A, sam, sak, (const TI*)g.B, sbn, sbk,
-                                                (TC*)g.C, g.ldc, g.R, g.ldr);
+                                                (TC*)g.C, g.ldc, g.R, g.ldr, g.K2, (const TI*)g.A2,
+                                                g.a_kmajor ? g.lda2 : 1, g.a_kmajor ? 1 : g.lda2, (const TI*)g.B2,
+                                                g.b_kmajor ? g.ldb2 : 1, g.b_kmajor ? 1 : g.ldb2, g.alpha);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
 }

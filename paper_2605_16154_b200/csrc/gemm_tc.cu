@@ -51,6 +51,10 @@ struct TcParams {
   const float2* rope_tab; int S, dh, d;
   int up_row0;                                // EPI_SWIGLU_FWD: first "up" row of B (= F)
   HeadLossArgs hl;                            // EPI_HEAD_LOSS
+  int kb_main;                                // k-blocks taken from the first operand pair; later ones come from the second
+  int kb_total;                               // all k-blocks of the contraction (first pair + continuation)
+  int ext_ksteps;                             // MMAs of 16 k-columns in a k-block of the continuation (K2 / 16)
+  float alpha;                                // scale of the product in the plain store epilogue
 };
 
 __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&v)[32]) {
@@ -471,6 +475,7 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               v[i] = *reinterpret_cast<const float4*>(stage + (i * 4 + (lane_ >> 3)) * EPI_STAGE_STRIDE + (lane_ & 7) * 4);
+              if (p.alpha != 1.f) { v[i].x *= p.alpha; v[i].y *= p.alpha; v[i].z *= p.alpha; v[i].w *= p.alpha; }
               if (p.R) { v[i].x += pre.r[i].x; v[i].y += pre.r[i].y; v[i].z += pre.r[i].z; v[i].w += pre.r[i].w; }
             }
             if (p.R && more) fetch_residual(p, row_base, col + 32, lane_, pre.r);
@@ -486,6 +491,10 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
             for (int i = 0; i < 4; ++i) {
               const float* sp = stage + (i * 8 + (lane_ >> 2)) * EPI_STAGE_STRIDE + (lane_ & 3) * 8;
               float4 a = *reinterpret_cast<const float4*>(sp), b = *reinterpret_cast<const float4*>(sp + 4);
+              if (p.alpha != 1.f) {
+                a.x *= p.alpha; a.y *= p.alpha; a.z *= p.alpha; a.w *= p.alpha;
+                b.x *= p.alpha; b.y *= p.alpha; b.z *= p.alpha; b.w *= p.alpha;
+              }
               if (p.R) {
                 a.x += pre.r[2 * i].x; a.y += pre.r[2 * i].y; a.z += pre.r[2 * i].z; a.w += pre.r[2 * i].w;
                 b.x += pre.r[2 * i + 1].x; b.y += pre.r[2 * i + 1].y; b.z += pre.r[2 * i + 1].z; b.w += pre.r[2 * i + 1].w;
@@ -511,7 +520,8 @@ __device__ __forceinline__ void epi_tile(const TcParams& p, uint32_t tmem_acc, i
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   using SM = TcSmem<BN>;
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -526,7 +536,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   float* epi_stage = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_kb_total = (p.K + TC_BK - 1) / TC_BK;
+  const int num_kb_total = p.kb_total;
   const int tiles_mn = p.tiles_m * p.tiles_n;
   const int total_tiles = tiles_mn * p.splits;
 
@@ -564,22 +574,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           uint8_t* sa = tiles + st * SM::STAGE_BYTES;
           uint8_t* sb = sa + SM::A_BYTES;
           mbar_expect_tx(&full[st], SM::STAGE_BYTES);
-          const int k0 = kb * TC_BK;
+          const bool ext = kb >= p.kb_main;                               // continuation: second operand pair
+          const CUtensorMap* mA = ext ? &tmA2 : &tmA;
+          const CUtensorMap* mB = ext ? &tmB2 : &tmB;
+          const int k0 = (ext ? kb - p.kb_main : kb) * TC_BK;
           if (p.a_kmajor) {
-            tma_load_2d(sa, &tmA, k0, m0, &full[st]);                     // box {64 k, 128 m}
+            tma_load_2d(sa, mA, k0, m0, &full[st]);                       // box {64 k, 128 m}
           } else {
 #pragma unroll
-            for (int b = 0; b < TC_BM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, m0 + b * 64, k0, &full[st]);  // box {64 m, 64 k}
+            for (int b = 0; b < TC_BM / 64; ++b) tma_load_2d(sa + b * 8192, mA, m0 + b * 64, k0, &full[st]);  // box {64 m, 64 k}
           }
           if (EPI == EPI_SWIGLU_FWD) {
             // n0 counts accumulator columns (256 per tile = 128 hidden units): gate rows, then the matching up rows
-            tma_load_2d(sb, &tmB, k0, n0 / 2, &full[st]);                 // box {64 k, 128 n}
-            tma_load_2d(sb + 128 * 128, &tmB, k0, p.up_row0 + n0 / 2, &full[st]);
+            tma_load_2d(sb, mB, k0, n0 / 2, &full[st]);                   // box {64 k, 128 n}
+            tma_load_2d(sb + 128 * 128, mB, k0, p.up_row0 + n0 / 2, &full[st]);
           } else if (p.b_kmajor) {
-            tma_load_2d(sb, &tmB, k0, n0, &full[st]);                     // box {64 k, BN n}
+            tma_load_2d(sb, mB, k0, n0, &full[st]);                       // box {64 k, BN n}
           } else {
 #pragma unroll
-            for (int b = 0; b < BN / 64; ++b) tma_load_2d(sb + b * 8192, &tmB, n0 + b * 64, k0, &full[st]);
+            for (int b = 0; b < BN / 64; ++b) tma_load_2d(sb + b * 8192, mB, n0 + b * 64, k0, &full[st]);
           }
         }
       }
@@ -609,8 +622,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_fence_after();
           const uint32_t sa = smem_u32(tiles + st * SM::STAGE_BYTES);
           const uint32_t sb = sa + SM::A_BYTES;
+          const int ksteps = kb >= p.kb_main ? p.ext_ksteps : TC_BK / 16;   // the continuation may be narrower than 64
 #pragma unroll
           for (int k = 0; k < TC_BK / 16; ++k) {
+            if (k >= ksteps) break;
             const uint64_t da = make_smem_desc(sa + k * a_step, a_lbo, 1024u);
             const uint64_t db = make_smem_desc(sb + k * b_step, b_lbo, 1024u);
             umma_bf16(tmem_acc, da, db, idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
@@ -706,7 +721,8 @@ constexpr int T2_SMEM_TOTAL = T2_STAGES * T2_STAGE_BYTES + 1024 + 256 + EPI_STAG
 
 template <int EPI>
 __global__ void __launch_bounds__(T2_THREADS, 1)
-gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   constexpr int BN = T2_BN;
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -724,7 +740,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int num_kb_total = (p.K + TC_BK - 1) / TC_BK;
+  const int num_kb_total = p.kb_total;
   const int tiles_mn = p.tiles_m * p.tiles_n;  // tiles of 256 x 256
   const int total_tiles = tiles_mn * p.splits;
 
@@ -769,23 +785,26 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           uint8_t* sa = tiles + st * T2_STAGE_BYTES;
           uint8_t* sb = sa + T2_A_BYTES;
           const uint32_t bar = bar0 + (uint32_t)st * 8u;
-          const int k0 = kb * TC_BK;
+          const bool ext = kb >= p.kb_main;                                     // continuation: second operand pair
+          const CUtensorMap* mA = ext ? &tmA2 : &tmA;
+          const CUtensorMap* mB = ext ? &tmB2 : &tmB;
+          const int k0 = (ext ? kb - p.kb_main : kb) * TC_BK;
           if (load_a) {
             if (leader) mbar_expect_tx(&full[st], 2 * T2_STAGE_BYTES);
             if (p.a_kmajor) {
-              tma_load_2d_pair(sa, &tmA, k0, m0, bar);                          // box {64 k, 128 m}
+              tma_load_2d_pair(sa, mA, k0, m0, bar);                            // box {64 k, 128 m}
             } else {
 #pragma unroll
-              for (int b = 0; b < 2; ++b) tma_load_2d_pair(sa + b * 8192, &tmA, m0 + b * 64, k0, bar);   // box {64 m, 64 k}
+              for (int b = 0; b < 2; ++b) tma_load_2d_pair(sa + b * 8192, mA, m0 + b * 64, k0, bar);   // box {64 m, 64 k}
             }
           } else if (EPI == EPI_SWIGLU_FWD) {
             // accumulator columns [0,128) = gate (leader's half of B), [128,256) = up (the peer's half)
-            tma_load_2d_pair(sb, &tmB, k0, (leader ? 0 : p.up_row0) + n0 / 2, bar);                 // box {64 k, 128 n}
+            tma_load_2d_pair(sb, mB, k0, (leader ? 0 : p.up_row0) + n0 / 2, bar);                   // box {64 k, 128 n}
           } else if (p.b_kmajor) {
-            tma_load_2d_pair(sb, &tmB, k0, nb0, bar);                           // box {64 k, 128 n}
+            tma_load_2d_pair(sb, mB, k0, nb0, bar);                             // box {64 k, 128 n}
           } else {
 #pragma unroll
-            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sb + b * 8192, &tmB, nb0 + b * 64, k0, bar);
+            for (int b = 0; b < 2; ++b) tma_load_2d_pair(sb + b * 8192, mB, nb0 + b * 64, k0, bar);
           }
           if (++st == T2_STAGES) { st = 0; ph ^= 1u; }
         }
@@ -825,9 +844,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           tc_fence_after();
           const uint32_t alo = da_lo + st_off, blo = db_lo + st_off;
           umma_bf16_pair(tmem_acc, desc(alo, da_hi), desc(blo, db_hi), idesc, kb > kb_lo ? 1u : 0u);
+          if (kb < p.kb_main) {
 #pragma unroll
-          for (int k = 1; k < TC_BK / 16; ++k)
-            umma_bf16_pair(tmem_acc, desc(alo + k * a_step16, da_hi), desc(blo + k * b_step16, db_hi), idesc, 1u);
+            for (int k = 1; k < TC_BK / 16; ++k)
+              umma_bf16_pair(tmem_acc, desc(alo + k * a_step16, da_hi), desc(blo + k * b_step16, db_hi), idesc, 1u);
+          } else {                               // continuation block: K2 / 16 MMAs, the rest of the tile is zero fill
+#pragma unroll 1
+            for (int k = 1; k < p.ext_ksteps; ++k)
+              umma_bf16_pair(tmem_acc, desc(alo + k * a_step16, da_hi), desc(blo + k * b_step16, db_hi), idesc, 1u);
+          }
           umma_commit_pair(&empty[st], 3);     // both CTAs may refill the stage
           st_off += T2_STAGE_BYTES >> 4;
           if (++st == T2_STAGES) { st = 0; st_off = 0; ph ^= 1u; }
@@ -924,6 +949,9 @@ bool gemm_tcgen05_supported(const GemmArgs& g) {
   if (g.c_dtype == DT_F32 && (g.ldc % 4)) return false;
   if (g.R && (((uintptr_t)g.R & 15) || (g.ldr % 4))) return false;
   if (g.R && (const void*)g.R == (const void*)g.C && g.c_dtype != DT_F32) return false;
+  if (g.K2 < 0 || g.K2 > TC_BK || (g.K2 % 16)) return false;
+  if (g.K2 > 0 && (!g.A2 || !g.B2 || (g.lda2 % 8) || (g.ldb2 % 8) || (((uintptr_t)g.A2 | (uintptr_t)g.B2) & 15))) return false;
+  if (g.alpha != 1.f && (g.epi.kind != EPI_NONE || (g.R && (const void*)g.R == (const void*)g.C))) return false;
     return encode_fn() != nullptr;
 }
 
@@ -938,6 +966,10 @@ static void fill_params(TcParams& p, const GemmArgs& g) {
   p.rope_tab = g.epi.rope_tab; p.S = g.epi.S; p.dh = g.epi.dh; p.d = g.epi.d;
   p.up_row0 = g.N / 2;
   p.hl = g.epi.hl;
+  p.kb_main = (g.K + TC_BK - 1) / TC_BK;
+  p.kb_total = p.kb_main + (g.K2 > 0 ? 1 : 0);
+  p.ext_ksteps = g.K2 / 16;
+  p.alpha = g.alpha;
   p.kb_per_split = 1; p.tiles_m = p.tiles_n = p.splits = 1;
 }
 
@@ -951,10 +983,18 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   const bool okB = g.b_kmajor ? make_tmap(&tmB, g.B, g.N, g.K, g.ldb, TC_BK, B_BOX_ROWS)
                               : make_tmap(&tmB, g.B, g.K, g.N, g.ldb, 64, TC_BK);
   if (!okA || !okB) return PCM_ERR_CUDA;
+  CUtensorMap tmA2 = tmA, tmB2 = tmB;                      // continuation of the contraction, laid out like A / B
+  if (g.K2 > 0) {
+    const bool okA2 = g.a_kmajor ? make_tmap(&tmA2, g.A2, g.M, g.K2, g.lda2, TC_BK, TC_BM)
+                                 : make_tmap(&tmA2, g.A2, g.K2, g.M, g.lda2, 64, TC_BK);
+    const bool okB2 = g.b_kmajor ? make_tmap(&tmB2, g.B2, g.N, g.K2, g.ldb2, TC_BK, B_BOX_ROWS)
+                                 : make_tmap(&tmB2, g.B2, g.K2, g.N, g.ldb2, 64, TC_BK);
+    if (!okA2 || !okB2) return PCM_ERR_CUDA;
+  }
   TcParams p;
   fill_params(p, g);
   const int tiles_m = (g.M + TC_BM - 1) / TC_BM, tiles_n = (g.N + BN - 1) / BN;
-  const int num_kb = (g.K + TC_BK - 1) / TC_BK;
+  const int num_kb = p.kb_total;
   int splits = 1;
   if (p.reduce) {
     // split the contraction until there are about two waves of CTAs, keeping >= 8 k-blocks per split
@@ -972,7 +1012,7 @@ static int launch_tc(const GemmArgs& g, cudaStream_t s) {
   p.tiles_m = tiles_m; p.tiles_n = tiles_n; p.splits = splits;
   const long long total = (long long)tiles_m * tiles_n * splits;
   const int grid = (int)(total < sm_count() ? total : sm_count());      // persistent: one CTA per SM walks the tile list
-  gemm_tc_kernel<BN, EPI><<<grid, TC_THREADS, TcSmem<BN>::TOTAL, s>>>(tmA, tmB, p);
+  gemm_tc_kernel<BN, EPI><<<grid, TC_THREADS, TcSmem<BN>::TOTAL, s>>>(tmA, tmB, tmA2, tmB2, p);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
 }
@@ -995,10 +1035,18 @@ static int launch_tc2(const GemmArgs& g, cudaStream_t s) {
   const bool okB = g.b_kmajor ? make_tmap(&tmB, g.B, g.N, g.K, g.ldb, TC_BK, T2_BN / 2)
                               : make_tmap(&tmB, g.B, g.K, g.N, g.ldb, 64, TC_BK);
   if (!okA || !okB) return PCM_ERR_CUDA;
+  CUtensorMap tmA2 = tmA, tmB2 = tmB;
+  if (g.K2 > 0) {
+    const bool okA2 = g.a_kmajor ? make_tmap(&tmA2, g.A2, g.M, g.K2, g.lda2, TC_BK, TC_BM)
+                                 : make_tmap(&tmA2, g.A2, g.K2, g.M, g.lda2, 64, TC_BK);
+    const bool okB2 = g.b_kmajor ? make_tmap(&tmB2, g.B2, g.N, g.K2, g.ldb2, TC_BK, T2_BN / 2)
+                                 : make_tmap(&tmB2, g.B2, g.K2, g.N, g.ldb2, 64, TC_BK);
+    if (!okA2 || !okB2) return PCM_ERR_CUDA;
+  }
   TcParams p;
   fill_params(p, g);
   const int tiles_m = (g.M + 2 * TC_BM - 1) / (2 * TC_BM), tiles_n = (g.N + T2_BN - 1) / T2_BN;
-  const int num_kb = (g.K + TC_BK - 1) / TC_BK;
+  const int num_kb = p.kb_total;
   const int n_pairs_max = sm_count() / 2;
   int splits = 1;
   if (p.reduce) {
@@ -1036,7 +1084,7 @@ static int launch_tc2(const GemmArgs& g, cudaStream_t s) {
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, tmA, tmB, p) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, gemm_tc2_kernel<EPI>, tmA, tmB, tmA2, tmB2, p) != cudaSuccess) {
     cudaGetLastError();
     return PCM_ERR_CUDA;
   }

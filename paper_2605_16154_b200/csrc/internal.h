@@ -39,6 +39,13 @@ struct GemmArgs {
   void* C; long long ldc; int c_dtype;
   const float* R; long long ldr;
   GemmEpilogue epi;
+  // Optional continuation of the contraction: sum_k A(m,k) B(n,k) + sum_k2 A2(m,k2) B2(n,k2), with A2 / B2 laid out
+  // like A / B (same major-ness, own row strides) and K2 <= 64 a multiple of 16.  This is how a low-rank adapter
+  // branch enters the accumulator before any fused epilogue: [x | x A^T] [W | B]^T.
+  const void* A2 = nullptr; long long lda2 = 0;
+  const void* B2 = nullptr; long long ldb2 = 0;
+  int K2 = 0;
+  float alpha = 1.f;            // the product is scaled by alpha before R is added (plain epilogue, no reduction)
 };
 
 enum GemmBackend { GEMM_AUTO = 0, GEMM_SIMT = 1, GEMM_TCGEN05 = 2 };

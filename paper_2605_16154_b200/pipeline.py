@@ -49,3 +49,8 @@ def select(ctx: B.Context, batch: B.pcm_batch, it: int):
     p, q = B.pcm_update_keep_probs(ctx, Cc, valid)
     kept_idx, kept_off, per_phase = B.pcm_sample_chunks(ctx, batch, q, it)
     return adv, Cc, valid, p, q, kept_idx, kept_off, per_phase
+
+
+def upload_lora(w: synth.Workload, model: B.Model, lora: Dict) -> B.Lora:
+    td = torch_dtype(w)
+    return B.Lora(model, int(lora["rank"]), float(lora["alpha"]), {k: dev(lora[k], td) for k in synth.LORA_NAMES})

@@ -231,6 +231,28 @@ def make_weights(w: Workload, seed: Optional[int] = None) -> Dict[str, np.ndarra
     return out
 
 
+LORA_NAMES = ("a_qkv", "b_qkv", "a_o", "b_o", "a_gu", "b_gu", "a_d", "b_d")
+
+
+def lora_shapes(w: Workload, rank: int) -> Dict[str, tuple]:
+    """A [L, rank, in_features], B [L, out_features, rank] for the four linear maps of a layer."""
+    d, L = w.d, w.L
+    return {"a_qkv": (L, rank, d), "b_qkv": (L, 3 * d, rank), "a_o": (L, rank, d), "b_o": (L, d, rank),
+            "a_gu": (L, rank, d), "b_gu": (L, 8 * d, rank), "a_d": (L, rank, 4 * d), "b_d": (L, d, rank)}
+
+
+def make_lora(w: Workload, rank: int = 32, alpha: float = 32.0, seed: Optional[int] = None, b_std: float = 0.02):
+    """Adapter tensors (App. E: rank 32, alpha 32).  A ~ N(0, 1/in_features), B ~ N(0, b_std^2): a fresh adapter
+    has B = 0 (b_std = 0); a non-zero B stands for an adapter part-way through training."""
+    seed = w.seed if seed is None else seed
+    rng = np.random.Generator(np.random.PCG64(seed + 15485863))
+    out = {"rank": rank, "alpha": float(alpha)}
+    for name, shape in lora_shapes(w, rank).items():
+        std = 1.0 / np.sqrt(shape[2]) if name.startswith("a_") else b_std
+        out[name] = round_to_dtype((std * rng.standard_normal(shape, dtype=np.float32)).astype(np.float32), w.dtype)
+    return out
+
+
 def logp_noise(seed: int, n_chunks: int, sigma: float = 0.1) -> np.ndarray:
     """fp32 [n_chunks, 56] noise added to a policy's log-probs to stand in for the behaviour policy."""
     rng = np.random.Generator(np.random.PCG64(seed + 104729))

@@ -31,6 +31,7 @@ def test_binding_struct_sizes_match_the_header_layout():
     assert ctypes.sizeof(B.grpo_packed) == 8 + 5 * 8
     assert ctypes.sizeof(B.grpo_loss_cfg) == 24
     assert ctypes.sizeof(B.grpo_stats) == 32
+    assert ctypes.sizeof(B.grpo_lora) == 8 + 8 * 8 and ctypes.sizeof(B.grpo_lora_grads) == 8 * 8
     assert set(B.EXPORTED) == set(_declared())
 
 
@@ -42,9 +43,14 @@ def test_host_side_argument_checks_need_no_gpu():
     full = B._lib.grpo_workspace_bytes(ctypes.byref(cfg), 64, 0)
     fwd = B._lib.grpo_workspace_bytes(ctypes.byref(cfg), 64, B.GRPO_FWD_ONLY)
     assert 0 < fwd < full
-    # activations kept per token per layer: 18 d bf16 + 2 d fp32 (+ small terms)
+    # activations kept per token per layer: 18 d bf16 + 2 d fp32 = 44 d bytes (+ small terms); in the last layer the
+    # 30 d bytes after the attention exist for the 56 scored rows of a chunk's 312 only
     per_token = full / (64 * 312)
-    assert 8 * 44 * 1024 < per_token < 8 * 44 * 1024 * 1.3
+    expect = (7 * 44 + 14 + 30 * 56 / 312) * 1024
+    assert expect < per_token < expect * 1.3
+    lora = B._lib.grpo_lora_workspace_bytes(ctypes.byref(cfg), 32, 64, 0)
+    assert full < lora < full * 1.02                     # adapters keep four [tokens][rank] products per layer
+    assert B._lib.grpo_lora_workspace_bytes(ctypes.byref(cfg), 12, 64, 0) == 0
     assert B._lib.pcm_create(None, None, 0) == -1
 
 
