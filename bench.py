@@ -37,10 +37,23 @@ UNIT = "chunks/s"
 ACT = 56
 
 
-def flops_per_kept_chunk(w) -> float:
-    """Linear layers fwd + dgrad + wgrad, causal attention fwd + bwd, head."""
+def flops_per_kept_chunk(w, lora_rank: int = 0) -> float:
+    """The work the path executes per kept chunk: linear layers forward + input gradient + weight gradient, causal
+    attention forward + backward, head.  In the last layer everything after the attention runs on the 56 scored
+    rows only (W_o, gate|up, down: 13 d^2 of a layer's 16 d^2 per token), so those rows are what is counted.
+    With adapters (rank r) the base weight gradients do not exist (4 d^2 instead of 6 per weight element) and each
+    projection adds four rank-r products (x A^T, dy B, u^T x, dy^T t) plus the two continuation blocks."""
     S, d, L = w.S, w.d, w.L
-    return 6.0 * S * 16 * d * d * L + 7.0 * S * S * d * L + 6.0 * ACT * d * 256
+    per_w = 6.0 if lora_rank == 0 else 4.0
+    full_rows = S * 16 * d * d * (L - 1) + S * 3 * d * d      # layers 0..L-2, and the last layer's QKV
+    scored_rows = ACT * 13 * d * d                            # last layer after the attention
+    lin = per_w * (full_rows + scored_rows)
+    if lora_rank:
+        io_all = (d + 3 * d) + (d + d) + (d + 8 * d) + (4 * d + d)          # in + out of the four projections
+        io_qkv = d + 3 * d
+        # per projection and row: 2 r (in + out) flops forward (t, continuation) and 4 r (in + out) backward (u, continuation, dA, dB)
+        lin += 6.0 * lora_rank * (S * io_all * (L - 1) + S * io_qkv + ACT * (io_all - io_qkv))
+    return lin + 7.0 * S * S * d * L + 6.0 * ACT * d * 256
 
 
 def measured_peaks():
@@ -111,7 +124,7 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # CPU oracle timing (baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample_step(w, rb, weights, seed, n_sample):
+def oracle_sample_step(w, rb, weights, seed, n_sample, lora_rank=0):
     """One oracle pass: PCM control plane on the whole batch, actor forward + backward on the first
     n_sample kept chunks.  Returns (seconds for the control plane, seconds for the actor sample, n_kept)."""
     from oracle import actor_oracle as ao
@@ -130,7 +143,8 @@ def oracle_sample_step(w, rb, weights, seed, n_sample):
     lpo_all = np.full((total, ACT), -np.log(256.0), dtype=np.float32)
     t1 = time.perf_counter()
     X, tgt, lpo, adv_c, _ = po.pack_chunks(lambda c: obs[c], rb["tok"], lpo_all, adv, rb["traj_off"], sample, weights["e_act"])
-    ao.fwd_bwd(weights, X, tgt, lpo, adv_c, w.H, w.P, w.eps_low, w.eps_high, 1.0 / (ACT * len(kept)))
+    lo = synth.make_lora(w, lora_rank, float(lora_rank)) if lora_rank else None
+    ao.fwd_bwd(weights, X, tgt, lpo, adv_c, w.H, w.P, w.eps_low, w.eps_high, 1.0 / (ACT * len(kept)), lora=lo)
     t_actor = time.perf_counter() - t1
     return t_pcm, t_actor, len(kept)
 
@@ -143,9 +157,9 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def config_of(w, n_kept, total, mb, iterations=None):
+def config_of(w, n_kept, total, mb, iterations=None, lora_rank=0):
     """The `config` object both arms print."""
-    c = {"workload": w.name, "kept_chunks_per_step": int(n_kept), "chunks_per_step": int(total),
+    c = {"workload": w.name, "trainable": f"LoRA rank {lora_rank}, alpha {lora_rank}, base frozen" if lora_rank else "all weights", "kept_chunks_per_step": int(n_kept), "chunks_per_step": int(total),
          "tokens_per_step": int(n_kept) * w.S, "mb_chunks": int(mb), "l2": "inputs_larger_than_l2",
          "multi_gpu": "independent replicas, no collective"}
     if iterations is not None:
@@ -175,7 +189,7 @@ def run_reference(args):
     n_sample = 1
     est = []
     for it in range(args.warmup + args.steps):
-        t_pcm, t_actor, n_kept = oracle_sample_step(w, rb, weights, w.seed, n_sample)
+        t_pcm, t_actor, n_kept = oracle_sample_step(w, rb, weights, w.seed, n_sample, args.lora)
         if it >= args.warmup:
             est.append(t_pcm + t_actor * n_kept / n_sample)
     ms = 1e3 * sum(est) / len(est)
@@ -186,7 +200,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": config_of(w, n_kept, total, default_mb(args, n_kept), launch_steps_online(args) if online else None),
+            "config": config_of(w, n_kept, total, default_mb(args, n_kept), launch_steps_online(args) if online else None,
+                                args.lora),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -199,12 +214,14 @@ def run_reference(args):
 class Harness:
     """Device state shared by the timed legs: model, workspace, preallocated outputs."""
 
-    def __init__(self, B, PL, synth, w, weights, n_kept_max, mb):
+    def __init__(self, B, PL, synth, w, weights, n_kept_max, mb, lora_rank=0):
         import torch
         self.B, self.w, self.mb = B, w, mb
         self.model = PL.upload_model(w, weights)
         self.model.alloc_grads()
-        self.ws = torch.empty(B.grpo_workspace_bytes(self.model, mb, 0) + 256, dtype=torch.uint8, device="cuda")
+        # adapters part-way through training (non-zero B), alpha = rank as in App. E
+        self.lora = PL.upload_lora(w, self.model, synth.make_lora(w, lora_rank, float(lora_rank))) if lora_rank else None
+        self.ws = torch.empty(B.grpo_workspace_bytes(self.model, mb, 0, self.lora) + 256, dtype=torch.uint8, device="cuda")
         self.loss = torch.zeros(1, dtype=torch.float32, device="cuda")
         self.outputs(n_kept_max, w.n_traj, w.budget)
 
@@ -229,7 +246,7 @@ class Harness:
         B, w = self.B, self.w
         B.grpo_pack_chunks(ctx, bt, self.model, kept_idx, kept_off, adv, self.packed)
         B.grpo_actor_fwd_bwd(self.model, self.packed, w.eps_low, w.eps_high, 0.0, mb_chunks=self.mb, workspace=self.ws,
-                             want_stats=False, logp=self.logp, loss=self.loss)
+                             want_stats=False, logp=self.logp, loss=self.loss, lora=self.lora)
 
     def step(self, ctx, bt, it):
         adv, kept_idx, kept_off, _ = self.select(ctx, bt, it)
@@ -306,7 +323,7 @@ def make_timers(torch, dist, dist_util, world):
     return barrier, timed
 
 
-def behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed):
+def behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed, lora=None):
     """Behaviour-policy log-probs: a forward-only pass of the library over every chunk, plus seeded noise."""
     ident = B.Context(w.n_phases, int(lengths.max()), w.G, max_traj=w.n_traj)
     d_lpo = torch.zeros((total, ACT), dtype=torch.float32, device="cuda")
@@ -317,7 +334,7 @@ def behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed)
         idx = torch.arange(c0, c1, dtype=torch.int32, device="cuda")
         off = torch.clamp(d_in["traj_off"].to(torch.int32) - c0, 0, c1 - c0).to(torch.int32).contiguous()
         pk_all = B.grpo_pack_chunks(ident, batch, model, idx, off, zero_adv, B.Packed(model, c1 - c0))
-        _, lp, _, _ = B.grpo_actor_fwd_bwd(model, pk_all, flags=B.GRPO_FWD_ONLY, mb_chunks=128)
+        _, lp, _, _ = B.grpo_actor_fwd_bwd(model, pk_all, flags=B.GRPO_FWD_ONLY, mb_chunks=128, lora=lora)
         d_lpo[c0:c1] = lp
         del pk_all
     ident.close()
@@ -345,12 +362,12 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
         h_obs[c0:c1] = torch.randn((c1 - c0, w.P, w.d), generator=gen, dtype=torch.float32).to(td)
     h = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in rb.items()}
 
-    hs = Harness(B, PL, synth, w, weights, n_kept, mb)
+    hs = Harness(B, PL, synth, w, weights, n_kept, mb, args.lora)
     model = hs.model
     ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=seed, max_traj=w.n_traj)
     d_in = {k: v.cuda() for k, v in h.items()}
     d_obs = h_obs.cuda()
-    d_lpo, batch = behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed)
+    d_lpo, batch = behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed, hs.lora)
     h_lpo = d_lpo.cpu().pin_memory()
     kept_host = torch.empty(w.n_traj * w.budget, dtype=torch.int32).pin_memory()
 
@@ -415,8 +432,8 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
         assert B.pcm_poll_status(ctx_full) == 0
         ctx_full.close()
         traj_mb = 8                                    # trajectories per micro-batch for the activation figure
-        act_masked = B.grpo_workspace_bytes(model, traj_mb * w.budget, 0)
-        act_full = B.grpo_workspace_bytes(model, traj_mb * int(lengths.max()), 0)
+        act_masked = B.grpo_workspace_bytes(model, traj_mb * w.budget, 0, hs.lora)
+        act_full = B.grpo_workspace_bytes(model, traj_mb * int(lengths.max()), 0, hs.lora)
         masked_full = {"ms_masked": ms_total / args.steps, "ms_full": ms_full, "speedup": ms_full / (ms_total / args.steps),
                        "kept_chunks_masked": n_kept, "kept_chunks_full": total, "steps_full": full_steps,
                        "activation_bytes": {"masked": int(act_masked), "full": int(act_full),
@@ -437,8 +454,8 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": config_of(w, n_kept, total, mb),
-            "roofline": roofline_of(prof, peaks, args.steps, flops_per_kept_chunk(w) * n_kept, ms_step, traffic),
+            "config": config_of(w, n_kept, total, mb, None, args.lora),
+            "roofline": roofline_of(prof, peaks, args.steps, flops_per_kept_chunk(w, args.lora) * n_kept, ms_step, traffic),
             "kernel_classes": class_table(prof, args.steps),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "ms_per_step": ms_e2e / args.steps},
@@ -456,7 +473,7 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
 
 
 def cpu_baseline_leg(args, w, rb, weights, seed):
-    t_pcm, t_actor, nk = oracle_sample_step(w, rb, weights, seed, args.cpu_sample)
+    t_pcm, t_actor, nk = oracle_sample_step(w, rb, weights, seed, args.cpu_sample, args.lora)
     est = t_pcm + t_actor * nk / args.cpu_sample
     return {"value": nk / est, "unit": UNIT, "cores": blas_threads(), "kind": "oracle (fp64 numpy, BLAS threads = cores)",
             "sample": (f"control plane on the full batch ({t_pcm:.2f} s) + actor fwd/bwd on {args.cpu_sample} of "
@@ -497,7 +514,7 @@ def run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local
         db = {k: v.cuda() for k, v in hb.items()}
         dev_b.append((db, B.make_batch(db["traj_off"], db["tok"], db["phase"], db["reward"], max_len, d_obs, db["lpo"])))
 
-    hs = Harness(B, PL, synth, w, weights, n_kept_max, mb)
+    hs = Harness(B, PL, synth, w, weights, n_kept_max, mb, args.lora)
     barrier, timed = make_timers(torch, dist, dist_util, world)
     # staging buffers of the end-to-end leg (sized for the largest iteration)
     stage = {"traj_off": torch.empty(w.n_traj + 1, dtype=torch.int32, device="cuda"),
@@ -593,14 +610,14 @@ def run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_iter,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(w, n_kept_total / n_iter, sum(totals) / n_iter, mb, n_iter),
+            "config": config_of(w, n_kept_total / n_iter, sum(totals) / n_iter, mb, n_iter, args.lora),
             "online": {"ms_mean": statistics.mean(per_it), "ms_min": min(per_it), "ms_max": max(per_it),
                        "kept_chunks_min": min(kept_per_it), "kept_chunks_max": max(kept_per_it),
                        "chunks_min": min(totals), "chunks_max": max(totals),
                        "keep_prob_refreshes": refreshes, "t_rc": w.t_rc,
                        "keep_probs_first": (q_np[0] / float(1 << 24)).round(4).tolist(),
                        "keep_probs_last": (q_np[-1] / float(1 << 24)).round(4).tolist()},
-            "roofline": roofline_of(prof, peaks, n_iter, flops_per_kept_chunk(w) * n_kept_total / n_iter, ms_step, None),
+            "roofline": roofline_of(prof, peaks, n_iter, flops_per_kept_chunk(w, args.lora) * n_kept_total / n_iter, ms_step, None),
             "kernel_classes": class_table(prof, n_iter),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d / n_iter),
                     "d2h_bytes_per_step": int(d2h / n_iter), "ms_per_step": ms_e2e / n_iter},
@@ -625,6 +642,8 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=2, help="kept chunks the CPU baseline leg runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-masked-full", action="store_true", help="skip the keep-every-chunk leg of the medium workload")
+    ap.add_argument("--lora", type=int, default=0, metavar="RANK",
+                    help="fine-tune low-rank adapters of this rank (alpha = rank) with the base weights frozen")
     args = ap.parse_args()
     from paper_2605_16154_b200 import launch
     if args.impl == "cuda" and launch.needs_relaunch(args.gpus, os.environ):

@@ -5,6 +5,7 @@
 #include <mutex>
 #include <new>
 
+#include "async_ptx.cuh"
 #include "internal.h"
 
 namespace pcm {
@@ -50,153 +51,157 @@ unsigned* ctx_status(pcm_ctx* c) { return c->status; }
 // ------------------------------------------------------------------------------------------------
 // Eq. 5, per group: integer token sums per (phase, outcome), then C_{c,g}
 // ------------------------------------------------------------------------------------------------
-// One CTA per group.  A warp walks whole trajectories.  Two consecutive chunks are 112 bytes = seven
-// 16-byte vectors, so lanes 0..27 load four chunk pairs per step (one per group of seven lanes); each lane owns the
-// same two 8-byte halves of every pair, i.e. the same 8 + 8 action dimensions of the pair's first or second
-// chunk.  Bytes are accumulated as packed 16-bit lanes; a run ends when the phase changes or after 256
-// chunks (255 * 257 < 2^16) and is flushed to 32-bit shared-memory counters.  Integer sums are exact, so
-// any order gives the same result.  A chunk at an odd index at either end of a trajectory (the vectors must
-// be 16-byte aligned) goes through a scalar path.
-__global__ void __launch_bounds__(256)
+// One CTA per group, a warp per trajectory.  The trajectory's tokens are staged in shared memory by asynchronous
+// copies (slabs of 32 chunks, two in flight per warp, about 170 KB per SM over all resident warps), so memory
+// parallelism does not depend on the phase structure.  The warp then finds the runs of equal
+// phase label in the slab (labels are read coalesced into registers while the copies fly, run starts come out of
+// a ballot, start positions and labels go through a small shared list) and sums four runs at a time: a chunk is
+// seven 8-byte vectors, lane = 7 * slot + vec owns vector `vec` (action dimensions 8 vec .. 8 vec + 7) of the
+// run its slot took.  Bytes are accumulated as packed 16-bit lanes (a run inside a slab has at most 32 chunks:
+// 32 * 255 < 2^16) and flushed with eight 32-bit shared-memory adds per lane: the per-run cost is shared by four
+// runs.  Integer sums are exact, so any order gives the same result.
+constexpr int SC_SLAB = 32;                              // chunks per staged slab: one label per lane
+constexpr int SC_SLAB_BYTES = SC_SLAB * ACT;             // 1792
+constexpr int SC_WARPS = 8;
+
+__device__ __forceinline__ void cp_async_8(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void score_add8(const uint2 w, unsigned& a0, unsigned& a1, unsigned& a2, unsigned& a3) {
+  a0 += w.x & 0x00FF00FFu; a1 += __byte_perm(w.x, 0, 0x4341);        // bytes {0, 2} and {1, 3} as 16-bit lanes
+  a2 += w.y & 0x00FF00FFu; a3 += __byte_perm(w.y, 0, 0x4341);
+}
+
+__global__ void __launch_bounds__(SC_WARPS * 32)
 score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restrict__ tok,
                     const uint8_t* __restrict__ phase, const uint8_t* __restrict__ reward, int G,
                     int n_phases, double* __restrict__ c_group, uint8_t* __restrict__ valid_group,
                     unsigned* __restrict__ status) {
-  extern __shared__ unsigned sm[];
+  extern __shared__ __align__(16) unsigned sm[];
+  const int n_cnt = (n_phases * 2 * (ACT + 1) + 3) & ~3; // counters, padded to 16 bytes
   unsigned* sums = sm;                                   // [n_phases][2][56]
   unsigned* cnt = sm + n_phases * 2 * ACT;               // [n_phases][2]
+  uint8_t* stage = reinterpret_cast<uint8_t*>(sm + n_cnt);   // [SC_WARPS][2][SC_SLAB_BYTES]
+  __shared__ unsigned char run_pos[SC_WARPS][SC_SLAB + 4];   // slab-local start of every run, then the slab's length
+  __shared__ unsigned char run_lab[SC_WARPS][SC_SLAB + 4];   // its phase label
   const int g = blockIdx.x;
   for (int i = threadIdx.x; i < n_phases * 2 * (ACT + 1); i += blockDim.x) sm[i] = 0;
   __syncthreads();
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  const int slot = lane / 7, vec = lane - slot * 7;      // slot 0..3 active (4 = idle lanes 28..31)
-  const uint32_t* tokw = reinterpret_cast<const uint32_t*>(tok);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int slot = lane / 7, vec = lane - slot * 7;      // lanes 28..31 (slot 4) idle in the sums
+  uint8_t* mybuf = stage + (size_t)warp * 2 * SC_SLAB_BYTES;
+  unsigned char* rp = run_pos[warp];
+  unsigned char* rl = run_lab[warp];
 
-  for (int i = g * G + warp; i < (g + 1) * G; i += nwarps) {
+  for (int i = g * G + warp; i < (g + 1) * G; i += SC_WARPS) {
     const int o = reward[i] ? 1 : 0;
     const int a = traj_off[i], b = traj_off[i + 1];
-    // scalar path for one chunk: 14 lanes x 4 tokens
-    auto single = [&](int ch) {
-      if (lane < WORDS) {
-        const int ph = phase[ch];
-        if (ph >= n_phases) {
-          atomicOr(status, STATUS_BAD_PHASE);
-        } else {
-          const uint32_t wv = __ldg(tokw + (size_t)ch * WORDS + lane);
-          unsigned* sp = sums + (ph * 2 + o) * ACT + lane * 4;
-          atomicAdd(sp + 0, wv & 0xFFu);
-          atomicAdd(sp + 1, (wv >> 8) & 0xFFu);
-          atomicAdd(sp + 2, (wv >> 16) & 0xFFu);
-          atomicAdd(sp + 3, wv >> 24);
-          if (lane == 0) atomicAdd(cnt + ph * 2 + o, 1u);
-        }
+    const int n_slab = (b - a + SC_SLAB - 1) / SC_SLAB;
+    // stage slab k (chunks a + 32 k ..) into buffer k & 1, one commit group per slab: 16-byte pieces when the slab
+    // starts at an even chunk (56 c is then a multiple of 16), 8-byte pieces otherwise and for an odd tail
+    auto issue = [&](int k) {
+      const int c0 = a + k * SC_SLAB, nc = min(SC_SLAB, b - c0);
+      const uint8_t* src = tok + (size_t)c0 * ACT;
+      uint8_t* dst = mybuf + (k & 1) * SC_SLAB_BYTES;
+      const int bytes = nc * ACT;
+      if ((c0 & 1) == 0) {
+        const int n16 = bytes >> 4;
+        for (int piece = lane; piece < n16; piece += 32) cp_async_16(dst + piece * 16, src + piece * 16);
+        if ((bytes & 8) && lane == 0) cp_async_8(dst + n16 * 16, src + n16 * 16);
+      } else {
+        for (int piece = lane; piece < (bytes >> 3); piece += 32) cp_async_8(dst + piece * 8, src + piece * 8);
       }
+      cp_async_commit();
     };
-    int lo = a;
-    if ((lo & 1) && lo < b) { single(lo); ++lo; }        // pairs start at an even chunk index (16-byte alignment)
-    const int n_pairs = (b - lo) >> 1;
-    if (((b - lo) & 1) && lo < b) single(b - 1);
-
-    if (slot < 4) {
-      // this lane's two 8-byte halves of a pair: which chunk of the pair they belong to and their first dimension
-      const int bo0 = 16 * vec, bo1 = 16 * vec + 8;
-      const int sel[2] = {bo0 >= ACT ? 1 : 0, bo1 >= ACT ? 1 : 0};
-      const int dim0[2] = {bo0 >= ACT ? bo0 - ACT : bo0, bo1 >= ACT ? bo1 - ACT : bo1};
-      const bool counts[2] = {vec == 0, vec == 6};        // one half per chunk also counts the chunk
-      unsigned acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
-      unsigned run[2] = {0, 0};
-      int cur[2] = {-1, -1};
-      auto flush = [&](int hf) {
-        if (run[hf]) {
-          unsigned* sp = sums + (cur[hf] * 2 + o) * ACT + dim0[hf];
-          atomicAdd(sp + 0, acc[hf][0] & 0xFFFFu); atomicAdd(sp + 2, acc[hf][0] >> 16);
-          atomicAdd(sp + 1, acc[hf][1] & 0xFFFFu); atomicAdd(sp + 3, acc[hf][1] >> 16);
-          atomicAdd(sp + 4, acc[hf][2] & 0xFFFFu); atomicAdd(sp + 6, acc[hf][2] >> 16);
-          atomicAdd(sp + 5, acc[hf][3] & 0xFFFFu); atomicAdd(sp + 7, acc[hf][3] >> 16);
-          if (counts[hf]) atomicAdd(cnt + cur[hf] * 2 + o, run[hf]);
+    if (n_slab > 0) issue(0);
+    if (n_slab > 1) issue(1);
+    for (int k = 0; k < n_slab; ++k) {
+      const int c0 = a + k * SC_SLAB, nc = min(SC_SLAB, b - c0);
+      // this slab's labels, one per lane, requested before the wait so that they overlap the copies
+      const int l0 = lane < nc ? (int)__ldg(phase + c0 + lane) : -2;
+      // runs: a chunk starts one when its label differs from its predecessor's; the slab's first chunk always does
+      int p0 = __shfl_up_sync(0xffffffffu, l0, 1);
+      if (lane == 0) p0 = -1;
+      const bool s0 = lane < nc && l0 != p0;
+      const unsigned m0 = __ballot_sync(0xffffffffu, s0);
+      const int n_runs = __popc(m0);
+      __syncwarp();                                      // the previous slab's list has been read by every lane
+      if (s0) { const int r = __popc(m0 & ((1u << lane) - 1u)); rp[r] = (unsigned char)lane; rl[r] = (unsigned char)l0; }
+      if (lane == 0) rp[n_runs] = (unsigned char)nc;
+      if (k + 1 < n_slab) cp_async_wait<1>(); else cp_async_wait<0>();
+      __syncwarp();
+      const uint2* base = reinterpret_cast<const uint2*>(mybuf + (k & 1) * SC_SLAB_BYTES) + vec;
+      for (int r0 = 0; r0 < n_runs; r0 += 4) {           // four runs per round, one per slot
+        const int r = r0 + slot;
+        const bool have = slot < 4 && r < n_runs;
+        int c = have ? rp[r] : 0;
+        int e = have ? rp[r + 1] : 0;
+        const int ph = have ? rl[r] : 0;
+        if (have && ph >= n_phases) {                    // a bad label: reported, its chunks are skipped
+          if (vec == 0) atomicOr(status, STATUS_BAD_PHASE);
+          e = c;
         }
-        acc[hf][0] = acc[hf][1] = acc[hf][2] = acc[hf][3] = 0;
-        run[hf] = 0;
-      };
-      constexpr int UNROLL = 4;                          // pair groups in flight per iteration
-      const uint4* tok16 = reinterpret_cast<const uint4*>(tok + (size_t)lo * ACT);
-      // each of the four lane groups walks its own contiguous quarter of the pairs: runs of equal phase stay long
-      const int per = (n_pairs + 3) >> 2;
-      const int p_end = min(n_pairs, (slot + 1) * per);
-      for (int p0 = slot * per; p0 < p_end; p0 += UNROLL) {
-        uint4 wv[UNROLL];
-        int ph[UNROLL][2];
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-          const int p = p0 + u;
-          if (p < p_end) {
-            wv[u] = __ldg(tok16 + (size_t)p * 7 + vec);
-            ph[u][0] = __ldg(phase + lo + 2 * p + sel[0]);
-            ph[u][1] = __ldg(phase + lo + 2 * p + sel[1]);
-          } else {
-            wv[u] = make_uint4(0, 0, 0, 0);
-            ph[u][0] = ph[u][1] = -1;
+        const int len = e - c;
+        unsigned a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+        while (__any_sync(0xffffffffu, c < e)) {
+          if (c + 1 < e) {
+            const uint2 w0 = base[c * 7], w1 = base[(c + 1) * 7];
+            score_add8(w0, a0, a1, a2, a3);
+            score_add8(w1, a0, a1, a2, a3);
+          } else if (c < e) {
+            score_add8(base[c * 7], a0, a1, a2, a3);
           }
+          c += 2;
         }
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-          const unsigned w4[4] = {wv[u].x, wv[u].y, wv[u].z, wv[u].w};
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            const int pv = ph[u][hf];
-            if (pv < 0) continue;
-            if (pv >= n_phases) {
-              atomicOr(status, STATUS_BAD_PHASE);
-              continue;
-            }
-            if (pv != cur[hf] || run[hf] == 256) {
-              flush(hf);
-              cur[hf] = pv;
-            }
-            acc[hf][0] += w4[2 * hf] & 0x00FF00FFu;
-            acc[hf][1] += (w4[2 * hf] >> 8) & 0x00FF00FFu;
-            acc[hf][2] += w4[2 * hf + 1] & 0x00FF00FFu;
-            acc[hf][3] += (w4[2 * hf + 1] >> 8) & 0x00FF00FFu;
-            ++run[hf];
-          }
+        if (len > 0) {
+          unsigned* sp = sums + (ph * 2 + o) * ACT + vec * 8;   // a0 = dims {0, 2}, a1 = {1, 3}, a2 = {4, 6}, a3 = {5, 7}
+          atomicAdd(sp + 0, a0 & 0xFFFFu); atomicAdd(sp + 2, a0 >> 16);
+          atomicAdd(sp + 1, a1 & 0xFFFFu); atomicAdd(sp + 3, a1 >> 16);
+          atomicAdd(sp + 4, a2 & 0xFFFFu); atomicAdd(sp + 6, a2 >> 16);
+          atomicAdd(sp + 5, a3 & 0xFFFFu); atomicAdd(sp + 7, a3 >> 16);
+          if (vec == 0) atomicAdd(cnt + ph * 2 + o, (unsigned)len);
         }
       }
-      flush(0);
-      flush(1);
+      __syncwarp();                                      // every lane is done with the buffer before it is refilled
+      if (k + 2 < n_slab) issue(k + 2);
     }
   }
   __syncthreads();
 
-  // C_{c,g}: individually rounded fp64 operations.  A warp per phase: the 56 squared differences are formed
-  // in parallel (two dimensions per lane), then lane 0 adds them in ascending-dimension order, which is the
-  // order the result is defined with.
-  __shared__ double sq[8][ACT];
-  for (int c = warp; c < n_phases; c += nwarps) {
+  // C_{c,g}: individually rounded fp64 operations.  All threads form the squared differences of the phases present
+  // in both outcomes; then lane c of the first warp adds phase c's 56 values in ascending-dimension order, which is
+  // the order the result is defined with (the chains of all phases run side by side).
+  double* sq = reinterpret_cast<double*>(stage);         // [n_phases][56], over the token slabs (no longer needed)
+  for (int idx = threadIdx.x; idx < n_phases * ACT; idx += blockDim.x) {
+    const int c = idx / ACT, dim = idx - c * ACT;
     const unsigned n_succ = cnt[c * 2 + 1], n_fail = cnt[c * 2 + 0];
-    const bool both = n_succ && n_fail;
+    if (n_succ && n_fail) {
+      const double m1 = __ddiv_rn((double)sums[(c * 2 + 1) * ACT + dim], (double)n_succ);
+      const double m0 = __ddiv_rn((double)sums[(c * 2 + 0) * ACT + dim], (double)n_fail);
+      const double diff = __dsub_rn(m1, m0);
+      sq[idx] = __dmul_rn(diff, diff);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < n_phases) {
+    const int c = threadIdx.x;
+    const bool both = cnt[c * 2 + 1] && cnt[c * 2 + 0];
+    double val = 0.0;
     if (both) {
-      const unsigned* s1 = sums + (c * 2 + 1) * ACT;
-      const unsigned* s0 = sums + (c * 2 + 0) * ACT;
-      for (int dim = lane; dim < ACT; dim += 32) {
-        const double m1 = __ddiv_rn((double)s1[dim], (double)n_succ);
-        const double m0 = __ddiv_rn((double)s0[dim], (double)n_fail);
-        const double diff = __dsub_rn(m1, m0);
-        sq[warp][dim] = __dmul_rn(diff, diff);
-      }
+      double acc = 0.0;
+      for (int dim = 0; dim < ACT; ++dim) acc = __dadd_rn(acc, sq[c * ACT + dim]);
+      val = __dmul_rn(__dsqrt_rn(acc), 2.0 / 256.0);
     }
-    __syncwarp();
-    if (lane == 0) {
-      double val = 0.0;
-      if (both) {
-        double acc = 0.0;
-        for (int dim = 0; dim < ACT; ++dim) acc = __dadd_rn(acc, sq[warp][dim]);
-        val = __dmul_rn(__dsqrt_rn(acc), 2.0 / 256.0);
-      }
-      c_group[(size_t)g * n_phases + c] = val;
-      valid_group[(size_t)g * n_phases + c] = both ? 1 : 0;
-    }
-    __syncwarp();
+    c_group[(size_t)g * n_phases + c] = val;
+    valid_group[(size_t)g * n_phases + c] = both ? 1 : 0;
   }
 }
 
@@ -568,6 +573,27 @@ static int check_batch(const pcm_ctx* ctx, const pcm_batch* b) {
 
 using namespace pcm;
 
+// score_groups_kernel with its shared memory: the counters plus two 32-chunk slabs per warp (29 KB, with 32 phases
+// 43 KB; the attribute is set once per device so that any count stays legal).  Allocates nothing.
+static int launch_score_groups(const pcm_batch* b, int G, int n_phases, int n_groups, double* c_group, uint8_t* valid_group,
+                               unsigned* status, cudaStream_t s) {
+  const size_t n_cnt = ((size_t)n_phases * 2 * (ACT + 1) + 3) & ~(size_t)3;
+  const size_t smem = n_cnt * sizeof(unsigned) + (size_t)SC_WARPS * 2 * SC_SLAB_BYTES;
+  static unsigned long long attr_devices = 0;
+  static std::mutex mu;
+  {
+    std::lock_guard<std::mutex> lk(mu);
+    if (attr_needed(&attr_devices))
+      PCM_CUDA_TRY(cudaFuncSetAttribute(score_groups_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(((size_t)PCM_MAX_PHASES * 2 * (ACT + 1) + 3) * sizeof(unsigned) +
+                                              (size_t)SC_WARPS * 2 * SC_SLAB_BYTES)));
+  }
+  score_groups_kernel<<<n_groups, SC_WARPS * 32, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, G, n_phases, c_group,
+                                                          valid_group, status);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
+}
+
 extern "C" {
 
 int pcm_create(pcm_ctx** out, const pcm_config* cfg, int32_t max_traj) {
@@ -656,11 +682,9 @@ int pcm_score_phases(pcm_ctx* ctx, const pcm_batch* b, double* C, uint8_t* valid
   if (((uintptr_t)b->tok) & 15) return PCM_ERR_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   const int G = ctx->cfg.group_size, Kc = ctx->cfg.n_phases, ng = b->n_traj / G;
-  const size_t smem = (size_t)Kc * 2 * (ACT + 1) * sizeof(unsigned);
   prof_begin(PC_SCORE, s);
-  score_groups_kernel<<<ng, 256, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, G, Kc, ctx->c_group,
-                                             ctx->valid_group, ctx->status);
-  PCM_LAUNCH_CHECK();
+  rc = launch_score_groups(b, G, Kc, ng, ctx->c_group, ctx->valid_group, ctx->status, s);
+  if (rc) return rc;
   prof_end(s, 0.0, (double)b->n_chunks * (ACT + 1));
   const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
   score_finalize_kernel<<<Kc + adv_blocks, 128, 0, s>>>(ctx->c_group, ctx->valid_group, ng, Kc, C, valid,
@@ -785,10 +809,8 @@ extern "C" int pcm_score_phases_static(int32_t n_phases, int32_t group_size, dou
   unsigned* status = reinterpret_cast<unsigned*>(base + NA_CGROUP_BYTES + NA_VALID_BYTES);
   cudaStream_t s = (cudaStream_t)stream;
   PCM_CUDA_TRY(cudaMemsetAsync(status, 0, sizeof(unsigned), s));   // the only part that must start at zero
-  const size_t smem = (size_t)n_phases * 2 * (ACT + 1) * sizeof(unsigned);
-  score_groups_kernel<<<ng, 256, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, group_size, n_phases, c_group,
-                                             valid_group, status);
-  PCM_LAUNCH_CHECK();
+  const int rc_launch = launch_score_groups(b, group_size, n_phases, ng, c_group, valid_group, status, s);
+  if (rc_launch) return rc_launch;
   const int adv_blocks = adv ? ceil_div(ng, 128) : 0;
   score_finalize_kernel<<<n_phases + adv_blocks, 128, 0, s>>>(c_group, valid_group, ng, n_phases, C, valid, n_valid_groups,
                                                        b->reward, group_size, adv_eps, adv);
