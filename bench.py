@@ -157,11 +157,12 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def config_of(w, n_kept, total, mb, iterations=None, lora_rank=0):
+def config_of(w, n_kept, total, mb, iterations=None, lora_rank=0, dp=False, world=1):
     """The `config` object both arms print."""
     c = {"workload": w.name, "trainable": f"LoRA rank {lora_rank}, alpha {lora_rank}, base frozen" if lora_rank else "all weights", "kept_chunks_per_step": int(n_kept), "chunks_per_step": int(total),
          "tokens_per_step": int(n_kept) * w.S, "mb_chunks": int(mb), "l2": "inputs_larger_than_l2",
-         "multi_gpu": "independent replicas, no collective"}
+         "multi_gpu": (f"data parallel over {world} ranks: one batch, kept chunks dealt out by trajectory, one fp32 gradient "
+                       "all-reduce per step") if dp else "independent replicas, no collective"}
     if iterations is not None:
         c["iterations"] = int(iterations)
         c["resampled"] = "rollouts redrawn every iteration from seeds 0..iterations-1, keep-probability state carried"
@@ -222,8 +223,15 @@ class Harness:
         # adapters part-way through training (non-zero B), alpha = rank as in App. E
         self.lora = PL.upload_lora(w, self.model, synth.make_lora(w, lora_rank, float(lora_rank))) if lora_rank else None
         self.ws = torch.empty(B.grpo_workspace_bytes(self.model, mb, 0, self.lora) + 256, dtype=torch.uint8, device="cuda")
+        if self.lora is not None:
+            self.lora.alloc_grads()
+        self.dp, self.loss_scale, self.dist_util = None, 0.0, None      # set by data_parallel()
         self.loss = torch.zeros(1, dtype=torch.float32, device="cuda")
         self.outputs(n_kept_max, w.n_traj, w.budget)
+
+    def data_parallel(self, dist_util, rank, world, n_kept_global):
+        """The ranks share one batch: this one takes its trajectories under the whole batch's loss scale."""
+        self.dist_util, self.dp, self.loss_scale = dist_util, (rank, world), 1.0 / (ACT * n_kept_global)
 
     def outputs(self, n_kept, n_traj, budget):
         import torch
@@ -240,13 +248,20 @@ class Harness:
         Cc, valid, _, adv = B.pcm_score_phases(ctx, bt)
         _, q = B.pcm_update_keep_probs(ctx, Cc, valid)
         kept_idx, kept_off, _ = B.pcm_sample_chunks(ctx, bt, q, it, out=self.samp)
+        if self.dp is not None:                      # data parallel: this rank's trajectories of the shared selection
+            kept_idx, kept_off = self.dist_util.partition_kept(kept_idx, kept_off, *self.dp)
         return adv, kept_idx, kept_off, q
 
     def update(self, ctx, bt, adv, kept_idx, kept_off):
         B, w = self.B, self.w
         B.grpo_pack_chunks(ctx, bt, self.model, kept_idx, kept_off, adv, self.packed)
-        B.grpo_actor_fwd_bwd(self.model, self.packed, w.eps_low, w.eps_high, 0.0, mb_chunks=self.mb, workspace=self.ws,
-                             want_stats=False, logp=self.logp, loss=self.loss, lora=self.lora)
+        B.grpo_actor_fwd_bwd(self.model, self.packed, w.eps_low, w.eps_high, self.loss_scale, mb_chunks=self.mb,
+                             workspace=self.ws, want_stats=False, logp=self.logp, loss=self.loss, lora=self.lora)
+        if self.dp is not None:                      # one sum over the ranks: full-batch gradient (and loss) everywhere
+            self.dist_util.allreduce_sum(self.lora.flat_grads if self.lora is not None else self.model.flat_grads)
+            if self.lora is not None:
+                self.dist_util.allreduce_sum(self.model.flat_grads)
+            self.dist_util.allreduce_sum(self.loss)
 
     def step(self, ctx, bt, it):
         adv, kept_idx, kept_off, _ = self.select(ctx, bt, it)
@@ -298,6 +313,7 @@ def run_cuda(args):
 
     w = synth.WORKLOADS[args.workload]
     if w.T == 0:
+        assert not args.dp, "--dp is implemented for the fixed-length workloads"
         run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank)
     else:
         run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank)
@@ -346,12 +362,14 @@ def behaviour_logp(torch, B, synth, w, model, d_in, d_obs, lengths, total, seed,
 def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank):
     """Fixed-length workloads (C0-C3): K steps over one resident batch."""
     td = PL.torch_dtype(w)
-    seed = dist_util.replica_seed(w.seed, rank)    # every rank works on its own batch (replicas, no exchange)
+    # replicas: every rank works on its own batch, no exchange.  --dp: all ranks share the batch of rank 0's seed
+    seed = w.seed if args.dp else dist_util.replica_seed(w.seed, rank)
     rb = synth.make_rollouts(w, seed)
     weights = synth.make_weights(w)
     lengths = np.diff(rb["traj_off"])
     total = int(rb["traj_off"][-1])
-    n_kept = PL.n_kept_of(w.budget, rb["traj_off"])
+    n_kept_global = PL.n_kept_of(w.budget, rb["traj_off"])
+    n_kept = dist_util.local_kept_count(lengths, w.budget, rank, world) if args.dp else n_kept_global
     mb = default_mb(args, n_kept)
 
     # host inputs in pinned memory (what an end-to-end caller owns)
@@ -363,6 +381,8 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
     h = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in rb.items()}
 
     hs = Harness(B, PL, synth, w, weights, n_kept, mb, args.lora)
+    if args.dp:
+        hs.data_parallel(dist_util, rank, world, n_kept_global)
     model = hs.model
     ctx = B.Context(w.n_phases, w.budget, w.G, w.t_rc, w.p_min, 1e-6, seed=seed, max_traj=w.n_traj)
     d_in = {k: v.cuda() for k, v in h.items()}
@@ -379,7 +399,7 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
             d_in[k].copy_(h[k], non_blocking=True)
         d_lpo.copy_(h_lpo, non_blocking=True)
         adv, kept_idx, kept_off, _ = hs.select(ctx, batch, it)
-        kept_host.copy_(kept_idx, non_blocking=True)
+        kept_host[:kept_idx.numel()].copy_(kept_idx, non_blocking=True)
         torch.cuda.current_stream().synchronize()
         for c in kept_host[:n_kept].tolist():
             d_obs[c].copy_(h_obs[c], non_blocking=True)
@@ -422,7 +442,7 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
 
     # ---- the same update with the mask keeping every chunk (plain GRPO), for the masked / full ratio ----
     masked_full = None
-    if w.name == "C1" and world == 1 and not args.no_masked_full:
+    if w.name == "C1" and world == 1 and not args.no_masked_full and not args.dp:
         full_steps = 3
         ctx_full = B.Context(w.n_phases, int(lengths.max()), w.G, w.t_rc, w.p_min, 1e-6, seed=seed, max_traj=w.n_traj)
         hs.outputs(total, w.n_traj, int(lengths.max()))
@@ -445,16 +465,21 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
     if rank == 0:
         peaks = measured_peaks()
         ms_step = ms_total / args.steps
-        value = dist_util.aggregate_throughput(n_kept, args.steps, ms_total, world)
-        e2e_value = dist_util.aggregate_throughput(n_kept, args.steps, ms_e2e, world)
+        if args.dp:                                   # one batch over all ranks: the whole job is n_kept_global per step
+            value = dist_util.aggregate_throughput(n_kept_global, args.steps, ms_total, 1)
+            e2e_value = dist_util.aggregate_throughput(n_kept_global, args.steps, ms_e2e, 1)
+        else:
+            value = dist_util.aggregate_throughput(n_kept, args.steps, ms_total, world)
+            e2e_value = dist_util.aggregate_throughput(n_kept, args.steps, ms_e2e, world)
         traffic = None
         if GEMM_TRAFFIC_CAPTURE and GEMM_TRAFFIC_CAPTURE["rows"] == min(mb, n_kept) * w.S and w.d == GEMM_TRAFFIC_CAPTURE["k"]:
             traffic = GEMM_TRAFFIC_CAPTURE["dram_bytes"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong" if args.dp else "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": config_of(w, n_kept, total, mb, None, args.lora),
+            "config": config_of(w, n_kept_global if args.dp else n_kept, total, mb, None, args.lora, args.dp, world),
             "roofline": roofline_of(prof, peaks, args.steps, flops_per_kept_chunk(w, args.lora) * n_kept, ms_step, traffic),
             "kernel_classes": class_table(prof, args.steps),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -642,6 +667,8 @@ def main():
     ap.add_argument("--cpu-sample", type=int, default=2, help="kept chunks the CPU baseline leg runs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-masked-full", action="store_true", help="skip the keep-every-chunk leg of the medium workload")
+    ap.add_argument("--dp", action="store_true",
+                    help="data parallel instead of replicas: the ranks share one batch and all-reduce the gradients")
     ap.add_argument("--lora", type=int, default=0, metavar="RANK",
                     help="fine-tune low-rank adapters of this rank (alpha = rank) with the base weights frozen")
     args = ap.parse_args()

@@ -316,8 +316,17 @@ class Model:
         return self.cfg.prefix_len + ACT_DIM
 
     def alloc_grads(self) -> Dict[str, torch.Tensor]:
+        """fp32 gradient tensors, views of one flat buffer (self.flat_grads) so that a data-parallel caller can
+        sum all of them over the ranks with a single all-reduce."""
         if self.grads is None:
-            self.grads = {k: torch.zeros(v.shape, dtype=torch.float32, device=v.device) for k, v in self.weights.items()}
+            sizes = [(k, self.weights[k].numel()) for k in _WEIGHTS]
+            pad = lambda n: (n + 63) // 64 * 64                      # every tensor starts 256-byte aligned
+            self.flat_grads = torch.zeros(sum(pad(n) for _, n in sizes), dtype=torch.float32,
+                                          device=self.weights["w_qkv"].device)
+            self.grads, off = {}, 0
+            for k, n in sizes:
+                self.grads[k] = self.flat_grads[off:off + n].view(self.weights[k].shape)
+                off += pad(n)
             self.c_grads = grpo_grads(*[_ptr(self.grads[k]) for k in _WEIGHTS])
         return self.grads
 
@@ -335,8 +344,16 @@ class Lora:
         self.c_grads: Optional[grpo_lora_grads] = None
 
     def alloc_grads(self) -> Dict[str, torch.Tensor]:
+        """fp32 adapter gradients, views of one flat buffer (self.flat_grads)."""
         if self.grads is None:
-            self.grads = {k: torch.zeros(v.shape, dtype=torch.float32, device=v.device) for k, v in self.tensors.items()}
+            sizes = [(k, self.tensors[k].numel()) for k in _LORA]
+            pad = lambda n: (n + 63) // 64 * 64
+            self.flat_grads = torch.zeros(sum(pad(n) for _, n in sizes), dtype=torch.float32,
+                                          device=self.tensors["a_qkv"].device)
+            self.grads, off = {}, 0
+            for k, n in sizes:
+                self.grads[k] = self.flat_grads[off:off + n].view(self.tensors[k].shape)
+                off += pad(n)
             self.c_grads = grpo_lora_grads(*[_ptr(self.grads[k]) for k in _LORA])
         return self.grads
 
