@@ -24,9 +24,10 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 
 # DRAM traffic of the dominant kernel, from one ncu capture of ONE launch at the shape the medium workload runs
-# (QKV projection, all 119 808 tokens in one micro-batch): dram__bytes_read.sum + dram__bytes_write.sum.  None until
-# such a capture exists for the kernel as it stands; never scaled from another size.
-GEMM_TRAFFIC_CAPTURE = None
+# (QKV projection, all 119 808 tokens in one micro-batch; profiles/gemm_tc2_kernel_M119808_N3072_K1024_traffic_ncu.md):
+# dram__bytes_read.sum 251.74 MB (= A + B, each byte once) + dram__bytes_write.sum 686.61 MB (49 MB of C are still in
+# L2 when the kernel ends).  Printed only when the run launches exactly this shape; never scaled from another size.
+GEMM_TRAFFIC_CAPTURE = {"rows": 119808, "n": 3072, "k": 1024, "dram_bytes": 938.35e6, "algorithmic_bytes": 987.76e6}
 
 # Context figures the paper reports for its own runs (7B policy with LoRA on 2 x H100, LIBERO): not targets.
 PAPER_CONTEXT = {"wall_clock_speedup": 2.38, "gradient_update_speedup": 4.8, "activation_memory_reduction": 0.60,
@@ -290,7 +291,8 @@ def roofline_of(prof, peaks, steps, step_flops, ms_step, traffic):
     step_tflops = step_flops / (ms_step * 1e9)
     return {"bound": "tensor", "kernel": "gemm_tc2_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
             "frac": achieved / peak if peak else None, "traffic": traffic,
-            "traffic_of": ("one QKV-projection launch at this workload's full micro-batch, ncu dram read + write"
+            "traffic_of": ("one QKV-projection launch [119808 x 3072 x 1024], ncu dram read + write; algorithmic 987.76 MB, "
+                           "of which 49 MB of the output are still in L2 when the kernel ends"
                            if traffic is not None else "no capture of the current kernel at this shape"),
             "peak_source": peaks["source"] + " bf16_tflops_sustained (kernel timed inside a long step)",
             "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
