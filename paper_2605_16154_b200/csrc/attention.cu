@@ -1,5 +1,6 @@
 // Dispatch of the attention entry points on the activation dtype: fp32 runs the SIMT kernels
-// (attention_f32.cu), bf16 the tensor-core kernels (attention_mma.cu).
+// (attention_f32.cu); bf16 runs the tcgen05 kernels (attention_tc.cu) when they take the shape (head dim 64 or
+// 128, S <= 384, 16-byte aligned tensors), else the warp-level mma.sync kernels (attention_mma.cu: head dim 32).
 #include <cstdlib>
 
 #include "internal.h"
