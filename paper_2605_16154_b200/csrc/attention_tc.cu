@@ -873,8 +873,10 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         const uint32_t acc0 = tmem_base + (uint32_t)C::ACC_COL, acc1 = acc0 + DH;
         const bool fresh = pc.it.first();
         if (MODE == BW_DKV) {
-          issue_acc(pc, acc0, dp_col, 0, fresh);                       // dK += dS^T Q_i (dS^T sits in the dP buffer)
-          if (NSBUF == 2 && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }   // the dP buffer is free again: next block's dP
+          // P^T and dS^T both sit in the block's score buffer, so the dP buffer is free: the next block's dP goes
+          // first and the compute warps start on it while the accumulating products of this block run
+          if (NSBUF == 2 && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }
+          issue_acc(pc, acc0, s_col + 16u, 0, fresh);                  // dK += dS^T Q_i
           if (fresh && k >= 1 && !mbar_wait_bounded(&accv_empty[(k - 1) & 1], (unsigned)((k - 1) >> 1) & 1u, WAIT_NS)) {
             fa_timeout(SITE_O_EMPTY); ok = false; break;
           }
@@ -1132,6 +1134,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         // 0 = every element of this warp's slice is kept, 1 = mixed, 2 = every element is masked
         int mode_mask = 0;
         if (it.diag(shp)) mode_mask = slice == quad ? 1 : ((MODE == BW_DQ ? slice > quad : slice < quad) ? 2 : 0);
+        uint32_t ds_first[8];                                       // BW_DKV: dS^T of the first half, stored after the second half's scores are read
 #pragma unroll 1
         for (int hc = 0; hc < 32; hc += 16) {
           uint32_t pp[8], pd8[8];
@@ -1163,13 +1166,21 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
               pd8[e >> 1] = pack_bf16x2(ds[0], ds[1]);
             }
           }
-          // packed results go over the first 16 columns of this warp's own slice (already consumed for hc = 0;
-          // for hc = 16 the columns written, 8..15, were read in the first half)
+          // packed results go over this warp's own 32 score columns, each column only after it has been read:
+          // P^T (BW_DQ: dS) into columns 0..15 (0..7 consumed in the first half, 8..15 in the second); BW_DKV keeps
+          // dS^T beside it in columns 16..31, which are free once the second half has been read.  Nothing is
+          // written into the dP buffer, so the next block's dP may be formed as soon as this block's has been read.
           if (MODE == BW_DQ) {
             tmem_st_32x8(s_addr + (uint32_t)(hc >> 1), pd8);           // dS over the scores
           } else {
             tmem_st_32x8(s_addr + (uint32_t)(hc >> 1), pp);            // P^T over S^T
-            tmem_st_32x8(dp_addr + (uint32_t)(hc >> 1), pd8);          // dS^T over dP^T
+            if (hc == 0) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ds_first[e] = pd8[e];
+            } else {
+              tmem_st_32x8(s_addr + 16u, ds_first);                    // dS^T, first half
+              tmem_st_32x8(s_addr + 24u, pd8);                         // dS^T, second half
+            }
           }
         }
         tmem_st_wait();

@@ -27,7 +27,9 @@ namespace pcm {
 
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                     // 64 bf16 = one 128-byte swizzle row
-constexpr int TC_STAGES = 3;
+// Ring depth of the single-CTA kernel: as deep as shared memory allows.  Its launches are the narrow or short GEMMs
+// (adapter products, the head), which are bound by getting their A operand out of HBM: bytes in flight, not MMAs.
+template <int BN> constexpr int tc_stages() { return BN == 128 ? 5 : 3; }
 constexpr int TC_EPI_WARPS = 8;                // two per tensor-memory lane quadrant, each takes half of the columns
 constexpr int EPI_STAGE_STRIDE = 36;            // floats per staged epilogue row (32 + 4 of padding: conflict free)
 constexpr int EPI_STAGE_FLOATS = 32 * EPI_STAGE_STRIDE;   // per epilogue warp
@@ -124,7 +126,9 @@ struct TcSmem {
   static constexpr int A_BYTES = TC_BM * TC_BK * 2;           // 16 KB
   static constexpr int B_BYTES = BN * TC_BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int TOTAL = TC_STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + EPI_STAGE_BYTES;
+  static constexpr int STAGES = tc_stages<BN>();
+  static constexpr int TOTAL = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */ + EPI_STAGE_BYTES;
+  static_assert(TOTAL <= 227 * 1024, "shared-memory plan does not fit");
 };
 
 // The plain epilogue stores through a per-warp shared-memory buffer: tcgen05.ld hands every thread one row
@@ -526,6 +530,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   using SM = TcSmem<BN>;
   const uint32_t raw_addr = smem_u32(smem_raw);
   uint8_t* tiles = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);       // swizzle atoms need 1024-byte alignment
+  constexpr int TC_STAGES = SM::STAGES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + TC_STAGES * SM::STAGE_BYTES);
   uint64_t* full = bars;                      // [TC_STAGES] producer -> MMA
   uint64_t* empty = bars + TC_STAGES;         // [TC_STAGES] MMA -> producer
