@@ -570,8 +570,8 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 // ------------------------------------------------------------------------------------------------
 // backward
 // ------------------------------------------------------------------------------------------------
-// Two launches of one kernel template, both built like the forward pass (TMA producer, one MMA thread,
-// compute warps on tensor memory, output warps with a TMA store), both recomputing the probabilities
+// Two launches of one kernel template, both built like the forward pass (TMA producer, MMA issue - here by two
+// threads -, compute warps on tensor memory, output warps with a TMA store), both recomputing the probabilities
 // from the saved log-sum-exp:
 //   BW_DQ   item = (sequence, head, query tile i): the tile's Q_i and dO_i stay in shared memory, the key
 //           blocks j <= i stream by.  Per block: S = Q_i K_j^T and dP = dO_i V_j^T into tensor memory;
@@ -579,15 +579,16 @@ fa_tc_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 //           it as packed bf16 over the scores; dQ_i += dS K_j with dS as the tensor-memory A operand.
 //           This launch also writes rowsum(dO o O) for the second one.
 //   BW_DKV  item = (sequence, head, key block j): K_j and V_j stay, the query tiles i >= j stream by.
-//           Per block: S^T = K_j Q_i^T and dP^T = V_j dO_i^T (rows = keys); P^T is written over S^T and
-//           dS^T over dP^T; dV_j += P^T dO_i and dK_j += dS^T Q_i.
+//           Per block: S^T = K_j Q_i^T and dP^T = V_j dO_i^T (rows = keys); P^T and dS^T are written over S^T,
+//           side by side; dV_j += P^T dO_i and dK_j += dS^T Q_i.
 // The streamed tile is the B operand twice: K-major for the first two products, MN-major (same bytes,
 // another descriptor) for the accumulating ones.  Scores are double-buffered for head dim 64, so the
 // tensor core forms the next block's scores while the compute warps work.  The output warps scale by
 // 1 / sqrt(dh), rotate dQ and dK back through the rotary embedding when a table is given, and store.
 enum { BW_DQ = 0, BW_DKV = 1 };
 constexpr int BW_COMPUTE_WARPS = 16;            // four per tensor-memory lane quadrant: one 32-column slice each
-constexpr int BW_THREADS = (2 + 4 + BW_COMPUTE_WARPS) * 32;
+constexpr int BW_ACC_WARP = 2 + 4 + BW_COMPUTE_WARPS;   // the warp whose lane 0 issues the accumulating products
+constexpr int BW_THREADS = (BW_ACC_WARP + 1) * 32;
 constexpr int BW_COMPUTE_BAR = 10;              // named barrier of the compute warps
 constexpr int BW_OUT_BAR = 11;                  // named barrier of the output warps
 
@@ -702,11 +703,19 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   uint64_t* str_full = bars + 6;               // [4] producer -> MMA: a block's streamed pair has landed
   uint64_t* str_empty = bars + 10;             // [4] MMA -> producer
   uint64_t* sdp_full = bars + 20;              // MMA -> compute: S and dP of a block are in tensor memory
-  uint64_t* p_ready = bars + 21;               // compute -> MMA: P / dS of the block are in tensor memory (16 warp arrivals)
+  // compute -> MMA threads: P / dS of the block are in tensor memory (16 warp arrivals).  Two barriers, used by
+  // alternate blocks: the accumulating threads may still be on their way to block b's phase when block b + 1
+  // completes, and a parity wait cannot tell a phase from the one two later on the same barrier; block b + 2, the
+  // next one on this barrier, cannot complete before every accumulating thread has seen block b (its scores need
+  // the score buffer those threads release).
+  uint64_t* p_ready0 = bars + 21;
   uint64_t* acc_full = bars + 14;              // [2] MMA -> output warps: the item's accumulators are complete
   uint64_t* acc_empty = bars + 16;             // [2] output warps -> MMA (4 warp arrivals): dQ / dK accumulator read; items alternate
   uint64_t* accv_empty = bars + 18;            // [2] the same for the dV accumulator
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 22);
+  uint64_t* s_free = bars + 22;                // [2] accumulating MMAs -> score MMAs: P / dS of the block that used the score buffer have been read
+  uint64_t* p_ready1 = bars + 24;
+  auto p_ready = [&](int block) { return (block & 1) ? p_ready1 : p_ready0; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   float* stat = reinterpret_cast<float*>(base + pl.stat_off);        // BW_DKV: [2][2][128] column statistics; BW_DQ: [4][128] partial row sums
 
@@ -718,7 +727,8 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
     for (int s = 0; s < 3; ++s) { mbar_init(&fix_full[s], 1); mbar_init(&fix_empty[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); mbar_init(&accv_empty[s], 4); }
     for (int s = 0; s < 4; ++s) { mbar_init(&str_full[s], 1); mbar_init(&str_empty[s], 1); }
-    mbar_init(sdp_full, 1); mbar_init(p_ready, BW_COMPUTE_WARPS);
+    mbar_init(sdp_full, 1); mbar_init(p_ready0, BW_COMPUTE_WARPS); mbar_init(p_ready1, BW_COMPUTE_WARPS);
+    mbar_init(&s_free[0], 1); mbar_init(&s_free[1], 1);
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmQKV);
@@ -786,9 +796,16 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       }
       if (!ok) *abort_flag = 1;
     }
-  } else if (warp == 1) {
+  } else if (warp == 1 || warp == BW_ACC_WARP) {
     if (lane == 0) {
-      // ------------------------------ MMA issuer ------------------------------
+      // ------------------------------ MMA issuers ------------------------------
+      // Two threads: a tcgen05.mma costs its issuing thread 70 to 140 cycles (most with the A operand in tensor
+      // memory) and a block needs 16 (dQ pass) or 24 (dK / dV pass) of them.  Warp 1 issues the products that open a
+      // block (scores, then dP) as far ahead as the buffers allow; the last warp issues the accumulating products
+      // once the compute warps have written P / dS, and releases operands and accumulators.  What one thread's
+      // products must wait for in the other's travels through barriers: p_ready (dP buffer consumed; P / dS written)
+      // and s_free (a score buffer's P / dS have been read by the accumulating products).  (A third thread, one per
+      // accumulator in the dK / dV pass, measured no faster.)
       bool ok = true;
       auto desc = [](uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; };
       const uint64_t dfk = smem_desc(smem_u32(base + pl.fix_off), 16u, 1024u);        // resident tiles: K-major A operands
@@ -798,7 +815,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       const uint32_t dsk_lo = (uint32_t)dsk, dsk_hi = (uint32_t)(dsk >> 32);
       const uint32_t dsm_lo = (uint32_t)dsm, dsm_hi = (uint32_t)(dsm >> 32);
       const uint32_t idesc_full = idesc_bf16(BN, 0), idesc_tail = idesc_bf16(nb_tail, 0), idesc_acc = idesc_bf16(DH, 1);
-      // ring positions of the three issue streams: scores (furthest ahead), dP, accumulation
+      // position of an issue stream in the operand rings
       struct Pos { BwIter it; int fs, ss, sph, fph; };
       auto pos_init = [&](Pos& q) { q.it.init(shp); q.fs = q.ss = q.sph = q.fph = 0; };
       auto pos_next = [&](Pos& q) {
@@ -807,96 +824,96 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
         if (++q.ss == C::STR_STAGES) { q.ss = 0; q.sph ^= 1; }
         if (item_end && ++q.fs == C::FIX_STAGES) { q.fs = 0; q.fph ^= 1; }
       };
-      Pos ps, pd, pc;                           // scores / dP / current (accumulating) block
-      pos_init(ps); pos_init(pd); pos_init(pc);
-      // first product of a block: scores into buffer sb.  Waits for the block's operands (first use of both).
-      auto issue_scores = [&](Pos& q, int sb) {
-        if (q.it.first() && !mbar_wait_bounded(&fix_full[q.fs], (unsigned)q.fph, WAIT_NS)) { fa_timeout(SITE_KV_FULL); ok = false; return; }
-        if (!mbar_wait_bounded(&str_full[q.ss], (unsigned)q.sph, WAIT_NS)) { fa_timeout(SITE_Q_FULL); ok = false; return; }
-        tc_fence_after();
-        const uint32_t a = dfk_lo + (uint32_t)q.fs * (FIXB >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4);
-        const uint32_t idesc = (q.it.stile(shp) == p.nq - 1) ? idesc_tail : idesc_full;
-        const uint32_t d_col = tmem_base + (uint32_t)(sb * BN);
+      if (warp == 1) {
+        // ---- opening products: S (or S^T) into score buffer n % NSBUF, dP (dP^T) into the dP buffer ----
+        Pos pa;
+        pos_init(pa);
+        for (int n = 0; pa.it.valid(shp) && ok; ++n) {
+          if (*abort_flag) { ok = false; break; }
+          const int sb = NSBUF == 2 ? (n & 1) : 0;
+          // operands of the block (first use of both pairs)
+          if (pa.it.first() && !mbar_wait_bounded(&fix_full[pa.fs], (unsigned)pa.fph, WAIT_NS)) { fa_timeout(SITE_KV_FULL); ok = false; break; }
+          if (!mbar_wait_bounded(&str_full[pa.ss], (unsigned)pa.sph, WAIT_NS)) { fa_timeout(SITE_Q_FULL); ok = false; break; }
+          // the score buffer: block n - NSBUF left P / dS in it until its accumulating products had read them
+          if (n >= NSBUF && !mbar_wait_bounded(&s_free[sb], (unsigned)(n / NSBUF - 1) & 1u, WAIT_NS)) { fa_timeout(SITE_S_FULL); ok = false; break; }
+          tc_fence_after();
+          const uint32_t idesc = (pa.it.stile(shp) == p.nq - 1) ? idesc_tail : idesc_full;
+          {
+            const uint32_t a = dfk_lo + (uint32_t)pa.fs * (FIXB >> 4), bq = dsk_lo + (uint32_t)pa.ss * (PAIR >> 4);
+            const uint32_t d_col = tmem_base + (uint32_t)(sb * BN);
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
-          const uint32_t o = (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
-          if (ks == 0) umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 0u);
-          else umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 1u);
-        }
-      };
-      // second product of a block: dP from the second tiles of both pairs; then both are announced
-      auto issue_dp = [&](Pos& q) {
-        const uint32_t a = dfk_lo + (uint32_t)q.fs * (FIXB >> 4) + (TILE >> 4), bq = dsk_lo + (uint32_t)q.ss * (PAIR >> 4) + (TILE >> 4);
-        const uint32_t idesc = (q.it.stile(shp) == p.nq - 1) ? idesc_tail : idesc_full;
-        const uint32_t d_col = tmem_base + (uint32_t)C::DP_COL;
+            for (int ks = 0; ks < DH / 16; ++ks) {
+              const uint32_t o = (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
+              if (ks == 0) umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 0u);
+              else umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 1u);
+            }
+          }
+          // the dP buffer: free once the compute warps have read the previous block's dP
+          if (n >= 1 && !mbar_wait_bounded(p_ready(n - 1), (unsigned)((n - 1) >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
+          tc_fence_after();
+          {
+            const uint32_t a = dfk_lo + (uint32_t)pa.fs * (FIXB >> 4) + (TILE >> 4), bq = dsk_lo + (uint32_t)pa.ss * (PAIR >> 4) + (TILE >> 4);
+            const uint32_t d_col = tmem_base + (uint32_t)C::DP_COL;
 #pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
-          const uint32_t o = (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
-          if (ks == 0) umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 0u);
-          else umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 1u);
+            for (int ks = 0; ks < DH / 16; ++ks) {
+              const uint32_t o = (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
+              if (ks == 0) umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 0u);
+              else umma_bf16(d_col, desc(a + o, dfk_hi), desc(bq + o, dsk_hi), idesc, 1u);
+            }
+          }
+          umma_commit(sdp_full);                                       // this thread's S and dP of block n are complete
+          pos_next(pa);
         }
-        umma_commit(sdp_full);
-      };
-      // accumulating product: D (+)= A[tensor memory, packed bf16 at a_col0] * streamed tile `which` read MN-major
-      auto issue_acc = [&](const Pos& q, uint32_t d_col, uint32_t a_col0, int which, bool fresh) {
-        const uint32_t bq = dsm_lo + (uint32_t)q.ss * (PAIR >> 4) + (uint32_t)which * (TILE >> 4);
-        const int nk = (q.it.stile(shp) == p.nq - 1 ? nb_tail : BN) >> 4;          // 16-row steps of the streamed tile
+      } else {
+        // ---- accumulating products: D (+)= A[tensor memory, packed bf16 at a_col0] * streamed tile read MN-major ----
+        Pos pc;
+        pos_init(pc);
+        auto issue_acc = [&](const Pos& q, uint32_t d_col, uint32_t a_col0, int which, bool fresh) {
+          const uint32_t bq = dsm_lo + (uint32_t)q.ss * (PAIR >> 4) + (uint32_t)which * (TILE >> 4);
+          const int nk = (q.it.stile(shp) == p.nq - 1 ? nb_tail : BN) >> 4;          // 16-row steps of the streamed tile
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk) {
-          if (kk < nk) {
-            const uint32_t a_col = a_col0 + (uint32_t)((kk >> 1) * 32 + (kk & 1) * 8);   // slice kk/2, half kk%2
-            umma_bf16_ts(d_col, a_col, desc(bq + (uint32_t)(kk * 128), dsm_hi), idesc_acc, (kk > 0 || !fresh) ? 1u : 0u);
+          for (int kk = 0; kk < BN / 16; ++kk) {
+            if (kk < nk) {
+              const uint32_t a_col = a_col0 + (uint32_t)((kk >> 1) * 32 + (kk & 1) * 8);   // slice kk/2, half kk%2
+              umma_bf16_ts(d_col, a_col, desc(bq + (uint32_t)(kk * 128), dsm_hi), idesc_acc, (kk > 0 || !fresh) ? 1u : 0u);
+            }
           }
-        }
-      };
-      // prologue: scores and dP of block 0, scores of block 1 when there is a second score buffer
-      if (ps.it.valid(shp)) {
-        issue_scores(ps, 0);
-        if (ok) { issue_dp(pd); pos_next(ps); pos_next(pd); }
-        if (NSBUF == 2 && ok && ps.it.valid(shp)) { issue_scores(ps, 1); if (ok) pos_next(ps); }
-      }
-      int sb = 0, rph = 0;                      // score buffer and p_ready parity of the current block
-      while (pc.it.valid(shp) && ok) {
-        if (*abort_flag) { ok = false; break; }
-        if (!mbar_wait_bounded(p_ready, (unsigned)rph, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
-        const int k = pc.it.k;
-        if (pc.it.first()) {
-          // BW_DQ alternates between two accumulators: the one of item k was last read for item k - 2;
-          // BW_DKV uses both accumulators for every item: wait for item k - 1
-          const int prev = MODE == BW_DQ ? k - 2 : k - 1;
-          if (prev >= 0 && !mbar_wait_bounded(&acc_empty[prev & 1], (unsigned)(prev >> 1) & 1u, WAIT_NS)) {
-            fa_timeout(SITE_O_EMPTY); ok = false; break;
+        };
+        int sb = 0;                               // score buffer of the current block
+        for (int b = 0; pc.it.valid(shp) && ok; ++b) {
+          if (*abort_flag) { ok = false; break; }
+          if (!mbar_wait_bounded(p_ready(b), (unsigned)(b >> 1) & 1u, WAIT_NS)) { fa_timeout(SITE_P_FULL); ok = false; break; }
+          const int k = pc.it.k;
+          if (pc.it.first()) {
+            // BW_DQ alternates between two accumulators: the one of item k was last read for item k - 2;
+            // BW_DKV uses both accumulators for every item: wait for item k - 1
+            const int prev = MODE == BW_DQ ? k - 2 : k - 1;
+            if (prev >= 0 && !mbar_wait_bounded(&acc_empty[prev & 1], (unsigned)(prev >> 1) & 1u, WAIT_NS)) {
+              fa_timeout(SITE_O_EMPTY); ok = false; break;
+            }
           }
-        }
-        tc_fence_after();
-        const uint32_t s_col = tmem_base + (uint32_t)(sb * BN), dp_col = tmem_base + (uint32_t)C::DP_COL;
-        const uint32_t acc0 = tmem_base + (uint32_t)C::ACC_COL, acc1 = acc0 + DH;
-        const bool fresh = pc.it.first();
-        if (MODE == BW_DKV) {
-          // P^T and dS^T both sit in the block's score buffer, so the dP buffer is free: the next block's dP goes
-          // first and the compute warps start on it while the accumulating products of this block run
-          if (NSBUF == 2 && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }
-          issue_acc(pc, acc0, s_col + 16u, 0, fresh);                  // dK += dS^T Q_i
-          if (fresh && k >= 1 && !mbar_wait_bounded(&accv_empty[(k - 1) & 1], (unsigned)((k - 1) >> 1) & 1u, WAIT_NS)) {
-            fa_timeout(SITE_O_EMPTY); ok = false; break;
+          tc_fence_after();
+          const uint32_t s_col = tmem_base + (uint32_t)(sb * BN);
+          const uint32_t acc0 = tmem_base + (uint32_t)C::ACC_COL, acc1 = acc0 + DH;
+          const bool fresh = pc.it.first();
+          if (MODE == BW_DKV) {
+            issue_acc(pc, acc0, s_col + 16u, 0, fresh);                // dK += dS^T Q_i (dS^T sits beside P^T in the score buffer)
+            if (fresh && k >= 1 && !mbar_wait_bounded(&accv_empty[(k - 1) & 1], (unsigned)((k - 1) >> 1) & 1u, WAIT_NS)) {
+              fa_timeout(SITE_O_EMPTY); ok = false; break;
+            }
+            issue_acc(pc, acc1, s_col, 1, fresh);                      // dV += P^T dO_i
+          } else {
+            issue_acc(pc, (k & 1) ? acc1 : acc0, s_col, 0, fresh);     // dQ += dS K_j
           }
-          issue_acc(pc, acc1, s_col, 1, fresh);                        // dV += P^T dO_i
-        } else {
-          if (NSBUF == 2 && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }   // dS went over the scores: dP is free
-          issue_acc(pc, (k & 1) ? acc1 : acc0, s_col, 0, fresh);       // dQ += dS K_j
+          umma_commit(&s_free[sb]);                                    // the score buffer may take the scores of block b + NSBUF
+          umma_commit(&str_empty[pc.ss]);                              // the streamed pair has been read for the last time
+          if (pc.it.last()) {
+            umma_commit(&acc_full[k & 1]);
+            umma_commit(&fix_empty[pc.fs]);
+          }
+          pos_next(pc);
+          if (++sb == NSBUF) sb = 0;
         }
-        umma_commit(&str_empty[pc.ss]);                                // the streamed pair has been read for the last time
-        if (pc.it.last()) {
-          umma_commit(&acc_full[k & 1]);
-          umma_commit(&fix_empty[pc.fs]);
-        }
-        pos_next(pc);
-        // this block's score buffer is free once the accumulation above has read it: scores of the block after next
-        // (or, with one buffer, scores and dP of the next block)
-        if (ps.it.valid(shp)) { issue_scores(ps, sb); if (ok) pos_next(ps); }
-        if (NSBUF == 1 && ok && pd.it.valid(shp)) { issue_dp(pd); pos_next(pd); }
-        if (++sb == NSBUF) sb = 0;
-        rph ^= 1;
       }
       if (!ok) *abort_flag = 1;
     }
@@ -1187,7 +1204,7 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0 && !dead) mbar_arrive(p_ready);
+      if (lane == 0 && !dead) mbar_arrive(p_ready(b));
       if (have_next) stat[((b + 1) & 1) * 2 * BM + ct] = next_stat * (ct < BM ? LOG2E : 1.f);
     }
   }
