@@ -198,28 +198,33 @@ rmsnorm_bwd_kernel(const DY* __restrict__ dy, const float* __restrict__ x, const
   }
 }
 
-// The same for d = 128 NV with the whole row in registers: every load of a row (x, dy, the incoming residual
+// The same for d = 128 NV WPR with the whole row in registers: every load of a row (x, dy, the incoming residual
 // gradient) is issued before the first use, nothing is read twice, gamma and the dgamma partial sums of this lane's
 // columns stay in registers for the life of the CTA.  Fewer, fatter warps: the kernel is HBM-bound and needs bytes
-// in flight, not occupancy.
-template <typename T, typename DY, int NV>
+// in flight, not occupancy.  WPR warps share a row (WPR = 2 for d = 2048: a warp holds 1024 columns): they add their
+// parts of the row's dot product through shared memory and a named barrier of their own.
+template <typename T, typename DY, int NV, int WPR>
 __global__ void __launch_bounds__(256)
 rmsnorm_bwd_rows_kernel(const DY* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ rstd,
                         const T* __restrict__ gamma, const float* dx_in, float* dx_out, T* __restrict__ dx_out_t,
                         float* __restrict__ part, long long rows, int map_S, int map_P) {
-  constexpr int d = NV * 128;
-  extern __shared__ float red[];                         // [8 warps][d]
+  constexpr int d = NV * 128 * WPR, RPB = 8 / WPR;        // row width; rows a CTA works on at a time
+  extern __shared__ float red[];                         // [8 warps][NV * 128]
+  __shared__ float dots[2][8];                           // partial dot products, double-buffered over a warp group's rows
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = warp / WPR, part_i = warp - grp * WPR;  // row slot of this warp, and which part of the row it holds
+  const int col0 = part_i * NV * 128 + lane * 4;
   float gm[NV][4], acc[NV][4];
 #pragma unroll
   for (int k = 0; k < NV; ++k) {
-    load4<T>(gamma + k * 128 + lane * 4, gm[k]);
+    load4<T>(gamma + col0 + k * 128, gm[k]);
     acc[k][0] = acc[k][1] = acc[k][2] = acc[k][3] = 0.f;
   }
-  for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
+  int it = 0;
+  for (long long r = (long long)blockIdx.x * RPB + grp; r < rows; r += (long long)gridDim.x * RPB, ++it) {
     const long long xr_i = map_row(r, map_S, map_P);
-    const float* xr = x + xr_i * d + lane * 4;
-    const DY* dyr = dy + r * d + lane * 4;
+    const float* xr = x + xr_i * d + col0;
+    const DY* dyr = dy + r * d + col0;
     float4 xv[NV], pv[NV];
     float gy[NV][4];
 #pragma unroll
@@ -229,7 +234,7 @@ rmsnorm_bwd_rows_kernel(const DY* __restrict__ dy, const float* __restrict__ x, 
     }
     if (dx_in) {
 #pragma unroll
-      for (int k = 0; k < NV; ++k) pv[k] = *reinterpret_cast<const float4*>(dx_in + xr_i * d + lane * 4 + k * 128);
+      for (int k = 0; k < NV; ++k) pv[k] = *reinterpret_cast<const float4*>(dx_in + xr_i * d + col0 + k * 128);
     } else {
 #pragma unroll
       for (int k = 0; k < NV; ++k) pv[k] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -241,6 +246,14 @@ rmsnorm_bwd_rows_kernel(const DY* __restrict__ dy, const float* __restrict__ x, 
       dot += gy[k][0] * gm[k][0] * xv[k].x + gy[k][1] * gm[k][1] * xv[k].y + gy[k][2] * gm[k][2] * xv[k].z +
              gy[k][3] * gm[k][3] * xv[k].w;
     dot = warp_sum(dot);
+    if constexpr (WPR > 1) {
+      // the group's warps run the same trip count (same r), so the barrier is reached by all of them
+      if (lane == 0) dots[it & 1][warp] = dot;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(WPR * 32) : "memory");
+      dot = 0.f;
+#pragma unroll
+      for (int w = 0; w < WPR; ++w) dot += dots[it & 1][grp * WPR + w];
+    }
     const float coef = dot * rs * rs * rs / (float)d;    // mean(dn * n) * rstd, with n = x * rstd
 #pragma unroll
     for (int k = 0; k < NV; ++k) {
@@ -252,18 +265,19 @@ rmsnorm_bwd_rows_kernel(const DY* __restrict__ dy, const float* __restrict__ x, 
         o[e] = rs * gy[k][e] * gm[k][e] - coef * xa[e] + pa[e];
         acc[k][e] += gy[k][e] * xa[e] * rs;
       }
-      *reinterpret_cast<float4*>(dx_out + xr_i * d + lane * 4 + k * 128) = make_float4(o[0], o[1], o[2], o[3]);
-      store4<T>(dx_out_t + xr_i * d + lane * 4 + k * 128, o[0], o[1], o[2], o[3]);
+      *reinterpret_cast<float4*>(dx_out + xr_i * d + col0 + k * 128) = make_float4(o[0], o[1], o[2], o[3]);
+      store4<T>(dx_out_t + xr_i * d + col0 + k * 128, o[0], o[1], o[2], o[3]);
     }
   }
 #pragma unroll
   for (int k = 0; k < NV; ++k)
-    *reinterpret_cast<float4*>(red + (size_t)warp * d + k * 128 + lane * 4) = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+    *reinterpret_cast<float4*>(red + (size_t)warp * (NV * 128) + k * 128 + lane * 4) = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
   __syncthreads();
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const int pi = c / (NV * 128), cc = c - pi * (NV * 128);   // which part of the row, column inside it
     float s = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) s += red[(size_t)w * d + c];
+    for (int g = 0; g < RPB; ++g) s += red[(size_t)(g * WPR + pi) * (NV * 128) + cc];
     part[(size_t)blockIdx.x * d + c] = s;
   }
 }
@@ -933,7 +947,8 @@ static int run(const grpo_model* m, const grpo_lora* lo, const grpo_packed* pk, 
     {
       PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
       PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_kernel<T, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
-      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_rows_kernel<T, T, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
+      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_rows_kernel<T, T, 8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
+      PCM_CUDA_TRY(cudaFuncSetAttribute(rmsnorm_bwd_rows_kernel<T, T, 8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)nb_smem));
     }
     // dy_is_t: the incoming gradient is stored in the activation type (the per-layer dh), else in fp32.
     // dx_out = dx_in + (gradient through the norm), in fp32 and in T.
@@ -942,8 +957,11 @@ static int run(const grpo_model* m, const grpo_lora* lo, const grpo_packed* pk, 
       const int blocks = (int)(rows / 8 + 1 < NORM_BWD_BLOCKS ? rows / 8 + 1 : NORM_BWD_BLOCKS);
       prof_begin(PC_NORM, s);
       if (dy_is_t && d == 1024)
-        rmsnorm_bwd_rows_kernel<T, T, 8><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, dx_out, dx_out_t,
-                                                                       w.norm_part, rows, 0, 0);
+        rmsnorm_bwd_rows_kernel<T, T, 8, 1><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, dx_out, dx_out_t,
+                                                                          w.norm_part, rows, 0, 0);
+      else if (dy_is_t && d == 2048)
+        rmsnorm_bwd_rows_kernel<T, T, 8, 2><<<blocks, 256, 8 * 1024 * sizeof(float), s>>>((const T*)dy, x, rstd, gamma, dx_in, dx_out,
+                                                                                          dx_out_t, w.norm_part, rows, 0, 0);
       else if (dy_is_t)
         rmsnorm_bwd_kernel<T, T><<<blocks, 256, nb_smem, s>>>((const T*)dy, x, rstd, gamma, dx_in, dx_out, dx_out_t, w.norm_part,
                                                                rows, d, 0, 0);
