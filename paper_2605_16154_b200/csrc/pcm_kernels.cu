@@ -52,15 +52,18 @@ unsigned* ctx_status(pcm_ctx* c) { return c->status; }
 // Eq. 5, per group: integer token sums per (phase, outcome), then C_{c,g}
 // ------------------------------------------------------------------------------------------------
 // One CTA per group, a warp per trajectory.  The trajectory's tokens are staged in shared memory by asynchronous
-// copies (slabs of 32 chunks, two in flight per warp, about 170 KB per SM over all resident warps), so memory
-// parallelism does not depend on the phase structure.  The warp then finds the runs of equal
-// phase label in the slab (labels are read coalesced into registers while the copies fly, run starts come out of
-// a ballot, start positions and labels go through a small shared list) and sums four runs at a time: a chunk is
-// seven 8-byte vectors, lane = 7 * slot + vec owns vector `vec` (action dimensions 8 vec .. 8 vec + 7) of the
-// run its slot took.  Bytes are accumulated as packed 16-bit lanes (a run inside a slab has at most 32 chunks:
-// 32 * 255 < 2^16) and flushed with eight 32-bit shared-memory adds per lane: the per-run cost is shared by four
-// runs.  Integer sums are exact, so any order gives the same result.
-constexpr int SC_SLAB = 32;                              // chunks per staged slab: one label per lane
+// copies (slabs of 32 chunks, two in flight per warp, about 170 KB per SM over all resident warps).  The sums
+// per (phase, dimension) of a slab are an integer contraction over its chunks,
+//     Sum[dim][phase] += tok^T[dim][chunk] * onehot[chunk][phase],
+// and run on the tensor cores as mma.sync m16n8k32 (u8 x u8 -> s32): per slab a lane reads eight 8-byte vectors,
+// transposes bytes in registers (the data has dimensions contiguous, the contraction index must be), builds the
+// one-hot operand from the slab's labels with byte compares, and issues 4 x NT MMAs (NT = ceil(n_phases / 8)).
+// Dimension 56 of the padded 64 is the constant 1, so the chunk counts come out of the same products.  Labels may
+// come in any order: nothing depends on runs.  Accumulators stay in registers for the whole trajectory and are
+// flushed once, with 32-bit shared-memory adds.  Integer sums are exact, so any order gives the same result.
+// (A byte costs one ALU operation per lane in a packed-add scheme, which left the kernel instruction-bound at less
+// than half of the copy bandwidth; the contraction costs a fraction of that.)
+constexpr int SC_SLAB = 32;                              // chunks per staged slab = the contraction length of one MMA
 constexpr int SC_SLAB_BYTES = SC_SLAB * ACT;             // 1792
 constexpr int SC_WARPS = 8;
 
@@ -74,12 +77,25 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-__device__ __forceinline__ void score_add8(const uint2 w, unsigned& a0, unsigned& a1, unsigned& a2, unsigned& a3) {
-  a0 += w.x & 0x00FF00FFu; a1 += __byte_perm(w.x, 0, 0x4341);        // bytes {0, 2} and {1, 3} as 16-bit lanes
-  a2 += w.y & 0x00FF00FFu; a3 += __byte_perm(w.y, 0, 0x4341);
+// D (16 x 8, s32) += A (16 x 32, u8, row) * B (32 x 8, u8, col).  Lane = 4 g + t: A registers hold rows g, g + 8 and
+// contraction indices 4 t .. 4 t + 3 (a0, a1) and 16 + 4 t .. (a2, a3), lowest byte first; B registers hold column g
+// and the same contraction indices; D registers hold rows g (c0, c1) and g + 8 (c2, c3), columns 2 t and 2 t + 1.
+__device__ __forceinline__ void imma_16x8x32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// r[m] = byte m of w0, w1, w2, w3 (lowest byte first): a 4 x 4 byte transpose
+__device__ __forceinline__ void transpose4(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint32_t (&r)[4]) {
+  const uint32_t t0 = __byte_perm(w0, w1, 0x5140), t1 = __byte_perm(w2, w3, 0x5140);
+  const uint32_t t2 = __byte_perm(w0, w1, 0x7362), t3 = __byte_perm(w2, w3, 0x7362);
+  r[0] = __byte_perm(t0, t1, 0x5410); r[1] = __byte_perm(t0, t1, 0x7632);
+  r[2] = __byte_perm(t2, t3, 0x5410); r[3] = __byte_perm(t2, t3, 0x7632);
 }
 
-__global__ void __launch_bounds__(SC_WARPS * 32)
+template <int NT>
+__global__ void __launch_bounds__(SC_WARPS * 32, NT <= 2 ? 4 : 2)
 score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restrict__ tok,
                     const uint8_t* __restrict__ phase, const uint8_t* __restrict__ reward, int G,
                     int n_phases, double* __restrict__ c_group, uint8_t* __restrict__ valid_group,
@@ -89,17 +105,15 @@ score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restr
   unsigned* sums = sm;                                   // [n_phases][2][56]
   unsigned* cnt = sm + n_phases * 2 * ACT;               // [n_phases][2]
   uint8_t* stage = reinterpret_cast<uint8_t*>(sm + n_cnt);   // [SC_WARPS][2][SC_SLAB_BYTES]
-  __shared__ unsigned char run_pos[SC_WARPS][SC_SLAB + 4];   // slab-local start of every run, then the slab's length
-  __shared__ unsigned char run_lab[SC_WARPS][SC_SLAB + 4];   // its phase label
+  __shared__ __align__(16) unsigned char lab_s[SC_WARPS][SC_SLAB];   // the current slab's labels, 0x40 = no chunk / bad label
   const int g = blockIdx.x;
   for (int i = threadIdx.x; i < n_phases * 2 * (ACT + 1); i += blockDim.x) sm[i] = 0;
   __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int slot = lane / 7, vec = lane - slot * 7;      // lanes 28..31 (slot 4) idle in the sums
+  const int gid = lane >> 2, tig = lane & 3;             // fragment coordinates: rows gid, gid + 8; contraction indices 4 tig ..
   uint8_t* mybuf = stage + (size_t)warp * 2 * SC_SLAB_BYTES;
-  unsigned char* rp = run_pos[warp];
-  unsigned char* rl = run_lab[warp];
+  unsigned char* lab = lab_s[warp];
 
   for (int i = g * G + warp; i < (g + 1) * G; i += SC_WARPS) {
     const int o = reward[i] ? 1 : 0;
@@ -123,56 +137,77 @@ score_groups_kernel(const int32_t* __restrict__ traj_off, const uint8_t* __restr
     };
     if (n_slab > 0) issue(0);
     if (n_slab > 1) issue(1);
+    // acc[j][n]: rows = dimensions 8 gid + 2 j (c0, c1) and 8 gid + 2 j + 1 (c2, c3); columns = phases 8 n + 2 tig, + 1
+    int acc[4][NT][4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int n = 0; n < NT; ++n) acc[j][n][0] = acc[j][n][1] = acc[j][n][2] = acc[j][n][3] = 0;
     for (int k = 0; k < n_slab; ++k) {
       const int c0 = a + k * SC_SLAB, nc = min(SC_SLAB, b - c0);
       // this slab's labels, one per lane, requested before the wait so that they overlap the copies
-      const int l0 = lane < nc ? (int)__ldg(phase + c0 + lane) : -2;
-      // runs: a chunk starts one when its label differs from its predecessor's; the slab's first chunk always does
-      int p0 = __shfl_up_sync(0xffffffffu, l0, 1);
-      if (lane == 0) p0 = -1;
-      const bool s0 = lane < nc && l0 != p0;
-      const unsigned m0 = __ballot_sync(0xffffffffu, s0);
-      const int n_runs = __popc(m0);
-      __syncwarp();                                      // the previous slab's list has been read by every lane
-      if (s0) { const int r = __popc(m0 & ((1u << lane) - 1u)); rp[r] = (unsigned char)lane; rl[r] = (unsigned char)l0; }
-      if (lane == 0) rp[n_runs] = (unsigned char)nc;
+      int l0 = lane < nc ? (int)__ldg(phase + c0 + lane) : 0x40;
+      const bool bad = lane < nc && l0 >= n_phases;        // reported; the chunk matches no phase and drops out
+      if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, STATUS_BAD_PHASE);
+      if (bad) l0 = 0x40;
+      __syncwarp();                                      // the previous slab's labels have been read by every lane
+      lab[lane] = (unsigned char)l0;
       if (k + 1 < n_slab) cp_async_wait<1>(); else cp_async_wait<0>();
       __syncwarp();
-      const uint2* base = reinterpret_cast<const uint2*>(mybuf + (k & 1) * SC_SLAB_BYTES) + vec;
-      for (int r0 = 0; r0 < n_runs; r0 += 4) {           // four runs per round, one per slot
-        const int r = r0 + slot;
-        const bool have = slot < 4 && r < n_runs;
-        int c = have ? rp[r] : 0;
-        int e = have ? rp[r + 1] : 0;
-        const int ph = have ? rl[r] : 0;
-        if (have && ph >= n_phases) {                    // a bad label: reported, its chunks are skipped
-          if (vec == 0) atomicOr(status, STATUS_BAD_PHASE);
-          e = c;
+      const uint8_t* buf = mybuf + (k & 1) * SC_SLAB_BYTES;
+      // A operand: T[h][m] = dimension 8 gid + m of chunks 16 h + 4 tig .. + 3.  The group gid = 7 holds the padding
+      // dimensions 56 .. 63: dimension 56 is the constant 1 (it counts chunks), the others are 0.
+      uint32_t T[2][8];
+      if (gid < 7) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint2 w[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) w[q] = *reinterpret_cast<const uint2*>(buf + (16 * h + 4 * tig + q) * ACT + 8 * gid);
+          uint32_t lo[4], hi[4];
+          transpose4(w[0].x, w[1].x, w[2].x, w[3].x, lo);
+          transpose4(w[0].y, w[1].y, w[2].y, w[3].y, hi);
+#pragma unroll
+          for (int m = 0; m < 4; ++m) { T[h][m] = lo[m]; T[h][4 + m] = hi[m]; }
         }
-        const int len = e - c;
-        unsigned a0 = 0, a1 = 0, a2 = 0, a3 = 0;
-        while (__any_sync(0xffffffffu, c < e)) {
-          if (c + 1 < e) {
-            const uint2 w0 = base[c * 7], w1 = base[(c + 1) * 7];
-            score_add8(w0, a0, a1, a2, a3);
-            score_add8(w1, a0, a1, a2, a3);
-          } else if (c < e) {
-            score_add8(base[c * 7], a0, a1, a2, a3);
-          }
-          c += 2;
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          T[h][0] = 0x01010101u;
+#pragma unroll
+          for (int m = 1; m < 8; ++m) T[h][m] = 0u;
         }
-        if (len > 0) {
-          unsigned* sp = sums + (ph * 2 + o) * ACT + vec * 8;   // a0 = dims {0, 2}, a1 = {1, 3}, a2 = {4, 6}, a3 = {5, 7}
-          atomicAdd(sp + 0, a0 & 0xFFFFu); atomicAdd(sp + 2, a0 >> 16);
-          atomicAdd(sp + 1, a1 & 0xFFFFu); atomicAdd(sp + 3, a1 >> 16);
-          atomicAdd(sp + 4, a2 & 0xFFFFu); atomicAdd(sp + 6, a2 >> 16);
-          atomicAdd(sp + 5, a3 & 0xFFFFu); atomicAdd(sp + 7, a3 >> 16);
-          if (vec == 0) atomicAdd(cnt + ph * 2 + o, (unsigned)len);
-        }
+      }
+      // B operand: one-hot of the labels against phase 8 n + gid
+      const uint32_t lab_lo = *reinterpret_cast<const uint32_t*>(lab + 4 * tig);
+      const uint32_t lab_hi = *reinterpret_cast<const uint32_t*>(lab + 16 + 4 * tig);
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        // byte-wise "label == phase": labels are below 0x60 (a phase, or the 0x40 of a chunk that takes no part), so
+        // x = label ^ phase is below 0x80 and x + 0x7f sets bit 7 exactly where x != 0, without carrying into the next byte
+        const uint32_t rep = (uint32_t)(8 * n + gid) * 0x01010101u;
+        const uint32_t b0 = (~((lab_lo ^ rep) + 0x7f7f7f7fu) >> 7) & 0x01010101u;
+        const uint32_t b1 = (~((lab_hi ^ rep) + 0x7f7f7f7fu) >> 7) & 0x01010101u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) imma_16x8x32(acc[j][n], T[0][2 * j], T[0][2 * j + 1], T[1][2 * j], T[1][2 * j + 1], b0, b1);
       }
       __syncwarp();                                      // every lane is done with the buffer before it is refilled
       if (k + 2 < n_slab) issue(k + 2);
     }
+    // flush the trajectory's sums: this lane holds dimensions 8 gid + 2 j, + 1 for phases 8 n + 2 tig, + 1
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int n = 0; n < NT; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int dim = 8 * gid + 2 * j + (e >> 1), ph = 8 * n + 2 * tig + (e & 1);
+          const int v = acc[j][n][e];
+          if (ph < n_phases && v != 0) {
+            if (dim < ACT) atomicAdd(sums + (ph * 2 + o) * ACT + dim, (unsigned)v);
+            else if (dim == ACT) atomicAdd(cnt + ph * 2 + o, (unsigned)v);
+          }
+        }
   }
   __syncthreads();
 
@@ -575,8 +610,9 @@ using namespace pcm;
 
 // score_groups_kernel with its shared memory: the counters plus two 32-chunk slabs per warp (29 KB, with 32 phases
 // 43 KB; the attribute is set once per device so that any count stays legal).  Allocates nothing.
-static int launch_score_groups(const pcm_batch* b, int G, int n_phases, int n_groups, double* c_group, uint8_t* valid_group,
-                               unsigned* status, cudaStream_t s) {
+template <int NT>
+static int launch_score_groups_nt(const pcm_batch* b, int G, int n_phases, int n_groups, double* c_group,
+                                  uint8_t* valid_group, unsigned* status, cudaStream_t s) {
   const size_t n_cnt = ((size_t)n_phases * 2 * (ACT + 1) + 3) & ~(size_t)3;
   const size_t smem = n_cnt * sizeof(unsigned) + (size_t)SC_WARPS * 2 * SC_SLAB_BYTES;
   static unsigned long long attr_devices = 0;
@@ -584,14 +620,24 @@ static int launch_score_groups(const pcm_batch* b, int G, int n_phases, int n_gr
   {
     std::lock_guard<std::mutex> lk(mu);
     if (attr_needed(&attr_devices))
-      PCM_CUDA_TRY(cudaFuncSetAttribute(score_groups_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      PCM_CUDA_TRY(cudaFuncSetAttribute(score_groups_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(((size_t)PCM_MAX_PHASES * 2 * (ACT + 1) + 3) * sizeof(unsigned) +
                                               (size_t)SC_WARPS * 2 * SC_SLAB_BYTES)));
   }
-  score_groups_kernel<<<n_groups, SC_WARPS * 32, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, G, n_phases, c_group,
-                                                          valid_group, status);
+  score_groups_kernel<NT><<<n_groups, SC_WARPS * 32, smem, s>>>(b->traj_off, b->tok, b->phase, b->reward, G, n_phases,
+                                                              c_group, valid_group, status);
   PCM_LAUNCH_CHECK();
   return PCM_OK;
+}
+
+static int launch_score_groups(const pcm_batch* b, int G, int n_phases, int n_groups, double* c_group, uint8_t* valid_group,
+                               unsigned* status, cudaStream_t s) {
+  switch ((n_phases + 7) / 8) {                          // phase columns come in MMA tiles of 8
+    case 1: return launch_score_groups_nt<1>(b, G, n_phases, n_groups, c_group, valid_group, status, s);
+    case 2: return launch_score_groups_nt<2>(b, G, n_phases, n_groups, c_group, valid_group, status, s);
+    case 3: return launch_score_groups_nt<3>(b, G, n_phases, n_groups, c_group, valid_group, status, s);
+    default: return launch_score_groups_nt<4>(b, G, n_phases, n_groups, c_group, valid_group, status, s);
+  }
 }
 
 extern "C" {
