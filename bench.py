@@ -125,9 +125,10 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # CPU oracle timing (baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample_step(w, rb, weights, seed, n_sample, lora_rank=0):
+def oracle_sample_step(w, rb, weights, seed, n_sample, lora_rank=0, adamw=False):
     """One oracle pass: PCM control plane on the whole batch, actor forward + backward on the first
-    n_sample kept chunks.  Returns (seconds for the control plane, seconds for the actor sample, n_kept)."""
+    n_sample kept chunks, then (adamw) one optimizer step on what was trained.  Returns (seconds for the
+    control plane, seconds for the actor sample, n_kept, seconds for the optimizer step)."""
     from oracle import actor_oracle as ao
     from oracle import pcm_oracle as po
     from paper_2605_16154_b200 import synth
@@ -145,9 +146,19 @@ def oracle_sample_step(w, rb, weights, seed, n_sample, lora_rank=0):
     t1 = time.perf_counter()
     X, tgt, lpo, adv_c, _ = po.pack_chunks(lambda c: obs[c], rb["tok"], lpo_all, adv, rb["traj_off"], sample, weights["e_act"])
     lo = synth.make_lora(w, lora_rank, float(lora_rank)) if lora_rank else None
-    ao.fwd_bwd(weights, X, tgt, lpo, adv_c, w.H, w.P, w.eps_low, w.eps_high, 1.0 / (ACT * len(kept)), lora=lo)
+    _, _, grads, _ = ao.fwd_bwd(weights, X, tgt, lpo, adv_c, w.H, w.P, w.eps_low, w.eps_high, 1.0 / (ACT * len(kept)), lora=lo)
     t_actor = time.perf_counter() - t1
-    return t_pcm, t_actor, len(kept)
+    t_opt = 0.0
+    if adamw:
+        from oracle import optim_oracle as oo
+        source = dict(weights, **{k: v for k, v in (lo or {}).items() if k not in ("rank", "alpha")})
+        params = {k: np.asarray(source[k], dtype=np.float64) for k, g in grads.items() if g is not None}
+        m = {k: np.zeros_like(v) for k, v in params.items()}
+        v = {k: np.zeros_like(v) for k, v in params.items()}
+        t2 = time.perf_counter()
+        oo.adamw_step(params, {k: grads[k] for k in params}, m, v, 1)
+        t_opt = time.perf_counter() - t2
+    return t_pcm, t_actor, len(kept), t_opt
 
 
 def blas_threads() -> int:
@@ -158,12 +169,13 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
-def config_of(w, n_kept, total, mb, iterations=None, lora_rank=0, dp=False, world=1):
+def config_of(w, n_kept, total, mb, iterations=None, lora_rank=0, dp=False, world=1, adamw=False):
     """The `config` object both arms print."""
     c = {"workload": w.name, "trainable": f"LoRA rank {lora_rank}, alpha {lora_rank}, base frozen" if lora_rank else "all weights", "kept_chunks_per_step": int(n_kept), "chunks_per_step": int(total),
          "tokens_per_step": int(n_kept) * w.S, "mb_chunks": int(mb), "l2": "inputs_larger_than_l2",
          "multi_gpu": (f"data parallel over {world} ranks: one batch, kept chunks dealt out by trajectory, one fp32 gradient "
                        "all-reduce per step") if dp else "independent replicas, no collective"}
+    c["optimizer"] = "gradient clipping at 2.0 + AdamW after every update (App. E)" if adamw else "none (gradients only)"
     if iterations is not None:
         c["iterations"] = int(iterations)
         c["resampled"] = "rollouts redrawn every iteration from seeds 0..iterations-1, keep-probability state carried"
@@ -191,19 +203,20 @@ def run_reference(args):
     n_sample = 1
     est = []
     for it in range(args.warmup + args.steps):
-        t_pcm, t_actor, n_kept = oracle_sample_step(w, rb, weights, w.seed, n_sample, args.lora)
+        t_pcm, t_actor, n_kept, t_opt = oracle_sample_step(w, rb, weights, w.seed, n_sample, args.lora, args.adamw)
         if it >= args.warmup:
-            est.append(t_pcm + t_actor * n_kept / n_sample)
+            est.append(t_pcm + t_actor * n_kept / n_sample + t_opt)
     ms = 1e3 * sum(est) / len(est)
     value = n_kept / (ms / 1e3)
     total = int(rb["traj_off"][-1])
     sample = (f"per step: control plane on the full batch + actor fwd/bwd on {n_sample} of {n_kept} kept chunks, "
-              f"scaled by {n_kept}/{n_sample} (chunks are independent sequences); ms_per_step is that estimate")
+              f"scaled by {n_kept}/{n_sample} (chunks are independent sequences)"
+              + (", + one optimizer step" if args.adamw else "") + "; ms_per_step is that estimate")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
             "config": config_of(w, n_kept, total, default_mb(args, n_kept), launch_steps_online(args) if online else None,
-                                args.lora),
+                                args.lora, adamw=args.adamw),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -216,7 +229,7 @@ def run_reference(args):
 class Harness:
     """Device state shared by the timed legs: model, workspace, preallocated outputs."""
 
-    def __init__(self, B, PL, synth, w, weights, n_kept_max, mb, lora_rank=0):
+    def __init__(self, B, PL, synth, w, weights, n_kept_max, mb, lora_rank=0, adamw=False):
         import torch
         self.B, self.w, self.mb = B, w, mb
         self.model = PL.upload_model(w, weights)
@@ -226,6 +239,9 @@ class Harness:
         self.ws = torch.empty(B.grpo_workspace_bytes(self.model, mb, 0, self.lora) + 256, dtype=torch.uint8, device="cuda")
         if self.lora is not None:
             self.lora.alloc_grads()
+        self.opt = None
+        if adamw:                                    # App. E: lr 1e-5, betas (0.9, 0.999), no decay, clip at 2.0
+            self.opt = B.LoraAdamW(self.model, self.lora) if self.lora is not None else B.AdamW(self.model)
         self.dp, self.loss_scale, self.dist_util = None, 0.0, None      # set by data_parallel()
         self.loss = torch.zeros(1, dtype=torch.float32, device="cuda")
         self.outputs(n_kept_max, w.n_traj, w.budget)
@@ -263,6 +279,8 @@ class Harness:
             if self.lora is not None:
                 self.dist_util.allreduce_sum(self.model.flat_grads)
             self.dist_util.allreduce_sum(self.loss)
+        if self.opt is not None:
+            self.opt.step()
 
     def step(self, ctx, bt, it):
         adv, kept_idx, kept_off, _ = self.select(ctx, bt, it)
@@ -382,7 +400,7 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
         h_obs[c0:c1] = torch.randn((c1 - c0, w.P, w.d), generator=gen, dtype=torch.float32).to(td)
     h = {k: torch.from_numpy(np.ascontiguousarray(v)).pin_memory() for k, v in rb.items()}
 
-    hs = Harness(B, PL, synth, w, weights, n_kept, mb, args.lora)
+    hs = Harness(B, PL, synth, w, weights, n_kept, mb, args.lora, args.adamw)
     if args.dp:
         hs.data_parallel(dist_util, rank, world, n_kept_global)
     model = hs.model
@@ -481,7 +499,7 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "strong" if args.dp else "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": config_of(w, n_kept_global if args.dp else n_kept, total, mb, None, args.lora, args.dp, world),
+            "config": config_of(w, n_kept_global if args.dp else n_kept, total, mb, None, args.lora, args.dp, world, args.adamw),
             "roofline": roofline_of(prof, peaks, args.steps, flops_per_kept_chunk(w, args.lora) * n_kept, ms_step, traffic),
             "kernel_classes": class_table(prof, args.steps),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -500,11 +518,12 @@ def run_fixed(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_
 
 
 def cpu_baseline_leg(args, w, rb, weights, seed):
-    t_pcm, t_actor, nk = oracle_sample_step(w, rb, weights, seed, args.cpu_sample, args.lora)
-    est = t_pcm + t_actor * nk / args.cpu_sample
+    t_pcm, t_actor, nk, t_opt = oracle_sample_step(w, rb, weights, seed, args.cpu_sample, args.lora, args.adamw)
+    est = t_pcm + t_actor * nk / args.cpu_sample + t_opt
     return {"value": nk / est, "unit": UNIT, "cores": blas_threads(), "kind": "oracle (fp64 numpy, BLAS threads = cores)",
             "sample": (f"control plane on the full batch ({t_pcm:.2f} s) + actor fwd/bwd on {args.cpu_sample} of "
-                       f"{nk} kept chunks ({t_actor:.2f} s), scaled by {nk}/{args.cpu_sample}")}
+                       f"{nk} kept chunks ({t_actor:.2f} s), scaled by {nk}/{args.cpu_sample}"
+                       + (f" + one optimizer step ({t_opt:.2f} s)" if args.adamw else ""))}
 
 
 def run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local_rank):
@@ -541,7 +560,7 @@ def run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local
         db = {k: v.cuda() for k, v in hb.items()}
         dev_b.append((db, B.make_batch(db["traj_off"], db["tok"], db["phase"], db["reward"], max_len, d_obs, db["lpo"])))
 
-    hs = Harness(B, PL, synth, w, weights, n_kept_max, mb, args.lora)
+    hs = Harness(B, PL, synth, w, weights, n_kept_max, mb, args.lora, args.adamw)
     barrier, timed = make_timers(torch, dist, dist_util, world)
     # staging buffers of the end-to-end leg (sized for the largest iteration)
     stage = {"traj_off": torch.empty(w.n_traj + 1, dtype=torch.int32, device="cuda"),
@@ -637,7 +656,7 @@ def run_online(args, torch, dist, B, dist_util, PL, synth, w, rank, world, local
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_iter,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(w, n_kept_total / n_iter, sum(totals) / n_iter, mb, n_iter, args.lora),
+            "config": config_of(w, n_kept_total / n_iter, sum(totals) / n_iter, mb, n_iter, args.lora, adamw=args.adamw),
             "online": {"ms_mean": statistics.mean(per_it), "ms_min": min(per_it), "ms_max": max(per_it),
                        "kept_chunks_min": min(kept_per_it), "kept_chunks_max": max(kept_per_it),
                        "chunks_min": min(totals), "chunks_max": max(totals),
@@ -673,6 +692,8 @@ def main():
                     help="data parallel instead of replicas: the ranks share one batch and all-reduce the gradients")
     ap.add_argument("--lora", type=int, default=0, metavar="RANK",
                     help="fine-tune low-rank adapters of this rank (alpha = rank) with the base weights frozen")
+    ap.add_argument("--adamw", action="store_true",
+                    help="follow every actor update with the optimizer step (clip + AdamW), inside the timed region")
     args = ap.parse_args()
     from paper_2605_16154_b200 import launch
     if args.impl == "cuda" and launch.needs_relaunch(args.gpus, os.environ):

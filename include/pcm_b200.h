@@ -351,6 +351,19 @@ int grpo_adamw_step(const grpo_model_cfg* cfg, const grpo_adamw_cfg* opt, int64_
                     grpo_grads* master, const grpo_grads* grads, grpo_grads* m, grpo_grads* v, float* grad_norm,
                     void* scratch, size_t scratch_bytes, pcm_stream stream);
 
+/* The same step for LoRA fine-tuning (App. E: the adapters are what is trained), after grpo_actor_fwd_bwd_lora.
+ * The eight adapter tensors of `lora` (cfg.dtype, device, WRITTEN by this call although the struct types them
+ * const) receive the rounded fp32 masters lora_master; lora_grads / lora_m / lora_v have the same shapes.
+ * The norm gains, head and action embedding, for which grpo_actor_fwd_bwd_lora also returns gradients, are
+ * trained along when model / master / grads / m / v are given (their g1, g2, gf, w_h, e_act; the four projection
+ * members are ignored), and stay frozen when all five are NULL (some but not all NULL: PCM_ERR_ARG).  One global
+ * norm and one clip coefficient over everything that is trained.  Arguments otherwise as grpo_adamw_step. */
+int grpo_adamw_step_lora(const grpo_model_cfg* cfg, const grpo_adamw_cfg* opt, int64_t step, grpo_lora* lora,
+                         grpo_lora_grads* lora_master, const grpo_lora_grads* lora_grads, grpo_lora_grads* lora_m,
+                         grpo_lora_grads* lora_v, grpo_model* model, grpo_grads* master, const grpo_grads* grads,
+                         grpo_grads* m, grpo_grads* v, float* grad_norm, void* scratch, size_t scratch_bytes,
+                         pcm_stream stream);
+
 /* ---- diagnostic entry points (per-kernel tests and measurements; not part of Algorithm 1) -------
  * grpo_gemm: C[m][n] = sum_k A(m,k) B(n,k) (+ R[m][n]) with the GEMM kernels the actor update uses.
  * a_kmajor != 0: A is stored [M][K] with row stride lda, else [K][M]; likewise B ([N][K] / [K][N]).

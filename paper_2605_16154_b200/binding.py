@@ -138,6 +138,12 @@ _lib.grpo_adamw_step.argtypes = [C.POINTER(grpo_model_cfg), C.POINTER(grpo_adamw
                                  C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.POINTER(grpo_grads),
                                  _P, _P, C.c_size_t, _P]
 _lib.grpo_adamw_step.restype = C.c_int
+_lib.grpo_adamw_step_lora.argtypes = [C.POINTER(grpo_model_cfg), C.POINTER(grpo_adamw_cfg), C.c_int64, C.POINTER(grpo_lora),
+                                      C.POINTER(grpo_lora_grads), C.POINTER(grpo_lora_grads), C.POINTER(grpo_lora_grads),
+                                      C.POINTER(grpo_lora_grads), C.POINTER(grpo_model), C.POINTER(grpo_grads),
+                                      C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.POINTER(grpo_grads), C.c_void_p,
+                                      C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.grpo_adamw_step_lora.restype = C.c_int
 _lib.pcm_launch_count.restype = C.c_int64
 _lib.pcm_first_use_on_device.argtypes = [C.POINTER(C.c_uint64), C.c_int32]
 _lib.pcm_first_use_on_device.restype = C.c_int32
@@ -152,7 +158,7 @@ EXPORTED = ("pcm_create", "pcm_destroy", "pcm_poll_status", "pcm_state_export", 
             "pcm_score_phases", "pcm_update_keep_probs", "pcm_sample_chunks", "grpo_pack_chunks",
             "grpo_workspace_bytes", "grpo_actor_fwd_bwd", "grpo_gemm", "grpo_attention", "pcm_launch_count",
             "pcm_profile_enable", "pcm_profile_read", "pcm_score_phases_static",
-            "grpo_adamw_scratch_bytes", "grpo_adamw_step", "pcm_label_phases", "pcm_score_phases_f32",
+            "grpo_adamw_scratch_bytes", "grpo_adamw_step", "grpo_adamw_step_lora", "pcm_label_phases", "pcm_score_phases_f32",
             "grpo_attention_wait_status", "pcm_first_use_on_device", "grpo_lora_workspace_bytes",
             "grpo_actor_fwd_bwd_lora")
 
@@ -506,4 +512,49 @@ class AdamW:
                _lib.grpo_adamw_step(C.byref(self.model.cfg), C.byref(self.cfg), self.step_count, C.byref(self.model.c_model),
                                     C.byref(self.c_master), C.byref(self.model.c_grads), C.byref(self.c_m), C.byref(self.c_v),
                                     _ptr(self.grad_norm), self.scratch.data_ptr() + off, self.scratch.numel() - off, _stream()))
+        return self.grad_norm
+
+
+_SMALL = ("g1", "g2", "gf", "w_h", "e_act")
+
+
+class LoraAdamW:
+    """AdamW for LoRA fine-tuning (grpo_adamw_step_lora): fp32 masters and moments for the adapters and, with
+    train_small, for the norm gains, head and action embedding as well; the projections stay frozen."""
+
+    def __init__(self, model: Model, lora: Lora, train_small: bool = True, lr: float = 1e-5, beta1: float = 0.9,
+                 beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.0, max_grad_norm: float = 2.0):
+        self.model, self.lora, self.train_small = model, lora, train_small
+        self.cfg = grpo_adamw_cfg(lr, beta1, beta2, eps, weight_decay, max_grad_norm)
+        self.master = {k: v.float().contiguous() for k, v in lora.tensors.items()}
+        if train_small:
+            self.master.update({k: model.weights[k].float().contiguous() for k in _SMALL})
+        self.m = {k: torch.zeros_like(v) for k, v in self.master.items()}
+        self.v = {k: torch.zeros_like(v) for k, v in self.master.items()}
+        lora_struct = lambda d: grpo_lora_grads(*[_ptr(d[k]) for k in _LORA])
+        small_struct = lambda d: grpo_grads(*[_ptr(d[k]) if k in _SMALL else None for k in _WEIGHTS])
+        self.c_lora = [lora_struct(d) for d in (self.master, self.m, self.v)]
+        self.c_small = [small_struct(d) for d in (self.master, self.m, self.v)] if train_small else None
+        n = int(_lib.grpo_adamw_scratch_bytes())
+        self.scratch = torch.empty(n + 256, dtype=torch.uint8, device="cuda")
+        self.grad_norm = torch.zeros(1, dtype=torch.float32, device="cuda")
+        self.step_count = 0
+
+    def step(self) -> torch.Tensor:
+        """Applies the current adapter (and small-tensor) gradients; returns the (device) norm before clipping."""
+        assert self.lora.c_grads is not None and self.model.c_grads is not None, "run grpo_actor_fwd_bwd with lora first"
+        self.step_count += 1
+        off = (-self.scratch.data_ptr()) % 256
+        ma, mm, mv = self.c_lora
+        if self.train_small:
+            sa, sm, sv = self.c_small
+            ref = lambda x: None if x is None else C.byref(x)
+            small = (ref(self.model.c_model), ref(sa), ref(self.model.c_grads), ref(sm), ref(sv))
+        else:
+            small = (None, None, None, None, None)
+        _check("grpo_adamw_step_lora",
+               _lib.grpo_adamw_step_lora(C.byref(self.model.cfg), C.byref(self.cfg), self.step_count, C.byref(self.lora.c),
+                                         C.byref(ma), C.byref(self.lora.c_grads), C.byref(mm), C.byref(mv), *small,
+                                         _ptr(self.grad_norm), self.scratch.data_ptr() + off, self.scratch.numel() - off,
+                                         _stream()))
         return self.grad_norm

@@ -78,3 +78,62 @@ def test_argument_errors():
     opt = B.AdamW(model, beta1=1.5)
     with pytest.raises(B.PcmError):
         opt.step()
+
+
+@pytest.mark.parametrize("train_small", [True, False])
+def test_lora_training_chain_matches_the_oracle(train_small):
+    """Three iterations of (actor update with adapters -> clip -> AdamW on what is trained), fp32 mode."""
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"].with_(gamma_std=0.1)
+    hp = host_problem(w)
+    lo = synth.make_lora(w, 8, 12.0, b_std=0.05)
+    model = PL.upload_model(w, hp["weights"])
+    lora = PL.upload_lora(w, model, lo)
+    pk = device_packed(B, PL, model, hp)
+    opt = B.LoraAdamW(model, lora, train_small=train_small, lr=1e-3, max_grad_norm=0.01)
+    small = ("g1", "g2", "gf", "w_h", "e_act") if train_small else ()
+    weights = {k: v.astype(np.float64) for k, v in hp["weights"].items()}
+    ad = {k: lo[k].astype(np.float64) for k in synth.LORA_NAMES}
+    start = {**{k: weights[k].copy() for k in small}, **{k: ad[k].copy() for k in ad}}
+    m = {k: np.zeros_like(v) for k, v in start.items()}
+    v = {k: np.zeros_like(v) for k, v in start.items()}
+    frozen_before = {k: model.weights[k].clone() for k in ("w_qkv", "w_o", "w_gu", "w_d")}
+    for step in range(1, 4):
+        B.grpo_actor_fwd_bwd(model, pk, lora=lora)
+        norm_gpu = float(opt.step().item())
+        Xo = hp["X"].copy().astype(np.float64)
+        Xo[:, w.P:] = weights["e_act"][hp["tgt"].astype(int)]
+        lo_now = dict(lo, **ad)
+        _, _, grads_o, _ = ao.fwd_bwd(weights, Xo, hp["tgt"], hp["lpo"], hp["adv_c"], w.H, w.P, 0.2, 0.2, lora=lo_now)
+        params = {**{k: weights[k] for k in small}, **ad}
+        norm_o = oo.adamw_step(params, {k: grads_o[k] for k in params}, m, v, step, lr=1e-3, max_norm=0.01)
+        for k in small:
+            weights[k] = params[k]
+        for k in ad:
+            ad[k] = params[k]
+        assert norm_o > 0.01
+        assert norm_gpu == pytest.approx(norm_o, rel=2e-5)
+        pk.X[:, w.P:] = model.weights["e_act"][pk.tgt.long()]
+        for k in params:
+            assert rel_fro(opt.master[k].cpu().numpy() - start[k], params[k] - start[k]) < 5e-4, (step, k)
+            live = lora.tensors[k] if k in lora.tensors else model.weights[k]
+            assert torch.equal(live, opt.master[k]), k
+    for k, t in frozen_before.items():
+        assert torch.equal(model.weights[k], t), k
+    if not train_small:
+        for k in ("g1", "g2", "gf", "w_h", "e_act"):
+            assert np.array_equal(model.weights[k].cpu().numpy(), hp["weights"][k].astype(np.float32)), k
+
+
+def test_lora_optimizer_wants_all_or_none_of_the_small_tensor_sets():
+    B, PL = _mods()
+    w = synth.WORKLOADS["C0"]
+    hp = host_problem(w)
+    model = PL.upload_model(w, hp["weights"])
+    lora = PL.upload_lora(w, model, synth.make_lora(w, 8, 8.0))
+    model.alloc_grads()
+    lora.alloc_grads()
+    opt = B.LoraAdamW(model, lora, train_small=True)
+    opt.c_small[1] = None                    # moments missing while the rest is given
+    with pytest.raises(B.PcmError):
+        opt.step()
