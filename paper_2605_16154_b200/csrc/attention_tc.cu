@@ -27,7 +27,7 @@ namespace pcm {
 
 __device__ unsigned g_fa_status = 0;          // bit 0: a bounded wait expired; bit 8 + site: which wait it was
 __device__ __forceinline__ void fa_timeout(int site) { atomicOr(&g_fa_status, 1u | (1u << (8 + site))); }
-enum { SITE_KV_EMPTY = 0, SITE_Q_EMPTY = 1, SITE_KV_FULL = 2, SITE_Q_FULL = 3, SITE_P_FULL = 4, SITE_O_EMPTY = 5, SITE_O_FULL = 6, SITE_S_FULL = 7 };
+enum { SITE_KV_EMPTY = 0, SITE_Q_EMPTY = 1, SITE_KV_FULL = 2, SITE_Q_FULL = 3, SITE_P_FULL = 4, SITE_O_EMPTY = 5, SITE_O_FULL = 6, SITE_S_FULL = 7, SITE_PLAN = 8 };
 
 namespace fatc {
 
@@ -618,6 +618,7 @@ struct BwParams {
   const __nv_bfloat16* out;                     // [n_seq*S][d]
   const __nv_bfloat16* dout;                    // [n_seq*S][d]
   const float2* rope_tab;                       // [S][dh/2] (cos, sin) or nullptr
+  __nv_bfloat16* dqkv;                          // [n_seq*S][3d]: the one-pass kernel stores rows itself
 };
 
 __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -1221,6 +1222,41 @@ fa_tc_bwd_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_constan
   }
 }
 
+#include "attention_tc_bwd1.cuh"
+
+// rowsum(dO o O) per (token, head) for head dim 64, written as dsum[sequence][head][position]: 16-byte chunks, eight
+// consecutive lanes per head, fully coalesced; HBM-bound (reads O and dO once).
+__global__ void __launch_bounds__(256)
+fa_rowsum64_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout, float* __restrict__ dsum,
+                   long long n_tokens, int S, int H) {
+  const int cpr = H * 8;                                              // 16-byte chunks per token row
+  const long long total = n_tokens * cpr;
+  const long long stride = (long long)gridDim.x * blockDim.x;        // a multiple of 32: a head's 8 chunks stay in one lane group
+  for (long long c0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; c0 - (threadIdx.x & 31) < total; c0 += stride) {   // warp-uniform
+    float part = 0.f;
+    if (c0 < total) {
+      const uint4 a = reinterpret_cast<const uint4*>(out)[c0], g = reinterpret_cast<const uint4*>(dout)[c0];
+      const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* gh = reinterpret_cast<const __nv_bfloat162*>(&g);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 af = __bfloat1622float2(ah[e]), gf = __bfloat1622float2(gh[e]);
+        part = fmaf(af.x, gf.x, part);
+        part = fmaf(af.y, gf.y, part);
+      }
+    }
+    part += __shfl_xor_sync(0xffffffffu, part, 1);
+    part += __shfl_xor_sync(0xffffffffu, part, 2);
+    part += __shfl_xor_sync(0xffffffffu, part, 4);
+    if ((threadIdx.x & 7) == 0 && c0 < total) {
+      const long long tok = c0 / cpr;
+      const int h = (int)(c0 - tok * cpr) >> 3;
+      const long long seq = tok / S;
+      dsum[(seq * H + h) * S + (tok - seq * S)] = part;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
@@ -1322,6 +1358,7 @@ static int bwd_launch(const void* qkv, const void* out, const void* dout, const 
   p.lse = lse; p.dsum = dsum;
   p.out = (const __nv_bfloat16*)out; p.dout = (const __nv_bfloat16*)dout;
   p.rope_tab = rope_tab;
+  p.dqkv = (__nv_bfloat16*)dqkv;
   CUtensorMap tmQKV, tmDO, tmOUT, tmDQKV;
   if (!make_seq_tmap(&tmQKV, qkv, n_seq, S, 3LL * d, 3LL * d, BM) || !make_seq_tmap(&tmDO, dout, n_seq, S, d, d, BM) ||
       !make_seq_tmap(&tmOUT, out, n_seq, S, d, d, BM) ||
@@ -1330,6 +1367,46 @@ static int bwd_launch(const void* qkv, const void* out, const void* dout, const 
   const int rc = bwd_launch_one<DH, BW_DQ>(tmQKV, tmDO, tmOUT, tmDQKV, p, s);     // also writes rowsum(dO o O) for the second launch
   if (rc != PCM_OK) return rc;
   return bwd_launch_one<DH, BW_DKV>(tmQKV, tmDO, tmOUT, tmDQKV, p, s);
+}
+
+// PCM_ATTN_BWD=2 keeps head dim 64 on the two-launch backward (dQ, then dK / dV), for comparison runs.
+static bool one_pass_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("PCM_ATTN_BWD");
+    v = (e && e[0] == '2') ? 0 : 1;
+  }
+  return v == 1;
+}
+
+static int bwd1_launch(const void* qkv, const void* out, const void* dout, const float* lse, float* dsum, void* dqkv,
+                       int n_seq, int S, int H, const float2* rope_tab, cudaStream_t s) {
+  constexpr int DH = 64;
+  const int d = H * DH;
+  BwParams p;
+  p.n_seq = n_seq; p.S = S; p.H = H; p.d = d;
+  p.nq = (S + BM - 1) / BM;
+  p.n_items = n_seq * H;
+  p.n_total = ((S + 15) / 16) * 16;
+  p.scale = 1.f / sqrtf((float)DH);
+  p.scale_log2 = LOG2E / sqrtf((float)DH);
+  p.lse = lse; p.dsum = dsum;
+  p.out = (const __nv_bfloat16*)out; p.dout = (const __nv_bfloat16*)dout;
+  p.rope_tab = rope_tab;
+  p.dqkv = (__nv_bfloat16*)dqkv;
+  CUtensorMap tmQKV, tmDO, tmDQKV;
+  if (!make_seq_tmap(&tmQKV, qkv, n_seq, S, 3LL * d, 3LL * d, BM) || !make_seq_tmap(&tmDO, dout, n_seq, S, d, d, BM) ||
+      !make_seq_tmap(&tmDQKV, dqkv, n_seq, S, 3LL * d, 3LL * d, BM))
+    return PCM_ERR_CUDA;
+  fa_rowsum64_kernel<<<sm_count() * 8, 256, 0, s>>>(p.out, p.dout, dsum, (long long)n_seq * S, S, H);
+  PCM_LAUNCH_CHECK();
+  static unsigned long long attr_devices = 0;
+  if (attr_needed(&attr_devices))
+    PCM_CUDA_TRY(cudaFuncSetAttribute(fa_tc_bwd1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)b1::SMEM_BYTES));
+  const int grid = p.n_items < sm_count() ? p.n_items : sm_count();
+  fa_tc_bwd1_kernel<<<grid, b1::THREADS, b1::SMEM_BYTES, s>>>(tmQKV, tmDO, tmDQKV, p);
+  PCM_LAUNCH_CHECK();
+  return PCM_OK;
 }
 
 }  // namespace fatc
@@ -1348,6 +1425,7 @@ int attention_bwd_bf16_tc(const void* qkv, const void* out, const void* dout, co
                           int n_seq, int S, int H, int dh, const float2* rope_tab, cudaStream_t s) {
   if (!attention_tc_supported(qkv, out, S, H, dh) || ((((uintptr_t)dout) | ((uintptr_t)dqkv)) & 15)) return PCM_ERR_SHAPE;
   if (n_seq < 1) return PCM_OK;
+  if (dh == 64 && fatc::one_pass_enabled()) return fatc::bwd1_launch(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s);
   return dh == 64 ? fatc::bwd_launch<64>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s)
                   : fatc::bwd_launch<128>(qkv, out, dout, lse, dsum, dqkv, n_seq, S, H, rope_tab, s);
 }
