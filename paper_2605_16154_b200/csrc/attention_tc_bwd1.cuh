@@ -385,18 +385,20 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
       }
       if (!__shfl_sync(0xffffffffu, ok, 0)) dead = true;
     };
-    // statistics of a block's 128 queries: lse * log2(e) (threads 0..127; +inf past the sequence gives probability 0)
-    // and rowsum(dO o O) (threads 128..255), both from global memory
+    // statistics of a block's 128 queries: lse (threads 0..127; +inf past the sequence gives probability 0) and
+    // rowsum(dO o O) (threads 128..255), both from global memory.  Raw values: the scaling by log2(e) happens where the
+    // value is stored, a block later, so that the load has that block to land.
     auto stat_of = [&](const B1Iter& q) -> float {
       const int qi = q.i * BM + (ct & (BM - 1));
       if (ct >= 2 * BM) return 0.f;
       const long long at = ((long long)(q.sh / p.H) * p.H + q.sh % p.H) * p.S + qi;
-      if (ct < BM) return qi < p.S ? p.lse[at] * LOG2E : INFINITY;
+      if (ct < BM) return qi < p.S ? p.lse[at] : INFINITY;
       return qi < p.S ? p.dsum[at] : 0.f;
     };
+    const float stat_scale = ct < BM ? LOG2E : 1.f;
     B1Iter it;
     it.init();
-    if (it.valid(n_sh) && ct < 2 * BM) cstat[ct] = stat_of(it);
+    if (it.valid(n_sh) && ct < 2 * BM) cstat[ct] = stat_of(it) * stat_scale;
     for (; it.valid(n_sh); it.next(nq)) {
       const int b = it.b;
       const float* cst = cstat + (b & 1) * 2 * BM;
@@ -470,7 +472,7 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0 && !dead) mbar_arrive(&pds_ready[b & 1]);
-      if (have_next && ct < 2 * BM) cstat[((b + 1) & 1) * 2 * BM + ct] = stat_next;
+      if (have_next && ct < 2 * BM) cstat[((b + 1) & 1) * 2 * BM + ct] = stat_next * stat_scale;
     }
   }
 
