@@ -21,9 +21,10 @@
  *   - Chunks are stored CSR style: trajectory i owns chunks traj_off[i] .. traj_off[i+1]-1.
  *   - A chunk is 56 action tokens (8 actions x 7 degrees of freedom, Sec. 5.1) over 256 bins.
  *   - Every linear weight is stored row-major [out_features][in_features] (y = x W^T).
- *   - Three environment variables, read once per process, exist for comparison runs and are not part of the
+ *   - Four environment variables, read once per process, exist for comparison runs and are not part of the
  *     interface: PCM_GEMM_BACKEND=simt|tcgen05 forces the GEMM kernel family, PCM_GEMM_PAIR=0 keeps the tensor-core
- *     GEMM on single CTAs, PCM_ATTN_TC=0 keeps bf16 attention on the warp-level kernels.
+ *     GEMM on single CTAs, PCM_ATTN_TC=0 keeps bf16 attention on the warp-level kernels, PCM_ATTN_BWD=2 keeps the
+ *     head-dim-64 attention backward on the two-launch kernels.
  */
 #ifndef PCM_B200_H
 #define PCM_B200_H
