@@ -85,24 +85,18 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
   }
   uint8_t* base = smem_raw + tiles_at;
   uint64_t* kv_full = bars;                    // [2] producer -> opening MMAs: K_j | V_j landed
-  uint64_t* kv_empty = bars + 2;               // [2] dQ's MMAs and the storing thread (dK, dV were staged there) -> producer
+  uint64_t* kv_empty = bars + 2;               // [2] dQ's MMAs (the key tile's last readers) -> producer
   uint64_t* q_full = bars + 4;                 // [3] producer -> opening MMAs, compute warps: Q_i | dO_i landed
-  uint64_t* q_empty = bars + 7;                // [3] dK / dV's MMAs of the tile's diagonal block and the storing thread (dQ_i was staged there) -> producer
+  uint64_t* q_empty = bars + 7;                // [3] dK / dV's MMAs of the tile's diagonal block and the storing thread (dQ_i, dK_i, dV_i were staged there) -> producer
   uint64_t* sdp_full = bars + 10;              // opening MMAs -> compute: S^T and dP^T of a block are in tensor memory
   uint64_t* sdp_read = bars + 11;              // compute (16 warps) -> opening MMAs: both have been read
   uint64_t* pds_ready = bars + 12;             // [2] compute (16 warps) -> accumulating MMAs: P^T and dS^T are in shared memory
-  uint64_t* p_free = bars + 14;                // accumulating MMAs -> compute: dV's products have read P^T
-  uint64_t* ds_free = bars + 15;               // accumulating MMAs -> compute: dK's and dQ's products have read dS^T
+  uint64_t* ds_free = bars + 15;               // accumulating MMAs (two threads) -> compute: the block's products have read P^T and dS^T
   uint64_t* dq_full = bars + 16;               // [2] accumulating MMAs -> output warps
   uint64_t* dq_empty = bars + 18;              // [2] output warps (4) -> accumulating MMAs
   uint64_t* dkv_full = bars + 20;
   uint64_t* dkv_empty = bars + 21;             // output warps (4): dK and dV have been read
   uint64_t* qi_done = bars + 22;               // dK / dV's MMAs -> output warps: a diagonal block's products have read Q_i | dO_i
-  // [2] dQ's MMAs -> output warps: a key tile's last product has read K_j.  Key tiles alternate between two barriers:
-  // the dQ thread does not wait for the output warps at a key tile of one block, so it can complete the next tile's
-  // phase before a late output warp has looked at this one's, and a parity wait cannot tell a phase from the one two
-  // later; the tile after next cannot complete before every output warp has released this tile's dK and dV.
-  uint64_t* kq_done = bars + 23;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
@@ -111,12 +105,12 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
   const int nb_tail = p.n_total - (nq - 1) * BN;                      // rows of a sequence's last tile that take part (multiple of 16)
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 2); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&kv_full[s], 1); mbar_init(&kv_empty[s], 1); }
     for (int s = 0; s < 3; ++s) { mbar_init(&q_full[s], 1); mbar_init(&q_empty[s], 2); }
     mbar_init(sdp_full, 1); mbar_init(sdp_read, BW_COMPUTE_WARPS);
     mbar_init(&pds_ready[0], BW_COMPUTE_WARPS); mbar_init(&pds_ready[1], BW_COMPUTE_WARPS);
-    mbar_init(p_free, 1); mbar_init(ds_free, 2);                      // dS^T is read by both accumulating threads
-    mbar_init(qi_done, 1); mbar_init(&kq_done[0], 1); mbar_init(&kq_done[1], 1);
+    mbar_init(ds_free, 2);                                            // dS^T is read by both accumulating threads
+    mbar_init(qi_done, 1);
     for (int s = 0; s < 2; ++s) { mbar_init(&dq_full[s], 1); mbar_init(&dq_empty[s], 4); }
     mbar_init(dkv_full, 1); mbar_init(dkv_empty, 4);
     *abort_flag = 0;
@@ -237,7 +231,6 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
             if (ks < nkq)
               umma_bf16(tmem_base + COL_DV, desc(dpk_lo + (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2), hi_k),
                         desc(q_lo + (TILE >> 4) + (uint32_t)(ks * 128), hi_m), idesc_kk, 1u);
-          umma_commit(p_free);
           umma_bf16(tmem_base + COL_DK, desc(dsk_lo, hi_k), desc(q_lo, hi_m), idesc_kk, acc);
 #pragma unroll
           for (int ks = 1; ks < BN / 16; ++ks)
@@ -267,7 +260,7 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
               umma_bf16(d_col, desc(dsm_lo + (uint32_t)(kk * 128), hi_m), desc(k_lo + (uint32_t)(kk * 128), hi_m), idesc_mm, 1u);
           umma_commit(ds_free);
           if (it.group_first()) umma_commit(&dq_full[slot]);                     // the diagonal block is dQ_i's last
-          if (it.group_last(nq)) { umma_commit(&kq_done[it.g & 1]); umma_commit(&kv_empty[it.g & 1]); }
+          if (it.group_last(nq)) umma_commit(&kv_empty[it.g & 1]);
         }
       }
       if (!ok) *abort_flag = 1;
@@ -276,9 +269,10 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
     // ------------------------------ output: warps 2..5, one lane quadrant each ------------------------------
     // A thread owns one row of an accumulator: 64 fp32 columns -> scale, inverse rotary embedding (dQ, dK) -> bf16 into
     // a staging tile in the swizzled layout of the gradient tensor map -> one TMA store (rows past the sequence are
-    // clipped).  The staging tile is an operand tile that has just been read for the last time: Q_i for dQ_i (after
-    // the diagonal block), K_j and V_j for dK_j and dV_j (after the key tile's last block); the storing thread hands
-    // it to the producer once the store has read it.  Accumulators are released as soon as they are in registers.
+    // clipped).  The staging tiles are the slot of query tile t, which no product reads after t's diagonal block: dQ_t
+    // right after that block, dK_t and dV_t (both halves of the slot) after key tile t's last block; then the storing
+    // thread hands the slot to the producer for the next item.  Accumulators are released as soon as they are in
+    // registers.
     const int quad = warp & 3, row = quad * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const bool storer = warp == 2 && lane == 0;
@@ -350,20 +344,18 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
         wait_warp(&dq_full[slot], (unsigned)(cnt >> 1) & 1u);
         emit((uint32_t)(COL_DQ + slot * DH), &dq_empty[slot], 0, it.i, seq, h, qi_done, (unsigned)it.g & 1u,
              base + Q_OFF + it.i * PAIR);
-        if (storer) {
-          bulk_wait_read_all();
-          if (!dead) mbar_arrive(&q_empty[it.i]);
-        }
+        if (storer) bulk_wait_read_all();                                 // dK_i will be staged over it
       }
       if (it.group_last(nq)) {
         wait_warp(dkv_full, (unsigned)it.g & 1u);
-        uint8_t* kv_stage = base + KV_OFF + (it.g & 1) * PAIR;
+        named_bar_sync(BW_OUT_BAR, 128);                                  // the store of dQ_j has read its staging tile
+        uint8_t* slot_j = base + Q_OFF + it.j * PAIR;
         // the two accumulators are released together: one arrival per warp, after dV has been read as well
-        emit((uint32_t)COL_DK, nullptr, 1, it.j, seq, h, &kq_done[it.g & 1], (unsigned)(it.g >> 1) & 1u, kv_stage);
-        emit((uint32_t)COL_DV, dkv_empty, 2, it.j, seq, h, nullptr, 0u, kv_stage + TILE);
+        emit((uint32_t)COL_DK, nullptr, 1, it.j, seq, h, nullptr, 0u, slot_j);
+        emit((uint32_t)COL_DV, dkv_empty, 2, it.j, seq, h, nullptr, 0u, slot_j + TILE);
         if (storer) {
           bulk_wait_read_all();
-          if (!dead) mbar_arrive(&kv_empty[it.g & 1]);
+          if (!dead) mbar_arrive(&q_empty[it.j]);                         // query tile j's slot goes back to the producer
         }
       }
     }
@@ -455,14 +447,14 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
       // the buffers are single: the previous block's products must have read them
       uint8_t* prow = base + P_OFF + (slice >> 1) * TILE + row * 128;
       uint8_t* drow = base + DS_OFF + (slice >> 1) * TILE + row * 128;
-      if (b >= 1) wait_warp(p_free, (unsigned)(b - 1) & 1u, SITE_P_FULL);
+      // (ds_free counts the commit that follows dK's products, which the same thread issues after dV's: it covers P^T too)
+      if (b >= 1) wait_warp(ds_free, (unsigned)(b - 1) & 1u, SITE_P_FULL);
       if (active) {
 #pragma unroll
         for (int c = 0; c < 4; ++c)
           *reinterpret_cast<uint4*>(prow + (((((slice & 1) << 2) + c) ^ (row & 7)) << 4)) =
               make_uint4(pp[4 * c], pp[4 * c + 1], pp[4 * c + 2], pp[4 * c + 3]);
       }
-      if (b >= 1) wait_warp(ds_free, (unsigned)(b - 1) & 1u, SITE_P_FULL);
       if (active) {
 #pragma unroll
         for (int c = 0; c < 4; ++c)
