@@ -425,18 +425,23 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
             if (lane == 0) mbar_arrive(sdp_read);
           }
 #pragma unroll
-          for (int e = 0; e < 16; e += 2) {
-            float pr[2], ds[2];
+          for (int e = 0; e < 16; e += 4) {
+            const int c0 = slice * 32 + hc + e;                        // statistics of four queries per 16-byte load
+            const float4 l4 = *reinterpret_cast<const float4*>(cst + c0);
+            const float4 d4 = *reinterpret_cast<const float4*>(cst + BM + c0);
+            const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dv[4] = {d4.x, d4.y, d4.z, d4.w};
+            float pr[4], ds[4];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const int c = slice * 32 + hc + e + u;
-              float pv = ex2_approx(fmaf(__uint_as_float(rs[e + u]), c2, -cst[c]));
-              if (mode_mask == 1) pv = c >= row ? pv : 0.f;
+            for (int u = 0; u < 4; ++u) {
+              float pv = ex2_approx(fmaf(__uint_as_float(rs[e + u]), c2, -lv[u]));
+              if (mode_mask == 1) pv = c0 + u >= row ? pv : 0.f;
               pr[u] = pv;
-              ds[u] = pv * (__uint_as_float(rd[e + u]) - cst[BM + c]);
+              ds[u] = pv * (__uint_as_float(rd[e + u]) - dv[u]);
             }
             pp[(hc + e) >> 1] = pack_bf16x2(pr[0], pr[1]);
+            pp[((hc + e) >> 1) + 1] = pack_bf16x2(pr[2], pr[3]);
             pd[(hc + e) >> 1] = pack_bf16x2(ds[0], ds[1]);
+            pd[((hc + e) >> 1) + 1] = pack_bf16x2(ds[2], ds[3]);
           }
         }
       } else {
