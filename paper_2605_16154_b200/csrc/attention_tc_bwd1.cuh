@@ -54,6 +54,12 @@ struct B1Iter {
   }
 };
 
+// Asks for a tile of a 3-D tensor map to be brought into L2 (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_3d(const void* tmap, int x, int y, int z) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tmap), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+
 // Named barrier that also ORs a flag over its participants: every thread gets the same answer, so a group of warps
 // leaves a loop together and none is left waiting at the barrier.
 __device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool flag) {
@@ -143,6 +149,17 @@ fa_tc_bwd1_kernel(const __grid_constant__ CUtensorMap tmQKV, const __grid_consta
         bool moved = false;
         if (kv_sh < n_sh && mbar_test_wait(&kv_empty[kv_g & 1], ((unsigned)(kv_g >> 1) & 1u) ^ 1u)) {
           const int h = kv_sh % p.H, seq = kv_sh / p.H, st = kv_g & 1;
+          if (kv_j == 0 && kv_sh + (int)gridDim.x < n_sh) {
+            // an item's first request: ask L2 for the whole next item, so that its loads, which can only be issued
+            // a block or two before they are needed, do not wait for DRAM
+            const int nsh = kv_sh + gridDim.x, nh = nsh % p.H, nseq = nsh / p.H;
+            for (int t = 0; t < nq; ++t) {
+              tma_prefetch_3d(&tmQKV, nh * DH, t * BM, nseq);
+              tma_prefetch_3d(&tmDO, nh * DH, t * BM, nseq);
+              tma_prefetch_3d(&tmQKV, p.d + nh * DH, t * BM, nseq);
+              tma_prefetch_3d(&tmQKV, 2 * p.d + nh * DH, t * BM, nseq);
+            }
+          }
           mbar_expect_tx(&kv_full[st], PAIR);
           uint8_t* dst = base + KV_OFF + st * PAIR;
           tma_load_3d(dst, &tmQKV, p.d + h * DH, kv_j * BM, seq, &kv_full[st]);
