@@ -177,3 +177,69 @@ def test_attention_at_the_full_batch_shape_on_sampled_sequences_and_heads():
         assert rel_fro(got[:, cols(2)], dv[0, 0]) < 2e-2, (s_i, h_i)
         lse_o = np.log(np.exp(q[0, 0] @ k[0, 0].T / np.sqrt(dh) + np.triu(np.full((S, S), -np.inf), 1)).sum(-1))
         assert np.max(np.abs(lse[s_i, h_i].cpu().numpy() - lse_o)) < 2e-2, (s_i, h_i)
+
+
+def test_attention_backward_repeats_bit_identically_over_many_items_per_cta():
+    """The one-pass backward keeps a dozen roles in step through barriers whose phases come around every other item;
+    a mis-counted phase shows up as a bounded wait that expires or as a tile taken too early.  Sizes from 2 to 40 items
+    per CTA, each run several times: every run must end without a device timeout and give the same bits (no atomics:
+    the order of every accumulation is fixed), and one run is checked against the oracle on sampled (sequence, head)s."""
+    from paper_2605_16154_b200 import binding as B
+    S, H, dh = 312, 16, 64
+    d = H * dh
+    for n_seq in (19, 74, 150):
+        g = torch.Generator(device="cuda").manual_seed(n_seq)
+        qkv = torch.randn((n_seq * S, 3 * d), generator=g, device="cuda").to(torch.bfloat16)
+        do = torch.randn((n_seq * S, d), generator=g, device="cuda").to(torch.bfloat16)
+        first = None
+        for rep in range(8):
+            _, _, dqkv = B.grpo_attention(qkv, n_seq, S, H, dh, dout=do)
+            if first is None:
+                first = dqkv.clone()
+            else:
+                assert torch.equal(dqkv, first), (n_seq, rep)
+        assert B.grpo_attention_wait_status() == 0
+        for s_i, h_i in ((0, 0), (n_seq - 1, H - 1), (n_seq // 2, 7)):
+            rows = slice(s_i * S, (s_i + 1) * S)
+            cols = lambda part: slice(part * d + h_i * dh, part * d + (h_i + 1) * dh)
+            blk = qkv[rows].float().cpu().numpy().astype(np.float64)
+            q, k, v = (blk[:, cols(i)][None, None] for i in range(3))
+            _, p = ao.causal_attention(q, k, v)
+            go = do[rows, h_i * dh:(h_i + 1) * dh].float().cpu().numpy().astype(np.float64)[None, None]
+            dq, dk, dv = ao.causal_attention_bwd(go, q, k, v, p)
+            got = first[rows].float().cpu().numpy()
+            for part, ref in enumerate((dq, dk, dv)):
+                assert rel_fro(got[:, cols(part)], ref[0, 0]) < 2e-2, (n_seq, s_i, h_i, part)
+
+
+def test_two_launch_attention_backward_stays_correct_at_head_dim_64():
+    """PCM_ATTN_BWD=2 (read once per process, hence a child process) keeps head dim 64 on the dQ / dK-dV launches, which
+    are also the head-dim-128 path: the same attention case as the parity tests, against the oracle."""
+    import os
+    import subprocess
+    import sys
+    code = r'''
+import numpy as np, torch
+from oracle import actor_oracle as ao
+from paper_2605_16154_b200 import binding as B
+n_seq, S, H, dh = 5, 312, 3, 64
+d = H * dh
+rng = np.random.default_rng(5)
+qkv = torch.from_numpy(rng.standard_normal((n_seq * S, 3 * d)).astype(np.float32)).cuda().to(torch.bfloat16)
+do = torch.from_numpy(rng.standard_normal((n_seq * S, d)).astype(np.float32)).cuda().to(torch.bfloat16)
+out, lse, dqkv = B.grpo_attention(qkv, n_seq, S, H, dh, dout=do)
+heads = lambda x: x.float().cpu().numpy().astype(np.float64).reshape(n_seq, S, H, dh).transpose(0, 2, 1, 3)
+q, k, v = heads(qkv[:, :d]), heads(qkv[:, d:2 * d]), heads(qkv[:, 2 * d:])
+o, p = ao.causal_attention(q, k, v)
+ref = ao.causal_attention_bwd(heads(do), q, k, v, p)
+back = lambda x: x.transpose(0, 2, 1, 3).reshape(n_seq * S, d)
+got = dqkv.float().cpu().numpy()
+err = max(np.linalg.norm(got[:, i * d:(i + 1) * d] - back(ref[i])) / np.linalg.norm(back(ref[i])) for i in range(3))
+assert err < 2e-2, err
+print("two-launch ok", err)
+'''
+    env = dict(os.environ, PCM_ATTN_BWD="2")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stdout + res.stderr
+    assert "two-launch ok" in res.stdout
