@@ -1,5 +1,6 @@
 // bf16 causal attention inside each chunk's sequence on the 5th-generation tensor cores: the forward pass
-// (described here) and, further down, the backward pass (one kernel template launched for dQ and for dK / dV).
+// (described here) and, further down, the backward pass: one kernel template launched for dQ and for dK / dV (head
+// dim 128, and head dim 64 on request), and the one-pass kernel of attention_tc_bwd1.cuh (head dim 64).
 //
 // Forward.  One persistent CTA per SM walks (sequence, head) items.  The whole K and V of an item (S <= 384 rows)
 // sit in shared memory (TMA, 128-byte swizzle); query tiles of 128 rows stream through a small ring.
